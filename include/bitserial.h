@@ -1,0 +1,172 @@
+/*
+ * bitserial.h -- C ABI of the bit-serial ultra-low-bit convolution library for NVIDIA B200 (sm_100a).
+ *
+ * Method (paper, Section V): weights (w bits) and activations (a bits) are split into bitplanes and
+ * packed into machine words.  A dot product is then
+ *       1-bit unipolar:   W . A = POPCOUNT(W & A)
+ *       multi-bit:        W . A = sum_{i<w} sum_{j<a} POPCOUNT(W[i] & A[j]) << (i + j)
+ * Extensions the paper leaves open and this library fixes:
+ *   - two's-complement operands: the top plane carries weight -2^(b-1);
+ *   - 1-bit bipolar operands {-1,+1} (stored bit 1 <-> +1): v = 2*bit - 1 is expanded algebraically,
+ *     which for two bipolar operands is the identity dot = K - 2*POPCOUNT(a XOR w);
+ *   - zero padding (value 0 has every plane 0, so out-of-image taps add nothing);
+ *   - a fused per-output-channel requantisation epilogue (Section IV quantiser applied to
+ *     scale*acc + bias), exact operation order documented at bs_conv_params.
+ * The quantiser (paper, Section IV) is  code = round(clip(x / s, qmin, qmax)), round-to-nearest-even,
+ * with [qmin, qmax] = [-2^(b-1), 2^(b-1)-1] (signed) or [0, 2^b-1] (unsigned).
+ *
+ * General conventions
+ *   - Every function returns a bs_status.  Nothing throws, aborts or prints.
+ *   - Every tensor pointer is DEVICE memory owned by the caller, 16-byte aligned, valid on the current
+ *     device; `stream` is a cudaStream_t passed as void* (NULL = the legacy default stream).  Calls
+ *     only enqueue work; they never synchronise and never allocate device memory.
+ *   - bs_conv_params / scalar arguments are HOST values, read before the call returns.
+ *   - Supported: bit-widths 1..4; sign BS_BIPOLAR only with 1 bit; square kernels R == S in
+ *     {1, 3, 5, 7}; stride in {1, 2}; 0 <= pad < R.  Bipolar activations need pad == 0 (zero is not
+ *     representable).  Shapes must keep |acc| < 2^31 (checked on the host).
+ *
+ * Packed storage (uint32 words, little-endian bit numbering):
+ *   activations  [N][H][W][Cw][a_bits]      Cw = ceil(C / 32)
+ *   weights      [O][R][S][Cw][w_bits]
+ *   matrix rows  [rows][Kw][bits]           Kw = ceil(K / 32)
+ *   Bit (c % 32) of word (c / 32) of plane j holds bit j of the stored pattern of channel c.  The
+ *   stored pattern of an unsigned or two's-complement code is its low `bits` bits; a bipolar code
+ *   stores 1 for +1 and 0 for -1.  Channels beyond C are stored as 0 in every plane.
+ *   A 1x1 convolution over N*H*W pixels and a matrix product over M = N*H*W rows use identical bytes.
+ */
+#ifndef BITSERIAL_H_
+#define BITSERIAL_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    BS_OK = 0,
+    BS_ERR_INVALID_ARG = 1, /* null pointer, non-positive size, bits outside 1..4, bad enum ...      */
+    BS_ERR_UNSUPPORTED = 2, /* well-formed but outside the supported set listed above                 */
+    BS_ERR_ALIGNMENT = 3,   /* a tensor pointer is not 16-byte aligned                                */
+    BS_ERR_CUDA = 4,        /* a CUDA runtime/driver call failed (launch error, no device, ...)       */
+    BS_ERR_TIMEOUT = 5      /* a bounded device-side wait ran out (reported by bs_check_status)       */
+} bs_status;
+
+typedef enum { BS_UNSIGNED = 0, BS_SIGNED = 1, BS_BIPOLAR = 2 } bs_sign_t;
+typedef enum { BS_NCHW = 0, BS_NHWC = 1 } bs_layout_t; /* for weights: OIHW = BS_NCHW, OHWI = BS_NHWC */
+
+/* Bytes of a packed activation tensor / packed weight tensor / packed row matrix (0 on bad input). */
+size_t bs_packed_act_bytes(int N, int C, int H, int W, int a_bits);
+size_t bs_packed_wgt_bytes(int O, int C, int R, int S, int w_bits);
+size_t bs_packed_rows_bytes(int rows, int K, int bits);
+
+/*
+ * bitpack_activations -- Section IV quantiser followed by the Section V bitplane split.
+ *   x          device, [N][C][H][W] (BS_NCHW) or [N][H][W][C] (BS_NHWC); float32 when x_is_fp32 != 0,
+ *              otherwise int8 codes already inside the code range of (a_bits, a_sign).
+ *   act_scale  the step s of the quantiser (> 0, finite); ignored for int8 input.
+ *              Bipolar: code = +1 when x >= 0 else -1.
+ *   packed_out device, bs_packed_act_bytes(N, C, H, W, a_bits) bytes, fully overwritten.
+ * Inputs must be finite.  One pass over x; bound by HBM bandwidth.
+ */
+int bitpack_activations(const void* x, int x_is_fp32, bs_layout_t layout, int N, int C, int H, int W,
+                        float act_scale, int a_bits, bs_sign_t a_sign, uint32_t* packed_out, void* stream);
+
+/* Inverse of the plane split (test and debugging aid): packed activations -> int8 codes in `layout`. */
+int bitunpack_activations(const uint32_t* packed, int N, int C, int H, int W, int a_bits, bs_sign_t a_sign,
+                          bs_layout_t layout, int8_t* codes_out, void* stream);
+
+/*
+ * pack_weights -- Section V bitplane split of quantised weights (done once per layer, off the hot loop).
+ *   w_codes    device int8, [O][C][R][S] (BS_NCHW) or [O][R][S][C] (BS_NHWC), inside the code range.
+ *   packed_out device, bs_packed_wgt_bytes(O, C, R, S, w_bits) bytes, fully overwritten.
+ */
+int pack_weights(const int8_t* w_codes, bs_layout_t layout, int O, int C, int R, int S, int w_bits,
+                 bs_sign_t w_sign, uint32_t* packed_out, void* stream);
+
+/* Plane split of a row-major int8 code matrix [rows][K] into [rows][Kw][bits] (operands of bitserial_gemm). */
+int bs_pack_rows(const int8_t* codes, int rows, int K, int bits, bs_sign_t sign, uint32_t* packed_out,
+                 void* stream);
+
+/*
+ * Convolution problem (host struct).  Output size P = (H + 2*pad - R)/stride + 1, Q likewise.
+ *
+ * Accumulator (exact int32):  acc[n][o][p][q] = sum_{c,r,s} a[n][c][p*stride-pad+r][q*stride-pad+s] * w[o][c][r][s]
+ * evaluated as the Section V plane-pair popcount sum with the sign handling described at the top.
+ *
+ * Epilogue, applied when out_packed != NULL, in exactly this order in IEEE binary32:
+ *     v = fmaf((float)acc, scale[o], bias[o]);
+ *     if (residual) v = fmaf(res_scale, (float)res_code, v);
+ *     if (relu)     v = fmaxf(v, 0.0f);
+ *     v = fminf(fmaxf(v, qmin), qmax);            (clip, then round: order of the Section IV quantiser)
+ *     code = (int) rintf(v);                      (ties to even; out_sign BS_BIPOLAR: code = v >= 0 ? +1 : -1)
+ * and the codes are split into out_bits planes and stored as packed activations [N][P][Q][Ow][out_bits]
+ * with Ow = ceil(out_c_total / 32), at channels [out_c_offset, out_c_offset + O) (concatenation for free).
+ */
+typedef struct {
+    int N, C, H, W;          /* input: batch, channels, height, width                                 */
+    int O, R, S;             /* filters and kernel size                                                */
+    int stride, pad;
+    int a_bits;  int a_sign; /* activation bits and bs_sign_t                                          */
+    int w_bits;  int w_sign; /* weight bits and bs_sign_t (1-bit signed weights are BS_BIPOLAR)        */
+    const float* scale;      /* device [O]; required iff out_packed != NULL                            */
+    const float* bias;       /* device [O]; required iff out_packed != NULL                            */
+    int relu;
+    int out_bits; int out_sign;      /* code range of the packed output (the next layer's activations) */
+    const uint32_t* residual;        /* device, packed activations [N][P][Q][ceil(res_c_total/32)][res_bits] or NULL */
+    float res_scale;
+    int res_bits; int res_sign;
+    int res_c_offset, res_c_total;   /* the residual code of output channel o is channel res_c_offset + o */
+    int out_c_offset, out_c_total;   /* out_c_offset is a multiple of 32; O is too unless the slice ends the tensor */
+    int i32_layout;                  /* bs_layout_t of out_i32: [N][O][P][Q] or [N][P][Q][O]              */
+} bs_conv_params;
+
+/*
+ * bitserial_conv2d -- Section V bit-serial convolution (implicit GEMM over packed bitplanes) with the
+ * fused epilogue.
+ *   act_packed  device, packed activations of shape (N, C, H, W, a_bits)
+ *   wgt_packed  device, packed weights of shape (O, C, R, S, w_bits)
+ *   out_i32     device or NULL: raw accumulators in p->i32_layout
+ *   out_packed  device or NULL: requantised, packed output (see bs_conv_params); the channel range
+ *               written is fully overwritten, other channels of a wider tensor are left untouched.
+ * At least one output must be non-NULL.  Asynchronous on `stream`.
+ */
+int bitserial_conv2d(const uint32_t* act_packed, const uint32_t* wgt_packed, const bs_conv_params* p,
+                     int32_t* out_i32, uint32_t* out_packed, void* stream);
+
+/*
+ * bitserial_gemm -- Section V bit-serial dot products on plain matrices:
+ *     out[m][n] = sum_{k<K} a[m][k] * w[n][k]
+ *   a_packed  device [M][Kw][a_bits], w_packed device [N][Kw][w_bits] (bs_pack_rows layout)
+ *   out_i32   device or NULL, row-major [M][N]
+ *   out_packed device or NULL, [M][ceil(N/32)][out_bits], epilogue as in bs_conv_params with
+ *             scale/bias indexed by n (scale, bias may be NULL when out_packed is NULL)
+ */
+int bitserial_gemm(const uint32_t* a_packed, const uint32_t* w_packed, int M, int N, int K, int a_bits,
+                   bs_sign_t a_sign, int w_bits, bs_sign_t w_sign, const float* scale, const float* bias,
+                   int relu, int out_bits, bs_sign_t out_sign, int32_t* out_i32, uint32_t* out_packed,
+                   void* stream);
+
+/*
+ * bs_check_status -- synchronises `stream`, then reads and clears the device status word of the current
+ * device.  Returns BS_ERR_TIMEOUT if any kernel since the last check gave up on a bounded wait (its
+ * outputs are then undefined), BS_ERR_CUDA if the stream reports an error, else BS_OK.
+ */
+int bs_check_status(void* stream);
+
+/*
+ * bs_popc_rate -- register-only micro-benchmark of the SM population-count pipe: every thread runs
+ * `iters` rounds of independent  acc += popc(x & y)  chains.  Writes the measured rate in
+ * popc32(AND) word-operations per second to *wordops_per_s (HOST pointer).  Synchronises the device.
+ * Used to state the arithmetic roofline of the convolution kernel beside its measured time.
+ */
+int bs_popc_rate(int iters, double* wordops_per_s);
+
+/* Human-readable name of a bs_status (static storage). */
+const char* bs_status_string(int status);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* BITSERIAL_H_ */

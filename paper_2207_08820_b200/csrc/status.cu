@@ -1,0 +1,89 @@
+// Device status word, status strings and the popcount-pipe micro-benchmark.
+#include "common.cuh"
+
+namespace bs {
+
+__device__ int g_status = 0;
+
+int* status_device_ptr()
+{
+    int* p = nullptr;
+    if (cudaGetSymbolAddress(reinterpret_cast<void**>(&p), g_status) != cudaSuccess) return nullptr;
+    return p;
+}
+
+// Register-only chains of acc += popc(x & y).  Operands change every round so nothing folds.
+__global__ void __launch_bounds__(256) popc_rate_kernel(int iters, unsigned seed, int* sink)
+{
+    unsigned x[8], acc[8];
+    unsigned y = seed ^ (threadIdx.x * 2654435761u + blockIdx.x);
+#pragma unroll
+    for (int k = 0; k < 8; ++k) { x[k] = y * (2 * k + 3) + k; acc[k] = 0; }
+    for (int it = 0; it < iters; ++it) {
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+#pragma unroll
+            for (int k = 0; k < 8; ++k) acc[k] += __popc(x[k] & y);
+            y = y * 1664525u + 1013904223u;
+        }
+    }
+    unsigned total = 0;
+#pragma unroll
+    for (int k = 0; k < 8; ++k) total += acc[k];
+    if (total == 0xFFFFFFFFu) atomicOr(sink, 0);   // never true in practice; keeps the chains alive
+}
+
+}  // namespace bs
+
+extern "C" int bs_popc_rate(int iters, double* wordops_per_s)
+{
+    if (iters <= 0 || wordops_per_s == nullptr) return BS_ERR_INVALID_ARG;
+    int dev = 0, sms = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return BS_ERR_CUDA;
+    if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return BS_ERR_CUDA;
+    int* sink = bs::status_device_ptr();
+    if (!sink) return BS_ERR_CUDA;
+    const int blocks = sms * 8, threads = 256;
+    cudaEvent_t e0, e1;
+    if (cudaEventCreate(&e0) != cudaSuccess || cudaEventCreate(&e1) != cudaSuccess) return BS_ERR_CUDA;
+    bs::popc_rate_kernel<<<blocks, threads>>>(iters / 4 + 1, 12345u, sink);   // warm-up
+    cudaEventRecord(e0);
+    bs::popc_rate_kernel<<<blocks, threads>>>(iters, 12345u, sink);
+    cudaEventRecord(e1);
+    cudaError_t err = cudaEventSynchronize(e1);
+    float ms = 0.f;
+    if (err == cudaSuccess) err = cudaEventElapsedTime(&ms, e0, e1);
+    cudaEventDestroy(e0);
+    cudaEventDestroy(e1);
+    if (err != cudaSuccess || cudaGetLastError() != cudaSuccess || ms <= 0.f) return BS_ERR_CUDA;
+    const double ops = static_cast<double>(blocks) * threads * static_cast<double>(iters) * 32.0;
+    *wordops_per_s = ops / (static_cast<double>(ms) * 1e-3);
+    return BS_OK;
+}
+
+extern "C" int bs_check_status(void* stream)
+{
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (cudaStreamSynchronize(st) != cudaSuccess) { cudaGetLastError(); return BS_ERR_CUDA; }
+    int h = 0;
+    if (cudaMemcpyFromSymbol(&h, bs::g_status, sizeof(int)) != cudaSuccess) return BS_ERR_CUDA;
+    if (h != 0) {
+        int zero = 0;
+        cudaMemcpyToSymbol(bs::g_status, &zero, sizeof(int));
+        return BS_ERR_TIMEOUT;
+    }
+    return BS_OK;
+}
+
+extern "C" const char* bs_status_string(int status)
+{
+    switch (status) {
+        case BS_OK: return "BS_OK";
+        case BS_ERR_INVALID_ARG: return "BS_ERR_INVALID_ARG";
+        case BS_ERR_UNSUPPORTED: return "BS_ERR_UNSUPPORTED";
+        case BS_ERR_ALIGNMENT: return "BS_ERR_ALIGNMENT";
+        case BS_ERR_CUDA: return "BS_ERR_CUDA";
+        case BS_ERR_TIMEOUT: return "BS_ERR_TIMEOUT";
+        default: return "BS_ERR_UNKNOWN";
+    }
+}
