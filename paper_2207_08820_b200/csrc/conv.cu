@@ -1,0 +1,306 @@
+// Host side of bitserial_conv2d / bitserial_gemm: validation, tile planning, TMA descriptors, launch.
+#include <array>
+#include <map>
+#include <mutex>
+
+#include "conv_launch.cuh"
+
+namespace bs {
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+static EncodeTiledFn encode_fn()
+{
+    static EncodeTiledFn fn = nullptr;
+    static std::once_flag once;
+    std::call_once(once, [] {
+        void* p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+            q == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeTiledFn>(p);
+    });
+    return fn;
+}
+
+static int sm_count()
+{
+    static int sms = 0;
+    if (sms == 0) {
+        int dev = 0;
+        if (cudaGetDevice(&dev) != cudaSuccess ||
+            cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms <= 0)
+            sms = 148;
+    }
+    return sms;
+}
+
+static int round_up(int v, int m) { return (v + m - 1) / m * m; }
+
+struct Plan {
+    int PB, NFG, NT, TWB, TH, TNI, CWC, nchunks, nstage;
+    int hh, hw, stageA_words, stageW_words, aux_off_words;
+    int tma_a, tma_w, boxA_w, nboxA, unitA, unitW;
+    size_t smem;
+    long long tiles;
+    double cost;
+};
+
+static int largest_unit(int a, int b)
+{
+    if (a % 4 == 0 && b % 4 == 0) return 4;
+    if (a % 2 == 0 && b % 2 == 0) return 2;
+    return 1;
+}
+
+// Fill the staging part of a plan; returns false if the tile cannot be staged in shared memory.
+static bool plan_staging(Plan& pl, int Cw, int RS, int R, int S, int stride, int A, int WB)
+{
+    const int TN = pl.NFG * CONV_FB;
+    const int TW = pl.TWB * pl.PB;
+    pl.hh = (pl.TH - 1) * stride + R;
+    pl.hw = (TW - 1) * stride + S;
+    pl.CWC = Cw < (RS == 1 ? 8 : 4) ? Cw : (RS == 1 ? 8 : 4);
+    pl.nchunks = ceil_div(Cw, pl.CWC);
+    const int recA = pl.CWC * A, recW = pl.CWC * WB;
+    pl.tma_a = (recA % 4 == 0) && ((Cw * A) % 4 == 0);
+    pl.tma_w = (recW % 4 == 0) && ((Cw * WB) % 4 == 0) && RS <= 256 && TN <= 256;
+    pl.boxA_w = pl.hw;
+    pl.nboxA = 1;
+    if (pl.tma_a) {
+        if (pl.hh > 256 || pl.TNI > 256 || recA > 256) pl.tma_a = 0;
+        else if (pl.hw > 256) {
+            // only a single-row, single-image tile keeps split boxes contiguous in shared memory
+            const int nb = ceil_div(pl.hw, 256);
+            if (pl.hh == 1 && pl.TNI == 1 && pl.hw % nb == 0) { pl.nboxA = nb; pl.boxA_w = pl.hw / nb; }
+            else pl.tma_a = 0;
+        }
+    }
+    pl.unitA = largest_unit(recA, Cw * A);
+    pl.unitW = largest_unit(recW, Cw * WB);
+    pl.stageA_words = round_up(pl.TNI * pl.hh * pl.hw * recA, 32);
+    pl.stageW_words = round_up(TN * RS * recW, 32);
+    const size_t stage_bytes = static_cast<size_t>(pl.stageA_words + pl.stageW_words) * 4;
+    pl.nstage = pl.nchunks < 3 ? pl.nchunks : 3;
+    while (pl.nstage > 1 && stage_bytes * pl.nstage > 96 * 1024) --pl.nstage;
+    const size_t ring = stage_bytes * pl.nstage;
+    const int used_pix = pl.TWB * pl.TH * pl.TNI * pl.PB;
+    const size_t codes = static_cast<size_t>(used_pix) * (TN + 4);
+    const size_t main_bytes = round_up(static_cast<int>(ring > codes ? ring : codes), 128);
+    pl.aux_off_words = static_cast<int>(main_bytes / 4);
+    pl.smem = main_bytes + MAX_STAGES * 8 + static_cast<size_t>(used_pix) * 4 + static_cast<size_t>(TN) * 4;
+    return pl.smem <= 200 * 1024;
+}
+
+static bool search_plan(Plan& best, int N, int P, int Q, int O, int Cw, int R, int S, int stride, int A, int WB)
+{
+    const int RS = R * S;
+    const int sms = sm_count();
+    bool found = false;
+    const int pbs[3] = {8, 7, 4};
+    const int nfgs[3] = {8, 4, 16};
+    const int nts[2] = {256, 128};
+    for (int PB : pbs) {
+        const int qb = ceil_div(Q, PB);
+        for (int NFG : nfgs) {
+            const int TN = NFG * CONV_FB;
+            const long long tiles_o = ceil_div(O, TN);
+            for (int NT : nts) {
+                const int NPG = NT / NFG;
+                for (int TWB = 1; TWB <= NPG && TWB <= qb; ++TWB) {
+                    const int max_th = NPG / TWB;
+                    for (int TH = 1; TH <= max_th && TH <= P; ++TH) {
+                        int TNI = NPG / (TWB * TH);
+                        if (TNI > N) TNI = N;
+                        if (TNI < 1) continue;
+                        Plan pl{};
+                        pl.PB = PB; pl.NFG = NFG; pl.NT = NT; pl.TWB = TWB; pl.TH = TH; pl.TNI = TNI;
+                        if (!plan_staging(pl, Cw, RS, R, S, stride, A, WB)) continue;
+                        pl.tiles = tiles_o * ceil_div(qb, TWB) * ceil_div(P, TH) * ceil_div(N, TNI);
+                        // time model: the busiest SM runs ceil(tiles / sms) CTAs; each CTA costs NT * PB thread-steps;
+                        // fewer than 8 resident warps leave the popcount pipe partly idle
+                        const long long per_sm = ceil_div_ll(pl.tiles, sms);
+                        long long resident = static_cast<long long>((200 * 1024) / pl.smem);
+                        if (resident > per_sm) resident = per_sm;
+                        if (resident * NT > 2048) resident = 2048 / NT;
+                        double warps = static_cast<double>(resident) * NT / 32.0;
+                        double eff = warps >= 8.0 ? 1.0 : warps / 8.0;
+                        pl.cost = static_cast<double>(per_sm) * NT * PB / eff;
+                        // mild preference for TMA-friendly, low-halo tiles
+                        pl.cost *= 1.0 + 0.02 * (static_cast<double>(pl.hh * pl.hw * TNI) / (TWB * PB * TH * TNI) - 1.0) / (stride * stride);
+                        if (!found || pl.cost < best.cost * 0.999) { best = pl; found = true; }
+                    }
+                }
+            }
+        }
+    }
+    return found;
+}
+
+// Plans depend on the shape only, so they are searched once per shape and remembered.
+static bool make_plan(Plan& out, int N, int P, int Q, int O, int Cw, int R, int S, int stride, int A, int WB)
+{
+    static std::map<std::array<int, 10>, std::pair<bool, Plan>> cache;
+    static std::mutex mu;
+    const std::array<int, 10> key = {N, P, Q, O, Cw, R, S, stride, A, WB};
+    std::lock_guard<std::mutex> lock(mu);
+    auto it = cache.find(key);
+    if (it == cache.end()) {
+        Plan pl{};
+        const bool ok = search_plan(pl, N, P, Q, O, Cw, R, S, stride, A, WB);
+        it = cache.emplace(key, std::make_pair(ok, pl)).first;
+    }
+    out = it->second.second;
+    return it->second.first;
+}
+
+static bool encode_map(CUtensorMap* tm, const void* base, int rank, const cuuint64_t* dims, const cuuint64_t* strides_bytes,
+                       const cuuint32_t* box)
+{
+    EncodeTiledFn fn = encode_fn();
+    if (!fn) return false;
+    cuuint32_t estr[5] = {1, 1, 1, 1, 1};
+    return fn(tm, CU_TENSOR_MAP_DATA_TYPE_UINT32, static_cast<cuuint32_t>(rank), const_cast<void*>(base), dims,
+              strides_bytes, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE,
+              CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+static int max_abs_code(int bits, int sign)
+{
+    if (sign == BS_BIPOLAR) return 1;
+    if (sign == BS_SIGNED) return 1 << (bits - 1);
+    return (1 << bits) - 1;
+}
+
+static int conv_impl(const uint32_t* act, const uint32_t* wgt, const bs_conv_params* p, int32_t* out_i32,
+                     uint32_t* out_packed, cudaStream_t st)
+{
+    if (!act || !wgt || !p || (!out_i32 && !out_packed)) return BS_ERR_INVALID_ARG;
+    if (p->N <= 0 || p->C <= 0 || p->H <= 0 || p->W <= 0 || p->O <= 0 || p->R <= 0 || p->S <= 0) return BS_ERR_INVALID_ARG;
+    if (!bits_ok(p->a_bits, p->a_sign) || !bits_ok(p->w_bits, p->w_sign)) return BS_ERR_INVALID_ARG;
+    if (p->stride < 1 || p->pad < 0) return BS_ERR_INVALID_ARG;
+    if (p->i32_layout != BS_NCHW && p->i32_layout != BS_NHWC) return BS_ERR_INVALID_ARG;
+    if (p->R != p->S || (p->R != 1 && p->R != 3 && p->R != 5 && p->R != 7)) return BS_ERR_UNSUPPORTED;
+    if (p->stride > 2 || p->pad >= p->R) return BS_ERR_UNSUPPORTED;
+    if (p->a_sign == BS_BIPOLAR && p->pad != 0) return BS_ERR_UNSUPPORTED;
+    if (p->H + 2 * p->pad < p->R || p->W + 2 * p->pad < p->S) return BS_ERR_INVALID_ARG;
+    if (!aligned16(act) || !aligned16(wgt) || (out_i32 && !aligned16(out_i32)) || (out_packed && !aligned16(out_packed)))
+        return BS_ERR_ALIGNMENT;
+    const long long kred = static_cast<long long>(p->C) * p->R * p->S;
+    if (kred * max_abs_code(p->a_bits, p->a_sign) * max_abs_code(p->w_bits, p->w_sign) >= (1LL << 31))
+        return BS_ERR_UNSUPPORTED;
+
+    ConvArgs g{};
+    g.P = (p->H + 2 * p->pad - p->R) / p->stride + 1;
+    g.Q = (p->W + 2 * p->pad - p->S) / p->stride + 1;
+    g.Cw = ceil_div(p->C, 32);
+    if (out_packed) {
+        if (!p->scale || !p->bias) return BS_ERR_INVALID_ARG;
+        if (!bits_ok(p->out_bits, p->out_sign)) return BS_ERR_INVALID_ARG;
+        if (p->out_c_offset < 0 || p->out_c_total < p->out_c_offset + p->O) return BS_ERR_INVALID_ARG;
+        if (p->out_c_offset % 32 != 0) return BS_ERR_UNSUPPORTED;
+        if (p->O % 32 != 0 && p->out_c_offset + p->O != p->out_c_total) return BS_ERR_UNSUPPORTED;
+        if (p->residual) {
+            if (!bits_ok(p->res_bits, p->res_sign)) return BS_ERR_INVALID_ARG;
+            if (p->res_c_offset < 0 || p->res_c_total < p->res_c_offset + p->O) return BS_ERR_INVALID_ARG;
+            if (!aligned16(p->residual)) return BS_ERR_ALIGNMENT;
+        }
+    }
+
+    const int A = p->a_bits, WB = p->w_bits;
+    Plan pl{};
+    if (!make_plan(pl, p->N, g.P, g.Q, p->O, g.Cw, p->R, p->S, p->stride, A, WB)) return BS_ERR_UNSUPPORTED;
+
+    g.act = act; g.wgt = wgt; g.out_i32 = out_i32; g.out_packed = out_packed;
+    g.scale = p->scale; g.bias = p->bias;
+    g.residual = out_packed ? p->residual : nullptr;
+    g.res_scale = p->res_scale;
+    g.status = status_device_ptr();
+    if (!g.status) return BS_ERR_CUDA;
+    g.N = p->N; g.C = p->C; g.H = p->H; g.W = p->W; g.O = p->O; g.R = p->R; g.S = p->S;
+    g.stride = p->stride; g.pad = p->pad;
+    g.a_sign = p->a_sign; g.w_sign = p->w_sign;
+    g.relu = p->relu; g.out_bits = p->out_bits; g.out_sign = p->out_sign;
+    g.out_cw_off = p->out_c_offset / 32; g.out_cw_total = ceil_div(p->out_c_total > 0 ? p->out_c_total : 1, 32);
+    g.res_bits = p->res_bits; g.res_sign = p->res_sign; g.res_c_off = p->res_c_offset;
+    g.res_cw_total = ceil_div(p->res_c_total > 0 ? p->res_c_total : 1, 32);
+    g.i32_nhwc = p->i32_layout == BS_NHWC;
+    g.NFG = pl.NFG; g.NPG = pl.NT / pl.NFG; g.TNI = pl.TNI; g.TH = pl.TH; g.TWB = pl.TWB;
+    g.used_pg = pl.TWB * pl.TH * pl.TNI;
+    g.hh = pl.hh; g.hw = pl.hw; g.CWC = pl.CWC; g.nchunks = pl.nchunks; g.nstage = pl.nstage;
+    g.stageA_words = pl.stageA_words; g.stageW_words = pl.stageW_words; g.aux_off_words = pl.aux_off_words;
+    const int TN = pl.NFG * CONV_FB, TW = pl.TWB * pl.PB;
+    g.tiles_o = ceil_div(p->O, TN); g.tiles_q = ceil_div(g.Q, TW); g.tiles_p = ceil_div(g.P, pl.TH);
+    g.tiles_n = ceil_div(p->N, pl.TNI);
+    g.tma_a = pl.tma_a; g.tma_w = pl.tma_w; g.boxA_w = pl.boxA_w; g.nboxA = pl.nboxA;
+    g.unitA = pl.unitA; g.unitW = pl.unitW;
+
+    const int alpha_a = p->a_sign == BS_BIPOLAR ? 2 : 1, alpha_w = p->w_sign == BS_BIPOLAR ? 2 : 1;
+    for (int i = 0; i < 4; ++i) {
+        const int ci = (p->w_sign == BS_SIGNED && i == WB - 1) ? -1 : 1;
+        g.cs_coef[i] = -alpha_w * ci * (1 << i);
+        for (int j = 0; j < 4; ++j) {
+            const int dj = (p->a_sign == BS_SIGNED && j == A - 1) ? -1 : 1;
+            g.coef[i][j] = alpha_a * alpha_w * ci * dj * (1 << (i + j));
+            g.rs_coef[j] = -alpha_a * dj * (1 << j);
+        }
+    }
+    g.need_rs = p->w_sign == BS_BIPOLAR;
+    g.need_cs = p->a_sign == BS_BIPOLAR;
+    g.kconst = (g.need_rs && g.need_cs) ? static_cast<int>(kred) : 0;
+
+    const long long tiles = static_cast<long long>(g.tiles_o) * g.tiles_q * g.tiles_p * g.tiles_n;
+    if (tiles > 0x7fffffffLL) return BS_ERR_UNSUPPORTED;
+
+    if (g.tma_a) {
+        const cuuint64_t fullA = static_cast<cuuint64_t>(g.Cw) * A;
+        cuuint64_t dims[4] = {fullA, static_cast<cuuint64_t>(p->W), static_cast<cuuint64_t>(p->H), static_cast<cuuint64_t>(p->N)};
+        cuuint64_t strides[3] = {fullA * 4, fullA * 4 * p->W, fullA * 4 * p->W * p->H};
+        cuuint32_t box[4] = {static_cast<cuuint32_t>(g.CWC * A), static_cast<cuuint32_t>(g.boxA_w),
+                             static_cast<cuuint32_t>(g.hh), static_cast<cuuint32_t>(g.TNI)};
+        if (!encode_map(&g.tmA, act, 4, dims, strides, box)) {
+            g.tma_a = 0; g.nboxA = 1; g.boxA_w = g.hw;   // descriptor refused: gather instead
+        }
+    }
+    if (g.tma_w) {
+        const cuuint64_t fullW = static_cast<cuuint64_t>(g.Cw) * WB;
+        const cuuint64_t RS = static_cast<cuuint64_t>(p->R) * p->S;
+        cuuint64_t dims[3] = {fullW, RS, static_cast<cuuint64_t>(p->O)};
+        cuuint64_t strides[2] = {fullW * 4, fullW * 4 * RS};
+        cuuint32_t box[3] = {static_cast<cuuint32_t>(g.CWC * WB), static_cast<cuuint32_t>(RS), static_cast<cuuint32_t>(TN)};
+        if (!encode_map(&g.tmW, wgt, 3, dims, strides, box)) g.tma_w = 0;
+    }
+
+    const unsigned grid = static_cast<unsigned>(tiles), block = static_cast<unsigned>(pl.NT);
+    switch (A) {
+        case 1: return launch_conv_a1(WB, pl.PB, g, grid, block, pl.smem, st);
+        case 2: return launch_conv_a2(WB, pl.PB, g, grid, block, pl.smem, st);
+        case 3: return launch_conv_a3(WB, pl.PB, g, grid, block, pl.smem, st);
+        default: return launch_conv_a4(WB, pl.PB, g, grid, block, pl.smem, st);
+    }
+}
+
+}  // namespace bs
+
+extern "C" int bitserial_conv2d(const uint32_t* act_packed, const uint32_t* wgt_packed, const bs_conv_params* p,
+                                int32_t* out_i32, uint32_t* out_packed, void* stream)
+{
+    return bs::conv_impl(act_packed, wgt_packed, p, out_i32, out_packed, static_cast<cudaStream_t>(stream));
+}
+
+extern "C" int bitserial_gemm(const uint32_t* a_packed, const uint32_t* w_packed, int M, int N, int K, int a_bits,
+                              bs_sign_t a_sign, int w_bits, bs_sign_t w_sign, const float* scale, const float* bias,
+                              int relu, int out_bits, bs_sign_t out_sign, int32_t* out_i32, uint32_t* out_packed,
+                              void* stream)
+{
+    if (M <= 0 || N <= 0 || K <= 0) return BS_ERR_INVALID_ARG;
+    // a matrix product is a 1x1 convolution over a 1 x M image with K channels and N filters
+    bs_conv_params p{};
+    p.N = 1; p.C = K; p.H = 1; p.W = M; p.O = N; p.R = 1; p.S = 1; p.stride = 1; p.pad = 0;
+    p.a_bits = a_bits; p.a_sign = a_sign; p.w_bits = w_bits; p.w_sign = w_sign;
+    p.scale = scale; p.bias = bias; p.relu = relu; p.out_bits = out_bits; p.out_sign = out_sign;
+    p.residual = nullptr; p.out_c_offset = 0; p.out_c_total = N; p.i32_layout = BS_NHWC;
+    return bs::conv_impl(a_packed, w_packed, &p, out_i32, out_packed, static_cast<cudaStream_t>(stream));
+}
