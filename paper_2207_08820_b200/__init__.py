@@ -5,17 +5,14 @@ The arithmetic lives in the CUDA library behind the C ABI declared in
 entry-point names.  Importing the package does not load the library; the first use of an API
 name does, and raises if the library is missing (there is no CPU fallback).
 """
-_API_MODULE = None
+import importlib
+
+_API_NAMES = ("bitpack_activations", "bitunpack_activations", "pack_weights", "bs_pack_rows",
+              "bitserial_conv2d", "bitserial_gemm", "bs_check_status", "bs_popc_rate",
+              "UNSIGNED", "SIGNED", "BIPOLAR", "NCHW", "NHWC")
 
 
 def __getattr__(name):
-    if name.startswith("__"):
-        raise AttributeError(name)
-    global _API_MODULE
-    if _API_MODULE is None:
-        from . import api as _api
-        _API_MODULE = _api
-    try:
-        return getattr(_API_MODULE, name)
-    except AttributeError:
-        raise AttributeError(f"module 'paper_2207_08820_b200' has no attribute {name!r}") from None
+    if name in _API_NAMES:
+        return getattr(importlib.import_module(__name__ + ".api"), name)
+    raise AttributeError(f"module {__name__!r} has no attribute {name!r}")

@@ -1,0 +1,78 @@
+"""Loads the CUDA library.  There is no fallback: a missing library is an error."""
+from __future__ import annotations
+
+import ctypes
+import os
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libbitserial_b200.so")
+_lib = None
+
+
+class BitserialError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        name = lib().bs_status_string(status).decode() if _lib is not None else str(status)
+        super().__init__(f"{where} failed: {name} ({status})")
+
+
+class ConvParams(ctypes.Structure):
+    """Mirror of ``bs_conv_params`` (include/bitserial.h)."""
+    _fields_ = [
+        ("N", ctypes.c_int), ("C", ctypes.c_int), ("H", ctypes.c_int), ("W", ctypes.c_int),
+        ("O", ctypes.c_int), ("R", ctypes.c_int), ("S", ctypes.c_int),
+        ("stride", ctypes.c_int), ("pad", ctypes.c_int),
+        ("a_bits", ctypes.c_int), ("a_sign", ctypes.c_int),
+        ("w_bits", ctypes.c_int), ("w_sign", ctypes.c_int),
+        ("scale", ctypes.c_void_p), ("bias", ctypes.c_void_p),
+        ("relu", ctypes.c_int),
+        ("out_bits", ctypes.c_int), ("out_sign", ctypes.c_int),
+        ("residual", ctypes.c_void_p), ("res_scale", ctypes.c_float),
+        ("res_bits", ctypes.c_int), ("res_sign", ctypes.c_int),
+        ("res_c_offset", ctypes.c_int), ("res_c_total", ctypes.c_int),
+        ("out_c_offset", ctypes.c_int), ("out_c_total", ctypes.c_int),
+        ("i32_layout", ctypes.c_int),
+    ]
+
+
+def lib() -> ctypes.CDLL:
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(LIB_PATH):
+        raise ImportError(
+            f"{LIB_PATH} is missing: build it with `python -m paper_2207_08820_b200.build` "
+            "(nvcc, sm_100a).  This library has no CPU or PyTorch fallback.")
+    L = ctypes.CDLL(LIB_PATH)
+    vp, i, f = ctypes.c_void_p, ctypes.c_int, ctypes.c_float
+    L.bs_packed_act_bytes.restype = ctypes.c_size_t
+    L.bs_packed_act_bytes.argtypes = [i] * 5
+    L.bs_packed_wgt_bytes.restype = ctypes.c_size_t
+    L.bs_packed_wgt_bytes.argtypes = [i] * 5
+    L.bs_packed_rows_bytes.restype = ctypes.c_size_t
+    L.bs_packed_rows_bytes.argtypes = [i] * 3
+    L.bitpack_activations.restype = i
+    L.bitpack_activations.argtypes = [vp, i, i, i, i, i, i, f, i, i, vp, vp]
+    L.bitunpack_activations.restype = i
+    L.bitunpack_activations.argtypes = [vp, i, i, i, i, i, i, i, vp, vp]
+    L.pack_weights.restype = i
+    L.pack_weights.argtypes = [vp, i, i, i, i, i, i, i, vp, vp]
+    L.bs_pack_rows.restype = i
+    L.bs_pack_rows.argtypes = [vp, i, i, i, i, vp, vp]
+    L.bitserial_conv2d.restype = i
+    L.bitserial_conv2d.argtypes = [vp, vp, ctypes.POINTER(ConvParams), vp, vp, vp]
+    L.bitserial_gemm.restype = i
+    L.bitserial_gemm.argtypes = [vp, vp, i, i, i, i, i, i, i, vp, vp, i, i, i, vp, vp, vp]
+    L.bs_check_status.restype = i
+    L.bs_check_status.argtypes = [vp]
+    L.bs_popc_rate.restype = i
+    L.bs_popc_rate.argtypes = [i, ctypes.POINTER(ctypes.c_double)]
+    L.bs_status_string.restype = ctypes.c_char_p
+    L.bs_status_string.argtypes = [i]
+    _lib = L
+    return L
+
+
+EXPORTED = ("bs_packed_act_bytes", "bs_packed_wgt_bytes", "bs_packed_rows_bytes", "bitpack_activations",
+            "bitunpack_activations", "pack_weights", "bs_pack_rows", "bitserial_conv2d", "bitserial_gemm",
+            "bs_check_status", "bs_popc_rate", "bs_status_string")

@@ -1,0 +1,179 @@
+"""Thin Python binding over the C ABI of ``include/bitserial.h``.
+
+Argument marshalling only: tensors are torch CUDA tensors used as device buffers, streams are torch
+streams, and every function forwards to the entry point of the same name.  No arithmetic of the method
+happens here and nothing falls back to PyTorch ops.
+"""
+from __future__ import annotations
+
+import ctypes
+from typing import Optional
+
+import torch
+
+from ._lib import BitserialError, ConvParams, lib
+
+UNSIGNED, SIGNED, BIPOLAR = 0, 1, 2
+NCHW, NHWC = 0, 1
+
+launch_count = 0   # kernels enqueued through this binding (every entry point below launches exactly one)
+
+
+def _stream_ptr(stream: Optional[torch.cuda.Stream]) -> int:
+    s = stream if stream is not None else torch.cuda.current_stream()
+    return s.cuda_stream
+
+
+def _ptr(t: Optional[torch.Tensor]) -> Optional[int]:
+    if t is None:
+        return None
+    if not t.is_cuda or not t.is_contiguous():
+        raise ValueError("expected a contiguous CUDA tensor")
+    return t.data_ptr()
+
+
+def _check(status: int, where: str) -> None:
+    global launch_count
+    if status != 0:
+        raise BitserialError(status, where)
+    launch_count += 1
+
+
+def packed_act_words(N, C, H, W, bits) -> int:
+    return lib().bs_packed_act_bytes(N, C, H, W, bits) // 4
+
+
+def packed_wgt_words(O, C, R, S, bits) -> int:
+    return lib().bs_packed_wgt_bytes(O, C, R, S, bits) // 4
+
+
+def packed_rows_words(rows, K, bits) -> int:
+    return lib().bs_packed_rows_bytes(rows, K, bits) // 4
+
+
+def _words(n: int, device) -> torch.Tensor:
+    return torch.empty(n, dtype=torch.int32, device=device)
+
+
+def bitpack_activations(x: torch.Tensor, act_scale: float, a_bits: int, a_sign: int = UNSIGNED,
+                        layout: int = NCHW, out: Optional[torch.Tensor] = None, stream=None) -> torch.Tensor:
+    """x: float32 or int8 (codes), [N,C,H,W] (NCHW) or [N,H,W,C] (NHWC).  Returns int32 words
+    viewed as [N, H, W, Cw, a_bits]."""
+    if x.dtype not in (torch.float32, torch.int8):
+        raise ValueError("x must be float32 or int8")
+    if layout == NCHW:
+        N, C, H, W = x.shape
+    else:
+        N, H, W, C = x.shape
+    Cw = (C + 31) // 32
+    if out is None:
+        out = _words(N * H * W * Cw * a_bits, x.device)
+    st = lib().bitpack_activations(_ptr(x), int(x.dtype == torch.float32), layout, N, C, H, W,
+                                   ctypes.c_float(act_scale), a_bits, a_sign, _ptr(out), _stream_ptr(stream))
+    _check(st, "bitpack_activations")
+    return out.view(N, H, W, Cw, a_bits)
+
+
+def bitunpack_activations(packed: torch.Tensor, C: int, a_bits: int, a_sign: int = UNSIGNED, layout: int = NCHW,
+                          stream=None) -> torch.Tensor:
+    N, H, W, Cw, b = packed.shape
+    shape = (N, C, H, W) if layout == NCHW else (N, H, W, C)
+    out = torch.empty(shape, dtype=torch.int8, device=packed.device)
+    st = lib().bitunpack_activations(_ptr(packed), N, C, H, W, a_bits, a_sign, layout, _ptr(out), _stream_ptr(stream))
+    _check(st, "bitunpack_activations")
+    return out
+
+
+def pack_weights(w_codes: torch.Tensor, w_bits: int, w_sign: int, layout: int = NCHW, stream=None) -> torch.Tensor:
+    """w_codes int8 [O,C,R,S] (layout NCHW = OIHW) or [O,R,S,C].  Returns int32 words [O,R,S,Cw,w_bits]."""
+    if layout == NCHW:
+        O, C, R, S = w_codes.shape
+    else:
+        O, R, S, C = w_codes.shape
+    Cw = (C + 31) // 32
+    out = _words(O * R * S * Cw * w_bits, w_codes.device)
+    st = lib().pack_weights(_ptr(w_codes), layout, O, C, R, S, w_bits, w_sign, _ptr(out), _stream_ptr(stream))
+    _check(st, "pack_weights")
+    return out.view(O, R, S, Cw, w_bits)
+
+
+def bs_pack_rows(codes: torch.Tensor, bits: int, sign: int, stream=None) -> torch.Tensor:
+    rows, K = codes.shape
+    Kw = (K + 31) // 32
+    out = _words(rows * Kw * bits, codes.device)
+    st = lib().bs_pack_rows(_ptr(codes), rows, K, bits, sign, _ptr(out), _stream_ptr(stream))
+    _check(st, "bs_pack_rows")
+    return out.view(rows, Kw, bits)
+
+
+def bitserial_conv2d(act_packed: torch.Tensor, wgt_packed: torch.Tensor, *, C: int, stride: int = 1, pad: int = 0,
+                     a_sign: int = UNSIGNED, w_sign: int = SIGNED, scale: Optional[torch.Tensor] = None,
+                     bias: Optional[torch.Tensor] = None, relu: bool = False, out_bits: int = 0,
+                     out_sign: int = UNSIGNED, residual: Optional[torch.Tensor] = None, res_scale: float = 0.0,
+                     res_bits: int = 0, res_sign: int = UNSIGNED, res_c_offset: int = 0, res_c_total: int = 0,
+                     out_i32: Optional[torch.Tensor] = None, want_i32: bool = False, i32_layout: int = NCHW,
+                     out_packed: Optional[torch.Tensor] = None, out_c_offset: int = 0, out_c_total: int = 0,
+                     stream=None):
+    """act_packed [N,H,W,Cw,a_bits], wgt_packed [O,R,S,Cw,w_bits].  Returns (out_i32 or None, out_packed or None).
+    A packed output is produced when ``out_bits`` > 0 (allocated here unless ``out_packed`` is given)."""
+    N, H, W, Cw, a_bits = act_packed.shape
+    O, R, S, Cw2, w_bits = wgt_packed.shape
+    if Cw != Cw2 or Cw != (C + 31) // 32:
+        raise ValueError("channel words of activations and weights disagree")
+    P = (H + 2 * pad - R) // stride + 1
+    Q = (W + 2 * pad - S) // stride + 1
+    dev = act_packed.device
+    if want_i32 and out_i32 is None:
+        shape = (N, O, P, Q) if i32_layout == NCHW else (N, P, Q, O)
+        out_i32 = torch.empty(shape, dtype=torch.int32, device=dev)
+    if out_bits > 0:
+        if out_c_total == 0:
+            out_c_total = out_c_offset + O
+        if out_packed is None:
+            out_packed = torch.zeros(N, P, Q, (out_c_total + 31) // 32, out_bits, dtype=torch.int32, device=dev)
+    p = ConvParams(N=N, C=C, H=H, W=W, O=O, R=R, S=S, stride=stride, pad=pad, a_bits=a_bits, a_sign=a_sign,
+                   w_bits=w_bits, w_sign=w_sign, scale=_ptr(scale), bias=_ptr(bias), relu=int(relu),
+                   out_bits=out_bits, out_sign=out_sign, residual=_ptr(residual), res_scale=res_scale,
+                   res_bits=res_bits, res_sign=res_sign, res_c_offset=res_c_offset,
+                   res_c_total=res_c_total if res_c_total else res_c_offset + O,
+                   out_c_offset=out_c_offset, out_c_total=out_c_total, i32_layout=i32_layout)
+    st = lib().bitserial_conv2d(_ptr(act_packed), _ptr(wgt_packed), ctypes.byref(p), _ptr(out_i32),
+                                _ptr(out_packed) if out_bits > 0 else None, _stream_ptr(stream))
+    _check(st, "bitserial_conv2d")
+    return out_i32, (out_packed if out_bits > 0 else None)
+
+
+def bitserial_gemm(a_packed: torch.Tensor, w_packed: torch.Tensor, K: int, *, a_sign: int = UNSIGNED,
+                   w_sign: int = SIGNED, scale: Optional[torch.Tensor] = None, bias: Optional[torch.Tensor] = None,
+                   relu: bool = False, out_bits: int = 0, out_sign: int = UNSIGNED,
+                   out_i32: Optional[torch.Tensor] = None, want_i32: bool = True,
+                   out_packed: Optional[torch.Tensor] = None, stream=None):
+    """a_packed [M,Kw,a_bits], w_packed [N,Kw,w_bits].  Returns (out_i32 [M,N] or None, out_packed or None)."""
+    M, Kw, a_bits = a_packed.shape
+    N, Kw2, w_bits = w_packed.shape
+    if Kw != Kw2 or Kw != (K + 31) // 32:
+        raise ValueError("reduction words of the operands disagree")
+    dev = a_packed.device
+    if want_i32 and out_i32 is None:
+        out_i32 = torch.empty(M, N, dtype=torch.int32, device=dev)
+    if out_bits > 0 and out_packed is None:
+        out_packed = torch.zeros(M, (N + 31) // 32, out_bits, dtype=torch.int32, device=dev)
+    st = lib().bitserial_gemm(_ptr(a_packed), _ptr(w_packed), M, N, K, a_bits, a_sign, w_bits, w_sign,
+                              _ptr(scale), _ptr(bias), int(relu), out_bits, out_sign, _ptr(out_i32),
+                              _ptr(out_packed) if out_bits > 0 else None, _stream_ptr(stream))
+    _check(st, "bitserial_gemm")
+    return out_i32, (out_packed if out_bits > 0 else None)
+
+
+def bs_check_status(stream=None) -> None:
+    st = lib().bs_check_status(_stream_ptr(stream))
+    if st != 0:
+        raise BitserialError(st, "bs_check_status")
+
+
+def bs_popc_rate(iters: int = 4096) -> float:
+    out = ctypes.c_double(0.0)
+    st = lib().bs_popc_rate(iters, ctypes.byref(out))
+    if st != 0:
+        raise BitserialError(st, "bs_popc_rate")
+    return out.value

@@ -1,0 +1,77 @@
+"""Runs a stack of quantised conv layers (``workloads.NetSpec``) through the C ABI.
+
+Host logic only: buffer planning, weight packing at set-up, one ``bitserial_conv2d`` call per layer
+(residual adds and concatenations are epilogue arguments), optional CUDA-graph replay.
+"""
+from __future__ import annotations
+
+from typing import Dict, Optional
+
+import numpy as np
+import torch
+
+from . import api
+from .workloads import NetSpec
+
+
+class BitserialNet:
+    def __init__(self, net: NetSpec, params: Dict[str, Dict], act_scale: float, device="cuda", batch: Optional[int] = None):
+        self.net = net
+        self.act_scale = float(act_scale)
+        self.device = torch.device(device)
+        self.batch = batch or net.batch
+        self.shapes = net.tensor_shapes()
+        self.layers = []
+        for L in net.layers:
+            p = params[L.name]
+            w = torch.from_numpy(np.ascontiguousarray(p["w"])).to(self.device)
+            self.layers.append(dict(
+                spec=L,
+                w=api.pack_weights(w, net.w_bits, p["w_sign"]),
+                w_sign=p["w_sign"],
+                scale=torch.from_numpy(p["scale"]).to(self.device),
+                bias=torch.from_numpy(p["bias"]).to(self.device)))
+        self.bufs: Dict[str, torch.Tensor] = {}
+        for name, (C, H, W) in self.shapes.items():
+            self.bufs[name] = torch.zeros(self.batch, H, W, (C + 31) // 32, net.a_bits, dtype=torch.int32, device=self.device)
+        self.graph = None
+        self.static_in = None
+        self.launches_per_forward = 1 + len(self.layers)
+
+    def _run(self, x: torch.Tensor) -> torch.Tensor:
+        net = self.net
+        api.bitpack_activations(x, self.act_scale, net.a_bits, api.UNSIGNED, api.NCHW, out=self.bufs[net.in_name].view(-1))
+        for item in self.layers:
+            L = item["spec"]
+            res = self.bufs[L.res] if L.res else None
+            api.bitserial_conv2d(
+                self.bufs[L.src], item["w"], C=L.C, stride=L.stride, pad=L.pad, a_sign=api.UNSIGNED,
+                w_sign=item["w_sign"], scale=item["scale"], bias=item["bias"], relu=L.relu, out_bits=net.a_bits,
+                out_sign=api.UNSIGNED, residual=res, res_scale=L.res_scale, res_bits=net.a_bits if L.res else 0,
+                res_sign=api.UNSIGNED, res_c_offset=0, res_c_total=self.shapes[L.res][0] if L.res else 0,
+                out_packed=self.bufs[L.dst], out_c_offset=L.dst_c_offset, out_c_total=self.shapes[L.dst][0])
+        return self.bufs[net.out_name]
+
+    def forward(self, x: torch.Tensor) -> torch.Tensor:
+        """x: float32 [batch, C, H, W] on the device.  Returns the packed output tensor of the stack."""
+        return self._run(x)
+
+    def capture(self, x: torch.Tensor) -> None:
+        """Record one forward pass into a CUDA graph replayed by :meth:`replay` (input copied into a static buffer)."""
+        self.static_in = x.clone()
+        self._run(self.static_in)            # warm-up outside capture: plans, descriptors, module loading
+        torch.cuda.synchronize()
+        self.graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(self.graph):
+            self._run(self.static_in)
+
+    def replay(self, x: Optional[torch.Tensor] = None) -> torch.Tensor:
+        if x is not None:
+            self.static_in.copy_(x, non_blocking=True)
+        self.graph.replay()
+        return self.bufs[self.net.out_name]
+
+    def unpacked(self, name: str) -> torch.Tensor:
+        """int8 NCHW codes of an activation tensor (debugging / tests)."""
+        C = self.shapes[name][0]
+        return api.bitunpack_activations(self.bufs[name], C, self.net.a_bits, api.UNSIGNED, api.NCHW)

@@ -34,6 +34,26 @@ def rand_codes(rng: np.random.Generator, shape, bits: int, sign: int) -> np.ndar
     return rng.integers(lo, hi + 1, size=shape, dtype=np.int8)
 
 
+def rand_weights_zero_mean(rng: np.random.Generator, shape, bits: int, sign: int) -> np.ndarray:
+    """Weights over the full code range with zero mean: the most negative code of a two's-complement
+    range has no positive partner, so it and its neighbour get half the probability of the others,
+    re-balanced so that the expectation is exactly zero (2 bits: p(-2), p(-1), p(0), p(1) = 1/7, 1/7,
+    2/7, 3/7).  Keeps every filter's sum near zero, so accumulators do not inherit the common-mode
+    brightness of a pixel and deep stacks keep all activation levels in use."""
+    if sign != SIGNED or bits < 2:
+        return rand_codes(rng, shape, bits, sign)
+    lo, hi = code_range(bits, sign)
+    vals = np.arange(lo, hi + 1)
+    p = np.ones(len(vals))
+    p[0] = p[1] = 0.5
+    # tilt the non-negative side so that sum(p * v) = 0
+    neg = float((p * vals)[vals < 0].sum())
+    pos = float((p * vals)[vals > 0].sum())
+    p[vals > 0] *= -neg / pos
+    p /= p.sum()
+    return rng.choice(vals, size=shape, p=p).astype(np.int8)
+
+
 def weight_sign(w_bits: int) -> int:
     """Signed weights; 1-bit signed weights are bipolar."""
     return BIPOLAR if w_bits == 1 else SIGNED
@@ -246,7 +266,7 @@ def network_params(net: NetSpec, seed: int) -> Dict[str, Dict]:
     ws = weight_sign(net.w_bits)
     params = {}
     for L in net.layers:
-        w = rand_codes(rng, (L.O, L.C, L.k, L.k), net.w_bits, ws)
+        w = rand_weights_zero_mean(rng, (L.O, L.C, L.k, L.k), net.w_bits, ws)
         scale, bias = calibrated_scale_bias(w, net.a_bits, UNSIGNED, net.a_bits,
                                             res_scale=L.res_scale if L.res else 0.0, res_bits=net.a_bits)
         params[L.name] = dict(w=w, scale=scale, bias=bias, w_sign=ws)

@@ -1,0 +1,112 @@
+"""Host-only checks of the C ABI: the library loads without a GPU, exports every symbol the header
+declares, agrees with the header on struct layout and size formulas, and rejects bad arguments on
+the host before touching a device."""
+import ctypes
+import os
+import re
+import subprocess
+import sys
+
+import pytest
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+HEADER = os.path.join(ROOT, "include", "bitserial.h")
+
+
+@pytest.fixture(scope="module")
+def L():
+    from paper_2207_08820_b200 import build
+    build.build()
+    from paper_2207_08820_b200 import _lib
+    return _lib.lib()
+
+
+def _declared_functions():
+    src = open(HEADER).read()
+    src = re.sub(r"/\*.*?\*/", "", src, flags=re.S)
+    names = re.findall(r"^\s*(?:int|size_t|const char\*)\s+(\w+)\s*\(", src, flags=re.M)
+    return sorted(set(names))
+
+
+def test_every_declared_symbol_is_exported(L):
+    names = _declared_functions()
+    assert {"bitpack_activations", "pack_weights", "bitserial_conv2d", "bitserial_gemm"} <= set(names)
+    for n in names:
+        assert hasattr(L, n), n
+
+
+def test_header_compiles_as_c_and_struct_matches_binding(tmp_path):
+    from paper_2207_08820_b200._lib import ConvParams
+    src = tmp_path / "t.c"
+    src.write_text('#include <stdio.h>\n#include <stddef.h>\n#include "bitserial.h"\n'
+                   'int main(void){printf("%zu %zu %zu %zu %zu\\n", sizeof(bs_conv_params), offsetof(bs_conv_params, scale),'
+                   ' offsetof(bs_conv_params, residual), offsetof(bs_conv_params, res_scale), offsetof(bs_conv_params, i32_layout));return 0;}\n')
+    exe = tmp_path / "t"
+    subprocess.run(["gcc", "-std=c99", "-Wall", "-Werror", "-I", os.path.join(ROOT, "include"), str(src), "-o", str(exe)], check=True)
+    out = subprocess.run([str(exe)], capture_output=True, text=True, check=True).stdout.split()
+    assert int(out[0]) == ctypes.sizeof(ConvParams)
+    assert int(out[1]) == ConvParams.scale.offset
+    assert int(out[2]) == ConvParams.residual.offset
+    assert int(out[3]) == ConvParams.res_scale.offset
+    assert int(out[4]) == ConvParams.i32_layout.offset
+
+
+def test_size_queries(L):
+    assert L.bs_packed_act_bytes(1, 64, 56, 56, 2) == 56 * 56 * 2 * 2 * 4
+    assert L.bs_packed_act_bytes(2, 33, 3, 5, 3) == 2 * 3 * 5 * 2 * 3 * 4
+    assert L.bs_packed_wgt_bytes(64, 64, 3, 3, 2) == 64 * 9 * 2 * 2 * 4
+    assert L.bs_packed_rows_bytes(10, 577, 1) == 10 * 19 * 4
+    assert L.bs_packed_act_bytes(1, 64, 56, 56, 5) == 0
+    assert L.bs_packed_wgt_bytes(0, 64, 3, 3, 2) == 0
+
+
+def test_bad_arguments_are_rejected_on_the_host(L):
+    from paper_2207_08820_b200._lib import ConvParams
+    buf = (ctypes.c_char * 4096)()
+    addr = (ctypes.addressof(buf) + 255) & ~255      # never dereferenced: validation fails first
+    INVALID, UNSUPPORTED, ALIGN = 1, 2, 3
+    assert L.bitpack_activations(None, 1, 0, 1, 64, 8, 8, 1.0, 2, 0, addr, None) == INVALID
+    assert L.bitpack_activations(addr, 1, 0, 1, 64, 8, 8, 1.0, 5, 0, addr, None) == INVALID
+    assert L.bitpack_activations(addr, 1, 0, 1, 64, 8, 8, 1.0, 2, 2, addr, None) == INVALID      # bipolar needs 1 bit
+    assert L.bitpack_activations(addr, 1, 0, 1, 64, 8, 8, 0.0, 2, 0, addr, None) == INVALID      # scale must be > 0
+    assert L.bitpack_activations(addr + 4, 1, 0, 1, 64, 8, 8, 1.0, 2, 0, addr, None) == ALIGN
+    assert L.pack_weights(addr, 0, 64, 64, 3, 3, 0, 1, addr, None) == INVALID
+    p = ConvParams(N=1, C=64, H=8, W=8, O=64, R=3, S=3, stride=1, pad=1, a_bits=2, a_sign=0, w_bits=2, w_sign=1,
+                   i32_layout=0)
+    assert L.bitserial_conv2d(addr, addr, ctypes.byref(p), None, None, None) == INVALID          # no output
+    p.R = 3; p.S = 1
+    assert L.bitserial_conv2d(addr, addr, ctypes.byref(p), addr, None, None) == UNSUPPORTED
+    p.S = 3; p.stride = 3
+    assert L.bitserial_conv2d(addr, addr, ctypes.byref(p), addr, None, None) == UNSUPPORTED
+    p.stride = 1; p.a_bits = 1; p.a_sign = 2
+    assert L.bitserial_conv2d(addr, addr, ctypes.byref(p), addr, None, None) == UNSUPPORTED      # bipolar acts with padding
+    p.a_bits = 2; p.a_sign = 0
+    assert L.bitserial_conv2d(addr, addr, ctypes.byref(p), None, addr, None) == INVALID          # packed output needs scale/bias
+    assert L.bitserial_conv2d(addr, addr + 8, ctypes.byref(p), addr, None, None) == ALIGN
+    p.C = 1 << 28                                                                                 # accumulator could overflow
+    p.a_bits = 4; p.w_bits = 4
+    assert L.bitserial_conv2d(addr, addr, ctypes.byref(p), addr, None, None) == UNSUPPORTED
+    assert L.bitserial_gemm(addr, addr, 0, 4, 4, 2, 0, 2, 1, None, None, 0, 0, 0, addr, None, None) == INVALID
+    assert L.bs_status_string(5) == b"BS_ERR_TIMEOUT"
+
+
+def test_binding_fails_loudly_without_library(tmp_path):
+    """Importing the binding with the shared library absent must raise, not fall back."""
+    code = ("import sys; sys.path.insert(0, %r)\n"
+            "from paper_2207_08820_b200 import _lib\n"
+            "_lib.LIB_PATH = %r\n"
+            "try:\n    _lib.lib()\nexcept ImportError as e:\n    print('RAISED'); sys.exit(0)\nsys.exit(1)\n"
+            % (ROOT, str(tmp_path / "nope.so")))
+    r = subprocess.run([sys.executable, "-c", code], capture_output=True, text=True)
+    assert r.returncode == 0 and "RAISED" in r.stdout
+
+
+def test_product_never_imports_oracle():
+    pkg = os.path.join(ROOT, "paper_2207_08820_b200")
+    for dirpath, _, files in os.walk(pkg):
+        if "_build" in dirpath:
+            continue
+        for f in files:
+            if f.endswith((".py", ".cu", ".cuh", ".h")):
+                text = open(os.path.join(dirpath, f)).read()
+                assert "import oracle" not in text and "from oracle" not in text and "bitserial_oracle" not in text, f
