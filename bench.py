@@ -1,0 +1,323 @@
+#!/usr/bin/env python
+"""Benchmark of the bit-serial convolution hot path.
+
+One step = one pass of the whole path over one batch: quantise + bitplane-pack the fp32 input, then every
+quantised conv layer of the residual stack (conv2_x..conv5_x of an 18-layer network at 224 px, batch 64 per
+GPU, 2-bit weights and activations) with the fused requantisation epilogue.  Prints ONE JSON line.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--workload NAME]
+
+N > 1 runs under torchrun, one rank per GPU, each rank its own batch (no data-path collective).
+`--impl reference` times the CPU oracle on a bounded sample of the same workload on the host cores.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+from paper_2207_08820_b200 import workloads as wl  # noqa: E402
+
+ACT_SCALE = 0.25
+METRIC = "bitserial_conv_effective_gops"
+UNIT = "GOPS"
+POPC_PER_CLK_PER_SM = 16          # population count throughput per SM per clock (CUDA programming guide, arithmetic table)
+
+
+def make_net(name: str, batch: int):
+    if name == "resnet18_body":
+        return wl.resnet18_body(batch), 3000
+    if name == "detection_backbone":
+        return wl.detection_backbone(batch), 4000
+    raise SystemExit(f"unknown workload {name}")
+
+
+def wordops_per_image(net) -> int:
+    """popc32(AND) word operations of the Section V plane-pair sum: outputs x reduction words x plane pairs."""
+    shapes = net.tensor_shapes()
+    total = 0
+    for L in net.layers:
+        _, P, Q = shapes[L.dst]
+        total += P * Q * L.O * L.k * L.k * ((L.C + 31) // 32) * net.a_bits * net.w_bits
+    return total
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            d = json.load(f)
+        return d, "measured"
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "sm_max_mhz": 1965.0}, "fallback"
+
+
+class ClockSampler:
+    """Samples nvidia-smi clocks and throttle reasons while the timed region runs."""
+    QUERY = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+             "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index = index
+        self.samples = []
+        self._stop = threading.Event()
+        self._thread = threading.Thread(target=self._run, daemon=True)
+
+    def _run(self):
+        while not self._stop.is_set():
+            try:
+                out = subprocess.run(["nvidia-smi", f"--query-gpu={self.QUERY}", "--format=csv,noheader,nounits",
+                                      "-i", str(self.index)], capture_output=True, text=True, timeout=5).stdout.strip()
+                if out:
+                    self.samples.append([c.strip() for c in out.split(",")])
+            except Exception:
+                pass
+            self._stop.wait(0.1)
+
+    def __enter__(self):
+        self._thread.start()
+        return self
+
+    def __exit__(self, *exc):
+        self._stop.set()
+        self._thread.join(timeout=10)
+
+    def summary(self):
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for s in self.samples:
+            try:
+                sm.append(float(s[0]))
+                mx.append(float(s[1]))
+            except (ValueError, IndexError):
+                continue
+            for n, v in zip(names, s[2:6]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "reasons": sorted(reasons), "samples": len(sm)}
+
+
+def run_reference(args):
+    """The CPU oracle, as it stands, on a bounded sample of the workload (host cores only)."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    import oracle
+    from oracle import network as onet
+    net, seed = make_net(args.workload, args.batch)
+    params = wl.network_params(net, seed)
+    sample = args.ref_images
+    x = wl.network_input(net, seed, ACT_SCALE, batch=sample)
+    macs = net.macs_per_image() * sample
+    for _ in range(args.warmup):
+        onet.run_stack(net, params, x[:1], ACT_SCALE)
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        onet.run_stack(net, params, x, ACT_SCALE)
+    dt = (time.perf_counter() - t0) / args.steps
+    gops = 2.0 * macs / dt / 1e9
+    cores = oracle.num_threads()
+    desc = f"{sample} of {net.batch} images of {net.name} per step, all layers, quantise + direct integer conv + epilogue"
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": gops, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": dt * 1e3, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "int32", "data": "synthetic",
+        "config": {"workload": f"{net.name}_batch{net.batch}_w{net.w_bits}a{net.a_bits}", "sample_images": sample},
+        "images_per_s": sample / dt,
+        "cpu_baseline": {"value": gops, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": desc},
+        "e2e": {"value": gops, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }))
+
+
+def run_ours(args):
+    import torch
+    import torch.distributed as dist
+
+    from paper_2207_08820_b200 import api
+    from paper_2207_08820_b200.net import BitserialNet
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the library has no CPU fallback")
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+
+    net, seed = make_net(args.workload, args.batch)
+    params = wl.network_params(net, seed)
+    x_host = torch.from_numpy(wl.network_input(net, seed + rank, ACT_SCALE)).pin_memory()
+    x_dev = x_host.cuda()
+    runner = BitserialNet(net, params, ACT_SCALE, batch=net.batch)
+
+    stream = torch.cuda.Stream()
+    with torch.cuda.stream(stream):
+        # two graphs so that the pack kernel and the conv kernels can be timed separately on this stream
+        in_buf = runner.bufs[net.in_name]
+        api.bitpack_activations(x_dev, ACT_SCALE, net.a_bits, api.UNSIGNED, api.NCHW, out=in_buf.view(-1))
+        runner.forward(x_dev)
+        api.bs_check_status(stream)
+        g_pack, g_conv = torch.cuda.CUDAGraph(), torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g_pack, stream=stream):
+            api.bitpack_activations(x_dev, ACT_SCALE, net.a_bits, api.UNSIGNED, api.NCHW, out=in_buf.view(-1))
+        with torch.cuda.graph(g_conv, stream=stream):
+            for item in runner.layers:
+                runner_conv(runner, item)
+    stream.synchronize()
+
+    flush = torch.empty(256 * 1024 * 1024, dtype=torch.uint8, device="cuda")   # larger than the 126 MB L2
+
+    def step(ev=None):
+        if ev:
+            ev[0].record(stream)
+        g_pack.replay()
+        if ev:
+            ev[1].record(stream)
+        g_conv.replay()
+        if ev:
+            ev[2].record(stream)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    out_packed = runner.bufs[net.out_name]
+    out_host = torch.empty(out_packed.shape, dtype=out_packed.dtype).pin_memory()
+
+    with torch.cuda.stream(stream):
+        for _ in range(args.warmup):
+            flush.zero_()
+            step()
+        barrier()
+        events = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(args.steps)]
+        with ClockSampler(local) as clocks:
+            barrier()
+            for k in range(args.steps):
+                flush.zero_()          # L2 flush between timed iterations (outside the event pairs)
+                step(events[k])
+            barrier()
+        t_pack = sum(e[0].elapsed_time(e[1]) for e in events) / args.steps
+        t_conv = sum(e[1].elapsed_time(e[2]) for e in events) / args.steps
+        t_step = sum(e[0].elapsed_time(e[2]) for e in events) / args.steps
+        api.bs_check_status(stream)
+
+        # end to end through the public API: pinned host input -> device, path, packed result -> host
+        e2e_events = [[torch.cuda.Event(enable_timing=True) for _ in range(2)] for _ in range(args.steps)]
+        for k in range(args.warmup + args.steps):
+            flush.zero_()
+            timed = k >= args.warmup
+            if timed:
+                e2e_events[k - args.warmup][0].record(stream)
+            x_dev.copy_(x_host, non_blocking=True)
+            step()
+            out_host.copy_(out_packed, non_blocking=True)
+            if timed:
+                e2e_events[k - args.warmup][1].record(stream)
+        barrier()
+        t_e2e = sum(e[0].elapsed_time(e[1]) for e in e2e_events) / args.steps
+
+    times = torch.tensor([t_step, t_e2e, t_conv, t_pack], dtype=torch.float64, device="cuda")
+    if world > 1:
+        dist.all_reduce(times, op=dist.ReduceOp.MAX)
+    t_step, t_e2e, t_conv, t_pack = times.tolist()
+
+    if rank == 0:
+        macs = net.macs_per_image() * net.batch
+        wops = wordops_per_image(net) * net.batch
+        gops = 2.0 * macs * world / (t_step * 1e-3) / 1e9
+        peaks, peak_kind = measured_peaks()
+        sms = torch.cuda.get_device_properties(local).multi_processor_count
+        popc_peak = POPC_PER_CLK_PER_SM * sms * peaks["sm_max_mhz"] * 1e6          # word-ops/s at the maximum SM clock
+        achieved = wops / (t_conv * 1e-3)
+        popc_measured = api.bs_popc_rate(4096)
+        in_bytes = x_host.numel() * 4
+        pack_bytes = in_bytes + in_buf.numel() * 4
+        line = {
+            "metric": METRIC, "value": gops, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+            "ms_per_step": t_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "int32", "data": "synthetic",
+            "config": {"workload": f"{net.name}_batch{net.batch}_w{net.w_bits}a{net.a_bits}",
+                       "global_batch": net.batch * world, "parallelism": f"replicas{world}", "layers": len(net.layers),
+                       "l2": "flushed between timed iterations (256 MB write)", "launch": "CUDA graphs (pack, convs)"},
+            "images_per_s": net.batch * world / (t_step * 1e-3),
+            "roofline": {"bound": "alu", "kernel": "bitserial_conv_kernel", "achieved": achieved / 1e12,
+                         "peak": popc_peak / 1e12, "unit": "Tword-op/s", "frac": achieved / popc_peak, "traffic": None,
+                         "peak_source": f"{POPC_PER_CLK_PER_SM} popc/clk/SM x {sms} SMs x {peaks['sm_max_mhz']:.0f} MHz ({peak_kind} clock)",
+                         "popc_pipe_measured": popc_measured / 1e12, "launches_per_step": len(net.layers),
+                         "avg_launch_ms": t_conv / len(net.layers)},
+            "pack": {"bound": "hbm", "ms": t_pack, "achieved": pack_bytes / (t_pack * 1e-3) / 1e9, "peak": peaks["hbm_gbs"],
+                     "unit": "GB/s", "frac": pack_bytes / (t_pack * 1e-3) / 1e9 / peaks["hbm_gbs"]},
+            "e2e": {"value": 2.0 * macs * world / (t_e2e * 1e-3) / 1e9, "unit": UNIT, "ms_per_step": t_e2e,
+                    "h2d_bytes_per_step": in_bytes, "d2h_bytes_per_step": out_host.numel() * 4},
+            "gpu_launches": runner.launches_per_forward * args.steps,
+            "clocks": clocks.summary(),
+        }
+        if world == 1 and not args.no_cpu_baseline:
+            line["cpu_baseline"] = cpu_baseline(net, params, seed, args.cpu_baseline_images)
+        print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def runner_conv(runner, item):
+    """One conv layer of the stack through the C ABI (same call BitserialNet.forward makes)."""
+    from paper_2207_08820_b200 import api
+    net, L = runner.net, item["spec"]
+    res = runner.bufs[L.res] if L.res else None
+    api.bitserial_conv2d(
+        runner.bufs[L.src], item["w"], C=L.C, stride=L.stride, pad=L.pad, a_sign=api.UNSIGNED, w_sign=item["w_sign"],
+        scale=item["scale"], bias=item["bias"], relu=L.relu, out_bits=net.a_bits, out_sign=api.UNSIGNED, residual=res,
+        res_scale=L.res_scale, res_bits=net.a_bits if L.res else 0, res_sign=api.UNSIGNED, res_c_offset=0,
+        res_c_total=runner.shapes[L.res][0] if L.res else 0, out_packed=runner.bufs[L.dst],
+        out_c_offset=L.dst_c_offset, out_c_total=runner.shapes[L.dst][0])
+
+
+def cpu_baseline(net, params, seed, sample):
+    import oracle
+    from oracle import network as onet
+    x = wl.network_input(net, seed, ACT_SCALE, batch=sample)
+    onet.run_stack(net, params, x[:1], ACT_SCALE)
+    t0 = time.perf_counter()
+    onet.run_stack(net, params, x, ACT_SCALE)
+    dt = time.perf_counter() - t0
+    return {"value": 2.0 * net.macs_per_image() * sample / dt / 1e9, "unit": UNIT, "cores": oracle.num_threads(),
+            "kind": "oracle", "images_per_s": sample / dt,
+            "sample": f"{sample} of {net.batch} images of {net.name}, all layers, one pass ({dt:.1f} s)"}
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="resnet18_body", choices=["resnet18_body", "detection_backbone"])
+    ap.add_argument("--batch", type=int, default=0, help="images per GPU (default: 64 / 16 as the workload defines)")
+    ap.add_argument("--ref-images", type=int, default=2, help="images per step of the reference arm (bounded CPU sample)")
+    ap.add_argument("--cpu-baseline-images", type=int, default=64, help="images of the one oracle pass timed beside the GPU run")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.batch == 0:
+        args.batch = 64 if args.workload == "resnet18_body" else 16
+    if args.warmup < 3 and args.impl == "ours":
+        args.warmup = 3
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()
