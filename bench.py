@@ -168,12 +168,22 @@ def run_ours(args):
         api.bitpack_activations(x_dev, ACT_SCALE, net.a_bits, api.UNSIGNED, api.NCHW, out=in_buf.view(-1))
         runner.forward(x_dev)
         api.bs_check_status(stream)
-        g_pack, g_conv = torch.cuda.CUDAGraph(), torch.cuda.CUDAGraph()
-        with torch.cuda.graph(g_pack, stream=stream):
+        def run_pack():
             api.bitpack_activations(x_dev, ACT_SCALE, net.a_bits, api.UNSIGNED, api.NCHW, out=in_buf.view(-1))
-        with torch.cuda.graph(g_conv, stream=stream):
+
+        def run_convs():
             for item in runner.layers:
                 runner_conv(runner, item)
+
+        if args.eager:
+            replay_pack, replay_conv = run_pack, run_convs
+        else:
+            g_pack, g_conv = torch.cuda.CUDAGraph(), torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g_pack, stream=stream):
+                run_pack()
+            with torch.cuda.graph(g_conv, stream=stream):
+                run_convs()
+            replay_pack, replay_conv = g_pack.replay, g_conv.replay
     stream.synchronize()
 
     flush = torch.empty(256 * 1024 * 1024, dtype=torch.uint8, device="cuda")   # larger than the 126 MB L2
@@ -181,10 +191,10 @@ def run_ours(args):
     def step(ev=None):
         if ev:
             ev[0].record(stream)
-        g_pack.replay()
+        replay_pack()
         if ev:
             ev[1].record(stream)
-        g_conv.replay()
+        replay_conv()
         if ev:
             ev[2].record(stream)
 
@@ -250,7 +260,7 @@ def run_ours(args):
             "dtype": "int32", "data": "synthetic",
             "config": {"workload": f"{net.name}_batch{net.batch}_w{net.w_bits}a{net.a_bits}",
                        "global_batch": net.batch * world, "parallelism": f"replicas{world}", "layers": len(net.layers),
-                       "l2": "flushed between timed iterations (256 MB write)", "launch": "CUDA graphs (pack, convs)"},
+                       "l2": "flushed between timed iterations (256 MB write)", "launch": "eager stream launches" if args.eager else "CUDA graphs (pack, convs)"},
             "images_per_s": net.batch * world / (t_step * 1e-3),
             "roofline": {"bound": "alu", "kernel": "bitserial_conv_kernel", "achieved": achieved / 1e12,
                          "peak": popc_peak / 1e12, "unit": "Tword-op/s", "frac": achieved / popc_peak, "traffic": None,
@@ -308,6 +318,7 @@ def main():
     ap.add_argument("--ref-images", type=int, default=2, help="images per step of the reference arm (bounded CPU sample)")
     ap.add_argument("--cpu-baseline-images", type=int, default=64, help="images of the one oracle pass timed beside the GPU run")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--eager", action="store_true", help="plain stream launches instead of CUDA graphs (for per-launch profiling)")
     args = ap.parse_args()
     if args.batch == 0:
         args.batch = 64 if args.workload == "resnet18_body" else 16

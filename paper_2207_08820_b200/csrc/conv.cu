@@ -1,5 +1,8 @@
 // Host side of bitserial_conv2d / bitserial_gemm: validation, tile planning, TMA descriptors, launch.
 #include <array>
+#include <cmath>
+#include <cstdio>
+#include <cstdlib>
 #include <map>
 #include <mutex>
 
@@ -40,7 +43,7 @@ static int sm_count()
 static int round_up(int v, int m) { return (v + m - 1) / m * m; }
 
 struct Plan {
-    int PB, NFG, NT, TWB, TH, TNI, CWC, nchunks, nstage;
+    int PB, FB, NFG, NT, TWB, TH, TNI, CWC, nchunks, nstage;
     int hh, hw, stageA_words, stageW_words, aux_off_words;
     int tma_a, tma_w, boxA_w, nboxA, unitA, unitW;
     size_t smem;
@@ -58,7 +61,7 @@ static int largest_unit(int a, int b)
 // Fill the staging part of a plan; returns false if the tile cannot be staged in shared memory.
 static bool plan_staging(Plan& pl, int Cw, int RS, int R, int S, int stride, int A, int WB)
 {
-    const int TN = pl.NFG * CONV_FB;
+    const int TN = pl.NFG * pl.FB;
     const int TW = pl.TWB * pl.PB;
     pl.hh = (pl.TH - 1) * stride + R;
     pl.hw = (TW - 1) * stride + S;
@@ -94,42 +97,62 @@ static bool plan_staging(Plan& pl, int Cw, int RS, int R, int S, int stride, int
     return pl.smem <= 200 * 1024;
 }
 
+// Per-thread (pixels, filters) register blocks that are instantiated (must match BS_TILE_LIST).
+static const int kTiles[][2] = {{8, 8}, {7, 8}, {4, 8}, {8, 4}, {7, 4}, {4, 4}, {8, 2}, {7, 2}, {4, 2}};
+
+// Exhaustive search over register blocks and CTA tilings with a small analytic time model:
+//   - the popcount pipe retires one warp instruction per 8 cycles per SM sub-partition, so a warp costs
+//     steps * PB * FB * pairs * 8 cycles, divided by an efficiency that is best for 48..160 popcounts per
+//     reduction step (larger bodies spill out of the instruction cache, smaller ones are load-issue bound);
+//   - the busiest SM runs ceil(tiles / SMs) CTAs one after the other on its four sub-partitions;
+//   - fewer than 8 resident warps leave the pipe partly idle.
 static bool search_plan(Plan& best, int N, int P, int Q, int O, int Cw, int R, int S, int stride, int A, int WB)
 {
     const int RS = R * S;
     const int sms = sm_count();
+    const double steps = static_cast<double>(RS) * Cw;
+    const int pairs = A * WB;
     bool found = false;
-    const int pbs[3] = {8, 7, 4};
-    const int nfgs[3] = {8, 4, 16};
-    const int nts[2] = {256, 128};
-    for (int PB : pbs) {
+    for (const auto& tile : kTiles) {
+        const int PB = tile[0], FB = tile[1];
         const int qb = ceil_div(Q, PB);
-        for (int NFG : nfgs) {
-            const int TN = NFG * CONV_FB;
+        const double work = static_cast<double>(PB) * FB * pairs;
+        double eff_block = 0.86;
+        if (work > 160.0) eff_block -= 0.06 * log2(work / 160.0);
+        if (work < 48.0) eff_block -= 0.08 * log2(48.0 / work);
+        const double warp_cycles = steps * work * 8.0 / eff_block + 0.5 * (PB * FB * 15.0 + 1500.0);
+        for (int NFG = 4; NFG <= 32; NFG *= 2) {
+            const int TN = NFG * FB;
+            if (TN % 32 != 0 || TN > 256) continue;          // packed output words must not straddle CTAs
+            if (PB > 4 * NFG) continue;                      // window sums: at most 4 tile pixels per thread
             const long long tiles_o = ceil_div(O, TN);
-            for (int NT : nts) {
-                const int NPG = NT / NFG;
+            for (int NPG = 1; NPG * NFG <= 256; NPG *= 2) {
                 for (int TWB = 1; TWB <= NPG && TWB <= qb; ++TWB) {
                     const int max_th = NPG / TWB;
                     for (int TH = 1; TH <= max_th && TH <= P; ++TH) {
                         int TNI = NPG / (TWB * TH);
                         if (TNI > N) TNI = N;
                         if (TNI < 1) continue;
+                        const int used = TWB * TH * TNI;
+                        if (2 * used <= NPG && NPG > 1) continue;           // a smaller NPG covers this tiling
                         Plan pl{};
-                        pl.PB = PB; pl.NFG = NFG; pl.NT = NT; pl.TWB = TWB; pl.TH = TH; pl.TNI = TNI;
+                        pl.PB = PB; pl.FB = FB; pl.NFG = NFG; pl.TWB = TWB; pl.TH = TH; pl.TNI = TNI;
+                        pl.NT = round_up(used * NFG, 32);
                         if (!plan_staging(pl, Cw, RS, R, S, stride, A, WB)) continue;
                         pl.tiles = tiles_o * ceil_div(qb, TWB) * ceil_div(P, TH) * ceil_div(N, TNI);
-                        // time model: the busiest SM runs ceil(tiles / sms) CTAs; each CTA costs NT * PB thread-steps;
-                        // fewer than 8 resident warps leave the popcount pipe partly idle
                         const long long per_sm = ceil_div_ll(pl.tiles, sms);
+                        const double cta_warps = pl.NT / 32.0;
                         long long resident = static_cast<long long>((200 * 1024) / pl.smem);
                         if (resident > per_sm) resident = per_sm;
-                        if (resident * NT > 2048) resident = 2048 / NT;
-                        double warps = static_cast<double>(resident) * NT / 32.0;
-                        double eff = warps >= 8.0 ? 1.0 : warps / 8.0;
-                        pl.cost = static_cast<double>(per_sm) * NT * PB / eff;
-                        // mild preference for TMA-friendly, low-halo tiles
-                        pl.cost *= 1.0 + 0.02 * (static_cast<double>(pl.hh * pl.hw * TNI) / (TWB * PB * TH * TNI) - 1.0) / (stride * stride);
+                        if (resident * pl.NT > 1536) resident = 1536 / pl.NT;
+                        if (resident < 1) resident = 1;
+                        const double warps = static_cast<double>(resident) * cta_warps;
+                        const double occ = warps >= 8.0 ? 1.0 : warps / 8.0;
+                        // warps of a CTA spread over the four sub-partitions; the fullest one sets the pace
+                        const double per_subpartition = 0.5 * (ceil(cta_warps / 4.0) + cta_warps / 4.0);
+                        pl.cost = static_cast<double>(per_sm) * (per_subpartition < 1.0 ? 1.0 : per_subpartition) * warp_cycles / occ;
+                        // staged halo bytes per useful pixel: a mild tie-breaker towards compact tiles
+                        pl.cost *= 1.0 + 0.01 * (static_cast<double>(pl.hh) * pl.hw / (TWB * PB * TH)) / (stride * stride);
                         if (!found || pl.cost < best.cost * 0.999) { best = pl; found = true; }
                     }
                 }
@@ -142,6 +165,18 @@ static bool search_plan(Plan& best, int N, int P, int Q, int O, int Cw, int R, i
 // Plans depend on the shape only, so they are searched once per shape and remembered.
 static bool make_plan(Plan& out, int N, int P, int Q, int O, int Cw, int R, int S, int stride, int A, int WB)
 {
+#ifdef BS_TUNING   // tile-plan tuning hook, compiled only into tuning builds: BS_PLAN="PB,FB,NFG,NT,TWB,TH,TNI"
+    if (const char* ov = getenv("BS_PLAN")) {
+        Plan pl{};
+        if (sscanf(ov, "%d,%d,%d,%d,%d,%d,%d", &pl.PB, &pl.FB, &pl.NFG, &pl.NT, &pl.TWB, &pl.TH, &pl.TNI) == 7) {
+            if (pl.TNI > N) pl.TNI = N;
+            pl.NT = round_up(pl.TWB * pl.TH * pl.TNI * pl.NFG, 32);
+            if (!plan_staging(pl, Cw, R * S, R, S, stride, A, WB)) return false;
+            out = pl;
+            return true;
+        }
+    }
+#endif
     static std::map<std::array<int, 10>, std::pair<bool, Plan>> cache;
     static std::mutex mu;
     const std::array<int, 10> key = {N, P, Q, O, Cw, R, S, stride, A, WB};
@@ -231,7 +266,7 @@ static int conv_impl(const uint32_t* act, const uint32_t* wgt, const bs_conv_par
     g.used_pg = pl.TWB * pl.TH * pl.TNI;
     g.hh = pl.hh; g.hw = pl.hw; g.CWC = pl.CWC; g.nchunks = pl.nchunks; g.nstage = pl.nstage;
     g.stageA_words = pl.stageA_words; g.stageW_words = pl.stageW_words; g.aux_off_words = pl.aux_off_words;
-    const int TN = pl.NFG * CONV_FB, TW = pl.TWB * pl.PB;
+    const int TN = pl.NFG * pl.FB, TW = pl.TWB * pl.PB;
     g.tiles_o = ceil_div(p->O, TN); g.tiles_q = ceil_div(g.Q, TW); g.tiles_p = ceil_div(g.P, pl.TH);
     g.tiles_n = ceil_div(p->N, pl.TNI);
     g.tma_a = pl.tma_a; g.tma_w = pl.tma_w; g.boxA_w = pl.boxA_w; g.nboxA = pl.nboxA;
@@ -250,6 +285,7 @@ static int conv_impl(const uint32_t* act, const uint32_t* wgt, const bs_conv_par
     g.need_rs = p->w_sign == BS_BIPOLAR;
     g.need_cs = p->a_sign == BS_BIPOLAR;
     g.kconst = (g.need_rs && g.need_cs) ? static_cast<int>(kred) : 0;
+    g.acc_small = kred * max_abs_code(p->a_bits, p->a_sign) * max_abs_code(p->w_bits, p->w_sign) < (1LL << 22);
 
     const long long tiles = static_cast<long long>(g.tiles_o) * g.tiles_q * g.tiles_p * g.tiles_n;
     if (tiles > 0x7fffffffLL) return BS_ERR_UNSUPPORTED;
@@ -274,12 +310,12 @@ static int conv_impl(const uint32_t* act, const uint32_t* wgt, const bs_conv_par
     }
 
     const unsigned grid = static_cast<unsigned>(tiles), block = static_cast<unsigned>(pl.NT);
-    switch (A) {
-        case 1: return launch_conv_a1(WB, pl.PB, g, grid, block, pl.smem, st);
-        case 2: return launch_conv_a2(WB, pl.PB, g, grid, block, pl.smem, st);
-        case 3: return launch_conv_a3(WB, pl.PB, g, grid, block, pl.smem, st);
-        default: return launch_conv_a4(WB, pl.PB, g, grid, block, pl.smem, st);
-    }
+    typedef int (*LaunchFn)(int, int, const ConvArgs&, unsigned, unsigned, size_t, cudaStream_t);
+    static const LaunchFn table[4][3] = {{launch_conv_a1_f2, launch_conv_a1_f4, launch_conv_a1_f8},
+                                         {launch_conv_a2_f2, launch_conv_a2_f4, launch_conv_a2_f8},
+                                         {launch_conv_a3_f2, launch_conv_a3_f4, launch_conv_a3_f8},
+                                         {launch_conv_a4_f2, launch_conv_a4_f4, launch_conv_a4_f8}};
+    return table[A - 1][pl.FB == 8 ? 2 : (pl.FB == 4 ? 1 : 0)](WB, pl.PB, g, grid, block, pl.smem, st);
 }
 
 }  // namespace bs

@@ -52,6 +52,7 @@ struct ConvArgs {
     int cs_coef[4];                          // per weight plane, used when the activations are bipolar
     int kconst;                              // + K when both operands are bipolar
     int need_rs, need_cs;
+    int acc_small;                           // |acc| < 2^22 guaranteed by the shape: the exact mantissa trick applies
 };
 
 // ----------------------------------------------------------------------------- PTX wrappers
@@ -126,6 +127,21 @@ __device__ __forceinline__ void cp_async_wait_pending(int pending)
     }
 }
 
+// ----------------------------------------------------------------------------- exact conversions off the XU pipe
+
+// (float)i for |i| < 2^22, exact: the integer is planted in the mantissa of 1.5 * 2^23 and the offset subtracted.
+// Keeps int->float conversions (which share the population-count pipe) out of the epilogue.
+__device__ __forceinline__ float int_to_float_exact(int i)
+{
+    return __int_as_float(0x4B400000 + i) - 12582912.0f;
+}
+// Round-to-nearest-even of a float already clamped to a small range (|v| <= 2^21): adding 1.5 * 2^23 rounds to an
+// integer in the mantissa with the IEEE default rounding, which is ties-to-even.
+__device__ __forceinline__ int small_float_to_int_rn(float v)
+{
+    return __float_as_int(v + 12582912.0f) - 0x4B400000;
+}
+
 // ----------------------------------------------------------------------------- operand loads
 
 template <int NB>
@@ -198,7 +214,7 @@ __device__ __forceinline__ void stage_issue(const ConvArgs& g, int chunk, uint32
 // ----------------------------------------------------------------------------- the kernel
 
 template <int A, int WB, int PB, int FB>
-__global__ void __launch_bounds__(256) bitserial_conv_kernel(const __grid_constant__ ConvArgs g)
+__global__ void __launch_bounds__(256, (PB * FB <= 32) ? 3 : 1) bitserial_conv_kernel(const __grid_constant__ ConvArgs g)
 {
     extern __shared__ __align__(128) uint32_t smem[];
     const int tid = threadIdx.x, nthreads = blockDim.x;
@@ -283,7 +299,8 @@ __global__ void __launch_bounds__(256) bitserial_conv_kernel(const __grid_consta
         }
         if (any_cp) __syncthreads();
 
-        // ---- plane-pair popcount MACs over all taps and words of this chunk
+        // ---- plane-pair popcount MACs over all taps and words of this chunk (idle pixel groups skip them)
+        if (pg_used)
         for (int tap = 0; tap < RS; ++tap) {
             const int r = tap / g.S, sx = tap - r * g.S;
             const uint32_t* pa = sA + a_off0 + (r * g.hw + sx) * recA;
@@ -405,24 +422,35 @@ __global__ void __launch_bounds__(256) bitserial_conv_kernel(const __grid_consta
             const int q = t.q0 + x;
             const bool pix_ok = row_ok && q < g.Q;
             const size_t pix = (static_cast<size_t>(n) * g.P + p) * g.Q + q;
+            // residual planes are fetched once per 32-channel word, not once per output
+            uint32_t rw[4] = {0, 0, 0, 0};
+            int rw_word = -1;
 #pragma unroll
             for (int u = 0; u < FB; ++u) {
                 const int of = fg + g.NFG * u;
                 const int o = t.o0 + of;
                 unsigned pat = 0;
                 if (pix_ok && o < g.O) {
-                    float val = fmaf(static_cast<float>(acc[v][u]), sc[u], bi[u]);
+                    float val = fmaf(g.acc_small ? int_to_float_exact(acc[v][u]) : static_cast<float>(acc[v][u]), sc[u], bi[u]);
                     if (g.residual) {
                         const int rc = g.res_c_off + o;
-                        const uint32_t* rw = g.residual + (pix * g.res_cw_total + (rc >> 5)) * g.res_bits;
-                        unsigned rp = 0;
-                        for (int j = 0; j < g.res_bits; ++j) rp |= ((rw[j] >> (rc & 31)) & 1u) << j;
-                        val = fmaf(g.res_scale, static_cast<float>(pattern_value(rp, g.res_bits, g.res_sign)), val);
+                        if ((rc >> 5) != rw_word) {
+                            rw_word = rc >> 5;
+                            const uint32_t* rp = g.residual + (pix * g.res_cw_total + rw_word) * g.res_bits;
+#pragma unroll
+                            for (int j = 0; j < 4; ++j)
+                                if (j < g.res_bits) rw[j] = rp[j];
+                        }
+                        unsigned rpat = 0;
+#pragma unroll
+                        for (int j = 0; j < 4; ++j)
+                            if (j < g.res_bits) rpat |= ((rw[j] >> (rc & 31)) & 1u) << j;
+                        val = fmaf(g.res_scale, static_cast<float>(pattern_value(rpat, g.res_bits, g.res_sign)), val);
                     }
                     if (g.relu) val = fmaxf(val, 0.0f);
                     int code;
                     if (g.out_sign == BS_BIPOLAR) code = val >= 0.0f ? 1 : -1;
-                    else code = __float2int_rn(fminf(fmaxf(val, fqmin), fqmax));
+                    else code = small_float_to_int_rn(fminf(fmaxf(val, fqmin), fqmax));
                     pat = stored_pattern(code, g.out_bits, g.out_sign);
                 }
                 if (pg_used) codes_s[((ni * g.TH + ty) * TW + x) * pitch + of] = static_cast<unsigned char>(pat);

@@ -72,29 +72,51 @@ bitpack_kernel(const T* __restrict__ x, uint32_t* __restrict__ out, int C, int H
         }
     } else {
         const bool vec = (HW % 4 == 0);
-        for (int cw = 0; cw < Cw; ++cw) {
-            // phase 1: 32 channels x TP pixels -> byte patterns
-            for (int item = threadIdx.x; item < 32 * (TP / 4); item += PACK_THREADS) {
-                const int cl = item / (TP / 4), q4 = item % (TP / 4);
-                const int c = cw * 32 + cl, px = q4 * 4;
-                unsigned packed4 = 0;
-                if (c < C && px < npix) {
+        // Each thread owns up to 4 items (channel cl, 4 consecutive pixels) per 32-channel word.  The loads of
+        // word cw + 1 are issued before the ballot phase of word cw so that global reads stay in flight.
+        constexpr int MAXI = 4;                       // TP <= 128  =>  32 * (TP / 4) / PACK_THREADS <= 4
+        const int q4n = TP / 4;
+        T v[MAXI][4];
+        auto load_items = [&](int cw) {
+#pragma unroll
+            for (int it = 0; it < MAXI; ++it) {
+                const int item = threadIdx.x + it * PACK_THREADS;
+                const int cl = item / q4n, px = (item % q4n) * 4;
+                const int c = cw * 32 + cl;
+#pragma unroll
+                for (int u = 0; u < 4; ++u) v[it][u] = T(0);
+                if (item < 32 * q4n && c < C && px < npix) {
                     const T* src = x + (static_cast<size_t>(n) * C + c) * HW + hw0 + px;
-                    T v[4];
                     if (vec) {   // npix is a multiple of 4 here, so all four are inside the image
                         typename In4<T>::type q = *reinterpret_cast<const typename In4<T>::type*>(src);
-                        v[0] = q.x; v[1] = q.y; v[2] = q.z; v[3] = q.w;
+                        v[it][0] = q.x; v[it][1] = q.y; v[it][2] = q.z; v[it][3] = q.w;
                     } else {
 #pragma unroll
-                        for (int u = 0; u < 4; ++u) v[u] = (px + u < npix) ? src[u] : T(0);
+                        for (int u = 0; u < 4; ++u)
+                            if (px + u < npix) v[it][u] = src[u];
                     }
+                }
+            }
+        };
+        load_items(0);
+        for (int cw = 0; cw < Cw; ++cw) {
+            // phase 1: 32 channels x TP pixels -> byte patterns
+#pragma unroll
+            for (int it = 0; it < MAXI; ++it) {
+                const int item = threadIdx.x + it * PACK_THREADS;
+                if (item >= 32 * q4n) continue;
+                const int cl = item / q4n, px = (item % q4n) * 4;
+                const int c = cw * 32 + cl;
+                unsigned packed4 = 0;
+                if (c < C) {
 #pragma unroll
                     for (int u = 0; u < 4; ++u)
                         if (px + u < npix)
-                            packed4 |= stored_pattern(to_code<T>(v[u], s, qmin, qmax, sign), bits, sign) << (8 * u);
+                            packed4 |= stored_pattern(to_code<T>(v[it][u], s, qmin, qmax, sign), bits, sign) << (8 * u);
                 }
                 *reinterpret_cast<unsigned*>(codes_s + cl * pitch + px) = packed4;
             }
+            if (cw + 1 < Cw) load_items(cw + 1);
             __syncthreads();
             // phase 2: one warp per pixel, lane = channel, one ballot per plane
             for (int px = warp; px < TP; px += NWARP) {
