@@ -1,145 +1,149 @@
 // Quantise + bitplane split of activations (Section IV quantiser, Section V plane split), the inverse
 // unpack, and the offline plane split of weights / matrix rows.
+#include <cmath>
+#include <cstring>
+
 #include "common.cuh"
 
 namespace bs {
 
 constexpr int PACK_THREADS = 256;
-constexpr int CODE_PITCH_PAD = 4;   // bytes added to each code row so that byte reads by 32 lanes hit 32 banks
+constexpr int PACK_WARPS = PACK_THREADS / 32;
+constexpr int PACK_UNROLL = 8;      // NHWC: pixels in flight per warp
 
-template <typename T> struct In4;
-template <> struct In4<float> { using type = float4; };
-template <> struct In4<int8_t> { using type = char4; };
+// Quantiser of Section IV prepared for the device.  For 1- and 2-bit codes the decision
+//     code = round_half_even(clip(x / s, qmin, qmax))
+// is monotone in x, so it equals qmin + #{k : x >= bound[k]} where bound[k] is the smallest binary32 value whose
+// code is >= qmin + k.  The host finds those bounds by bisection over the ordered float bit patterns using the very
+// same IEEE division, clip and rint, so the comparison form takes exactly the decision of the formula while costing
+// three compares instead of a division.  Wider codes evaluate the formula directly.
+struct QuantParams {
+    float bound[3];
+    float scale;
+    int bits, sign, qmin, qmax;
+    int by_bounds;      // 1: compare against bound[]; 0: evaluate the formula
+    int flip;           // plane bits to flip: pattern = (count ^ flip) for two's-complement codes
+    float null_value;   // an input whose plane bits (before flipping) are all zero
+};
 
-template <typename T>
-__device__ __forceinline__ int to_code(T v, float s, int qmin, int qmax, int sign);
-template <>
-__device__ __forceinline__ int to_code<float>(float v, float s, int qmin, int qmax, int sign)
-{
-    return quantize_code(v, s, qmin, qmax, sign);
-}
-template <>
-__device__ __forceinline__ int to_code<int8_t>(int8_t v, float, int, int, int) { return v; }
+// Plane bits of one input element.  BITS is the code width; BOUNDS selects the comparison form of the quantiser.
+// Bits that a two's-complement offset flips (QuantParams::flip) are NOT applied here: the callers flip whole words.
+template <typename T, int BITS, bool BOUNDS>
+struct PlaneBits {
+    bool p[BITS];
+    __device__ __forceinline__ PlaneBits(T x, const QuantParams& q)
+    {
+        if constexpr (sizeof(T) == 1) {
+#pragma unroll
+            for (int j = 0; j < BITS; ++j) p[j] = (static_cast<int>(x) >> j) & 1;
+            if (q.sign == BS_BIPOLAR) p[0] = x > 0;
+        } else if constexpr (BOUNDS) {
+            const bool c1 = x >= q.bound[0];
+            if constexpr (BITS == 1) {
+                p[0] = c1;
+            } else {
+                const bool c2 = x >= q.bound[1], c3 = x >= q.bound[2];
+                p[0] = (c1 != c2) != c3;      // count = c1 + c2 + c3 with c1 >= c2 >= c3: bit 0 is the parity, bit 1 is c2
+                p[1] = c2;
+            }
+        } else {
+            const unsigned pat = stored_pattern(quantize_code(x, q.scale, q.qmin, q.qmax, q.sign), BITS, q.sign);
+#pragma unroll
+            for (int j = 0; j < BITS; ++j) p[j] = (pat >> j) & 1u;
+        }
+    }
+};
 
-// One block packs TP consecutive pixels (flattened y*W + x) of one image, all channels.
-//   NCHW: per 32-channel word, lanes read 4 consecutive pixels of one channel (coalesced, vectorised
-//         when H*W % 4 == 0), quantise, park the patterns as bytes in shared memory; then one warp per
-//         pixel reads lane = channel and __ballot_sync gives one word per plane.
-//   NHWC: lane = channel directly; ballot straight from the quantised value.
-// The packed pixel records of the tile are contiguous in global memory and leave through 128-bit stores.
-template <typename T, bool NHWC>
+// Input value that sets no plane bit (used for channels and pixels outside the tensor).
+template <typename T> __device__ __forceinline__ T null_input(const QuantParams& q);
+template <> __device__ __forceinline__ float null_input<float>(const QuantParams& q) { return q.null_value; }
+template <> __device__ __forceinline__ int8_t null_input<int8_t>(const QuantParams& q) { return static_cast<int8_t>(q.null_value); }
+
+// One warp packs 32 consecutive pixels (flattened y*W + x) of one image, all channels, with no block-wide barrier.
+//   NCHW: lane = pixel.  Every channel row is read with one coalesced 128-byte request per warp, a whole 32-channel
+//         word in flight; each lane sets bit c of its own plane words from the plane bits of channel c.
+//   NHWC: lane = channel.  One coalesced request per (pixel, 32-channel word); __ballot_sync over the 32 channels
+//         yields one plane word per vote.
+// The packed records of the 32 pixels are contiguous in global memory; they are parked in the warp's slice of
+// shared memory and leave through coalesced 128-bit stores.
+template <typename T, bool NHWC, int BITS, bool BOUNDS>
 __global__ void __launch_bounds__(PACK_THREADS)
-bitpack_kernel(const T* __restrict__ x, uint32_t* __restrict__ out, int C, int HW, int Cw, int bits, int sign,
-               float s, int TP)
+bitpack_kernel(const T* __restrict__ x, uint32_t* __restrict__ out, int C, int HW, int Cw, long long ntiles,
+               int tiles_per_img, const QuantParams q)
 {
-    extern __shared__ __align__(16) unsigned char smem_raw[];
-    uint32_t* out_s = reinterpret_cast<uint32_t*>(smem_raw);                     // [TP][Cw][bits]
-    const int rec = Cw * bits;
-    unsigned char* codes_s = smem_raw + static_cast<size_t>(TP) * rec * 4;       // [32][TP + pad] (NCHW only)
-    const int pitch = TP + CODE_PITCH_PAD;
-
-    const int n = blockIdx.y;
-    const int hw0 = blockIdx.x * TP;
-    const int npix = min(TP, HW - hw0);
+    extern __shared__ __align__(16) uint32_t pack_smem[];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    constexpr int NWARP = PACK_THREADS / 32;
-    int qmin, qmax;
-    code_limits(bits, sign, qmin, qmax);
+    const long long tile = static_cast<long long>(blockIdx.x) * PACK_WARPS + warp;
+    if (tile >= ntiles) return;                       // whole warps leave; only __syncwarp is used below
+    constexpr int rec_bits = BITS;
+    const int rec = Cw * rec_bits;
+    uint32_t* stage = pack_smem + static_cast<size_t>(warp) * 32 * rec;      // [32 pixels][rec]
+    const long long n = tile / tiles_per_img;
+    const int hw0 = static_cast<int>(tile % tiles_per_img) * 32;
+    const int npix = min(32, HW - hw0);
+    const T nullv = null_input<T>(q);
 
     if (NHWC) {
         const T* xin = x + (static_cast<size_t>(n) * HW + hw0) * C;
         for (int cw = 0; cw < Cw; ++cw) {
             const int c = cw * 32 + lane;
             const bool cvalid = c < C;
-            for (int px0 = warp; px0 < TP; px0 += NWARP * 4) {
-                T v[4];
+            const unsigned valid_word = __ballot_sync(0xffffffffu, cvalid);
+            for (int p0 = 0; p0 < 32; p0 += PACK_UNROLL) {
+                T v[PACK_UNROLL];
 #pragma unroll
-                for (int u = 0; u < 4; ++u) {
-                    const int px = px0 + u * NWARP;
-                    v[u] = (cvalid && px < npix) ? xin[static_cast<size_t>(px) * C + c] : T(0);
-                }
+                for (int u = 0; u < PACK_UNROLL; ++u)
+                    v[u] = (cvalid && p0 + u < npix) ? xin[static_cast<size_t>(p0 + u) * C + c] : nullv;
 #pragma unroll
-                for (int u = 0; u < 4; ++u) {
-                    const int px = px0 + u * NWARP;
-                    unsigned pat = 0;
-                    if (cvalid && px < npix) pat = stored_pattern(to_code<T>(v[u], s, qmin, qmax, sign), bits, sign);
-                    for (int j = 0; j < bits; ++j) {
-                        const unsigned word = __ballot_sync(0xffffffffu, (pat >> j) & 1u);
-                        if (lane == j && px < TP) out_s[(px * Cw + cw) * bits + j] = word;
+                for (int u = 0; u < PACK_UNROLL; ++u) {
+                    const PlaneBits<T, BITS, BOUNDS> pb(v[u], q);
+                    const unsigned fl = (p0 + u < npix) ? valid_word : 0u;
+#pragma unroll
+                    for (int j = 0; j < BITS; ++j) {
+                        unsigned word = __ballot_sync(0xffffffffu, pb.p[j]);
+                        if ((q.flip >> j) & 1) word ^= fl;
+                        if (lane == j) stage[(p0 + u) * rec + cw * BITS + j] = word;
                     }
                 }
             }
         }
     } else {
-        const bool vec = (HW % 4 == 0);
-        // Each thread owns up to 4 items (channel cl, 4 consecutive pixels) per 32-channel word.  The loads of
-        // word cw + 1 are issued before the ballot phase of word cw so that global reads stay in flight.
-        constexpr int MAXI = 4;                       // TP <= 128  =>  32 * (TP / 4) / PACK_THREADS <= 4
-        const int q4n = TP / 4;
-        T v[MAXI][4];
-        auto load_items = [&](int cw) {
-#pragma unroll
-            for (int it = 0; it < MAXI; ++it) {
-                const int item = threadIdx.x + it * PACK_THREADS;
-                const int cl = item / q4n, px = (item % q4n) * 4;
-                const int c = cw * 32 + cl;
-#pragma unroll
-                for (int u = 0; u < 4; ++u) v[it][u] = T(0);
-                if (item < 32 * q4n && c < C && px < npix) {
-                    const T* src = x + (static_cast<size_t>(n) * C + c) * HW + hw0 + px;
-                    if (vec) {   // npix is a multiple of 4 here, so all four are inside the image
-                        typename In4<T>::type q = *reinterpret_cast<const typename In4<T>::type*>(src);
-                        v[it][0] = q.x; v[it][1] = q.y; v[it][2] = q.z; v[it][3] = q.w;
-                    } else {
-#pragma unroll
-                        for (int u = 0; u < 4; ++u)
-                            if (px + u < npix) v[it][u] = src[u];
-                    }
-                }
-            }
-        };
-        load_items(0);
+        const bool pvalid = lane < npix;
+        const T* xin = x + static_cast<size_t>(n) * C * HW + hw0 + lane;
         for (int cw = 0; cw < Cw; ++cw) {
-            // phase 1: 32 channels x TP pixels -> byte patterns
+            uint32_t words[BITS];
 #pragma unroll
-            for (int it = 0; it < MAXI; ++it) {
-                const int item = threadIdx.x + it * PACK_THREADS;
-                if (item >= 32 * q4n) continue;
-                const int cl = item / q4n, px = (item % q4n) * 4;
-                const int c = cw * 32 + cl;
-                unsigned packed4 = 0;
-                if (c < C) {
+            for (int j = 0; j < BITS; ++j) words[j] = 0u;
+            T v[32];
 #pragma unroll
-                    for (int u = 0; u < 4; ++u)
-                        if (px + u < npix)
-                            packed4 |= stored_pattern(to_code<T>(v[it][u], s, qmin, qmax, sign), bits, sign) << (8 * u);
-                }
-                *reinterpret_cast<unsigned*>(codes_s + cl * pitch + px) = packed4;
+            for (int u = 0; u < 32; ++u) {
+                const int c = cw * 32 + u;
+                v[u] = (pvalid && c < C) ? xin[static_cast<size_t>(c) * HW] : nullv;
             }
-            if (cw + 1 < Cw) load_items(cw + 1);
-            __syncthreads();
-            // phase 2: one warp per pixel, lane = channel, one ballot per plane
-            for (int px = warp; px < TP; px += NWARP) {
-                const unsigned pat = codes_s[lane * pitch + px];
-                for (int j = 0; j < bits; ++j) {
-                    const unsigned word = __ballot_sync(0xffffffffu, (pat >> j) & 1u);
-                    if (lane == j) out_s[(px * Cw + cw) * bits + j] = word;
-                }
+#pragma unroll
+            for (int u = 0; u < 32; ++u) {
+                const PlaneBits<T, BITS, BOUNDS> pb(v[u], q);
+#pragma unroll
+                for (int j = 0; j < BITS; ++j)
+                    if (pb.p[j]) words[j] |= 1u << u;
             }
-            __syncthreads();
+            const int nvalid = min(32, C - cw * 32);
+            const unsigned fl = pvalid ? (nvalid == 32 ? 0xffffffffu : ((1u << nvalid) - 1u)) : 0u;
+#pragma unroll
+            for (int j = 0; j < BITS; ++j)
+                stage[lane * rec + cw * BITS + j] = ((q.flip >> j) & 1) ? (words[j] ^ fl) : words[j];
         }
     }
-    __syncthreads();
-    // write-out: npix * rec contiguous words; the tile start is 16-byte aligned when TP*rec % 4 == 0
+    __syncwarp();
+    // write-out: npix * rec contiguous words
     uint32_t* dst = out + (static_cast<size_t>(n) * HW + hw0) * rec;
     const int nwords = npix * rec;
-    if ((static_cast<size_t>(HW) * rec) % 4 == 0 && (static_cast<size_t>(TP) * rec) % 4 == 0) {
+    if ((static_cast<size_t>(HW) * rec) % 4 == 0 && (32 * rec) % 4 == 0) {
         const int nvec = nwords / 4;
-        for (int k = threadIdx.x; k < nvec; k += PACK_THREADS)
-            reinterpret_cast<uint4*>(dst)[k] = reinterpret_cast<const uint4*>(out_s)[k];
-        for (int k = nvec * 4 + threadIdx.x; k < nwords; k += PACK_THREADS) dst[k] = out_s[k];
+        for (int k = lane; k < nvec; k += 32) reinterpret_cast<uint4*>(dst)[k] = reinterpret_cast<const uint4*>(stage)[k];
+        for (int k = nvec * 4 + lane; k < nwords; k += 32) dst[k] = stage[k];
     } else {
-        for (int k = threadIdx.x; k < nwords; k += PACK_THREADS) dst[k] = out_s[k];
+        for (int k = lane; k < nwords; k += 32) dst[k] = stage[k];
     }
 }
 
@@ -203,24 +207,94 @@ extern "C" size_t bs_packed_rows_bytes(int rows, int K, int bits)
     return static_cast<size_t>(rows) * ceil_div(K, 32) * bits * sizeof(uint32_t);
 }
 
-template <typename T, bool NHWC>
-static int launch_bitpack(const void* x, uint32_t* out, int N, int C, int HW, int bits, int sign, float s,
-                          cudaStream_t st)
+// Host copy of the Section IV quantiser (IEEE binary32 division, clip, round-half-even) used to derive the bounds.
+static int host_quantize(float x, float s, int qmin, int qmax)
+{
+    volatile float t = x / s;
+    float c = fminf(fmaxf(t, static_cast<float>(qmin)), static_cast<float>(qmax));
+    return static_cast<int>(nearbyintf(c));
+}
+
+// Ordered integer key of a float (monotone in the float order) and back.
+static uint32_t float_key(float f)
+{
+    uint32_t u;
+    memcpy(&u, &f, 4);
+    return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
+}
+static float key_float(uint32_t k)
+{
+    uint32_t u = (k & 0x80000000u) ? (k & 0x7fffffffu) : ~k;
+    float f;
+    memcpy(&f, &u, 4);
+    return f;
+}
+
+static QuantParams make_quant_params(float s, int bits, int sign, bool quantise)
+{
+    QuantParams q{};
+    q.scale = s; q.bits = bits; q.sign = sign;
+    code_limits(bits, sign, q.qmin, q.qmax);
+    q.flip = 0;
+    q.by_bounds = 0;
+    q.null_value = (sign == BS_UNSIGNED) ? 0.0f : (sign == BS_BIPOLAR ? -1.0f : 0.0f);   // formula mode / int8 codes
+    if (!quantise) return q;
+    if (sign == BS_BIPOLAR) {                 // +1 iff x >= 0
+        q.null_value = -INFINITY;
+        q.by_bounds = 1;
+        q.bound[0] = 0.0f;
+        return q;
+    }
+    if (bits <= 2) {
+        q.by_bounds = 1;
+        q.null_value = -INFINITY;
+        const uint32_t lo_key = float_key(-INFINITY), hi_key = float_key(INFINITY);
+        for (int k = 1; k <= q.qmax - q.qmin; ++k) {
+            // smallest x (in float order) with code >= qmin + k; the code is monotone in x and reaches qmax at +inf
+            uint32_t lo = lo_key, hi = hi_key;
+            while (lo < hi) {
+                const uint32_t mid = lo + (hi - lo) / 2;
+                if (host_quantize(key_float(mid), s, q.qmin, q.qmax) >= q.qmin + k) hi = mid;
+                else lo = mid + 1;
+            }
+            q.bound[k - 1] = key_float(lo);
+        }
+        if (bits == 1) q.bound[1] = q.bound[2] = INFINITY;
+        // pattern = (qmin + count) mod 2^bits; for two's-complement 2-bit codes qmin = -2 flips bit 1 only
+        q.flip = (sign == BS_SIGNED) ? (static_cast<unsigned>(q.qmin) & ((1u << bits) - 1u)) : 0;
+    }
+    return q;
+}
+
+template <typename T, bool NHWC, int BITS, bool BOUNDS>
+static int launch_bitpack_one(const void* x, uint32_t* out, int N, int C, int HW, const QuantParams& q, cudaStream_t st)
 {
     const int Cw = ceil_div(C, 32);
-    const int rec = Cw * bits;
-    int TP = 128;
-    auto smem_for = [&](int tp) { return static_cast<size_t>(tp) * rec * 4 + (NHWC ? 0 : 32 * (tp + CODE_PITCH_PAD)); };
-    if (smem_for(TP) > 64 * 1024) TP = 32;
-    const size_t smem = smem_for(TP);
+    const int rec = Cw * q.bits;
+    const size_t smem = static_cast<size_t>(PACK_WARPS) * 32 * rec * 4;
     if (smem > 200 * 1024) return BS_ERR_UNSUPPORTED;
-    auto kern = bitpack_kernel<T, NHWC>;
+    auto kern = bitpack_kernel<T, NHWC, BITS, BOUNDS>;
     if (smem > 48 * 1024 &&
         cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)) != cudaSuccess)
         return BS_ERR_CUDA;
-    dim3 grid(ceil_div(HW, TP), N);
-    kern<<<grid, PACK_THREADS, smem, st>>>(static_cast<const T*>(x), out, C, HW, Cw, bits, sign, s, TP);
+    const int tiles_per_img = ceil_div(HW, 32);
+    const long long ntiles = static_cast<long long>(N) * tiles_per_img;
+    const long long blocks = ceil_div_ll(ntiles, PACK_WARPS);
+    if (blocks > 0x7fffffffLL) return BS_ERR_UNSUPPORTED;
+    kern<<<static_cast<unsigned>(blocks), PACK_THREADS, smem, st>>>(static_cast<const T*>(x), out, C, HW, Cw, ntiles,
+                                                                  tiles_per_img, q);
     return cudaGetLastError() == cudaSuccess ? BS_OK : BS_ERR_CUDA;
+}
+
+template <typename T, bool NHWC>
+static int launch_bitpack(const void* x, uint32_t* out, int N, int C, int HW, const QuantParams& q, cudaStream_t st)
+{
+    switch (q.bits) {
+        case 1: return launch_bitpack_one<T, NHWC, 1, true>(x, out, N, C, HW, q, st);
+        case 2: return launch_bitpack_one<T, NHWC, 2, true>(x, out, N, C, HW, q, st);
+        case 3: return launch_bitpack_one<T, NHWC, 3, false>(x, out, N, C, HW, q, st);
+        default: return launch_bitpack_one<T, NHWC, 4, false>(x, out, N, C, HW, q, st);
+    }
 }
 
 extern "C" int bitpack_activations(const void* x, int x_is_fp32, bs_layout_t layout, int N, int C, int H, int W,
@@ -230,14 +304,15 @@ extern "C" int bitpack_activations(const void* x, int x_is_fp32, bs_layout_t lay
     if (!bits_ok(a_bits, a_sign) || (layout != BS_NCHW && layout != BS_NHWC)) return BS_ERR_INVALID_ARG;
     if (x_is_fp32 && !(act_scale > 0.0f && act_scale < 3.0e38f)) return BS_ERR_INVALID_ARG;
     if (!aligned16(x) || !aligned16(packed_out)) return BS_ERR_ALIGNMENT;
-    if (static_cast<long long>(H) * W > 0x7fffffffLL || N > 65535) return BS_ERR_UNSUPPORTED;
+    if (static_cast<long long>(H) * W > 0x7fffffffLL) return BS_ERR_UNSUPPORTED;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const int HW = H * W;
+    const QuantParams q = make_quant_params(x_is_fp32 ? act_scale : 1.0f, a_bits, a_sign, x_is_fp32 != 0);
     if (x_is_fp32)
-        return layout == BS_NHWC ? launch_bitpack<float, true>(x, packed_out, N, C, HW, a_bits, a_sign, act_scale, st)
-                                 : launch_bitpack<float, false>(x, packed_out, N, C, HW, a_bits, a_sign, act_scale, st);
-    return layout == BS_NHWC ? launch_bitpack<int8_t, true>(x, packed_out, N, C, HW, a_bits, a_sign, 1.0f, st)
-                             : launch_bitpack<int8_t, false>(x, packed_out, N, C, HW, a_bits, a_sign, 1.0f, st);
+        return layout == BS_NHWC ? launch_bitpack<float, true>(x, packed_out, N, C, HW, q, st)
+                                 : launch_bitpack<float, false>(x, packed_out, N, C, HW, q, st);
+    return layout == BS_NHWC ? launch_bitpack<int8_t, true>(x, packed_out, N, C, HW, q, st)
+                             : launch_bitpack<int8_t, false>(x, packed_out, N, C, HW, q, st);
 }
 
 extern "C" int bitunpack_activations(const uint32_t* packed, int N, int C, int H, int W, int a_bits, bs_sign_t a_sign,
