@@ -142,7 +142,7 @@ def run_ours(args):
     import torch
     import torch.distributed as dist
 
-    from paper_2207_08820_b200 import api
+    from paper_2207_08820_b200 import api, replicas
     from paper_2207_08820_b200.net import BitserialNet
 
     world = int(os.environ.get("WORLD_SIZE", "1"))
@@ -156,7 +156,7 @@ def run_ours(args):
 
     net, seed = make_net(args.workload, args.batch)
     params = wl.network_params(net, seed)
-    x_host = torch.from_numpy(wl.network_input(net, seed + rank, ACT_SCALE)).pin_memory()
+    x_host = torch.from_numpy(wl.network_input(net, replicas.rank_seed(seed, rank), ACT_SCALE)).pin_memory()
     x_dev = x_host.cuda()
     runner = BitserialNet(net, params, ACT_SCALE, batch=net.batch)
 
@@ -237,10 +237,7 @@ def run_ours(args):
         barrier()
         t_e2e = sum(e[0].elapsed_time(e[1]) for e in e2e_events) / args.steps
 
-    times = torch.tensor([t_step, t_e2e, t_conv, t_pack], dtype=torch.float64, device="cuda")
-    if world > 1:
-        dist.all_reduce(times, op=dist.ReduceOp.MAX)
-    t_step, t_e2e, t_conv, t_pack = times.tolist()
+    t_step, t_e2e, t_conv, t_pack = replicas.max_over_ranks([t_step, t_e2e, t_conv, t_pack], torch.device("cuda", local))
 
     if rank == 0:
         macs = net.macs_per_image() * net.batch

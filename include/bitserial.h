@@ -149,6 +149,26 @@ int bitserial_gemm(const uint32_t* a_packed, const uint32_t* w_packed, int M, in
                    void* stream);
 
 /*
+ * Reduction split over several thread blocks (for problems with few output tiles and a long reduction, e.g. a
+ * 256 x 256 matrix product with K = 4608, or a 7 x 7 layer with 512 channels).  The Section V sum is associative,
+ * so partial popcount sums of disjoint channel-word ranges are added in a caller-provided workspace and the last
+ * block of a tile applies the epilogue; results are bit-identical to the unsplit entry points.
+ *   workspace        device, 16-byte aligned, at least bs_*_workspace_bytes(...) bytes; it must be ZERO before the
+ *                    first call and every call leaves it zero again, so one cudaMemset at allocation suffices.
+ *                    Calls that share a workspace must not overlap on the GPU (use one stream, or one workspace
+ *                    per stream).  A NULL or too small workspace falls back to the unsplit kernel.
+ *   bs_*_workspace_bytes  bytes the planner wants for this shape (0: no split would be used).  Host-only, no launch.
+ */
+size_t bs_conv_workspace_bytes(const bs_conv_params* p);
+size_t bs_gemm_workspace_bytes(int M, int N, int K, int a_bits, bs_sign_t a_sign, int w_bits, bs_sign_t w_sign);
+int bitserial_conv2d_ws(const uint32_t* act_packed, const uint32_t* wgt_packed, const bs_conv_params* p,
+                        int32_t* out_i32, uint32_t* out_packed, void* workspace, size_t workspace_bytes, void* stream);
+int bitserial_gemm_ws(const uint32_t* a_packed, const uint32_t* w_packed, int M, int N, int K, int a_bits,
+                      bs_sign_t a_sign, int w_bits, bs_sign_t w_sign, const float* scale, const float* bias,
+                      int relu, int out_bits, bs_sign_t out_sign, int32_t* out_i32, uint32_t* out_packed,
+                      void* workspace, size_t workspace_bytes, void* stream);
+
+/*
  * bs_check_status -- synchronises `stream`, then reads and clears the device status word of the current
  * device.  Returns BS_ERR_TIMEOUT if any kernel since the last check gave up on a bounded wait (its
  * outputs are then undefined), BS_ERR_CUDA if the stream reports an error, else BS_OK.

@@ -63,6 +63,14 @@ def lib() -> ctypes.CDLL:
     L.bitserial_conv2d.argtypes = [vp, vp, ctypes.POINTER(ConvParams), vp, vp, vp]
     L.bitserial_gemm.restype = i
     L.bitserial_gemm.argtypes = [vp, vp, i, i, i, i, i, i, i, vp, vp, i, i, i, vp, vp, vp]
+    L.bitserial_conv2d_ws.restype = i
+    L.bitserial_conv2d_ws.argtypes = [vp, vp, ctypes.POINTER(ConvParams), vp, vp, vp, ctypes.c_size_t, vp]
+    L.bitserial_gemm_ws.restype = i
+    L.bitserial_gemm_ws.argtypes = [vp, vp, i, i, i, i, i, i, i, vp, vp, i, i, i, vp, vp, vp, ctypes.c_size_t, vp]
+    L.bs_conv_workspace_bytes.restype = ctypes.c_size_t
+    L.bs_conv_workspace_bytes.argtypes = [ctypes.POINTER(ConvParams)]
+    L.bs_gemm_workspace_bytes.restype = ctypes.c_size_t
+    L.bs_gemm_workspace_bytes.argtypes = [i] * 7
     L.bs_check_status.restype = i
     L.bs_check_status.argtypes = [vp]
     L.bs_popc_rate.restype = i
@@ -75,4 +83,5 @@ def lib() -> ctypes.CDLL:
 
 EXPORTED = ("bs_packed_act_bytes", "bs_packed_wgt_bytes", "bs_packed_rows_bytes", "bitpack_activations",
             "bitunpack_activations", "pack_weights", "bs_pack_rows", "bitserial_conv2d", "bitserial_gemm",
+            "bitserial_conv2d_ws", "bitserial_gemm_ws", "bs_conv_workspace_bytes", "bs_gemm_workspace_bytes",
             "bs_check_status", "bs_popc_rate", "bs_status_string")

@@ -113,9 +113,10 @@ def bitserial_conv2d(act_packed: torch.Tensor, wgt_packed: torch.Tensor, *, C: i
                      res_bits: int = 0, res_sign: int = UNSIGNED, res_c_offset: int = 0, res_c_total: int = 0,
                      out_i32: Optional[torch.Tensor] = None, want_i32: bool = False, i32_layout: int = NCHW,
                      out_packed: Optional[torch.Tensor] = None, out_c_offset: int = 0, out_c_total: int = 0,
-                     stream=None):
+                     workspace: Optional[torch.Tensor] = None, stream=None):
     """act_packed [N,H,W,Cw,a_bits], wgt_packed [O,R,S,Cw,w_bits].  Returns (out_i32 or None, out_packed or None).
-    A packed output is produced when ``out_bits`` > 0 (allocated here unless ``out_packed`` is given)."""
+    A packed output is produced when ``out_bits`` > 0 (allocated here unless ``out_packed`` is given).
+    ``workspace`` (zeroed device tensor, see :func:`conv_workspace`) enables the reduction split (``bitserial_conv2d_ws``)."""
     N, H, W, Cw, a_bits = act_packed.shape
     O, R, S, Cw2, w_bits = wgt_packed.shape
     if Cw != Cw2 or Cw != (C + 31) // 32:
@@ -137,8 +138,13 @@ def bitserial_conv2d(act_packed: torch.Tensor, wgt_packed: torch.Tensor, *, C: i
                    res_bits=res_bits, res_sign=res_sign, res_c_offset=res_c_offset,
                    res_c_total=res_c_total if res_c_total else res_c_offset + O,
                    out_c_offset=out_c_offset, out_c_total=out_c_total, i32_layout=i32_layout)
-    st = lib().bitserial_conv2d(_ptr(act_packed), _ptr(wgt_packed), ctypes.byref(p), _ptr(out_i32),
-                                _ptr(out_packed) if out_bits > 0 else None, _stream_ptr(stream))
+    if workspace is not None:
+        st = lib().bitserial_conv2d_ws(_ptr(act_packed), _ptr(wgt_packed), ctypes.byref(p), _ptr(out_i32),
+                                       _ptr(out_packed) if out_bits > 0 else None, _ptr(workspace),
+                                       workspace.numel() * workspace.element_size(), _stream_ptr(stream))
+    else:
+        st = lib().bitserial_conv2d(_ptr(act_packed), _ptr(wgt_packed), ctypes.byref(p), _ptr(out_i32),
+                                    _ptr(out_packed) if out_bits > 0 else None, _stream_ptr(stream))
     _check(st, "bitserial_conv2d")
     return out_i32, (out_packed if out_bits > 0 else None)
 
@@ -147,8 +153,9 @@ def bitserial_gemm(a_packed: torch.Tensor, w_packed: torch.Tensor, K: int, *, a_
                    w_sign: int = SIGNED, scale: Optional[torch.Tensor] = None, bias: Optional[torch.Tensor] = None,
                    relu: bool = False, out_bits: int = 0, out_sign: int = UNSIGNED,
                    out_i32: Optional[torch.Tensor] = None, want_i32: bool = True,
-                   out_packed: Optional[torch.Tensor] = None, stream=None):
-    """a_packed [M,Kw,a_bits], w_packed [N,Kw,w_bits].  Returns (out_i32 [M,N] or None, out_packed or None)."""
+                   out_packed: Optional[torch.Tensor] = None, workspace: Optional[torch.Tensor] = None, stream=None):
+    """a_packed [M,Kw,a_bits], w_packed [N,Kw,w_bits].  Returns (out_i32 [M,N] or None, out_packed or None).
+    ``workspace`` (zeroed device tensor, see :func:`gemm_workspace`) enables the reduction split (``bitserial_gemm_ws``)."""
     M, Kw, a_bits = a_packed.shape
     N, Kw2, w_bits = w_packed.shape
     if Kw != Kw2 or Kw != (K + 31) // 32:
@@ -158,11 +165,32 @@ def bitserial_gemm(a_packed: torch.Tensor, w_packed: torch.Tensor, K: int, *, a_
         out_i32 = torch.empty(M, N, dtype=torch.int32, device=dev)
     if out_bits > 0 and out_packed is None:
         out_packed = torch.zeros(M, (N + 31) // 32, out_bits, dtype=torch.int32, device=dev)
-    st = lib().bitserial_gemm(_ptr(a_packed), _ptr(w_packed), M, N, K, a_bits, a_sign, w_bits, w_sign,
-                              _ptr(scale), _ptr(bias), int(relu), out_bits, out_sign, _ptr(out_i32),
-                              _ptr(out_packed) if out_bits > 0 else None, _stream_ptr(stream))
+    if workspace is not None:
+        st = lib().bitserial_gemm_ws(_ptr(a_packed), _ptr(w_packed), M, N, K, a_bits, a_sign, w_bits, w_sign,
+                                     _ptr(scale), _ptr(bias), int(relu), out_bits, out_sign, _ptr(out_i32),
+                                     _ptr(out_packed) if out_bits > 0 else None, _ptr(workspace),
+                                     workspace.numel() * workspace.element_size(), _stream_ptr(stream))
+    else:
+        st = lib().bitserial_gemm(_ptr(a_packed), _ptr(w_packed), M, N, K, a_bits, a_sign, w_bits, w_sign,
+                                  _ptr(scale), _ptr(bias), int(relu), out_bits, out_sign, _ptr(out_i32),
+                                  _ptr(out_packed) if out_bits > 0 else None, _stream_ptr(stream))
     _check(st, "bitserial_gemm")
     return out_i32, (out_packed if out_bits > 0 else None)
+
+
+def gemm_workspace(M: int, N: int, K: int, a_bits: int, a_sign: int, w_bits: int, w_sign: int, device="cuda"):
+    """Zeroed workspace for the reduction split of this matrix product, or None when the planner would not split."""
+    nbytes = lib().bs_gemm_workspace_bytes(M, N, K, a_bits, a_sign, w_bits, w_sign)
+    return torch.zeros((nbytes + 3) // 4, dtype=torch.int32, device=device) if nbytes else None
+
+
+def conv_workspace(N: int, C: int, H: int, W: int, O: int, k: int, stride: int, pad: int, a_bits: int, a_sign: int,
+                   w_bits: int, w_sign: int, device="cuda"):
+    """Zeroed workspace for the reduction split of this convolution, or None when the planner would not split."""
+    p = ConvParams(N=N, C=C, H=H, W=W, O=O, R=k, S=k, stride=stride, pad=pad, a_bits=a_bits, a_sign=a_sign,
+                   w_bits=w_bits, w_sign=w_sign)
+    nbytes = lib().bs_conv_workspace_bytes(ctypes.byref(p))
+    return torch.zeros((nbytes + 3) // 4, dtype=torch.int32, device=device) if nbytes else None
 
 
 def bs_check_status(stream=None) -> None:

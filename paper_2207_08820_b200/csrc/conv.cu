@@ -46,7 +46,8 @@ struct Plan {
     int PB, FB, NFG, NT, TWB, TH, TNI, CWC, nchunks, nstage;
     int hh, hw, stageA_words, stageW_words, aux_off_words;
     int tma_a, tma_w, boxA_w, nboxA, unitA, unitW;
-    size_t smem;
+    int ksplit, chunks_per_split;
+    size_t smem, ws_bytes;
     long long tiles;
     double cost;
 };
@@ -106,11 +107,11 @@ static const int kTiles[][2] = {{8, 8}, {7, 8}, {4, 8}, {8, 4}, {7, 4}, {4, 4}, 
 //     reduction step (larger bodies spill out of the instruction cache, smaller ones are load-issue bound);
 //   - the busiest SM runs ceil(tiles / SMs) CTAs one after the other on its four sub-partitions;
 //   - fewer than 8 resident warps leave the pipe partly idle.
-static bool search_plan(Plan& best, int N, int P, int Q, int O, int Cw, int R, int S, int stride, int A, int WB)
+static bool search_plan(Plan& best, int N, int P, int Q, int O, int Cw, int R, int S, int stride, int A, int WB,
+                        bool allow_split)
 {
     const int RS = R * S;
     const int sms = sm_count();
-    const double steps = static_cast<double>(RS) * Cw;
     const int pairs = A * WB;
     bool found = false;
     for (const auto& tile : kTiles) {
@@ -120,7 +121,6 @@ static bool search_plan(Plan& best, int N, int P, int Q, int O, int Cw, int R, i
         double eff_block = 0.86;
         if (work > 160.0) eff_block -= 0.06 * log2(work / 160.0);
         if (work < 48.0) eff_block -= 0.08 * log2(48.0 / work);
-        const double warp_cycles = steps * work * 8.0 / eff_block + 0.5 * (PB * FB * 15.0 + 1500.0);
         for (int NFG = 4; NFG <= 32; NFG *= 2) {
             const int TN = NFG * FB;
             if (TN % 32 != 0 || TN > 256) continue;          // packed output words must not straddle CTAs
@@ -140,20 +140,38 @@ static bool search_plan(Plan& best, int N, int P, int Q, int O, int Cw, int R, i
                         pl.NT = round_up(used * NFG, 32);
                         if (!plan_staging(pl, Cw, RS, R, S, stride, A, WB)) continue;
                         pl.tiles = tiles_o * ceil_div(qb, TWB) * ceil_div(P, TH) * ceil_div(N, TNI);
-                        const long long per_sm = ceil_div_ll(pl.tiles, sms);
                         const double cta_warps = pl.NT / 32.0;
-                        long long resident = static_cast<long long>((200 * 1024) / pl.smem);
-                        if (resident > per_sm) resident = per_sm;
-                        if (resident * pl.NT > 1536) resident = 1536 / pl.NT;
-                        if (resident < 1) resident = 1;
-                        const double warps = static_cast<double>(resident) * cta_warps;
-                        const double occ = warps >= 8.0 ? 1.0 : warps / 8.0;
                         // warps of a CTA spread over the four sub-partitions; the fullest one sets the pace
-                        const double per_subpartition = 0.5 * (ceil(cta_warps / 4.0) + cta_warps / 4.0);
-                        pl.cost = static_cast<double>(per_sm) * (per_subpartition < 1.0 ? 1.0 : per_subpartition) * warp_cycles / occ;
-                        // staged halo bytes per useful pixel: a mild tie-breaker towards compact tiles
-                        pl.cost *= 1.0 + 0.01 * (static_cast<double>(pl.hh) * pl.hw / (TWB * PB * TH)) / (stride * stride);
-                        if (!found || pl.cost < best.cost * 0.999) { best = pl; found = true; }
+                        double per_subpartition = 0.5 * (ceil(cta_warps / 4.0) + cta_warps / 4.0);
+                        if (per_subpartition < 1.0) per_subpartition = 1.0;
+                        const double halo = 1.0 + 0.01 * (static_cast<double>(pl.hh) * pl.hw / (TWB * PB * TH)) / (stride * stride);
+                        // reduction split: only when the tiles alone cannot fill the machine
+                        const int max_split = allow_split ? pl.nchunks : 1;
+                        for (int ksplit = 1; ksplit <= max_split; ksplit *= 2) {
+                            if (ksplit > 1 && pl.tiles * (ksplit / 2) >= 2LL * sms) break;
+                            const int cps = ceil_div(pl.nchunks, ksplit);
+                            const int eff_split = ceil_div(pl.nchunks, cps);
+                            const double split_steps = static_cast<double>(cps) * pl.CWC * RS;
+                            const double wc = split_steps * work * 8.0 / eff_block + 0.5 * (PB * FB * 15.0 + 1500.0) +
+                                              (eff_split > 1 ? PB * FB * 40.0 + 2000.0 : 0.0);
+                            const long long ctas = pl.tiles * eff_split;
+                            const long long per_sm = ceil_div_ll(ctas, sms);
+                            long long resident = static_cast<long long>((200 * 1024) / pl.smem);
+                            if (resident > per_sm) resident = per_sm;
+                            if (resident * pl.NT > 1536) resident = 1536 / pl.NT;
+                            if (resident < 1) resident = 1;
+                            const double warps = static_cast<double>(resident) * cta_warps;
+                            const double occ = warps >= 8.0 ? 1.0 : warps / 8.0;
+                            const double cost = static_cast<double>(per_sm) * per_subpartition * wc / occ * halo;
+                            if (!found || cost < best.cost * 0.999) {
+                                best = pl;
+                                best.cost = cost;
+                                best.ksplit = eff_split;
+                                best.chunks_per_split = cps;
+                                best.ws_bytes = eff_split > 1 ? static_cast<size_t>(pl.tiles) * (static_cast<size_t>(PB) * FB * pl.NT + 1) * 4 : 0;
+                                found = true;
+                            }
+                        }
                     }
                 }
             }
@@ -163,7 +181,8 @@ static bool search_plan(Plan& best, int N, int P, int Q, int O, int Cw, int R, i
 }
 
 // Plans depend on the shape only, so they are searched once per shape and remembered.
-static bool make_plan(Plan& out, int N, int P, int Q, int O, int Cw, int R, int S, int stride, int A, int WB)
+static bool make_plan(Plan& out, int N, int P, int Q, int O, int Cw, int R, int S, int stride, int A, int WB,
+                      bool allow_split)
 {
 #ifdef BS_TUNING   // tile-plan tuning hook, compiled only into tuning builds: BS_PLAN="PB,FB,NFG,NT,TWB,TH,TNI"
     if (const char* ov = getenv("BS_PLAN")) {
@@ -172,19 +191,20 @@ static bool make_plan(Plan& out, int N, int P, int Q, int O, int Cw, int R, int 
             if (pl.TNI > N) pl.TNI = N;
             pl.NT = round_up(pl.TWB * pl.TH * pl.TNI * pl.NFG, 32);
             if (!plan_staging(pl, Cw, R * S, R, S, stride, A, WB)) return false;
+            pl.ksplit = 1; pl.chunks_per_split = pl.nchunks; pl.ws_bytes = 0;
             out = pl;
             return true;
         }
     }
 #endif
-    static std::map<std::array<int, 10>, std::pair<bool, Plan>> cache;
+    static std::map<std::array<int, 11>, std::pair<bool, Plan>> cache;
     static std::mutex mu;
-    const std::array<int, 10> key = {N, P, Q, O, Cw, R, S, stride, A, WB};
+    const std::array<int, 11> key = {N, P, Q, O, Cw, R, S, stride, A, WB, allow_split ? 1 : 0};
     std::lock_guard<std::mutex> lock(mu);
     auto it = cache.find(key);
     if (it == cache.end()) {
         Plan pl{};
-        const bool ok = search_plan(pl, N, P, Q, O, Cw, R, S, stride, A, WB);
+        const bool ok = search_plan(pl, N, P, Q, O, Cw, R, S, stride, A, WB, allow_split);
         it = cache.emplace(key, std::make_pair(ok, pl)).first;
     }
     out = it->second.second;
@@ -209,10 +229,13 @@ static int max_abs_code(int bits, int sign)
     return (1 << bits) - 1;
 }
 
+// `query_ws` != NULL: validate, plan with the reduction split allowed, report the workspace it wants, launch nothing.
 static int conv_impl(const uint32_t* act, const uint32_t* wgt, const bs_conv_params* p, int32_t* out_i32,
-                     uint32_t* out_packed, cudaStream_t st)
+                     uint32_t* out_packed, void* workspace, size_t workspace_bytes, cudaStream_t st,
+                     size_t* query_ws = nullptr)
 {
-    if (!act || !wgt || !p || (!out_i32 && !out_packed)) return BS_ERR_INVALID_ARG;
+    if (!p) return BS_ERR_INVALID_ARG;
+    if (!query_ws && (!act || !wgt || (!out_i32 && !out_packed))) return BS_ERR_INVALID_ARG;
     if (p->N <= 0 || p->C <= 0 || p->H <= 0 || p->W <= 0 || p->O <= 0 || p->R <= 0 || p->S <= 0) return BS_ERR_INVALID_ARG;
     if (!bits_ok(p->a_bits, p->a_sign) || !bits_ok(p->w_bits, p->w_sign)) return BS_ERR_INVALID_ARG;
     if (p->stride < 1 || p->pad < 0) return BS_ERR_INVALID_ARG;
@@ -221,7 +244,8 @@ static int conv_impl(const uint32_t* act, const uint32_t* wgt, const bs_conv_par
     if (p->stride > 2 || p->pad >= p->R) return BS_ERR_UNSUPPORTED;
     if (p->a_sign == BS_BIPOLAR && p->pad != 0) return BS_ERR_UNSUPPORTED;
     if (p->H + 2 * p->pad < p->R || p->W + 2 * p->pad < p->S) return BS_ERR_INVALID_ARG;
-    if (!aligned16(act) || !aligned16(wgt) || (out_i32 && !aligned16(out_i32)) || (out_packed && !aligned16(out_packed)))
+    if (!aligned16(act) || !aligned16(wgt) || (out_i32 && !aligned16(out_i32)) || (out_packed && !aligned16(out_packed)) ||
+        (workspace && !aligned16(workspace)))
         return BS_ERR_ALIGNMENT;
     const long long kred = static_cast<long long>(p->C) * p->R * p->S;
     if (kred * max_abs_code(p->a_bits, p->a_sign) * max_abs_code(p->w_bits, p->w_sign) >= (1LL << 31))
@@ -246,7 +270,12 @@ static int conv_impl(const uint32_t* act, const uint32_t* wgt, const bs_conv_par
 
     const int A = p->a_bits, WB = p->w_bits;
     Plan pl{};
-    if (!make_plan(pl, p->N, g.P, g.Q, p->O, g.Cw, p->R, p->S, p->stride, A, WB)) return BS_ERR_UNSUPPORTED;
+    const bool want_split = query_ws != nullptr || (workspace != nullptr && workspace_bytes > 0);
+    if (!make_plan(pl, p->N, g.P, g.Q, p->O, g.Cw, p->R, p->S, p->stride, A, WB, want_split)) return BS_ERR_UNSUPPORTED;
+    if (query_ws) { *query_ws = pl.ws_bytes; return BS_OK; }
+    if (pl.ws_bytes > workspace_bytes &&      // the workspace is too small for the split plan: run unsplit
+        !make_plan(pl, p->N, g.P, g.Q, p->O, g.Cw, p->R, p->S, p->stride, A, WB, false))
+        return BS_ERR_UNSUPPORTED;
 
     g.act = act; g.wgt = wgt; g.out_i32 = out_i32; g.out_packed = out_packed;
     g.scale = p->scale; g.bias = p->bias;
@@ -285,9 +314,14 @@ static int conv_impl(const uint32_t* act, const uint32_t* wgt, const bs_conv_par
     g.need_rs = p->w_sign == BS_BIPOLAR;
     g.need_cs = p->a_sign == BS_BIPOLAR;
     g.kconst = (g.need_rs && g.need_cs) ? static_cast<int>(kred) : 0;
+    g.ksplit = pl.ksplit; g.chunks_per_split = pl.chunks_per_split;
+    if (pl.ksplit > 1) {
+        g.ws_acc = static_cast<int*>(workspace);
+        g.ws_cnt = reinterpret_cast<unsigned*>(g.ws_acc + static_cast<size_t>(pl.tiles) * pl.PB * pl.FB * pl.NT);
+    }
     g.acc_small = kred * max_abs_code(p->a_bits, p->a_sign) * max_abs_code(p->w_bits, p->w_sign) < (1LL << 22);
 
-    const long long tiles = static_cast<long long>(g.tiles_o) * g.tiles_q * g.tiles_p * g.tiles_n;
+    const long long tiles = static_cast<long long>(g.tiles_o) * g.tiles_q * g.tiles_p * g.tiles_n * pl.ksplit;
     if (tiles > 0x7fffffffLL) return BS_ERR_UNSUPPORTED;
 
     if (g.tma_a) {
@@ -320,10 +354,37 @@ static int conv_impl(const uint32_t* act, const uint32_t* wgt, const bs_conv_par
 
 }  // namespace bs
 
+static bs_conv_params gemm_as_conv(int M, int N, int K, int a_bits, int a_sign, int w_bits, int w_sign, const float* scale,
+                                   const float* bias, int relu, int out_bits, int out_sign)
+{
+    // a matrix product is a 1x1 convolution over a 1 x M image with K channels and N filters
+    bs_conv_params p{};
+    p.N = 1; p.C = K; p.H = 1; p.W = M; p.O = N; p.R = 1; p.S = 1; p.stride = 1; p.pad = 0;
+    p.a_bits = a_bits; p.a_sign = a_sign; p.w_bits = w_bits; p.w_sign = w_sign;
+    p.scale = scale; p.bias = bias; p.relu = relu; p.out_bits = out_bits; p.out_sign = out_sign;
+    p.residual = nullptr; p.out_c_offset = 0; p.out_c_total = N; p.i32_layout = BS_NHWC;
+    return p;
+}
+
 extern "C" int bitserial_conv2d(const uint32_t* act_packed, const uint32_t* wgt_packed, const bs_conv_params* p,
                                 int32_t* out_i32, uint32_t* out_packed, void* stream)
 {
-    return bs::conv_impl(act_packed, wgt_packed, p, out_i32, out_packed, static_cast<cudaStream_t>(stream));
+    return bs::conv_impl(act_packed, wgt_packed, p, out_i32, out_packed, nullptr, 0, static_cast<cudaStream_t>(stream));
+}
+
+extern "C" int bitserial_conv2d_ws(const uint32_t* act_packed, const uint32_t* wgt_packed, const bs_conv_params* p,
+                                   int32_t* out_i32, uint32_t* out_packed, void* workspace, size_t workspace_bytes,
+                                   void* stream)
+{
+    return bs::conv_impl(act_packed, wgt_packed, p, out_i32, out_packed, workspace, workspace_bytes,
+                         static_cast<cudaStream_t>(stream));
+}
+
+extern "C" size_t bs_conv_workspace_bytes(const bs_conv_params* p)
+{
+    size_t need = 0;
+    if (bs::conv_impl(nullptr, nullptr, p, nullptr, nullptr, nullptr, 0, nullptr, &need) != BS_OK) return 0;
+    return need;
 }
 
 extern "C" int bitserial_gemm(const uint32_t* a_packed, const uint32_t* w_packed, int M, int N, int K, int a_bits,
@@ -332,11 +393,26 @@ extern "C" int bitserial_gemm(const uint32_t* a_packed, const uint32_t* w_packed
                               void* stream)
 {
     if (M <= 0 || N <= 0 || K <= 0) return BS_ERR_INVALID_ARG;
-    // a matrix product is a 1x1 convolution over a 1 x M image with K channels and N filters
-    bs_conv_params p{};
-    p.N = 1; p.C = K; p.H = 1; p.W = M; p.O = N; p.R = 1; p.S = 1; p.stride = 1; p.pad = 0;
-    p.a_bits = a_bits; p.a_sign = a_sign; p.w_bits = w_bits; p.w_sign = w_sign;
-    p.scale = scale; p.bias = bias; p.relu = relu; p.out_bits = out_bits; p.out_sign = out_sign;
-    p.residual = nullptr; p.out_c_offset = 0; p.out_c_total = N; p.i32_layout = BS_NHWC;
-    return bs::conv_impl(a_packed, w_packed, &p, out_i32, out_packed, static_cast<cudaStream_t>(stream));
+    const bs_conv_params p = gemm_as_conv(M, N, K, a_bits, a_sign, w_bits, w_sign, scale, bias, relu, out_bits, out_sign);
+    return bs::conv_impl(a_packed, w_packed, &p, out_i32, out_packed, nullptr, 0, static_cast<cudaStream_t>(stream));
+}
+
+extern "C" int bitserial_gemm_ws(const uint32_t* a_packed, const uint32_t* w_packed, int M, int N, int K, int a_bits,
+                                 bs_sign_t a_sign, int w_bits, bs_sign_t w_sign, const float* scale, const float* bias,
+                                 int relu, int out_bits, bs_sign_t out_sign, int32_t* out_i32, uint32_t* out_packed,
+                                 void* workspace, size_t workspace_bytes, void* stream)
+{
+    if (M <= 0 || N <= 0 || K <= 0) return BS_ERR_INVALID_ARG;
+    const bs_conv_params p = gemm_as_conv(M, N, K, a_bits, a_sign, w_bits, w_sign, scale, bias, relu, out_bits, out_sign);
+    return bs::conv_impl(a_packed, w_packed, &p, out_i32, out_packed, workspace, workspace_bytes,
+                         static_cast<cudaStream_t>(stream));
+}
+
+extern "C" size_t bs_gemm_workspace_bytes(int M, int N, int K, int a_bits, bs_sign_t a_sign, int w_bits, bs_sign_t w_sign)
+{
+    if (M <= 0 || N <= 0 || K <= 0) return 0;
+    const bs_conv_params p = gemm_as_conv(M, N, K, a_bits, a_sign, w_bits, w_sign, nullptr, nullptr, 0, 0, 0);
+    size_t need = 0;
+    if (bs::conv_impl(nullptr, nullptr, &p, nullptr, nullptr, nullptr, 0, nullptr, &need) != BS_OK) return 0;
+    return need;
 }

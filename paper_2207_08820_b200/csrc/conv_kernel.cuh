@@ -52,6 +52,10 @@ struct ConvArgs {
     int cs_coef[4];                          // per weight plane, used when the activations are bipolar
     int kconst;                              // + K when both operands are bipolar
     int need_rs, need_cs;
+    // split of the reduction over several CTAs of one tile (needs a zeroed workspace; left zeroed on exit)
+    int ksplit, chunks_per_split;
+    int* ws_acc;                             // [tiles][PB*FB][threads] partial accumulators
+    unsigned* ws_cnt;                        // [tiles] arrival counters
     int acc_small;                           // |acc| < 2^22 guaranteed by the shape: the exact mantissa trick applies
 };
 
@@ -229,10 +233,15 @@ __global__ void __launch_bounds__(256, (PB * FB <= 32) ? 3 : 1) bitserial_conv_k
     int* rs_s = reinterpret_cast<int*>(bars + MAX_STAGES);     // [used_pix]
     int* cs_s = rs_s + used_pix;                               // [TN]
 
-    // tile origin: filter tile fastest, then columns, rows, images
+    // reduction split fastest, then filter tile, columns, rows, images
+    const int ks = static_cast<int>(blockIdx.x % static_cast<unsigned>(g.ksplit));
+    const int tile_id = static_cast<int>(blockIdx.x / static_cast<unsigned>(g.ksplit));
+    const int c_begin = ks * g.chunks_per_split;
+    const int c_end = min(g.nchunks, c_begin + g.chunks_per_split);
+    const int my_chunks = c_end - c_begin;
     TileOrigin t;
     {
-        int b = blockIdx.x;
+        int b = tile_id;
         t.o0 = (b % g.tiles_o) * TN;       b /= g.tiles_o;
         t.q0 = (b % g.tiles_q) * TW;       b /= g.tiles_q;
         t.p0 = (b % g.tiles_p) * g.TH;     b /= g.tiles_p;
@@ -265,7 +274,7 @@ __global__ void __launch_bounds__(256, (PB * FB <= 32) ? 3 : 1) bitserial_conv_k
 
     // prologue: fill the ring (every thread commits exactly nstage groups, possibly empty)
     for (int s = 0; s < g.nstage; ++s) {
-        if (s < g.nchunks) stage_issue<A, WB>(g, s, stageA + static_cast<size_t>(s) * g.stageA_words,
+        if (s < my_chunks) stage_issue<A, WB>(g, c_begin + s, stageA + static_cast<size_t>(s) * g.stageA_words,
                                               stageW + static_cast<size_t>(s) * g.stageW_words, &bars[s], t, TN);
         else cp_async_commit();
     }
@@ -286,7 +295,7 @@ __global__ void __launch_bounds__(256, (PB * FB <= 32) ? 3 : 1) bitserial_conv_k
     int cs_acc = 0;
     bool dead = false;   // set once a bounded wait ran out; later waits are skipped so the CTA still ends
 
-    for (int c = 0; c < g.nchunks; ++c) {
+    for (int c = 0; c < my_chunks; ++c) {
         const int s = c % g.nstage;
         const uint32_t* sA = stageA + static_cast<size_t>(s) * g.stageA_words;
         const uint32_t* sW = stageW + static_cast<size_t>(s) * g.stageW_words;
@@ -352,8 +361,8 @@ __global__ void __launch_bounds__(256, (PB * FB <= 32) ? 3 : 1) bitserial_conv_k
             cs_acc += sum;
         }
         __syncthreads();   // everyone is done with stage s
-        if (c + g.nstage < g.nchunks)
-            stage_issue<A, WB>(g, c + g.nstage, stageA + static_cast<size_t>(s) * g.stageA_words,
+        if (c + g.nstage < my_chunks)
+            stage_issue<A, WB>(g, c_begin + c + g.nstage, stageA + static_cast<size_t>(s) * g.stageA_words,
                                stageW + static_cast<size_t>(s) * g.stageW_words, &bars[s], t, TN);
         else
             cp_async_commit();
@@ -375,13 +384,38 @@ __global__ void __launch_bounds__(256, (PB * FB <= 32) ? 3 : 1) bitserial_conv_k
 #pragma unroll
     for (int v = 0; v < PB; ++v) {
         const int x = tb + g.TWB * v;
-        int add = g.kconst;
+        int add = ks == 0 ? g.kconst : 0;
         if (g.need_rs) add += rs_s[(ni * g.TH + ty) * TW + x];
 #pragma unroll
         for (int u = 0; u < FB; ++u) {
             acc[v][u] += add;
             if (g.need_cs) acc[v][u] += cs_s[fg + g.NFG * u];
         }
+    }
+
+    // ---- reduction split: add partial sums into the workspace; the last CTA of the tile picks up the totals,
+    //      clears what it read (the workspace stays zero for the next launch) and runs the epilogue
+    if (g.ksplit > 1) {
+        int* ws = g.ws_acc + static_cast<size_t>(tile_id) * (PB * FB) * nthreads + tid;
+#pragma unroll
+        for (int v = 0; v < PB; ++v)
+#pragma unroll
+            for (int u = 0; u < FB; ++u) atomicAdd(ws + (v * FB + u) * nthreads, acc[v][u]);
+        __threadfence();
+        __syncthreads();
+        __shared__ unsigned s_arrival;
+        if (tid == 0) s_arrival = atomicAdd(g.ws_cnt + tile_id, 1u);
+        __syncthreads();
+        if (s_arrival != static_cast<unsigned>(g.ksplit - 1)) return;
+        __threadfence();
+#pragma unroll
+        for (int v = 0; v < PB; ++v)
+#pragma unroll
+            for (int u = 0; u < FB; ++u) {
+                acc[v][u] = __ldcg(ws + (v * FB + u) * nthreads);
+                __stcg(ws + (v * FB + u) * nthreads, 0);
+            }
+        if (tid == 0) g.ws_cnt[tile_id] = 0u;
     }
 
     // ---- raw accumulators
