@@ -169,6 +169,34 @@ int bitserial_gemm_ws(const uint32_t* a_packed, const uint32_t* w_packed, int M,
                       void* workspace, size_t workspace_bytes, void* stream);
 
 /*
+ * bitserial_gemm_noalloc -- bitserial_gemm with the reduction split, for callers that must not allocate device
+ * memory.  (The paper has no counterpart: this is a deployment convenience of this library, not part of the method.)
+ *
+ * Who needs it: host programs that hand all device memory to their own pool at start-up, inference loops that
+ * are forbidden to call cudaMalloc/cudaFree after initialisation (those calls synchronise the whole device and
+ * can fail late), and plugins that run inside another framework's stream and have no allocator of their own.
+ * Such callers cannot provide the workspace bitserial_gemm_ws asks for, so the scratch for the partial sums is a
+ * 2 MiB array built into the library image (bs_gemm_noalloc_max_scratch_bytes()); every GPU that loads the
+ * library holds those 2 MiB until the process exits.  This call never calls cudaMalloc, cudaFree or any
+ * allocating routine.
+ *
+ *   Arguments, outputs and results are exactly those of bitserial_gemm (bit-identical).
+ *   Limit: shapes whose split plan needs more than the built-in scratch (roughly M*N above 400 thousand outputs
+ *   when the planner splits) return BS_ERR_UNSUPPORTED and launch nothing; use bitserial_gemm or bitserial_gemm_ws.
+ *   Shapes the planner does not split run the ordinary kernel and touch no scratch.
+ *   First call on a device: looks up the device address of the built-in array (once per device, with that device
+ *   current).  Make that first call before starting any stream capture.
+ *   Sharing: all calls on a device use the same array, which keeps the previous call's contents; each call clears
+ *   the part it needs on `stream` before its kernel.  Two calls that overlap on the GPU (different streams without
+ *   ordering) race on the array and give wrong results; serialise them.
+ */
+size_t bs_gemm_noalloc_max_scratch_bytes(void);
+int bitserial_gemm_noalloc(const uint32_t* a_packed, const uint32_t* w_packed, int M, int N, int K, int a_bits,
+                           bs_sign_t a_sign, int w_bits, bs_sign_t w_sign, const float* scale, const float* bias,
+                           int relu, int out_bits, bs_sign_t out_sign, int32_t* out_i32, uint32_t* out_packed,
+                           void* stream);
+
+/*
  * bs_check_status -- synchronises `stream`, then reads and clears the device status word of the current
  * device.  Returns BS_ERR_TIMEOUT if any kernel since the last check gave up on a bounded wait (its
  * outputs are then undefined), BS_ERR_CUDA if the stream reports an error, else BS_OK.

@@ -71,6 +71,10 @@ def lib() -> ctypes.CDLL:
     L.bs_conv_workspace_bytes.argtypes = [ctypes.POINTER(ConvParams)]
     L.bs_gemm_workspace_bytes.restype = ctypes.c_size_t
     L.bs_gemm_workspace_bytes.argtypes = [i] * 7
+    L.bitserial_gemm_noalloc.restype = i
+    L.bitserial_gemm_noalloc.argtypes = [vp, vp, i, i, i, i, i, i, i, vp, vp, i, i, i, vp, vp, vp]
+    L.bs_gemm_noalloc_max_scratch_bytes.restype = ctypes.c_size_t
+    L.bs_gemm_noalloc_max_scratch_bytes.argtypes = []
     L.bs_check_status.restype = i
     L.bs_check_status.argtypes = [vp]
     L.bs_popc_rate.restype = i
@@ -84,4 +88,5 @@ def lib() -> ctypes.CDLL:
 EXPORTED = ("bs_packed_act_bytes", "bs_packed_wgt_bytes", "bs_packed_rows_bytes", "bitpack_activations",
             "bitunpack_activations", "pack_weights", "bs_pack_rows", "bitserial_conv2d", "bitserial_gemm",
             "bitserial_conv2d_ws", "bitserial_gemm_ws", "bs_conv_workspace_bytes", "bs_gemm_workspace_bytes",
+            "bitserial_gemm_noalloc", "bs_gemm_noalloc_max_scratch_bytes",
             "bs_check_status", "bs_popc_rate", "bs_status_string")

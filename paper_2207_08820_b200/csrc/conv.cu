@@ -416,3 +416,66 @@ extern "C" size_t bs_gemm_workspace_bytes(int M, int N, int K, int a_bits, bs_si
     if (bs::conv_impl(nullptr, nullptr, &p, nullptr, nullptr, nullptr, 0, nullptr, &need) != BS_OK) return 0;
     return need;
 }
+
+// ---------------------------------------------------------------------------------------------------------------
+// Matrix product with the reduction split for callers that cannot allocate device memory.
+//
+// The split needs a scratch area for partial sums.  Here it lives in the library image itself: a file-scope device
+// array that every GPU loading the library holds until the process exits.  In host code the array's name is only a
+// host-side stand-in for the symbol, not a device address, so the address is looked up once per device with
+// cudaGetSymbolAddress (with that device current) and that pointer is what the kernel receives.
+// ---------------------------------------------------------------------------------------------------------------
+#define BS_STATIC_SCRATCH_BYTES (2u * 1024u * 1024u)
+
+static __device__ __align__(256) unsigned char bs_static_scratch[BS_STATIC_SCRATCH_BYTES];
+
+namespace bs {
+
+constexpr int kMaxDevices = 64;
+static void* g_scratch_ptr[kMaxDevices];   // per device, filled on the first call made with that device current
+static std::mutex g_scratch_mu;
+
+// Device address of the static scratch array on the current device, or nullptr with *status set.
+static void* static_scratch_ptr(int* status)
+{
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) { *status = BS_ERR_CUDA; return nullptr; }
+    std::lock_guard<std::mutex> lock(g_scratch_mu);
+    if (!g_scratch_ptr[dev]) {
+        void* p = nullptr;
+        if (cudaGetSymbolAddress(&p, bs_static_scratch) != cudaSuccess || !p) {
+            cudaGetLastError();
+            *status = BS_ERR_CUDA;
+            return nullptr;
+        }
+        g_scratch_ptr[dev] = p;
+    }
+    return g_scratch_ptr[dev];
+}
+
+}  // namespace bs
+
+extern "C" size_t bs_gemm_noalloc_max_scratch_bytes(void) { return BS_STATIC_SCRATCH_BYTES; }
+
+extern "C" int bitserial_gemm_noalloc(const uint32_t* a_packed, const uint32_t* w_packed, int M, int N, int K, int a_bits,
+                                      bs_sign_t a_sign, int w_bits, bs_sign_t w_sign, const float* scale,
+                                      const float* bias, int relu, int out_bits, bs_sign_t out_sign, int32_t* out_i32,
+                                      uint32_t* out_packed, void* stream)
+{
+    if (M <= 0 || N <= 0 || K <= 0) return BS_ERR_INVALID_ARG;
+    const bs_conv_params p = gemm_as_conv(M, N, K, a_bits, a_sign, w_bits, w_sign, scale, bias, relu, out_bits, out_sign);
+    // how much scratch the split plan of this shape wants (host-only planning; also validates the shape)
+    size_t need = 0;
+    int st = bs::conv_impl(nullptr, nullptr, &p, nullptr, nullptr, nullptr, 0, nullptr, &need);
+    if (st != BS_OK) return st;
+    if (need > BS_STATIC_SCRATCH_BYTES) return BS_ERR_UNSUPPORTED;   // beyond the built-in scratch: use bitserial_gemm_ws
+    cudaStream_t cs = static_cast<cudaStream_t>(stream);
+    void* scratch = nullptr;
+    if (need > 0) {
+        scratch = bs::static_scratch_ptr(&st);
+        if (!scratch) return st;
+        // the array keeps whatever the previous call left; partial sums and arrival counters must start at zero
+        if (cudaMemsetAsync(scratch, 0, need, cs) != cudaSuccess) { cudaGetLastError(); return BS_ERR_CUDA; }
+    }
+    return bs::conv_impl(a_packed, w_packed, &p, out_i32, out_packed, scratch, need, cs);
+}
