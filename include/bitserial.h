@@ -197,6 +197,30 @@ int bitserial_gemm_noalloc(const uint32_t* a_packed, const uint32_t* w_packed, i
                            void* stream);
 
 /*
+ * Tensor-core formulation (exactly equivalent integer MMA).  The Section V plane-pair popcount sum is the integer
+ * dot product of the unpacked codes, so the same int32 accumulators are produced by an int8 x int8 -> int32 matrix
+ * product: activations stay bit-packed in memory and are expanded to int8 inside the kernel, filters are expanded
+ * once by bs_tc_prepare_weights.  Results (accumulators and requantised codes) are bit-identical to
+ * bitserial_conv2d / bitserial_gemm; the epilogue is the one documented at bs_conv_params.
+ *   Supported subset (bs_tc_supported returns 1): C a multiple of 32 whose packed pixel record and channel chunk are
+ *   16-byte multiples (a_bits 2: C % 64 == 0; a_bits 4: C % 32 == 0; a_bits 1 or 3: C % 128 == 0), res_c_offset a
+ *   multiple of 32; everything else as bitserial_conv2d.  Unsupported shapes return BS_ERR_UNSUPPORTED: use the
+ *   popcount entry points.
+ *   bs_tc_weights_bytes    bytes of the prepared int8 filter tensor (0 on bad input).
+ *   bs_tc_prepare_weights  packed weights [O][R][S][Cw][w_bits] -> int8 tiles [C/CK][ceil(O/128)*16][R*S][CK/16][8][16];
+ *                          the channel chunk CK depends on a_bits (the activation width the filters will meet).
+ */
+size_t bs_tc_weights_bytes(int O, int C, int R, int S);
+int bs_tc_prepare_weights(const uint32_t* wgt_packed, int O, int C, int R, int S, int w_bits, bs_sign_t w_sign,
+                          int a_bits, int8_t* wgt_tc_out, void* stream);
+int bs_tc_supported(const bs_conv_params* p);
+int bitserial_conv2d_tc(const uint32_t* act_packed, const int8_t* wgt_tc, const bs_conv_params* p, int32_t* out_i32,
+                        uint32_t* out_packed, void* stream);
+int bitserial_gemm_tc(const uint32_t* a_packed, const int8_t* w_tc, int M, int N, int K, int a_bits, bs_sign_t a_sign,
+                      int w_bits, bs_sign_t w_sign, const float* scale, const float* bias, int relu, int out_bits,
+                      bs_sign_t out_sign, int32_t* out_i32, uint32_t* out_packed, void* stream);
+
+/*
  * bs_check_status -- synchronises `stream`, then reads and clears the device status word of the current
  * device.  Returns BS_ERR_TIMEOUT if any kernel since the last check gave up on a bounded wait (its
  * outputs are then undefined), BS_ERR_CUDA if the stream reports an error, else BS_OK.

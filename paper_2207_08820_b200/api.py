@@ -113,10 +113,11 @@ def bitserial_conv2d(act_packed: torch.Tensor, wgt_packed: torch.Tensor, *, C: i
                      res_bits: int = 0, res_sign: int = UNSIGNED, res_c_offset: int = 0, res_c_total: int = 0,
                      out_i32: Optional[torch.Tensor] = None, want_i32: bool = False, i32_layout: int = NCHW,
                      out_packed: Optional[torch.Tensor] = None, out_c_offset: int = 0, out_c_total: int = 0,
-                     workspace: Optional[torch.Tensor] = None, stream=None):
+                     workspace: Optional[torch.Tensor] = None, wgt_tc: Optional[torch.Tensor] = None, stream=None):
     """act_packed [N,H,W,Cw,a_bits], wgt_packed [O,R,S,Cw,w_bits].  Returns (out_i32 or None, out_packed or None).
     A packed output is produced when ``out_bits`` > 0 (allocated here unless ``out_packed`` is given).
-    ``workspace`` (zeroed device tensor, see :func:`conv_workspace`) enables the reduction split (``bitserial_conv2d_ws``)."""
+    ``workspace`` (zeroed device tensor, see :func:`conv_workspace`) enables the reduction split (``bitserial_conv2d_ws``).
+    ``wgt_tc`` (from :func:`tc_prepare_weights`) selects the tensor-core entry point ``bitserial_conv2d_tc``."""
     N, H, W, Cw, a_bits = act_packed.shape
     O, R, S, Cw2, w_bits = wgt_packed.shape
     if Cw != Cw2 or Cw != (C + 31) // 32:
@@ -138,7 +139,10 @@ def bitserial_conv2d(act_packed: torch.Tensor, wgt_packed: torch.Tensor, *, C: i
                    res_bits=res_bits, res_sign=res_sign, res_c_offset=res_c_offset,
                    res_c_total=res_c_total if res_c_total else res_c_offset + O,
                    out_c_offset=out_c_offset, out_c_total=out_c_total, i32_layout=i32_layout)
-    if workspace is not None:
+    if wgt_tc is not None:
+        st = lib().bitserial_conv2d_tc(_ptr(act_packed), _ptr(wgt_tc), ctypes.byref(p), _ptr(out_i32),
+                                       _ptr(out_packed) if out_bits > 0 else None, _stream_ptr(stream))
+    elif workspace is not None:
         st = lib().bitserial_conv2d_ws(_ptr(act_packed), _ptr(wgt_packed), ctypes.byref(p), _ptr(out_i32),
                                        _ptr(out_packed) if out_bits > 0 else None, _ptr(workspace),
                                        workspace.numel() * workspace.element_size(), _stream_ptr(stream))
@@ -176,6 +180,38 @@ def bitserial_gemm(a_packed: torch.Tensor, w_packed: torch.Tensor, K: int, *, a_
                                   _ptr(out_packed) if out_bits > 0 else None, _stream_ptr(stream))
     _check(st, "bitserial_gemm")
     return out_i32, (out_packed if out_bits > 0 else None)
+
+
+def tc_prepare_weights(wgt_packed: torch.Tensor, C: int, w_sign: int, a_bits: int, stream=None) -> torch.Tensor:
+    """Packed weights [O,R,S,Cw,w_bits] -> int8 filter tiles for the tensor-core entry points."""
+    O, R, S, Cw, w_bits = wgt_packed.shape
+    nbytes = lib().bs_tc_weights_bytes(O, C, R, S)
+    if nbytes == 0:
+        raise BitserialError(2, "bs_tc_weights_bytes")
+    out = torch.empty(nbytes, dtype=torch.int8, device=wgt_packed.device)
+    st = lib().bs_tc_prepare_weights(_ptr(wgt_packed), O, C, R, S, w_bits, w_sign, a_bits, _ptr(out), _stream_ptr(stream))
+    _check(st, "bs_tc_prepare_weights")
+    return out
+
+
+def tc_supported(N, C, H, W, O, k, stride, pad, a_bits, a_sign, w_bits, w_sign) -> bool:
+    p = ConvParams(N=N, C=C, H=H, W=W, O=O, R=k, S=k, stride=stride, pad=pad, a_bits=a_bits, a_sign=a_sign,
+                   w_bits=w_bits, w_sign=w_sign)
+    return bool(lib().bs_tc_supported(ctypes.byref(p)))
+
+
+def bitserial_gemm_tc(a_packed: torch.Tensor, w_tc: torch.Tensor, N: int, K: int, w_bits: int, *, a_sign: int = UNSIGNED,
+                      w_sign: int = SIGNED, scale=None, bias=None, relu: bool = False, out_bits: int = 0,
+                      out_sign: int = UNSIGNED, want_i32: bool = True, stream=None):
+    """Tensor-core matrix product: a_packed [M,Kw,a_bits], w_tc from tc_prepare_weights on the [N,1,1,Kw,w_bits] rows."""
+    M, Kw, a_bits = a_packed.shape
+    dev = a_packed.device
+    out_i32 = torch.empty(M, N, dtype=torch.int32, device=dev) if want_i32 else None
+    out_packed = torch.zeros(M, (N + 31) // 32, out_bits, dtype=torch.int32, device=dev) if out_bits > 0 else None
+    st = lib().bitserial_gemm_tc(_ptr(a_packed), _ptr(w_tc), M, N, K, a_bits, a_sign, w_bits, w_sign, _ptr(scale), _ptr(bias),
+                                 int(relu), out_bits, out_sign, _ptr(out_i32), _ptr(out_packed), _stream_ptr(stream))
+    _check(st, "bitserial_gemm_tc")
+    return out_i32, out_packed
 
 
 def gemm_workspace(M: int, N: int, K: int, a_bits: int, a_sign: int, w_bits: int, w_sign: int, device="cuda"):

@@ -1,0 +1,622 @@
+// Exact integer tensor-core formulation of the bit-serial convolution (tcgen05.mma kind::i8, accumulators in TMEM).
+//
+// The Section V plane-pair popcount sum equals the integer dot product of the unpacked codes, so the same int32
+// accumulators come out of an int8 x int8 -> int32 matrix product on the 5th-generation tensor cores.  Activations
+// stay bit-packed in HBM (the library's format); a CTA
+//   - TMA-loads the packed halo of a channel chunk and a pre-expanded int8 filter slice (cp.async.bulk),
+//   - expands the bitplanes to int8 in shared memory, directly in the K-major core-matrix layout UMMA reads
+//     ([16-channel group][halo pixel][16 bytes]); a tap (r, s) of the implicit GEMM is then only a different
+//     descriptor start address, no im2col copy,
+//   - one elected thread issues tcgen05.mma (M = 128 pixels, N = filters of the tile, K = 32 channels each),
+//   - four warps read the accumulator rows back with tcgen05.ld (one pixel per thread), apply the same fused
+//     requantisation epilogue as the popcount kernel and build the output plane words thread-locally.
+// Every wait on an mbarrier is bounded; a wait that runs out sets the device status word and the CTA drains.
+#include <array>
+#include <map>
+#include <mutex>
+
+#include "conv_kernel.cuh"
+
+namespace bs {
+
+constexpr int TC_THREADS = 192;       // warps 0-3: expand + epilogue, warp 4: TMA producer, warp 5: MMA issuer
+constexpr int TC_M = 128;             // pixels per tile = 16 row groups x 8 columns (or 128 flat pixels)
+constexpr int TC_MAX_STAGES = 2;
+
+struct TcArgs {
+    CUtensorMap tmA;                  // packed activations: (Cw*A, W, H, N) words, or flat (Cw*A, N*H*W)
+    const int8_t* wgt;                // prepared int8 filters [chunk][O/8][tap][CK/16][8][16]
+    int32_t* out_i32;
+    uint32_t* out_packed;
+    const float* scale;
+    const float* bias;
+    const uint32_t* residual;
+    int* status;
+    float res_scale;
+    int N, H, W, O, R, S, stride, pad, P, Q;
+    int A;                            // activation bits
+    int relu, out_bits, out_sign, out_cw_off, out_cw_total;
+    int res_bits, res_sign, res_c_off, res_cw_total;
+    int i32_nhwc, acc_small;
+    // tiling
+    int flat;                         // 1: 128 consecutive pixels of the flattened image (1x1, stride 1)
+    int TN, CK, CWC, nchunks, nsp, nse;
+    int TNI, GI, hh, hw;              // packed box: TNI images x hh rows x hw columns; GI row groups per image
+    int HWP, HWH, HPE;                // expanded layout: row pitch, half-row offset (stride 2), pixels per 16-channel plane
+    int tiles_o, tiles_q, tiles_p, tiles_n;
+    int opad8;                        // padded filter count / 8 in the prepared weights
+    int pa_bytes, pa_tx_bytes, b_bytes, e_bytes;   // per stage (pa_tx_bytes: bytes the activation box delivers)
+    int off_e, off_sb, off_bar;       // shared-memory offsets (bytes)
+    int tmem_cols;
+    unsigned idesc;
+    unsigned mul[4];                  // byte value of plane j (2^j, or 256 - 2^(A-1) for a two's-complement top plane)
+    unsigned xormask;                 // 0xFFFFFFFF for bipolar activations
+};
+
+// ----------------------------------------------------------------------------- tcgen05 wrappers
+
+__device__ __forceinline__ void mbar_arrive(uint64_t* bar)
+{
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ void tmem_alloc(uint32_t* slot, unsigned ncols)
+{
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(slot)), "r"(ncols) : "memory");
+}
+__device__ __forceinline__ void tmem_relinquish() { asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory"); }
+__device__ __forceinline__ void tmem_dealloc(uint32_t taddr, unsigned ncols)
+{
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void umma_i8(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate)
+{
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::i8 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
+}
+__device__ __forceinline__ void umma_commit(uint64_t* bar)
+{
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&v)[32])
+{
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+        : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]),
+          "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]),
+          "=r"(v[16]), "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]),
+          "=r"(v[24]), "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
+        : "r"(taddr) : "memory");
+}
+__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+
+__device__ __forceinline__ void bulk_load(void* dst, const void* src, unsigned bytes, uint64_t* bar)
+{
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 ::"r"(smem_u32(dst)), "l"(src), "r"(bytes), "r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ void tma_load_2d(void* dst, const CUtensorMap* tm, uint64_t* bar, int c0, int c1)
+{
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cta.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+        ::"r"(smem_u32(dst)), "l"(reinterpret_cast<uint64_t>(tm)), "r"(smem_u32(bar)), "r"(c0), "r"(c1) : "memory");
+}
+
+// K-major, no-swizzle shared-memory matrix descriptor: 8-row x 16-byte core matrices of 128 contiguous bytes;
+// lbo = byte distance between the two core matrices of one K = 32 step, sbo = byte distance between 8-row groups.
+__device__ __forceinline__ uint64_t umma_desc(uint32_t smem_addr, uint32_t lbo, uint32_t sbo)
+{
+    return static_cast<uint64_t>((smem_addr >> 4) & 0x3FFFu) | (static_cast<uint64_t>((lbo >> 4) & 0x3FFFu) << 16) |
+           (static_cast<uint64_t>((sbo >> 4) & 0x3FFFu) << 32) | (1ull << 46);
+}
+
+// ----------------------------------------------------------------------------- the kernel
+
+template <int A>
+__global__ void __launch_bounds__(TC_THREADS) bitserial_conv_tc_kernel(const __grid_constant__ TcArgs g)
+{
+    extern __shared__ __align__(128) unsigned char tc_smem[];
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int RS = g.R * g.S;
+    const int stage_p_bytes = g.pa_bytes + g.b_bytes;
+    float* s_scale = reinterpret_cast<float*>(tc_smem + g.off_sb);
+    float* s_bias = s_scale + g.TN;
+    uint64_t* bars = reinterpret_cast<uint64_t*>(tc_smem + g.off_bar);
+    uint64_t* full_p = bars;                       // [TC_MAX_STAGES]
+    uint64_t* empty_p = bars + TC_MAX_STAGES;
+    uint64_t* full_e = bars + 2 * TC_MAX_STAGES;
+    uint64_t* empty_e = bars + 3 * TC_MAX_STAGES;
+    uint64_t* accum_full = bars + 4 * TC_MAX_STAGES;
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 4 * TC_MAX_STAGES + 1);
+
+    // tile origin: filter tile fastest
+    int n0, p0, q0, o0;
+    {
+        int b = blockIdx.x;
+        o0 = (b % g.tiles_o) * g.TN;   b /= g.tiles_o;
+        q0 = (b % g.tiles_q) * (g.flat ? TC_M : 8);   b /= g.tiles_q;
+        p0 = (b % g.tiles_p) * 16;     b /= g.tiles_p;
+        n0 = b * g.TNI;
+    }
+
+    if (tid == 0) {
+        for (int s = 0; s < TC_MAX_STAGES; ++s) {
+            mbar_init(&full_p[s], 1);
+            mbar_init(&empty_p[s], 1);
+            mbar_init(&full_e[s], 128);
+            mbar_init(&empty_e[s], 1);
+        }
+        mbar_init(accum_full, 1);
+        fence_barrier_init();
+        fence_proxy_async();
+    }
+    if (warp == 5) {
+        tmem_alloc(tmem_slot, static_cast<unsigned>(g.tmem_cols));
+        tmem_relinquish();
+    }
+    if (tid < g.TN) {
+        const int o = o0 + tid;
+        s_scale[tid] = (g.out_packed && o < g.O) ? g.scale[o] : 0.f;
+        s_bias[tid] = (g.out_packed && o < g.O) ? g.bias[o] : 0.f;
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+
+    if (warp == 4) {
+        // ------------------------------------------------------------------ producer
+        if (lane == 0) {
+            for (int c = 0; c < g.nchunks; ++c) {
+                const int s = c % g.nsp, k = c / g.nsp;
+                if (k >= 1 && !mbar_wait_bounded(&empty_p[s], (k - 1) & 1)) { atomicOr(g.status, STATUS_TIMEOUT); break; }
+                unsigned char* pa = tc_smem + s * stage_p_bytes;
+                unsigned char* pb = pa + g.pa_bytes;
+                mbar_expect_tx(&full_p[s], static_cast<unsigned>(g.pa_tx_bytes + g.b_bytes));
+                if (g.flat) tma_load_2d(pa, &g.tmA, &full_p[s], c * g.CWC * A, q0);
+                else tma_load_4d(pa, &g.tmA, &full_p[s], c * g.CWC * A, q0 * g.stride - g.pad, p0 * g.stride - g.pad, n0);
+                const size_t src = (static_cast<size_t>(c) * g.opad8 + (o0 >> 3)) * RS * (g.CK >> 4) * 128;
+                bulk_load(pb, g.wgt + src, static_cast<unsigned>(g.b_bytes), &full_p[s]);
+            }
+        }
+        __syncwarp();
+    } else if (warp == 5) {
+        // ------------------------------------------------------------------ MMA issuer
+        if (lane == 0) {
+            const uint32_t e_base = smem_u32(tc_smem + g.off_e);
+            const uint32_t lbo_a = static_cast<uint32_t>(g.HPE) * 16u;
+            const uint32_t sbo_a = g.flat ? 128u : static_cast<uint32_t>(g.stride * g.HWP) * 16u;
+            const uint32_t k16 = static_cast<uint32_t>(g.CK >> 4);
+            const uint32_t sbo_b = static_cast<uint32_t>(RS) * k16 * 128u;
+            bool ok = true;
+            for (int c = 0; c < g.nchunks && ok; ++c) {
+                const int s = c % g.nsp, e = c % g.nse;
+                ok = mbar_wait_bounded(&full_p[s], (c / g.nsp) & 1) && mbar_wait_bounded(&full_e[e], (c / g.nse) & 1);
+                if (!ok) { atomicOr(g.status, STATUS_TIMEOUT); break; }
+                tc_fence_after();
+                const uint32_t ea = e_base + static_cast<uint32_t>(e) * g.e_bytes;
+                const uint32_t ba = smem_u32(tc_smem + s * stage_p_bytes + g.pa_bytes);
+                for (int tap = 0; tap < RS; ++tap) {
+                    const int r = tap / g.S, sx = tap - r * g.S;
+                    const int xoff = g.stride == 2 ? (sx & 1) * g.HWH + (sx >> 1) : sx;
+                    const uint32_t a_tap = ea + static_cast<uint32_t>(r * g.HWP + xoff) * 16u;
+                    const uint32_t b_tap = ba + static_cast<uint32_t>(tap) * k16 * 128u;
+                    for (uint32_t kp = 0; kp < k16 / 2; ++kp) {
+                        const uint64_t ad = umma_desc(a_tap + 2 * kp * lbo_a, lbo_a, sbo_a);
+                        const uint64_t bd = umma_desc(b_tap + 2 * kp * 128u, 128u, sbo_b);
+                        umma_i8(tmem_base, ad, bd, g.idesc, (c | tap | static_cast<int>(kp)) != 0);
+                    }
+                }
+                umma_commit(&empty_e[e]);
+                umma_commit(&empty_p[s]);
+            }
+            umma_commit(accum_full);      // arrives when every MMA issued above has completed
+        }
+        __syncwarp();
+    } else {
+        // ------------------------------------------------------------------ expanders (warps 0-3)
+        const int items = g.flat ? TC_M * g.CWC : g.TNI * g.hh * g.hw * g.CWC;
+        bool ok = true;
+        for (int c = 0; c < g.nchunks; ++c) {
+            const int s = c % g.nsp, e = c % g.nse, k = c / g.nse;
+            if (ok) ok = mbar_wait_bounded(&full_p[s], (c / g.nsp) & 1);
+            if (ok && k >= 1) ok = mbar_wait_bounded(&empty_e[e], (k - 1) & 1);
+            if (!ok) atomicOr(g.status, STATUS_TIMEOUT);
+            const uint32_t* pa = reinterpret_cast<const uint32_t*>(tc_smem + s * stage_p_bytes);
+            unsigned char* eb = tc_smem + g.off_e + e * g.e_bytes;
+            for (int it = tid; it < items; it += 128) {
+                const int cw = it % g.CWC, hp = it / g.CWC;
+                int ep = hp;
+                if (!g.flat) {
+                    const int hy = hp / g.hw, hx = hp - hy * g.hw;
+                    ep = hy * g.HWP + (g.stride == 2 ? (hx & 1) * g.HWH + (hx >> 1) : hx);
+                }
+                uint32_t w[A];
+                load_planes<A>(pa + static_cast<size_t>(hp) * g.CWC * A + cw * A, w);
+                uint32_t out[8];
+#pragma unroll
+                for (int nb = 0; nb < 8; ++nb) {
+                    uint32_t acc = 0;
+#pragma unroll
+                    for (int j = 0; j < A; ++j) {
+                        const uint32_t sp = (((w[j] >> (4 * nb)) & 0xFu) * 0x00204081u) & 0x01010101u;
+                        acc += sp * g.mul[j];
+                    }
+                    out[nb] = acc ^ g.xormask;
+                }
+                uint4* d0 = reinterpret_cast<uint4*>(eb + static_cast<size_t>(2 * cw) * g.HPE * 16 + static_cast<size_t>(ep) * 16);
+                uint4* d1 = reinterpret_cast<uint4*>(eb + static_cast<size_t>(2 * cw + 1) * g.HPE * 16 + static_cast<size_t>(ep) * 16);
+                *d0 = make_uint4(out[0], out[1], out[2], out[3]);
+                *d1 = make_uint4(out[4], out[5], out[6], out[7]);
+            }
+            fence_proxy_async();          // make the generic-proxy writes visible to the tensor core's reads
+            mbar_arrive(&full_e[e]);
+        }
+
+        // ------------------------------------------------------------------ epilogue: one accumulator row per thread
+        if (ok) ok = mbar_wait_bounded(accum_full, 0);
+        if (!ok) atomicOr(g.status, STATUS_TIMEOUT);
+        tc_fence_after();
+        const int m = tid;                               // TMEM lane = tile pixel
+        int n, p, q;
+        bool valid;
+        if (g.flat) {
+            const long long pix = static_cast<long long>(q0) + m;
+            valid = pix < static_cast<long long>(g.N) * g.P * g.Q;
+            const int hwsz = g.P * g.Q;
+            n = static_cast<int>(pix / hwsz);
+            const int rem = static_cast<int>(pix - static_cast<long long>(n) * hwsz);
+            p = rem / g.Q; q = rem - p * g.Q;
+        } else {
+            const int grp = m >> 3, tx = m & 7;
+            const int ni = grp / g.GI, ty = grp - ni * g.GI;
+            n = n0 + ni; p = p0 + ty; q = q0 + tx;
+            valid = n < g.N && p < g.P && q < g.Q && ni < g.TNI && (g.GI == 16 || ty < g.P);
+        }
+        const size_t pix = (static_cast<size_t>(n) * g.P + p) * g.Q + q;
+        int qmin, qmax;
+        code_limits(g.out_bits > 0 ? g.out_bits : 1, g.out_sign, qmin, qmax);
+        const float fqmin = static_cast<float>(qmin), fqmax = static_cast<float>(qmax);
+        for (int cc = 0; cc < g.TN / 32; ++cc) {
+            uint32_t v[32];
+            tmem_ld32(tmem_base + (static_cast<uint32_t>(warp * 32) << 16) + static_cast<uint32_t>(cc * 32), v);
+            tmem_ld_wait();
+            const int ob = o0 + cc * 32;
+            if (valid && ob < g.O) {
+            if (g.out_i32) {
+#pragma unroll
+                for (int f = 0; f < 32; ++f) {
+                    const int o = ob + f;
+                    if (o < g.O) {
+                        const size_t idx = g.i32_nhwc ? pix * g.O + o : ((static_cast<size_t>(n) * g.O + o) * g.P + p) * g.Q + q;
+                        g.out_i32[idx] = static_cast<int>(v[f]);
+                    }
+                }
+            }
+            if (g.out_packed) {
+                uint32_t rw[4] = {0, 0, 0, 0};
+                if (g.residual) {
+                    const uint32_t* rp = g.residual + (pix * g.res_cw_total + ((g.res_c_off + ob) >> 5)) * g.res_bits;
+#pragma unroll
+                    for (int j = 0; j < 4; ++j)
+                        if (j < g.res_bits) rw[j] = rp[j];
+                }
+                uint32_t ow[4] = {0, 0, 0, 0};
+#pragma unroll
+                for (int f = 0; f < 32; ++f) {
+                    if (ob + f < g.O) {
+                        const int acc = static_cast<int>(v[f]);
+                        float val = fmaf(g.acc_small ? int_to_float_exact(acc) : static_cast<float>(acc), s_scale[cc * 32 + f], s_bias[cc * 32 + f]);
+                        if (g.residual) {
+                            unsigned rpat = 0;
+#pragma unroll
+                            for (int j = 0; j < 4; ++j)
+                                if (j < g.res_bits) rpat |= ((rw[j] >> f) & 1u) << j;
+                            val = fmaf(g.res_scale, static_cast<float>(pattern_value(rpat, g.res_bits, g.res_sign)), val);
+                        }
+                        if (g.relu) val = fmaxf(val, 0.0f);
+                        int code;
+                        if (g.out_sign == BS_BIPOLAR) code = val >= 0.0f ? 1 : -1;
+                        else code = small_float_to_int_rn(fminf(fmaxf(val, fqmin), fqmax));
+                        const unsigned pat = stored_pattern(code, g.out_bits, g.out_sign);
+#pragma unroll
+                        for (int j = 0; j < 4; ++j)
+                            if (j < g.out_bits) ow[j] |= ((pat >> j) & 1u) << f;
+                    }
+                }
+                uint32_t* dst = g.out_packed + (pix * g.out_cw_total + g.out_cw_off + (ob >> 5)) * g.out_bits;
+#pragma unroll
+                for (int j = 0; j < 4; ++j)
+                    if (j < g.out_bits) dst[j] = ow[j];
+            }
+            }
+            __syncwarp();                 // the next tcgen05.ld is warp-collective
+        }
+        tc_fence_before();
+    }
+    __syncthreads();
+    if (warp == 5) {
+        tc_fence_after();
+        tmem_dealloc(tmem_base, static_cast<unsigned>(g.tmem_cols));
+    }
+}
+
+
+// One thread per 16-byte vector of the prepared filter layout [chunk][O/8][tap][CK/16][8 filters][16 channels].
+__global__ void tc_prepare_weights_kernel(const uint32_t* __restrict__ packed, int8_t* __restrict__ out, long long nvec,
+                                          int O, int RS, int Cw, int WB, int sign, int CK, int opad8)
+{
+    const long long idx = static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x;
+    if (idx >= nvec) return;
+    const int k16n = CK >> 4;
+    long long t = idx;
+    const int row = static_cast<int>(t % 8);        t /= 8;
+    const int k16 = static_cast<int>(t % k16n);     t /= k16n;
+    const int tap = static_cast<int>(t % RS);       t /= RS;
+    const int og = static_cast<int>(t % opad8);     t /= opad8;
+    const int kc = static_cast<int>(t);
+    const int o = og * 8 + row;
+    const int c0 = kc * CK + k16 * 16;
+    uint32_t vals[4] = {0, 0, 0, 0};
+    if (o < O) {
+        const uint32_t* w = packed + ((static_cast<size_t>(o) * RS + tap) * Cw + (c0 >> 5)) * WB;
+        for (int ch = 0; ch < 16; ++ch) {
+            unsigned pat = 0;
+            for (int i = 0; i < WB; ++i) pat |= ((w[i] >> ((c0 & 31) + ch)) & 1u) << i;
+            const unsigned byte = static_cast<unsigned>(pattern_value(pat, WB, sign)) & 0xFFu;
+            vals[ch >> 2] |= byte << (8 * (ch & 3));
+        }
+    }
+    reinterpret_cast<uint4*>(out)[idx] = make_uint4(vals[0], vals[1], vals[2], vals[3]);
+}
+
+static int round_up_i(int v, int m) { return (v + m - 1) / m * m; }
+
+// Channel chunk per pipeline stage: the smallest of 32/64/128 whose packed record (CK/32 * A words) is a
+// 16-byte multiple (a TMA box requirement); 0 if C does not allow it.
+static int tc_chunk_channels(int C, int A)
+{
+    for (int ck = 32; ck <= 128; ck *= 2)
+        if (((ck / 32) * A) % 4 == 0 && C % ck == 0) return ck;
+    return 0;
+}
+
+static typename std::add_pointer<CUresult(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                                          const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                          CUtensorMapL2promotion, CUtensorMapFloatOOBfill)>::type
+tc_encode_fn()
+{
+    typedef CUresult (*Fn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                           const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                           CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+    static Fn fn = nullptr;
+    static std::once_flag once;
+    std::call_once(once, [] {
+        void* p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+            q == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<Fn>(p);
+    });
+    return fn;
+}
+
+static int tc_max_abs(int bits, int sign)
+{
+    if (sign == BS_BIPOLAR) return 1;
+    if (sign == BS_SIGNED) return 1 << (bits - 1);
+    return (1 << bits) - 1;
+}
+
+// Validation shared by the support query and the launch.  Returns BS_OK when the tensor-core path can run `p`.
+static int tc_validate(const bs_conv_params* p)
+{
+    if (!p) return BS_ERR_INVALID_ARG;
+    if (p->N <= 0 || p->C <= 0 || p->H <= 0 || p->W <= 0 || p->O <= 0 || p->R <= 0 || p->S <= 0) return BS_ERR_INVALID_ARG;
+    if (!bits_ok(p->a_bits, p->a_sign) || !bits_ok(p->w_bits, p->w_sign)) return BS_ERR_INVALID_ARG;
+    if (p->stride < 1 || p->pad < 0) return BS_ERR_INVALID_ARG;
+    if (p->i32_layout != BS_NCHW && p->i32_layout != BS_NHWC) return BS_ERR_INVALID_ARG;
+    if (p->R != p->S || (p->R != 1 && p->R != 3 && p->R != 5 && p->R != 7)) return BS_ERR_UNSUPPORTED;
+    if (p->stride > 2 || p->pad >= p->R) return BS_ERR_UNSUPPORTED;
+    if (p->a_sign == BS_BIPOLAR && p->pad != 0) return BS_ERR_UNSUPPORTED;
+    if (p->H + 2 * p->pad < p->R || p->W + 2 * p->pad < p->S) return BS_ERR_INVALID_ARG;
+    if (p->C % 32 != 0 || tc_chunk_channels(p->C, p->a_bits) == 0) return BS_ERR_UNSUPPORTED;
+    if ((ceil_div(p->C, 32) * p->a_bits) % 4 != 0) return BS_ERR_UNSUPPORTED;
+    const long long kred = static_cast<long long>(p->C) * p->R * p->S;
+    if (kred * tc_max_abs(p->a_bits, p->a_sign) * tc_max_abs(p->w_bits, p->w_sign) >= (1LL << 31)) return BS_ERR_UNSUPPORTED;
+    return BS_OK;
+}
+
+static int tc_conv_impl(const uint32_t* act, const int8_t* wgt, const bs_conv_params* p, int32_t* out_i32, uint32_t* out_packed,
+                        cudaStream_t st)
+{
+    int rc = tc_validate(p);
+    if (rc != BS_OK) return rc;
+    if (!act || !wgt || (!out_i32 && !out_packed)) return BS_ERR_INVALID_ARG;
+    if (!aligned16(act) || !aligned16(wgt) || (out_i32 && !aligned16(out_i32)) || (out_packed && !aligned16(out_packed)))
+        return BS_ERR_ALIGNMENT;
+    TcArgs g{};
+    g.P = (p->H + 2 * p->pad - p->R) / p->stride + 1;
+    g.Q = (p->W + 2 * p->pad - p->S) / p->stride + 1;
+    if (out_packed) {
+        if (!p->scale || !p->bias) return BS_ERR_INVALID_ARG;
+        if (!bits_ok(p->out_bits, p->out_sign)) return BS_ERR_INVALID_ARG;
+        if (p->out_c_offset < 0 || p->out_c_total < p->out_c_offset + p->O) return BS_ERR_INVALID_ARG;
+        if (p->out_c_offset % 32 != 0) return BS_ERR_UNSUPPORTED;
+        if (p->O % 32 != 0 && p->out_c_offset + p->O != p->out_c_total) return BS_ERR_UNSUPPORTED;
+        if (p->residual) {
+            if (!bits_ok(p->res_bits, p->res_sign)) return BS_ERR_INVALID_ARG;
+            if (p->res_c_offset < 0 || p->res_c_total < p->res_c_offset + p->O) return BS_ERR_INVALID_ARG;
+            if (p->res_c_offset % 32 != 0) return BS_ERR_UNSUPPORTED;
+            if (!aligned16(p->residual)) return BS_ERR_ALIGNMENT;
+        }
+    }
+    const int A = p->a_bits, RS = p->R * p->S, Cw = p->C / 32;
+    g.wgt = wgt; g.out_i32 = out_i32; g.out_packed = out_packed; g.scale = p->scale; g.bias = p->bias;
+    g.residual = out_packed ? p->residual : nullptr; g.res_scale = p->res_scale;
+    g.status = status_device_ptr();
+    if (!g.status) return BS_ERR_CUDA;
+    g.N = p->N; g.H = p->H; g.W = p->W; g.O = p->O; g.R = p->R; g.S = p->S; g.stride = p->stride; g.pad = p->pad; g.A = A;
+    g.relu = p->relu; g.out_bits = p->out_bits; g.out_sign = p->out_sign;
+    g.out_cw_off = p->out_c_offset / 32; g.out_cw_total = ceil_div(p->out_c_total > 0 ? p->out_c_total : 1, 32);
+    g.res_bits = p->res_bits; g.res_sign = p->res_sign; g.res_c_off = p->res_c_offset;
+    g.res_cw_total = ceil_div(p->res_c_total > 0 ? p->res_c_total : 1, 32);
+    g.i32_nhwc = p->i32_layout == BS_NHWC;
+    const long long kred = static_cast<long long>(p->C) * RS;
+    g.acc_small = kred * tc_max_abs(p->a_bits, p->a_sign) * tc_max_abs(p->w_bits, p->w_sign) < (1LL << 22);
+
+    g.CK = tc_chunk_channels(p->C, A);
+    g.CWC = g.CK / 32;
+    g.nchunks = p->C / g.CK;
+    g.nsp = g.nse = g.nchunks < TC_MAX_STAGES ? g.nchunks : TC_MAX_STAGES;
+    g.opad8 = round_up_i(p->O, 128) / 8;
+    g.flat = (p->R == 1 && p->stride == 1 && p->pad == 0);
+    long long tiles_m;
+    if (g.flat) {
+        const long long npix = static_cast<long long>(p->N) * p->H * p->W;
+        if (npix > 0x7fffffffLL) return BS_ERR_UNSUPPORTED;
+        g.tiles_q = static_cast<int>(ceil_div_ll(npix, TC_M)); g.tiles_p = 1; g.tiles_n = 1;
+        g.TNI = 1; g.GI = 16; g.hh = 1; g.hw = TC_M; g.HWP = TC_M; g.HWH = 0; g.HPE = TC_M;
+        g.pa_tx_bytes = TC_M * g.CWC * A * 4;
+        tiles_m = g.tiles_q;
+    } else {
+        g.hw = 7 * p->stride + p->S;
+        g.HWH = (g.hw + 1) / 2;
+        g.HWP = p->stride == 2 ? 2 * g.HWH : g.hw;
+        if (g.P <= 16) {        // whole image height in one tile; stack as many images as fit in the 16 row groups
+            g.hh = round_up_i((g.P - 1) * p->stride + p->R, p->stride);
+            g.GI = g.hh / p->stride;
+            g.TNI = (16 - g.P) / g.GI + 1;
+            if (g.TNI > p->N) g.TNI = p->N;
+            g.tiles_p = 1;
+        } else {
+            g.hh = round_up_i(15 * p->stride + p->R, p->stride);
+            g.GI = 16; g.TNI = 1;
+            g.tiles_p = ceil_div(g.P, 16);
+        }
+        g.tiles_q = ceil_div(g.Q, 8);
+        g.tiles_n = ceil_div(p->N, g.TNI);
+        const int rows_box = g.TNI * g.hh;
+        const int rows_read = 15 * p->stride + p->R;
+        g.HPE = (rows_box > rows_read ? rows_box : rows_read) * g.HWP;
+        g.pa_tx_bytes = g.TNI * g.hh * g.hw * g.CWC * A * 4;
+        tiles_m = static_cast<long long>(g.tiles_q) * g.tiles_p * g.tiles_n;
+    }
+    g.pa_bytes = round_up_i(g.pa_tx_bytes, 128);
+    g.e_bytes = round_up_i((g.CK / 16) * g.HPE * 16, 128);
+    // filters per tile: as many as keep the grid at two or more waves and the stages in shared memory
+    const int sms = 148;
+    int TN = 128;
+    while (TN > 32 && (TN / 2 >= round_up_i(p->O, 32) || tiles_m * ceil_div(p->O, TN) < 2LL * sms)) TN /= 2;
+    for (;; TN /= 2) {
+        g.TN = TN;
+        g.b_bytes = TN * RS * g.CK;
+        const size_t total = static_cast<size_t>(g.nsp) * (g.pa_bytes + g.b_bytes) + static_cast<size_t>(g.nse) * g.e_bytes +
+                             2 * TN * 4 + (4 * TC_MAX_STAGES + 2) * 8 + 128;
+        if (total <= 200 * 1024 || TN == 32) break;
+    }
+    g.off_e = g.nsp * (g.pa_bytes + g.b_bytes);
+    g.off_sb = g.off_e + g.nse * g.e_bytes;
+    g.off_bar = round_up_i(g.off_sb + 2 * g.TN * 4, 16);
+    const size_t smem = static_cast<size_t>(g.off_bar) + (4 * TC_MAX_STAGES + 2) * 8;
+    if (smem > 220 * 1024) return BS_ERR_UNSUPPORTED;
+    g.tiles_o = ceil_div(p->O, g.TN);
+    g.tmem_cols = g.TN < 32 ? 32 : g.TN;       // TN is 32, 64 or 128: already a power of two
+    g.idesc = (2u << 4) | (1u << 7) | (1u << 10) | (static_cast<unsigned>(g.TN >> 3) << 17) | (static_cast<unsigned>(TC_M >> 4) << 24);
+    for (int j = 0; j < 4; ++j) g.mul[j] = 1u << j;
+    g.xormask = 0;
+    if (p->a_sign == BS_SIGNED) g.mul[A - 1] = 256u - (1u << (A - 1));
+    if (p->a_sign == BS_BIPOLAR) { g.mul[0] = 0xFEu; g.xormask = 0xFFFFFFFFu; }
+
+    auto enc = tc_encode_fn();
+    if (!enc) return BS_ERR_CUDA;
+    const cuuint64_t fullA = static_cast<cuuint64_t>(Cw) * A;
+    cuuint32_t estr[4] = {1, 1, 1, 1};
+    CUresult cr;
+    if (g.flat) {
+        cuuint64_t dims[2] = {fullA, static_cast<cuuint64_t>(p->N) * p->H * p->W};
+        cuuint64_t strides[1] = {fullA * 4};
+        cuuint32_t box[2] = {static_cast<cuuint32_t>(g.CWC * A), static_cast<cuuint32_t>(TC_M)};
+        cr = enc(&g.tmA, CU_TENSOR_MAP_DATA_TYPE_UINT32, 2, const_cast<uint32_t*>(act), dims, strides, box, estr,
+                 CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                 CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    } else {
+        cuuint64_t dims[4] = {fullA, static_cast<cuuint64_t>(p->W), static_cast<cuuint64_t>(p->H), static_cast<cuuint64_t>(p->N)};
+        cuuint64_t strides[3] = {fullA * 4, fullA * 4 * p->W, fullA * 4 * p->W * p->H};
+        cuuint32_t box[4] = {static_cast<cuuint32_t>(g.CWC * A), static_cast<cuuint32_t>(g.hw), static_cast<cuuint32_t>(g.hh),
+                             static_cast<cuuint32_t>(g.TNI)};
+        cr = enc(&g.tmA, CU_TENSOR_MAP_DATA_TYPE_UINT32, 4, const_cast<uint32_t*>(act), dims, strides, box, estr,
+                 CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                 CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    }
+    if (cr != CUDA_SUCCESS) return BS_ERR_CUDA;
+
+    const long long grid = tiles_m * g.tiles_o;
+    if (grid > 0x7fffffffLL) return BS_ERR_UNSUPPORTED;
+    void (*kern)(TcArgs) = nullptr;
+    switch (A) {
+        case 1: kern = bitserial_conv_tc_kernel<1>; break;
+        case 2: kern = bitserial_conv_tc_kernel<2>; break;
+        case 3: kern = bitserial_conv_tc_kernel<3>; break;
+        default: kern = bitserial_conv_tc_kernel<4>; break;
+    }
+    if (smem > 48 * 1024 &&
+        cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)) != cudaSuccess) {
+        cudaGetLastError();
+        return BS_ERR_CUDA;
+    }
+    kern<<<static_cast<unsigned>(grid), TC_THREADS, smem, st>>>(g);
+    return cudaGetLastError() == cudaSuccess ? BS_OK : BS_ERR_CUDA;
+}
+
+}  // namespace bs
+
+extern "C" size_t bs_tc_weights_bytes(int O, int C, int R, int S)
+{
+    if (O <= 0 || C <= 0 || R <= 0 || S <= 0 || C % 32 != 0) return 0;
+    return static_cast<size_t>((O + 127) / 128 * 128) * R * S * C;
+}
+
+extern "C" int bs_tc_prepare_weights(const uint32_t* wgt_packed, int O, int C, int R, int S, int w_bits, bs_sign_t w_sign,
+                                     int a_bits, int8_t* out, void* stream)
+{
+    if (!wgt_packed || !out || O <= 0 || C <= 0 || R <= 0 || S <= 0) return BS_ERR_INVALID_ARG;
+    if (!bs::bits_ok(w_bits, w_sign) || a_bits < 1 || a_bits > 4) return BS_ERR_INVALID_ARG;
+    if (!bs::aligned16(wgt_packed) || !bs::aligned16(out)) return BS_ERR_ALIGNMENT;
+    const int CK = C % 32 == 0 ? bs::tc_chunk_channels(C, a_bits) : 0;
+    if (CK == 0) return BS_ERR_UNSUPPORTED;
+    const int opad8 = (O + 127) / 128 * 16;
+    const long long nvec = static_cast<long long>(C / CK) * opad8 * R * S * (CK / 16) * 8;
+    const long long blocks = (nvec + 255) / 256;
+    if (blocks > 0x7fffffffLL) return BS_ERR_UNSUPPORTED;
+    bs::tc_prepare_weights_kernel<<<static_cast<unsigned>(blocks), 256, 0, static_cast<cudaStream_t>(stream)>>>(
+        wgt_packed, out, nvec, O, R * S, C / 32, w_bits, w_sign, CK, opad8);
+    return cudaGetLastError() == cudaSuccess ? BS_OK : BS_ERR_CUDA;
+}
+
+extern "C" int bs_tc_supported(const bs_conv_params* p) { return bs::tc_validate(p) == BS_OK ? 1 : 0; }
+
+extern "C" int bitserial_conv2d_tc(const uint32_t* act_packed, const int8_t* wgt_tc, const bs_conv_params* p, int32_t* out_i32,
+                                   uint32_t* out_packed, void* stream)
+{
+    return bs::tc_conv_impl(act_packed, wgt_tc, p, out_i32, out_packed, static_cast<cudaStream_t>(stream));
+}
+
+extern "C" int bitserial_gemm_tc(const uint32_t* a_packed, const int8_t* w_tc, int M, int N, int K, int a_bits, bs_sign_t a_sign,
+                                 int w_bits, bs_sign_t w_sign, const float* scale, const float* bias, int relu, int out_bits,
+                                 bs_sign_t out_sign, int32_t* out_i32, uint32_t* out_packed, void* stream)
+{
+    if (M <= 0 || N <= 0 || K <= 0) return BS_ERR_INVALID_ARG;
+    bs_conv_params p{};
+    p.N = 1; p.C = K; p.H = 1; p.W = M; p.O = N; p.R = 1; p.S = 1; p.stride = 1; p.pad = 0;
+    p.a_bits = a_bits; p.a_sign = a_sign; p.w_bits = w_bits; p.w_sign = w_sign;
+    p.scale = scale; p.bias = bias; p.relu = relu; p.out_bits = out_bits; p.out_sign = out_sign;
+    p.out_c_offset = 0; p.out_c_total = N; p.i32_layout = BS_NHWC;
+    return bs::tc_conv_impl(a_packed, w_tc, &p, out_i32, out_packed, static_cast<cudaStream_t>(stream));
+}

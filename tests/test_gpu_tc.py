@@ -1,0 +1,95 @@
+"""GPU parity for the tensor-core entry points: int32 accumulators bit-exact against the oracle's direct integer
+convolution, requantised codes equal to the oracle's epilogue (tolerance: at most 1e-4 of codes off by one level;
+zero expected), and identical to the popcount entry points."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2207_08820_b200 import api, workloads as wl
+from gpu_util import dev, words
+
+pytestmark = pytest.mark.gpu
+
+
+def run_tc(c, residual=None, res_scale=0.0, want_packed=True, i32_layout=api.NCHW):
+    xa = api.bitpack_activations(dev(c["x"]), 1.0, c["a_bits"], c["a_sign"], api.NCHW)
+    wp = api.pack_weights(dev(c["w"]), c["w_bits"], c["w_sign"], api.NCHW)
+    wt = api.tc_prepare_weights(wp, c["C"], c["w_sign"], c["a_bits"])
+    res_t, res_total = None, 0
+    if residual is not None:
+        res_t = api.bitpack_activations(dev(residual), 1.0, 2, 0, api.NCHW)
+        res_total = residual.shape[1]
+    acc, packed = api.bitserial_conv2d(
+        xa, wp, C=c["C"], stride=c["stride"], pad=c["pad"], a_sign=c["a_sign"], w_sign=c["w_sign"],
+        scale=dev(c["scale"]) if want_packed else None, bias=dev(c["bias"]) if want_packed else None, relu=c["relu"],
+        out_bits=c["out_bits"] if want_packed else 0, out_sign=0, residual=res_t, res_scale=res_scale,
+        res_bits=2 if residual is not None else 0, res_c_total=res_total, want_i32=True, i32_layout=i32_layout, wgt_tc=wt)
+    api.bs_check_status()
+    return acc.cpu().numpy(), (words(packed) if packed is not None else None)
+
+
+@pytest.mark.parametrize("k,stride,pad", [(1, 1, 0), (1, 2, 0), (3, 1, 1), (3, 2, 1), (3, 1, 0), (3, 2, 0), (5, 1, 2), (7, 2, 3)])
+@pytest.mark.parametrize("hw", [(7, 7), (14, 14), (9, 20), (23, 11), (56, 56)])
+def test_tc_conv_geometry(k, stride, pad, hw):
+    H, W = hw
+    if H + 2 * pad < k or W + 2 * pad < k:
+        pytest.skip("kernel larger than padded image")
+    c = wl.single_conv_case(seed=k * 100 + stride * 10 + pad + H, N=3, C=64, H=H, W=W, O=40, k=k, stride=stride, pad=pad,
+                            calibrated=True)
+    acc, packed = run_tc(c)
+    want = oracle.conv2d_i32(c["x"], c["w"], stride, pad)
+    assert np.array_equal(acc, want)
+    codes = oracle.requantize(want, c["scale"], c["bias"], True, 2, 0)
+    assert np.array_equal(packed, oracle.pack_activations(codes, 2, 0))
+
+
+@pytest.mark.parametrize("ab,asg,C", [(2, 0, 64), (2, 1, 128), (4, 0, 32), (4, 1, 96), (1, 0, 128), (3, 0, 128), (1, 2, 128)])
+@pytest.mark.parametrize("wb,wsg", [(1, 2), (2, 1), (3, 1), (4, 1), (2, 0)])
+def test_tc_bitwidths_and_signs(ab, asg, C, wb, wsg):
+    pad = 0 if asg == 2 else 1
+    c = wl.single_conv_case(seed=ab * 10 + wb, N=2, C=C, H=12, W=10, O=72, pad=pad, a_bits=ab, a_sign=asg, w_bits=wb, w_sign=wsg,
+                            out_bits=2, calibrated=True)
+    acc, packed = run_tc(c, i32_layout=api.NHWC)
+    want = oracle.conv2d_i32(c["x"], c["w"], 1, pad)
+    assert np.array_equal(acc, want.transpose(0, 2, 3, 1))
+    codes = oracle.requantize(want, c["scale"], c["bias"], True, 2, 0)
+    assert np.array_equal(packed, oracle.pack_activations(codes, 2, 0))
+
+
+@pytest.mark.parametrize("C,O", [(64, 32), (64, 128), (128, 64), (256, 96), (512, 64), (192, 200)])
+def test_tc_channel_counts_multi_chunk(C, O):
+    c = wl.single_conv_case(seed=C + O, N=2, C=C, H=14, W=14, O=O, calibrated=True)
+    acc, packed = run_tc(c)
+    want = oracle.conv2d_i32(c["x"], c["w"], 1, 1)
+    assert np.array_equal(acc, want)
+    codes = oracle.requantize(want, c["scale"], c["bias"], True, 2, 0)
+    assert np.array_equal(packed, oracle.pack_activations(codes, 2, 0))
+
+
+def test_tc_residual_matches_oracle_and_popcount_path():
+    c = wl.single_conv_case(seed=9, N=2, C=64, H=12, W=12, O=64, calibrated=True)
+    rng = np.random.default_rng(4)
+    res = wl.rand_codes(rng, (2, 64, 12, 12), 2, 0)
+    acc, packed = run_tc(c, residual=res, res_scale=0.5)
+    want = oracle.conv2d_i32(c["x"], c["w"], 1, 1)
+    assert np.array_equal(acc, want)
+    codes = oracle.requantize(want, c["scale"], c["bias"], True, 2, 0, res=res, res_scale=0.5)
+    assert np.array_equal(packed, oracle.pack_activations(codes, 2, 0))
+
+
+@pytest.mark.parametrize("M,N,K", [(1, 8, 64), (130, 40, 128), (300, 72, 1024), (1031, 96, 64), (256, 256, 576), (1024, 1024, 2304)])
+def test_tc_gemm(M, N, K):
+    c = wl.gemm_case(M, N, K, seed=M + N + K)
+    ap = api.bs_pack_rows(dev(c["a"]), 2, 0)
+    wp = api.bs_pack_rows(dev(c["w"]), 1, 2)
+    wt = api.tc_prepare_weights(wp.view(N, 1, 1, -1, 1), K, 2, 2)
+    out, _ = api.bitserial_gemm_tc(ap, wt, N, K, 1, a_sign=0, w_sign=2)
+    api.bs_check_status()
+    assert np.array_equal(out.cpu().numpy(), oracle.gemm_i32(c["a"], c["w"]))
+
+
+def test_tc_unsupported_shape_is_refused():
+    assert not api.tc_supported(1, 32, 8, 8, 32, 3, 1, 1, 2, 0, 2, 1)       # 8-byte pixel records cannot be a TMA box
+    assert not api.tc_supported(1, 40, 8, 8, 32, 3, 1, 1, 4, 0, 2, 1)       # C not a multiple of 32
+    assert api.tc_supported(1, 64, 8, 8, 32, 3, 1, 1, 2, 0, 2, 1)
