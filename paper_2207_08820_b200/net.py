@@ -15,8 +15,12 @@ from .workloads import NetSpec
 
 
 class BitserialNet:
-    def __init__(self, net: NetSpec, params: Dict[str, Dict], act_scale: float, device="cuda", batch: Optional[int] = None):
+    def __init__(self, net: NetSpec, params: Dict[str, Dict], act_scale: float, device="cuda", batch: Optional[int] = None,
+                 engine: str = "popc"):
+        """engine: "popc" = popcount kernels on the integer pipes; "tc" = tensor-core entry point for every layer it
+        supports (others fall back to the popcount kernel)."""
         self.net = net
+        self.engine = engine
         self.act_scale = float(act_scale)
         self.device = torch.device(device)
         self.batch = batch or net.batch
@@ -25,9 +29,14 @@ class BitserialNet:
         for L in net.layers:
             p = params[L.name]
             w = torch.from_numpy(np.ascontiguousarray(p["w"])).to(self.device)
+            wp = api.pack_weights(w, net.w_bits, p["w_sign"])
+            _, H, W = self.shapes[L.src]
+            use_tc = engine == "tc" and api.tc_supported(self.batch, L.C, H, W, L.O, L.k, L.stride, L.pad, net.a_bits,
+                                                         api.UNSIGNED, net.w_bits, p["w_sign"])
             self.layers.append(dict(
                 spec=L,
-                w=api.pack_weights(w, net.w_bits, p["w_sign"]),
+                w=wp,
+                w_tc=api.tc_prepare_weights(wp, L.C, p["w_sign"], net.a_bits) if use_tc else None,
                 w_sign=p["w_sign"],
                 scale=torch.from_numpy(p["scale"]).to(self.device),
                 bias=torch.from_numpy(p["bias"]).to(self.device)))
@@ -49,7 +58,8 @@ class BitserialNet:
                 w_sign=item["w_sign"], scale=item["scale"], bias=item["bias"], relu=L.relu, out_bits=net.a_bits,
                 out_sign=api.UNSIGNED, residual=res, res_scale=L.res_scale, res_bits=net.a_bits if L.res else 0,
                 res_sign=api.UNSIGNED, res_c_offset=0, res_c_total=self.shapes[L.res][0] if L.res else 0,
-                out_packed=self.bufs[L.dst], out_c_offset=L.dst_c_offset, out_c_total=self.shapes[L.dst][0])
+                out_packed=self.bufs[L.dst], out_c_offset=L.dst_c_offset, out_c_total=self.shapes[L.dst][0],
+                wgt_tc=item["w_tc"])
         return self.bufs[net.out_name]
 
     def forward(self, x: torch.Tensor) -> torch.Tensor:

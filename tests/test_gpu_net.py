@@ -16,10 +16,10 @@ pytestmark = pytest.mark.gpu
 ACT_SCALE = 0.25
 
 
-def compare_stack(net, batch, seed, sample=None, graph=False):
+def compare_stack(net, batch, seed, sample=None, graph=False, engine="popc"):
     params = wl.network_params(net, seed)
     x = wl.network_input(net, seed, ACT_SCALE, batch=batch)
-    runner = BitserialNet(net, params, ACT_SCALE, batch=batch)
+    runner = BitserialNet(net, params, ACT_SCALE, batch=batch, engine=engine)
     xd = dev(x)
     if graph:
         runner.capture(xd)
@@ -56,3 +56,19 @@ def test_resnet18_body_full_batch_graph_sampled():
 
 def test_detection_backbone_full_size_sampled():
     compare_stack(wl.detection_backbone(16), 16, seed=4000, sample=[0, 15], graph=True)
+
+
+def test_resnet18_body_tensor_core_small_batch():
+    compare_stack(wl.resnet18_body(2), 2, seed=3000, engine="tc")
+
+
+def test_detection_backbone_tensor_core_small():
+    compare_stack(wl.detection_backbone(1, hw=64), 1, seed=4000, engine="tc")
+
+
+def test_resnet18_body_tensor_core_full_batch_graph_sampled():
+    compare_stack(wl.resnet18_body(64), 64, seed=3000, sample=[0, 31, 63], graph=True, engine="tc")
+
+
+def test_detection_backbone_tensor_core_full_size_sampled():
+    compare_stack(wl.detection_backbone(16), 16, seed=4000, sample=[0, 15], graph=True, engine="tc")
