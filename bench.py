@@ -158,7 +158,7 @@ def run_ours(args):
     params = wl.network_params(net, seed)
     x_host = torch.from_numpy(wl.network_input(net, replicas.rank_seed(seed, rank), ACT_SCALE)).pin_memory()
     x_dev = x_host.cuda()
-    runner = BitserialNet(net, params, ACT_SCALE, batch=net.batch)
+    runner = BitserialNet(net, params, ACT_SCALE, batch=net.batch, engine=args.engine)
 
     stream = torch.cuda.Stream()
     with torch.cuda.stream(stream):
@@ -287,7 +287,7 @@ def runner_conv(runner, item):
         scale=item["scale"], bias=item["bias"], relu=L.relu, out_bits=net.a_bits, out_sign=api.UNSIGNED, residual=res,
         res_scale=L.res_scale, res_bits=net.a_bits if L.res else 0, res_sign=api.UNSIGNED, res_c_offset=0,
         res_c_total=runner.shapes[L.res][0] if L.res else 0, out_packed=runner.bufs[L.dst],
-        out_c_offset=L.dst_c_offset, out_c_total=runner.shapes[L.dst][0])
+        out_c_offset=L.dst_c_offset, out_c_total=runner.shapes[L.dst][0], wgt_tc=item["w_tc"])
 
 
 def cpu_baseline(net, params, seed, sample):
@@ -314,6 +314,8 @@ def main():
     ap.add_argument("--ref-images", type=int, default=2, help="images per step of the reference arm (bounded CPU sample)")
     ap.add_argument("--cpu-baseline-images", type=int, default=64, help="images of the one oracle pass timed beside the GPU run")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--engine", default="popc", choices=["popc", "tc"],
+                    help="popc: popcount kernels on the integer pipes; tc: exact int8 tensor-core formulation")
     ap.add_argument("--eager", action="store_true", help="plain stream launches instead of CUDA graphs (for per-launch profiling)")
     args = ap.parse_args()
     if args.batch == 0:

@@ -16,6 +16,7 @@
 #include <mutex>
 
 #include "conv_kernel.cuh"
+#include "requant_bounds.h"
 
 namespace bs {
 
@@ -51,6 +52,7 @@ struct TcArgs {
     unsigned idesc;
     unsigned mul[4];                  // byte value of plane j (2^j, or 256 - 2^(A-1) for a two's-complement top plane)
     unsigned xormask;                 // 0xFFFFFFFF for bipolar activations
+    RequantBounds rb;                 // comparison form of the epilogue (1- and 2-bit outputs)
 };
 
 // ----------------------------------------------------------------------------- tcgen05 wrappers
@@ -125,8 +127,8 @@ __global__ void __launch_bounds__(TC_THREADS) bitserial_conv_tc_kernel(const __g
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int RS = g.R * g.S;
     const int stage_p_bytes = g.pa_bytes + g.b_bytes;
-    float* s_scale = reinterpret_cast<float*>(tc_smem + g.off_sb);
-    float* s_bias = s_scale + g.TN;
+    float2* s_sb = reinterpret_cast<float2*>(tc_smem + g.off_sb);           // (scale, bias) per filter of the tile
+    float4* s_bounds = reinterpret_cast<float4*>(tc_smem + g.off_sb + g.TN * 8);   // comparison bounds per residual pattern
     uint64_t* bars = reinterpret_cast<uint64_t*>(tc_smem + g.off_bar);
     uint64_t* full_p = bars;                       // [TC_MAX_STAGES]
     uint64_t* empty_p = bars + TC_MAX_STAGES;
@@ -162,9 +164,9 @@ __global__ void __launch_bounds__(TC_THREADS) bitserial_conv_tc_kernel(const __g
     }
     if (tid < g.TN) {
         const int o = o0 + tid;
-        s_scale[tid] = (g.out_packed && o < g.O) ? g.scale[o] : 0.f;
-        s_bias[tid] = (g.out_packed && o < g.O) ? g.bias[o] : 0.f;
+        s_sb[tid] = (g.out_packed && o < g.O) ? make_float2(g.scale[o], g.bias[o]) : make_float2(0.f, 0.f);
     }
+    if (tid < 16) s_bounds[tid] = make_float4(g.rb.bound[tid][0], g.rb.bound[tid][1], g.rb.bound[tid][2], 0.f);
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
@@ -283,6 +285,7 @@ __global__ void __launch_bounds__(TC_THREADS) bitserial_conv_tc_kernel(const __g
         int qmin, qmax;
         code_limits(g.out_bits > 0 ? g.out_bits : 1, g.out_sign, qmin, qmax);
         const float fqmin = static_cast<float>(qmin), fqmax = static_cast<float>(qmax);
+        const float4 bnd0 = s_bounds[0];
         for (int cc = 0; cc < g.TN / 32; ++cc) {
             uint32_t v[32];
             tmem_ld32(tmem_base + (static_cast<uint32_t>(warp * 32) << 16) + static_cast<uint32_t>(cc * 32), v);
@@ -308,11 +311,38 @@ __global__ void __launch_bounds__(TC_THREADS) bitserial_conv_tc_kernel(const __g
                         if (j < g.res_bits) rw[j] = rp[j];
                 }
                 uint32_t ow[4] = {0, 0, 0, 0};
+                if (g.rb.enabled) {
+                    // comparison form: t = fmaf(acc, scale, bias) against the bounds of the residual pattern
+                    const unsigned valid_mask = (g.O - ob >= 32) ? 0xffffffffu : ((1u << (g.O - ob)) - 1u);
+#pragma unroll
+                    for (int f = 0; f < 32; ++f) {
+                        const int acc = static_cast<int>(v[f]);
+                        const float2 sb = s_sb[cc * 32 + f];
+                        const float t = fmaf(g.acc_small ? int_to_float_exact(acc) : static_cast<float>(acc), sb.x, sb.y);
+                        float b0, b1, b2;
+                        if (g.residual) {
+                            unsigned rpat = 0;
+#pragma unroll
+                            for (int j = 0; j < 4; ++j)
+                                if (j < g.res_bits) rpat |= ((rw[j] >> f) & 1u) << j;
+                            const float4 bb = s_bounds[rpat];
+                            b0 = bb.x; b1 = bb.y; b2 = bb.z;
+                        } else {
+                            b0 = bnd0.x; b1 = bnd0.y; b2 = bnd0.z;
+                        }
+                        const bool c1 = t >= b0, c2 = t >= b1, c3 = t >= b2;
+                        if ((c1 != c2) != c3) ow[0] |= 1u << f;
+                        if (c2) ow[1] |= 1u << f;
+                    }
+                    ow[0] = (ow[0] ^ ((g.rb.flip & 1u) ? 0xffffffffu : 0u)) & valid_mask;
+                    ow[1] = (ow[1] ^ ((g.rb.flip & 2u) ? 0xffffffffu : 0u)) & valid_mask;
+                } else {
 #pragma unroll
                 for (int f = 0; f < 32; ++f) {
                     if (ob + f < g.O) {
                         const int acc = static_cast<int>(v[f]);
-                        float val = fmaf(g.acc_small ? int_to_float_exact(acc) : static_cast<float>(acc), s_scale[cc * 32 + f], s_bias[cc * 32 + f]);
+                        const float2 sb = s_sb[cc * 32 + f];
+                        float val = fmaf(g.acc_small ? int_to_float_exact(acc) : static_cast<float>(acc), sb.x, sb.y);
                         if (g.residual) {
                             unsigned rpat = 0;
 #pragma unroll
@@ -329,6 +359,7 @@ __global__ void __launch_bounds__(TC_THREADS) bitserial_conv_tc_kernel(const __g
                         for (int j = 0; j < 4; ++j)
                             if (j < g.out_bits) ow[j] |= ((pat >> j) & 1u) << f;
                     }
+                }
                 }
                 uint32_t* dst = g.out_packed + (pix * g.out_cw_total + g.out_cw_off + (ob >> 5)) * g.out_bits;
 #pragma unroll
@@ -518,12 +549,12 @@ static int tc_conv_impl(const uint32_t* act, const int8_t* wgt, const bs_conv_pa
         g.TN = TN;
         g.b_bytes = TN * RS * g.CK;
         const size_t total = static_cast<size_t>(g.nsp) * (g.pa_bytes + g.b_bytes) + static_cast<size_t>(g.nse) * g.e_bytes +
-                             2 * TN * 4 + (4 * TC_MAX_STAGES + 2) * 8 + 128;
+                             2 * TN * 4 + 256 + (4 * TC_MAX_STAGES + 2) * 8 + 128;
         if (total <= 200 * 1024 || TN == 32) break;
     }
     g.off_e = g.nsp * (g.pa_bytes + g.b_bytes);
     g.off_sb = g.off_e + g.nse * g.e_bytes;
-    g.off_bar = round_up_i(g.off_sb + 2 * g.TN * 4, 16);
+    g.off_bar = round_up_i(g.off_sb + 2 * g.TN * 4 + 256, 16);
     const size_t smem = static_cast<size_t>(g.off_bar) + (4 * TC_MAX_STAGES + 2) * 8;
     if (smem > 220 * 1024) return BS_ERR_UNSUPPORTED;
     g.tiles_o = ceil_div(p->O, g.TN);
@@ -533,6 +564,10 @@ static int tc_conv_impl(const uint32_t* act, const int8_t* wgt, const bs_conv_pa
     g.xormask = 0;
     if (p->a_sign == BS_SIGNED) g.mul[A - 1] = 256u - (1u << (A - 1));
     if (p->a_sign == BS_BIPOLAR) { g.mul[0] = 0xFEu; g.xormask = 0xFFFFFFFFu; }
+
+    g.rb = cached_requant_bounds(g.residual != nullptr, p->res_scale, p->res_bits, p->res_sign, p->relu,
+                               out_packed ? p->out_bits : 0, p->out_sign);
+    if (!out_packed) g.rb.enabled = 0;
 
     auto enc = tc_encode_fn();
     if (!enc) return BS_ERR_CUDA;
