@@ -47,7 +47,8 @@ struct TcArgs {
     int tiles_o, tiles_q, tiles_p, tiles_n;
     int opad8;                        // padded filter count / 8 in the prepared weights
     int pa_bytes, pa_tx_bytes, b_bytes, e_bytes;   // per stage (pa_tx_bytes: bytes the activation box delivers)
-    int off_e, off_sb, off_bar;       // shared-memory offsets (bytes)
+    int off_p, off_e, off_sb, off_bar;   // shared-memory offsets (bytes)
+    int persistent;
     int tmem_cols;
     unsigned idesc;
     unsigned mul[4];                  // byte value of plane j (2^j, or 256 - 2^(A-1) for a two's-complement top plane)
@@ -118,7 +119,185 @@ __device__ __forceinline__ uint64_t umma_desc(uint32_t smem_addr, uint32_t lbo, 
            (static_cast<uint64_t>((sbo >> 4) & 0x3FFFu) << 32) | (1ull << 46);
 }
 
-// ----------------------------------------------------------------------------- the kernel
+// ----------------------------------------------------------------------------- building blocks
+
+struct TcTile { int n0, p0, q0; };
+
+__device__ __forceinline__ TcTile tc_decode_tile(const TcArgs& g, int mt)
+{
+    TcTile t;
+    t.q0 = (mt % g.tiles_q) * (g.flat ? TC_M : 8);   mt /= g.tiles_q;
+    t.p0 = (mt % g.tiles_p) * 16;                    mt /= g.tiles_p;
+    t.n0 = mt * g.TNI;
+    return t;
+}
+
+// Expansion of one staged chunk: bitplanes of (pixel, 32-channel word) -> 32 int8 values, written as two 16-byte rows
+// of the K-major core-matrix layout [16-channel group][halo pixel][16 bytes].  `et` = 0..127 within the expander group.
+template <int A>
+__device__ __forceinline__ void tc_expand_chunk(const TcArgs& g, const uint32_t* pa, unsigned char* eb, int et)
+{
+    const int items = g.flat ? TC_M * g.CWC : g.TNI * g.hh * g.hw * g.CWC;
+    for (int it = et; it < items; it += 128) {
+        const int cw = it % g.CWC, hp = it / g.CWC;
+        int ep = hp;
+        if (!g.flat) {
+            const int hy = hp / g.hw, hx = hp - hy * g.hw;
+            ep = hy * g.HWP + (g.stride == 2 ? (hx & 1) * g.HWH + (hx >> 1) : hx);
+        }
+        uint32_t w[A];
+        load_planes<A>(pa + static_cast<size_t>(hp) * g.CWC * A + cw * A, w);
+        uint32_t out[8];
+#pragma unroll
+        for (int nb = 0; nb < 8; ++nb) {
+            uint32_t acc = 0;
+#pragma unroll
+            for (int j = 0; j < A; ++j) {
+                const uint32_t sp = (((w[j] >> (4 * nb)) & 0xFu) * 0x00204081u) & 0x01010101u;
+                acc += sp * g.mul[j];
+            }
+            out[nb] = acc ^ g.xormask;
+        }
+        uint4* d0 = reinterpret_cast<uint4*>(eb + static_cast<size_t>(2 * cw) * g.HPE * 16 + static_cast<size_t>(ep) * 16);
+        uint4* d1 = reinterpret_cast<uint4*>(eb + static_cast<size_t>(2 * cw + 1) * g.HPE * 16 + static_cast<size_t>(ep) * 16);
+        *d0 = make_uint4(out[0], out[1], out[2], out[3]);
+        *d1 = make_uint4(out[4], out[5], out[6], out[7]);
+    }
+}
+
+// All MMAs of one chunk: R*S taps x CK/32 steps of K = 32; a tap only moves the descriptor start address.
+__device__ __forceinline__ void tc_issue_chunk(const TcArgs& g, uint32_t ea, uint32_t ba, uint32_t tmem_acc, bool first_chunk)
+{
+    const int RS = g.R * g.S;
+    const uint32_t lbo_a = static_cast<uint32_t>(g.HPE) * 16u;
+    const uint32_t sbo_a = g.flat ? 128u : static_cast<uint32_t>(g.stride * g.HWP) * 16u;
+    const uint32_t k16 = static_cast<uint32_t>(g.CK >> 4);
+    const uint32_t sbo_b = static_cast<uint32_t>(RS) * k16 * 128u;
+    for (int tap = 0; tap < RS; ++tap) {
+        const int r = tap / g.S, sx = tap - r * g.S;
+        const int xoff = g.stride == 2 ? (sx & 1) * g.HWH + (sx >> 1) : sx;
+        const uint32_t a_tap = ea + static_cast<uint32_t>(r * g.HWP + xoff) * 16u;
+        const uint32_t b_tap = ba + static_cast<uint32_t>(tap) * k16 * 128u;
+        for (uint32_t kp = 0; kp < k16 / 2; ++kp) {
+            const uint64_t ad = umma_desc(a_tap + 2 * kp * lbo_a, lbo_a, sbo_a);
+            const uint64_t bd = umma_desc(b_tap + 2 * kp * 128u, 128u, sbo_b);
+            umma_i8(tmem_acc, ad, bd, g.idesc, (first_chunk ? (tap | static_cast<int>(kp)) : 1) != 0);
+        }
+    }
+}
+
+// Epilogue of one tile: thread `tid` (0..127, warp = TMEM lane quadrant) owns accumulator row tid = one output pixel.
+__device__ __forceinline__ void tc_epilogue_tile(const TcArgs& g, uint32_t tmem_acc, int tid, int warp, const TcTile& tile, int o0,
+                                                 const float2* s_sb, const float4* s_bounds)
+{
+    const int n0 = tile.n0, p0 = tile.p0, q0 = tile.q0;
+    const int m = tid;                               // TMEM lane = tile pixel
+    int n, p, q;
+    bool valid;
+    if (g.flat) {
+        const long long pix = static_cast<long long>(q0) + m;
+        valid = pix < static_cast<long long>(g.N) * g.P * g.Q;
+        const int hwsz = g.P * g.Q;
+        n = static_cast<int>(pix / hwsz);
+        const int rem = static_cast<int>(pix - static_cast<long long>(n) * hwsz);
+        p = rem / g.Q; q = rem - p * g.Q;
+    } else {
+        const int grp = m >> 3, tx = m & 7;
+        const int ni = grp / g.GI, ty = grp - ni * g.GI;
+        n = n0 + ni; p = p0 + ty; q = q0 + tx;
+        valid = n < g.N && p < g.P && q < g.Q && ni < g.TNI && (g.GI == 16 || ty < g.P);
+    }
+    const size_t pix = (static_cast<size_t>(n) * g.P + p) * g.Q + q;
+    int qmin, qmax;
+    code_limits(g.out_bits > 0 ? g.out_bits : 1, g.out_sign, qmin, qmax);
+    const float fqmin = static_cast<float>(qmin), fqmax = static_cast<float>(qmax);
+    const float4 bnd0 = s_bounds[0];
+    for (int cc = 0; cc < g.TN / 32; ++cc) {
+        uint32_t v[32];
+        tmem_ld32(tmem_acc + (static_cast<uint32_t>(warp * 32) << 16) + static_cast<uint32_t>(cc * 32), v);
+        tmem_ld_wait();
+        const int ob = o0 + cc * 32;
+        if (valid && ob < g.O) {
+        if (g.out_i32) {
+#pragma unroll
+            for (int f = 0; f < 32; ++f) {
+                const int o = ob + f;
+                if (o < g.O) {
+                    const size_t idx = g.i32_nhwc ? pix * g.O + o : ((static_cast<size_t>(n) * g.O + o) * g.P + p) * g.Q + q;
+                    g.out_i32[idx] = static_cast<int>(v[f]);
+                }
+            }
+        }
+        if (g.out_packed) {
+            uint32_t rw[4] = {0, 0, 0, 0};
+            if (g.residual) {
+                const uint32_t* rp = g.residual + (pix * g.res_cw_total + ((g.res_c_off + ob) >> 5)) * g.res_bits;
+#pragma unroll
+                for (int j = 0; j < 4; ++j)
+                    if (j < g.res_bits) rw[j] = rp[j];
+            }
+            uint32_t ow[4] = {0, 0, 0, 0};
+            if (g.rb.enabled) {
+                // comparison form: t = fmaf(acc, scale, bias) against the bounds of the residual pattern
+                const unsigned valid_mask = (g.O - ob >= 32) ? 0xffffffffu : ((1u << (g.O - ob)) - 1u);
+#pragma unroll
+                for (int f = 0; f < 32; ++f) {
+                    const int acc = static_cast<int>(v[f]);
+                    const float2 sb = s_sb[cc * 32 + f];
+                    const float t = fmaf(g.acc_small ? int_to_float_exact(acc) : static_cast<float>(acc), sb.x, sb.y);
+                    float b0, b1, b2;
+                    if (g.residual) {
+                        unsigned rpat = 0;
+#pragma unroll
+                        for (int j = 0; j < 4; ++j)
+                            if (j < g.res_bits) rpat |= ((rw[j] >> f) & 1u) << j;
+                        const float4 bb = s_bounds[rpat];
+                        b0 = bb.x; b1 = bb.y; b2 = bb.z;
+                    } else {
+                        b0 = bnd0.x; b1 = bnd0.y; b2 = bnd0.z;
+                    }
+                    const bool c1 = t >= b0, c2 = t >= b1, c3 = t >= b2;
+                    if ((c1 != c2) != c3) ow[0] |= 1u << f;
+                    if (c2) ow[1] |= 1u << f;
+                }
+                ow[0] = (ow[0] ^ ((g.rb.flip & 1u) ? 0xffffffffu : 0u)) & valid_mask;
+                ow[1] = (ow[1] ^ ((g.rb.flip & 2u) ? 0xffffffffu : 0u)) & valid_mask;
+            } else {
+#pragma unroll
+            for (int f = 0; f < 32; ++f) {
+                if (ob + f < g.O) {
+                    const int acc = static_cast<int>(v[f]);
+                    const float2 sb = s_sb[cc * 32 + f];
+                    float val = fmaf(g.acc_small ? int_to_float_exact(acc) : static_cast<float>(acc), sb.x, sb.y);
+                    if (g.residual) {
+                        unsigned rpat = 0;
+#pragma unroll
+                        for (int j = 0; j < 4; ++j)
+                            if (j < g.res_bits) rpat |= ((rw[j] >> f) & 1u) << j;
+                        val = fmaf(g.res_scale, static_cast<float>(pattern_value(rpat, g.res_bits, g.res_sign)), val);
+                    }
+                    if (g.relu) val = fmaxf(val, 0.0f);
+                    int code;
+                    if (g.out_sign == BS_BIPOLAR) code = val >= 0.0f ? 1 : -1;
+                    else code = small_float_to_int_rn(fminf(fmaxf(val, fqmin), fqmax));
+                    const unsigned pat = stored_pattern(code, g.out_bits, g.out_sign);
+#pragma unroll
+                    for (int j = 0; j < 4; ++j)
+                        if (j < g.out_bits) ow[j] |= ((pat >> j) & 1u) << f;
+                }
+            }
+            }
+            uint32_t* dst = g.out_packed + (pix * g.out_cw_total + g.out_cw_off + (ob >> 5)) * g.out_bits;
+#pragma unroll
+            for (int j = 0; j < 4; ++j)
+                if (j < g.out_bits) dst[j] = ow[j];
+        }
+        }
+        __syncwarp();                 // the next tcgen05.ld is warp-collective
+    }
+}
+
+// ----------------------------------------------------------------------------- one tile per CTA (filters streamed per chunk)
 
 template <int A>
 __global__ void __launch_bounds__(TC_THREADS) bitserial_conv_tc_kernel(const __grid_constant__ TcArgs g)
@@ -137,15 +316,8 @@ __global__ void __launch_bounds__(TC_THREADS) bitserial_conv_tc_kernel(const __g
     uint64_t* accum_full = bars + 4 * TC_MAX_STAGES;
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 4 * TC_MAX_STAGES + 1);
 
-    // tile origin: filter tile fastest
-    int n0, p0, q0, o0;
-    {
-        int b = blockIdx.x;
-        o0 = (b % g.tiles_o) * g.TN;   b /= g.tiles_o;
-        q0 = (b % g.tiles_q) * (g.flat ? TC_M : 8);   b /= g.tiles_q;
-        p0 = (b % g.tiles_p) * 16;     b /= g.tiles_p;
-        n0 = b * g.TNI;
-    }
+    const int o0 = static_cast<int>(blockIdx.x % static_cast<unsigned>(g.tiles_o)) * g.TN;   // filter tile fastest
+    const TcTile tile = tc_decode_tile(g, static_cast<int>(blockIdx.x / static_cast<unsigned>(g.tiles_o)));
 
     if (tid == 0) {
         for (int s = 0; s < TC_MAX_STAGES; ++s) {
@@ -181,8 +353,8 @@ __global__ void __launch_bounds__(TC_THREADS) bitserial_conv_tc_kernel(const __g
                 unsigned char* pa = tc_smem + s * stage_p_bytes;
                 unsigned char* pb = pa + g.pa_bytes;
                 mbar_expect_tx(&full_p[s], static_cast<unsigned>(g.pa_tx_bytes + g.b_bytes));
-                if (g.flat) tma_load_2d(pa, &g.tmA, &full_p[s], c * g.CWC * A, q0);
-                else tma_load_4d(pa, &g.tmA, &full_p[s], c * g.CWC * A, q0 * g.stride - g.pad, p0 * g.stride - g.pad, n0);
+                if (g.flat) tma_load_2d(pa, &g.tmA, &full_p[s], c * g.CWC * A, tile.q0);
+                else tma_load_4d(pa, &g.tmA, &full_p[s], c * g.CWC * A, tile.q0 * g.stride - g.pad, tile.p0 * g.stride - g.pad, tile.n0);
                 const size_t src = (static_cast<size_t>(c) * g.opad8 + (o0 >> 3)) * RS * (g.CK >> 4) * 128;
                 bulk_load(pb, g.wgt + src, static_cast<unsigned>(g.b_bytes), &full_p[s]);
             }
@@ -192,29 +364,15 @@ __global__ void __launch_bounds__(TC_THREADS) bitserial_conv_tc_kernel(const __g
         // ------------------------------------------------------------------ MMA issuer
         if (lane == 0) {
             const uint32_t e_base = smem_u32(tc_smem + g.off_e);
-            const uint32_t lbo_a = static_cast<uint32_t>(g.HPE) * 16u;
-            const uint32_t sbo_a = g.flat ? 128u : static_cast<uint32_t>(g.stride * g.HWP) * 16u;
-            const uint32_t k16 = static_cast<uint32_t>(g.CK >> 4);
-            const uint32_t sbo_b = static_cast<uint32_t>(RS) * k16 * 128u;
-            bool ok = true;
-            for (int c = 0; c < g.nchunks && ok; ++c) {
+            for (int c = 0; c < g.nchunks; ++c) {
                 const int s = c % g.nsp, e = c % g.nse;
-                ok = mbar_wait_bounded(&full_p[s], (c / g.nsp) & 1) && mbar_wait_bounded(&full_e[e], (c / g.nse) & 1);
-                if (!ok) { atomicOr(g.status, STATUS_TIMEOUT); break; }
-                tc_fence_after();
-                const uint32_t ea = e_base + static_cast<uint32_t>(e) * g.e_bytes;
-                const uint32_t ba = smem_u32(tc_smem + s * stage_p_bytes + g.pa_bytes);
-                for (int tap = 0; tap < RS; ++tap) {
-                    const int r = tap / g.S, sx = tap - r * g.S;
-                    const int xoff = g.stride == 2 ? (sx & 1) * g.HWH + (sx >> 1) : sx;
-                    const uint32_t a_tap = ea + static_cast<uint32_t>(r * g.HWP + xoff) * 16u;
-                    const uint32_t b_tap = ba + static_cast<uint32_t>(tap) * k16 * 128u;
-                    for (uint32_t kp = 0; kp < k16 / 2; ++kp) {
-                        const uint64_t ad = umma_desc(a_tap + 2 * kp * lbo_a, lbo_a, sbo_a);
-                        const uint64_t bd = umma_desc(b_tap + 2 * kp * 128u, 128u, sbo_b);
-                        umma_i8(tmem_base, ad, bd, g.idesc, (c | tap | static_cast<int>(kp)) != 0);
-                    }
+                if (!(mbar_wait_bounded(&full_p[s], (c / g.nsp) & 1) && mbar_wait_bounded(&full_e[e], (c / g.nse) & 1))) {
+                    atomicOr(g.status, STATUS_TIMEOUT);
+                    break;
                 }
+                tc_fence_after();
+                tc_issue_chunk(g, e_base + static_cast<uint32_t>(e) * g.e_bytes, smem_u32(tc_smem + s * stage_p_bytes + g.pa_bytes),
+                               tmem_base, c == 0);
                 umma_commit(&empty_e[e]);
                 umma_commit(&empty_p[s]);
             }
@@ -222,157 +380,173 @@ __global__ void __launch_bounds__(TC_THREADS) bitserial_conv_tc_kernel(const __g
         }
         __syncwarp();
     } else {
-        // ------------------------------------------------------------------ expanders (warps 0-3)
-        const int items = g.flat ? TC_M * g.CWC : g.TNI * g.hh * g.hw * g.CWC;
+        // ------------------------------------------------------------------ expanders (warps 0-3), then epilogue
         bool ok = true;
         for (int c = 0; c < g.nchunks; ++c) {
             const int s = c % g.nsp, e = c % g.nse, k = c / g.nse;
             if (ok) ok = mbar_wait_bounded(&full_p[s], (c / g.nsp) & 1);
             if (ok && k >= 1) ok = mbar_wait_bounded(&empty_e[e], (k - 1) & 1);
             if (!ok) atomicOr(g.status, STATUS_TIMEOUT);
-            const uint32_t* pa = reinterpret_cast<const uint32_t*>(tc_smem + s * stage_p_bytes);
-            unsigned char* eb = tc_smem + g.off_e + e * g.e_bytes;
-            for (int it = tid; it < items; it += 128) {
-                const int cw = it % g.CWC, hp = it / g.CWC;
-                int ep = hp;
-                if (!g.flat) {
-                    const int hy = hp / g.hw, hx = hp - hy * g.hw;
-                    ep = hy * g.HWP + (g.stride == 2 ? (hx & 1) * g.HWH + (hx >> 1) : hx);
-                }
-                uint32_t w[A];
-                load_planes<A>(pa + static_cast<size_t>(hp) * g.CWC * A + cw * A, w);
-                uint32_t out[8];
-#pragma unroll
-                for (int nb = 0; nb < 8; ++nb) {
-                    uint32_t acc = 0;
-#pragma unroll
-                    for (int j = 0; j < A; ++j) {
-                        const uint32_t sp = (((w[j] >> (4 * nb)) & 0xFu) * 0x00204081u) & 0x01010101u;
-                        acc += sp * g.mul[j];
-                    }
-                    out[nb] = acc ^ g.xormask;
-                }
-                uint4* d0 = reinterpret_cast<uint4*>(eb + static_cast<size_t>(2 * cw) * g.HPE * 16 + static_cast<size_t>(ep) * 16);
-                uint4* d1 = reinterpret_cast<uint4*>(eb + static_cast<size_t>(2 * cw + 1) * g.HPE * 16 + static_cast<size_t>(ep) * 16);
-                *d0 = make_uint4(out[0], out[1], out[2], out[3]);
-                *d1 = make_uint4(out[4], out[5], out[6], out[7]);
-            }
+            tc_expand_chunk<A>(g, reinterpret_cast<const uint32_t*>(tc_smem + s * stage_p_bytes), tc_smem + g.off_e + e * g.e_bytes, tid);
             fence_proxy_async();          // make the generic-proxy writes visible to the tensor core's reads
             mbar_arrive(&full_e[e]);
         }
-
-        // ------------------------------------------------------------------ epilogue: one accumulator row per thread
         if (ok) ok = mbar_wait_bounded(accum_full, 0);
         if (!ok) atomicOr(g.status, STATUS_TIMEOUT);
         tc_fence_after();
-        const int m = tid;                               // TMEM lane = tile pixel
-        int n, p, q;
-        bool valid;
-        if (g.flat) {
-            const long long pix = static_cast<long long>(q0) + m;
-            valid = pix < static_cast<long long>(g.N) * g.P * g.Q;
-            const int hwsz = g.P * g.Q;
-            n = static_cast<int>(pix / hwsz);
-            const int rem = static_cast<int>(pix - static_cast<long long>(n) * hwsz);
-            p = rem / g.Q; q = rem - p * g.Q;
-        } else {
-            const int grp = m >> 3, tx = m & 7;
-            const int ni = grp / g.GI, ty = grp - ni * g.GI;
-            n = n0 + ni; p = p0 + ty; q = q0 + tx;
-            valid = n < g.N && p < g.P && q < g.Q && ni < g.TNI && (g.GI == 16 || ty < g.P);
-        }
-        const size_t pix = (static_cast<size_t>(n) * g.P + p) * g.Q + q;
-        int qmin, qmax;
-        code_limits(g.out_bits > 0 ? g.out_bits : 1, g.out_sign, qmin, qmax);
-        const float fqmin = static_cast<float>(qmin), fqmax = static_cast<float>(qmax);
-        const float4 bnd0 = s_bounds[0];
-        for (int cc = 0; cc < g.TN / 32; ++cc) {
-            uint32_t v[32];
-            tmem_ld32(tmem_base + (static_cast<uint32_t>(warp * 32) << 16) + static_cast<uint32_t>(cc * 32), v);
-            tmem_ld_wait();
-            const int ob = o0 + cc * 32;
-            if (valid && ob < g.O) {
-            if (g.out_i32) {
-#pragma unroll
-                for (int f = 0; f < 32; ++f) {
-                    const int o = ob + f;
-                    if (o < g.O) {
-                        const size_t idx = g.i32_nhwc ? pix * g.O + o : ((static_cast<size_t>(n) * g.O + o) * g.P + p) * g.Q + q;
-                        g.out_i32[idx] = static_cast<int>(v[f]);
-                    }
-                }
-            }
-            if (g.out_packed) {
-                uint32_t rw[4] = {0, 0, 0, 0};
-                if (g.residual) {
-                    const uint32_t* rp = g.residual + (pix * g.res_cw_total + ((g.res_c_off + ob) >> 5)) * g.res_bits;
-#pragma unroll
-                    for (int j = 0; j < 4; ++j)
-                        if (j < g.res_bits) rw[j] = rp[j];
-                }
-                uint32_t ow[4] = {0, 0, 0, 0};
-                if (g.rb.enabled) {
-                    // comparison form: t = fmaf(acc, scale, bias) against the bounds of the residual pattern
-                    const unsigned valid_mask = (g.O - ob >= 32) ? 0xffffffffu : ((1u << (g.O - ob)) - 1u);
-#pragma unroll
-                    for (int f = 0; f < 32; ++f) {
-                        const int acc = static_cast<int>(v[f]);
-                        const float2 sb = s_sb[cc * 32 + f];
-                        const float t = fmaf(g.acc_small ? int_to_float_exact(acc) : static_cast<float>(acc), sb.x, sb.y);
-                        float b0, b1, b2;
-                        if (g.residual) {
-                            unsigned rpat = 0;
-#pragma unroll
-                            for (int j = 0; j < 4; ++j)
-                                if (j < g.res_bits) rpat |= ((rw[j] >> f) & 1u) << j;
-                            const float4 bb = s_bounds[rpat];
-                            b0 = bb.x; b1 = bb.y; b2 = bb.z;
-                        } else {
-                            b0 = bnd0.x; b1 = bnd0.y; b2 = bnd0.z;
-                        }
-                        const bool c1 = t >= b0, c2 = t >= b1, c3 = t >= b2;
-                        if ((c1 != c2) != c3) ow[0] |= 1u << f;
-                        if (c2) ow[1] |= 1u << f;
-                    }
-                    ow[0] = (ow[0] ^ ((g.rb.flip & 1u) ? 0xffffffffu : 0u)) & valid_mask;
-                    ow[1] = (ow[1] ^ ((g.rb.flip & 2u) ? 0xffffffffu : 0u)) & valid_mask;
-                } else {
-#pragma unroll
-                for (int f = 0; f < 32; ++f) {
-                    if (ob + f < g.O) {
-                        const int acc = static_cast<int>(v[f]);
-                        const float2 sb = s_sb[cc * 32 + f];
-                        float val = fmaf(g.acc_small ? int_to_float_exact(acc) : static_cast<float>(acc), sb.x, sb.y);
-                        if (g.residual) {
-                            unsigned rpat = 0;
-#pragma unroll
-                            for (int j = 0; j < 4; ++j)
-                                if (j < g.res_bits) rpat |= ((rw[j] >> f) & 1u) << j;
-                            val = fmaf(g.res_scale, static_cast<float>(pattern_value(rpat, g.res_bits, g.res_sign)), val);
-                        }
-                        if (g.relu) val = fmaxf(val, 0.0f);
-                        int code;
-                        if (g.out_sign == BS_BIPOLAR) code = val >= 0.0f ? 1 : -1;
-                        else code = small_float_to_int_rn(fminf(fmaxf(val, fqmin), fqmax));
-                        const unsigned pat = stored_pattern(code, g.out_bits, g.out_sign);
-#pragma unroll
-                        for (int j = 0; j < 4; ++j)
-                            if (j < g.out_bits) ow[j] |= ((pat >> j) & 1u) << f;
-                    }
-                }
-                }
-                uint32_t* dst = g.out_packed + (pix * g.out_cw_total + g.out_cw_off + (ob >> 5)) * g.out_bits;
-#pragma unroll
-                for (int j = 0; j < 4; ++j)
-                    if (j < g.out_bits) dst[j] = ow[j];
-            }
-            }
-            __syncwarp();                 // the next tcgen05.ld is warp-collective
-        }
+        tc_epilogue_tile(g, tmem_base, tid, warp, tile, o0, s_sb, s_bounds);
         tc_fence_before();
     }
     __syncthreads();
     if (warp == 5) {
+        tc_fence_after();
+        tmem_dealloc(tmem_base, static_cast<unsigned>(g.tmem_cols));
+    }
+}
+
+// ----------------------------------------------------------------------------- persistent CTAs, filters resident
+//
+// A CTA keeps the int8 filters of its filter tile (all channel chunks) in shared memory and walks over pixel tiles.
+// Warps 0-3: epilogue (TMEM lane quadrants), warps 4-7: bitplane expansion, warp 8: TMA producer, warp 9: MMA issuer.
+// Packed and expanded activation chunks travel through two mbarrier rings; two TMEM accumulator buffers let the
+// epilogue of tile i overlap the MMAs of tile i + 1.
+
+constexpr int TCP_THREADS = 320;
+constexpr int TCP_NSP = 4;            // packed-chunk ring
+constexpr int TCP_NSE = 3;            // expanded-chunk ring (at most)
+
+template <int A>
+__global__ void __launch_bounds__(TCP_THREADS) bitserial_conv_tc_persistent_kernel(const __grid_constant__ TcArgs g)
+{
+    extern __shared__ __align__(128) unsigned char tc_smem[];
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int RS = g.R * g.S;
+    unsigned char* s_w = tc_smem;                                              // [nchunks][b_bytes]
+    unsigned char* s_p = tc_smem + g.off_p;                                    // [TCP_NSP][pa_bytes]
+    unsigned char* s_e = tc_smem + g.off_e;                                    // [nse][e_bytes]
+    float2* s_sb = reinterpret_cast<float2*>(tc_smem + g.off_sb);
+    float4* s_bounds = reinterpret_cast<float4*>(tc_smem + g.off_sb + g.TN * 8);
+    uint64_t* bars = reinterpret_cast<uint64_t*>(tc_smem + g.off_bar);
+    uint64_t* full_p = bars;                        // [TCP_NSP]
+    uint64_t* empty_p = bars + TCP_NSP;             // [TCP_NSP]
+    uint64_t* full_e = bars + 2 * TCP_NSP;          // [TCP_NSE]
+    uint64_t* empty_e = full_e + TCP_NSE;           // [TCP_NSE]
+    uint64_t* full_acc = empty_e + TCP_NSE;         // [2]
+    uint64_t* empty_acc = full_acc + 2;             // [2]
+    uint64_t* wgt_full = empty_acc + 2;             // [1]
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(wgt_full + 1);
+
+    const int o0 = static_cast<int>(blockIdx.x % static_cast<unsigned>(g.tiles_o)) * g.TN;
+    const int first_tile = static_cast<int>(blockIdx.x / static_cast<unsigned>(g.tiles_o));
+    const int tile_step = static_cast<int>(gridDim.x / static_cast<unsigned>(g.tiles_o));
+    const int tiles_m = g.tiles_q * g.tiles_p * g.tiles_n;
+
+    if (tid == 0) {
+        for (int s = 0; s < TCP_NSP; ++s) { mbar_init(&full_p[s], 1); mbar_init(&empty_p[s], 128); }
+        for (int s = 0; s < TCP_NSE; ++s) { mbar_init(&full_e[s], 128); mbar_init(&empty_e[s], 1); }
+        for (int s = 0; s < 2; ++s) { mbar_init(&full_acc[s], 1); mbar_init(&empty_acc[s], 128); }
+        mbar_init(wgt_full, 1);
+        fence_barrier_init();
+        fence_proxy_async();
+    }
+    if (warp == 9) {
+        tmem_alloc(tmem_slot, static_cast<unsigned>(g.tmem_cols));
+        tmem_relinquish();
+    }
+    if (tid < g.TN) {
+        const int o = o0 + tid;
+        s_sb[tid] = (g.out_packed && o < g.O) ? make_float2(g.scale[o], g.bias[o]) : make_float2(0.f, 0.f);
+    }
+    if (tid < 16) s_bounds[tid] = make_float4(g.rb.bound[tid][0], g.rb.bound[tid][1], g.rb.bound[tid][2], 0.f);
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+
+    if (warp == 8) {
+        // ------------------------------------------------------------------ producer: filters once, then packed chunks
+        if (lane == 0) {
+            mbar_expect_tx(wgt_full, static_cast<unsigned>(g.nchunks * g.b_bytes));
+            for (int c = 0; c < g.nchunks; ++c) {
+                const size_t src = (static_cast<size_t>(c) * g.opad8 + (o0 >> 3)) * RS * (g.CK >> 4) * 128;
+                bulk_load(s_w + static_cast<size_t>(c) * g.b_bytes, g.wgt + src, static_cast<unsigned>(g.b_bytes), wgt_full);
+            }
+            int it = 0;
+            bool ok = true;
+            for (int mt = first_tile; mt < tiles_m && ok; mt += tile_step) {
+                const TcTile tile = tc_decode_tile(g, mt);
+                for (int c = 0; c < g.nchunks; ++c, ++it) {
+                    const int s = it % TCP_NSP, k = it / TCP_NSP;
+                    if (k >= 1 && !mbar_wait_bounded(&empty_p[s], (k - 1) & 1)) { ok = false; break; }
+                    unsigned char* pa = s_p + s * g.pa_bytes;
+                    mbar_expect_tx(&full_p[s], static_cast<unsigned>(g.pa_tx_bytes));
+                    if (g.flat) tma_load_2d(pa, &g.tmA, &full_p[s], c * g.CWC * A, tile.q0);
+                    else tma_load_4d(pa, &g.tmA, &full_p[s], c * g.CWC * A, tile.q0 * g.stride - g.pad, tile.p0 * g.stride - g.pad, tile.n0);
+                }
+            }
+            if (!ok) atomicOr(g.status, STATUS_TIMEOUT);
+        }
+        __syncwarp();
+    } else if (warp == 9) {
+        // ------------------------------------------------------------------ MMA issuer
+        if (lane == 0) {
+            bool ok = mbar_wait_bounded(wgt_full, 0);       // also keeps the CTA alive until the filter copy has landed
+            int it = 0, i = 0;
+            for (int mt = first_tile; mt < tiles_m && ok; mt += tile_step, ++i) {
+                const int buf = i & 1, use = i >> 1;
+                if (use >= 1) ok = mbar_wait_bounded(&empty_acc[buf], (use - 1) & 1);
+                if (!ok) break;
+                tc_fence_after();
+                const uint32_t tmem_acc = tmem_base + static_cast<uint32_t>(buf * g.TN);
+                for (int c = 0; c < g.nchunks; ++c, ++it) {
+                    const int e = it % g.nse;
+                    if (!mbar_wait_bounded(&full_e[e], (it / g.nse) & 1)) { ok = false; break; }
+                    tc_fence_after();
+                    tc_issue_chunk(g, smem_u32(s_e + e * g.e_bytes), smem_u32(s_w + static_cast<size_t>(c) * g.b_bytes), tmem_acc, c == 0);
+                    umma_commit(&empty_e[e]);
+                }
+                if (ok) umma_commit(&full_acc[buf]);
+            }
+            if (!ok) atomicOr(g.status, STATUS_TIMEOUT);
+        }
+        __syncwarp();
+    } else if (warp >= 4) {
+        // ------------------------------------------------------------------ expanders (warps 4-7)
+        const int et = tid - 128;
+        int it = 0;
+        bool ok = true;
+        for (int mt = first_tile; mt < tiles_m && ok; mt += tile_step) {
+            for (int c = 0; c < g.nchunks; ++c, ++it) {
+                const int s = it % TCP_NSP, e = it % g.nse, k = it / g.nse;
+                ok = mbar_wait_bounded(&full_p[s], (it / TCP_NSP) & 1);
+                if (ok && k >= 1) ok = mbar_wait_bounded(&empty_e[e], (k - 1) & 1);
+                if (!ok) break;
+                tc_expand_chunk<A>(g, reinterpret_cast<const uint32_t*>(s_p + s * g.pa_bytes), s_e + e * g.e_bytes, et);
+                fence_proxy_async();
+                mbar_arrive(&full_e[e]);
+                mbar_arrive(&empty_p[s]);
+            }
+        }
+        if (!ok) atomicOr(g.status, STATUS_TIMEOUT);
+    } else {
+        // ------------------------------------------------------------------ epilogue (warps 0-3)
+        int i = 0;
+        bool ok = true;
+        for (int mt = first_tile; mt < tiles_m && ok; mt += tile_step, ++i) {
+            const int buf = i & 1, use = i >> 1;
+            ok = mbar_wait_bounded(&full_acc[buf], use & 1);
+            if (!ok) break;
+            tc_fence_after();
+            const TcTile tile = tc_decode_tile(g, mt);
+            tc_epilogue_tile(g, tmem_base + static_cast<uint32_t>(buf * g.TN), tid, warp, tile, o0, s_sb, s_bounds);
+            tc_fence_before();
+            mbar_arrive(&empty_acc[buf]);
+        }
+        if (!ok) atomicOr(g.status, STATUS_TIMEOUT);
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 9) {
         tc_fence_after();
         tmem_dealloc(tmem_base, static_cast<unsigned>(g.tmem_cols));
     }
@@ -541,24 +715,51 @@ static int tc_conv_impl(const uint32_t* act, const int8_t* wgt, const bs_conv_pa
     }
     g.pa_bytes = round_up_i(g.pa_tx_bytes, 128);
     g.e_bytes = round_up_i((g.CK / 16) * g.HPE * 16, 128);
-    // filters per tile: as many as keep the grid at two or more waves and the stages in shared memory
     const int sms = 148;
-    int TN = 128;
-    while (TN > 32 && (TN / 2 >= round_up_i(p->O, 32) || tiles_m * ceil_div(p->O, TN) < 2LL * sms)) TN /= 2;
-    for (;; TN /= 2) {
-        g.TN = TN;
-        g.b_bytes = TN * RS * g.CK;
-        const size_t total = static_cast<size_t>(g.nsp) * (g.pa_bytes + g.b_bytes) + static_cast<size_t>(g.nse) * g.e_bytes +
-                             2 * TN * 4 + 256 + (4 * TC_MAX_STAGES + 2) * 8 + 128;
-        if (total <= 200 * 1024 || TN == 32) break;
+    // Persistent plan: the filters of a tile (all channel chunks) stay resident in shared memory.  Largest filter tile
+    // that fits and still leaves one (pixel tile, filter tile) pair per SM.
+    size_t smem = 0;
+    g.persistent = 0;
+    const int bar_bytes = (2 * TCP_NSP + 2 * TCP_NSE + 5) * 8 + 16;
+    for (int TN = 128; TN >= 32; TN /= 2) {
+        if (TN / 2 >= round_up_i(p->O, 32)) continue;                      // tile twice as wide as the filter bank
+        const long long pairs = tiles_m * ceil_div(p->O, TN);
+        if (TN > 32 && pairs < sms) continue;
+        const size_t wbytes = static_cast<size_t>(g.nchunks) * TN * RS * g.CK;
+        for (int nse = TCP_NSE; nse >= 2; --nse) {
+            const size_t total = wbytes + static_cast<size_t>(TCP_NSP) * g.pa_bytes + static_cast<size_t>(nse) * g.e_bytes +
+                                 static_cast<size_t>(TN) * 8 + 256 + bar_bytes + 128;
+            if (total <= 220 * 1024) {
+                g.persistent = 1; g.TN = TN; g.b_bytes = TN * RS * g.CK; g.nse = nse; g.nsp = TCP_NSP;
+                g.off_p = static_cast<int>(wbytes);
+                g.off_e = g.off_p + TCP_NSP * g.pa_bytes;
+                g.off_sb = g.off_e + nse * g.e_bytes;
+                g.off_bar = round_up_i(g.off_sb + TN * 8 + 256, 16);
+                smem = static_cast<size_t>(g.off_bar) + bar_bytes;
+                break;
+            }
+        }
+        if (g.persistent) break;
     }
-    g.off_e = g.nsp * (g.pa_bytes + g.b_bytes);
-    g.off_sb = g.off_e + g.nse * g.e_bytes;
-    g.off_bar = round_up_i(g.off_sb + 2 * g.TN * 4 + 256, 16);
-    const size_t smem = static_cast<size_t>(g.off_bar) + (4 * TC_MAX_STAGES + 2) * 8;
-    if (smem > 220 * 1024) return BS_ERR_UNSUPPORTED;
+    if (!g.persistent) {
+        // one tile per CTA, filters streamed with every chunk: as many filters as keep the grid at two or more waves
+        int TN = 128;
+        while (TN > 32 && (TN / 2 >= round_up_i(p->O, 32) || tiles_m * ceil_div(p->O, TN) < 2LL * sms)) TN /= 2;
+        for (;; TN /= 2) {
+            g.TN = TN;
+            g.b_bytes = TN * RS * g.CK;
+            const size_t total = static_cast<size_t>(g.nsp) * (g.pa_bytes + g.b_bytes) + static_cast<size_t>(g.nse) * g.e_bytes +
+                                 2 * TN * 4 + 256 + (4 * TC_MAX_STAGES + 2) * 8 + 128;
+            if (total <= 200 * 1024 || TN == 32) break;
+        }
+        g.off_e = g.nsp * (g.pa_bytes + g.b_bytes);
+        g.off_sb = g.off_e + g.nse * g.e_bytes;
+        g.off_bar = round_up_i(g.off_sb + 2 * g.TN * 4 + 256, 16);
+        smem = static_cast<size_t>(g.off_bar) + (4 * TC_MAX_STAGES + 2) * 8;
+        if (smem > 220 * 1024) return BS_ERR_UNSUPPORTED;
+    }
     g.tiles_o = ceil_div(p->O, g.TN);
-    g.tmem_cols = g.TN < 32 ? 32 : g.TN;       // TN is 32, 64 or 128: already a power of two
+    g.tmem_cols = g.persistent ? 2 * g.TN : g.TN;      // TN is 32, 64 or 128: powers of two, at least 32 columns
     g.idesc = (2u << 4) | (1u << 7) | (1u << 10) | (static_cast<unsigned>(g.TN >> 3) << 17) | (static_cast<unsigned>(TC_M >> 4) << 24);
     for (int j = 0; j < 4; ++j) g.mul[j] = 1u << j;
     g.xormask = 0;
@@ -592,6 +793,27 @@ static int tc_conv_impl(const uint32_t* act, const int8_t* wgt, const bs_conv_pa
     }
     if (cr != CUDA_SUCCESS) return BS_ERR_CUDA;
 
+    if (g.persistent) {
+        const int cps = smem <= 110 * 1024 ? 2 : 1;                        // CTAs that fit on one SM
+        long long per_o = (static_cast<long long>(sms) * cps) / g.tiles_o;
+        if (per_o < 1) per_o = 1;
+        if (per_o > tiles_m) per_o = tiles_m;
+        const long long grid = per_o * g.tiles_o;
+        void (*kern)(TcArgs) = nullptr;
+        switch (A) {
+            case 1: kern = bitserial_conv_tc_persistent_kernel<1>; break;
+            case 2: kern = bitserial_conv_tc_persistent_kernel<2>; break;
+            case 3: kern = bitserial_conv_tc_persistent_kernel<3>; break;
+            default: kern = bitserial_conv_tc_persistent_kernel<4>; break;
+        }
+        if (smem > 48 * 1024 &&
+            cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)) != cudaSuccess) {
+            cudaGetLastError();
+            return BS_ERR_CUDA;
+        }
+        kern<<<static_cast<unsigned>(grid), TCP_THREADS, smem, st>>>(g);
+        return cudaGetLastError() == cudaSuccess ? BS_OK : BS_ERR_CUDA;
+    }
     const long long grid = tiles_m * g.tiles_o;
     if (grid > 0x7fffffffLL) return BS_ERR_UNSUPPORTED;
     void (*kern)(TcArgs) = nullptr;
