@@ -25,7 +25,8 @@ constexpr int TC_M = 128;             // pixels per tile = 16 row groups x 8 col
 constexpr int TC_MAX_STAGES = 2;
 
 struct TcArgs {
-    CUtensorMap tmA;                  // packed activations: (Cw*A, W, H, N) words, or flat (Cw*A, N*H*W)
+    CUtensorMap tmA;                  // packed activations: (W*Cw*A, H, N) words when a halo row fits one box row, else (Cw*A, W, H, N)
+    const uint32_t* act;              // packed activations (flat mode copies whole pixel records with cp.async.bulk)
     const int8_t* wgt;                // prepared int8 filters [chunk][O/8][tap][CK/16][8][16]
     int32_t* out_i32;
     uint32_t* out_packed;
@@ -42,6 +43,8 @@ struct TcArgs {
     // tiling
     int flat;                         // 1: 128 consecutive pixels of the flattened image (1x1, stride 1)
     int TN, CK, CWC, nchunks, nsp, nse;
+    int fullA;                        // words of one packed pixel record (Cw * A)
+    int pmode;                        // how a tile's packed halo is fetched: 0 flat bulk copy, 1 rows merged with W, 2 4-D box
     int TNI, GI, hh, hw;              // packed box: TNI images x hh rows x hw columns; GI row groups per image
     int HWP, HWH, HPE;                // expanded layout: row pitch, half-row offset (stride 2), pixels per 16-channel plane
     int tiles_o, tiles_q, tiles_p, tiles_n;
@@ -132,10 +135,30 @@ __device__ __forceinline__ TcTile tc_decode_tile(const TcArgs& g, int mt)
     return t;
 }
 
-// Expansion of one staged chunk: bitplanes of (pixel, 32-channel word) -> 32 int8 values, written as two 16-byte rows
+// Fetch the packed halo of one tile (whole pixel records, all channel chunks) and arm `bar` with its byte count.
+// Rows of a TMA box cost a fixed overhead each, so the copy is shaped to have few, long rows: a flat tile is one
+// contiguous cp.async.bulk; otherwise a halo row (hw pixels x record) is one box row whenever it fits 256 elements.
+__device__ __forceinline__ void tc_load_tile(const TcArgs& g, void* dst, uint64_t* bar, const TcTile& tile)
+{
+    if (g.pmode == 0) {
+        const long long npix = static_cast<long long>(g.N) * g.P * g.Q;
+        long long rows = npix - tile.q0;
+        if (rows > TC_M) rows = TC_M;
+        const unsigned bytes = static_cast<unsigned>(rows) * static_cast<unsigned>(g.fullA) * 4u;
+        mbar_expect_tx(bar, bytes);
+        bulk_load(dst, g.act + static_cast<size_t>(tile.q0) * g.fullA, bytes, bar);
+    } else {
+        mbar_expect_tx(bar, static_cast<unsigned>(g.pa_tx_bytes));
+        const int x0 = tile.q0 * g.stride - g.pad, y0 = tile.p0 * g.stride - g.pad;
+        if (g.pmode == 1) tma_load_3d(dst, &g.tmA, bar, x0 * g.fullA, y0, tile.n0);
+        else tma_load_4d(dst, &g.tmA, bar, 0, x0, y0, tile.n0);
+    }
+}
+
+// Expansion of channel chunk c of the staged tile: bitplanes of (pixel, 32-channel word) -> 32 int8 values, written as two 16-byte rows
 // of the K-major core-matrix layout [16-channel group][halo pixel][16 bytes].  `et` = 0..127 within the expander group.
 template <int A>
-__device__ __forceinline__ void tc_expand_chunk(const TcArgs& g, const uint32_t* pa, unsigned char* eb, int et)
+__device__ __forceinline__ void tc_expand_chunk(const TcArgs& g, const uint32_t* pa, unsigned char* eb, int et, int c)
 {
     const int items = g.flat ? TC_M * g.CWC : g.TNI * g.hh * g.hw * g.CWC;
     for (int it = et; it < items; it += 128) {
@@ -146,7 +169,7 @@ __device__ __forceinline__ void tc_expand_chunk(const TcArgs& g, const uint32_t*
             ep = hy * g.HWP + (g.stride == 2 ? (hx & 1) * g.HWH + (hx >> 1) : hx);
         }
         uint32_t w[A];
-        load_planes<A>(pa + static_cast<size_t>(hp) * g.CWC * A + cw * A, w);
+        load_planes<A>(pa + static_cast<size_t>(hp) * g.fullA + (c * g.CWC + cw) * A, w);
         uint32_t out[8];
 #pragma unroll
         for (int nb = 0; nb < 8; ++nb) {
@@ -166,22 +189,47 @@ __device__ __forceinline__ void tc_expand_chunk(const TcArgs& g, const uint32_t*
 }
 
 // All MMAs of one chunk: R*S taps x CK/32 steps of K = 32; a tap only moves the descriptor start address.
-__device__ __forceinline__ void tc_issue_chunk(const TcArgs& g, uint32_t ea, uint32_t ba, uint32_t tmem_acc, bool first_chunk)
+// The loop is issued by a single thread, so it is kept to a few 32-bit adds per MMA: the constant descriptor halves
+// are prepared once (TcIssue) and the start-address fields advance in 16-byte units.
+struct TcIssue {
+    uint64_t a_hi, b_hi;      // descriptor bits above the start-address field
+    uint32_t lbo16;           // A: distance between the two K halves, in 16-byte units
+    uint32_t k16;             // 16-channel groups per chunk
+    uint32_t idesc;
+};
+
+__device__ __forceinline__ TcIssue tc_make_issue(const TcArgs& g)
 {
-    const int RS = g.R * g.S;
+    TcIssue is;
     const uint32_t lbo_a = static_cast<uint32_t>(g.HPE) * 16u;
     const uint32_t sbo_a = g.flat ? 128u : static_cast<uint32_t>(g.stride * g.HWP) * 16u;
-    const uint32_t k16 = static_cast<uint32_t>(g.CK >> 4);
-    const uint32_t sbo_b = static_cast<uint32_t>(RS) * k16 * 128u;
-    for (int tap = 0; tap < RS; ++tap) {
-        const int r = tap / g.S, sx = tap - r * g.S;
-        const int xoff = g.stride == 2 ? (sx & 1) * g.HWH + (sx >> 1) : sx;
-        const uint32_t a_tap = ea + static_cast<uint32_t>(r * g.HWP + xoff) * 16u;
-        const uint32_t b_tap = ba + static_cast<uint32_t>(tap) * k16 * 128u;
-        for (uint32_t kp = 0; kp < k16 / 2; ++kp) {
-            const uint64_t ad = umma_desc(a_tap + 2 * kp * lbo_a, lbo_a, sbo_a);
-            const uint64_t bd = umma_desc(b_tap + 2 * kp * 128u, 128u, sbo_b);
-            umma_i8(tmem_acc, ad, bd, g.idesc, (first_chunk ? (tap | static_cast<int>(kp)) : 1) != 0);
+    is.k16 = static_cast<uint32_t>(g.CK >> 4);
+    const uint32_t sbo_b = static_cast<uint32_t>(g.R * g.S) * is.k16 * 128u;
+    is.a_hi = umma_desc(0, lbo_a, sbo_a);
+    is.b_hi = umma_desc(0, 128u, sbo_b);
+    is.lbo16 = lbo_a >> 4;
+    is.idesc = g.idesc;
+    return is;
+}
+
+__device__ __forceinline__ void tc_issue_chunk(const TcArgs& g, const TcIssue& is, uint32_t ea, uint32_t ba, uint32_t tmem_acc,
+                                               bool first_chunk)
+{
+    const uint32_t ea16 = ea >> 4;
+    uint32_t b16 = ba >> 4;
+    uint32_t accumulate = first_chunk ? 0u : 1u;
+    const uint32_t kpn = is.k16 >> 1;
+    for (int r = 0; r < g.R; ++r) {
+        const uint32_t row16 = ea16 + static_cast<uint32_t>(r * g.HWP);
+        for (int sx = 0; sx < g.S; ++sx) {
+            const uint32_t a16 = row16 + static_cast<uint32_t>(g.stride == 2 ? (sx & 1) * g.HWH + (sx >> 1) : sx);
+            for (uint32_t kp = 0; kp < kpn; ++kp) {
+                const uint64_t ad = is.a_hi | static_cast<uint64_t>((a16 + 2 * kp * is.lbo16) & 0x3FFFu);
+                const uint64_t bd = is.b_hi | static_cast<uint64_t>((b16 + 16 * kp) & 0x3FFFu);
+                umma_i8(tmem_acc, ad, bd, is.idesc, accumulate);
+                accumulate = 1u;
+            }
+            b16 += is.k16 * 8;
         }
     }
 }
@@ -305,7 +353,7 @@ __global__ void __launch_bounds__(TC_THREADS) bitserial_conv_tc_kernel(const __g
     extern __shared__ __align__(128) unsigned char tc_smem[];
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int RS = g.R * g.S;
-    const int stage_p_bytes = g.pa_bytes + g.b_bytes;
+    const int stage_p_bytes = g.b_bytes;                                    // filter ring; the packed tile sits at off_p
     float2* s_sb = reinterpret_cast<float2*>(tc_smem + g.off_sb);           // (scale, bias) per filter of the tile
     float4* s_bounds = reinterpret_cast<float4*>(tc_smem + g.off_sb + g.TN * 8);   // comparison bounds per residual pattern
     uint64_t* bars = reinterpret_cast<uint64_t*>(tc_smem + g.off_bar);
@@ -314,7 +362,8 @@ __global__ void __launch_bounds__(TC_THREADS) bitserial_conv_tc_kernel(const __g
     uint64_t* full_e = bars + 2 * TC_MAX_STAGES;
     uint64_t* empty_e = bars + 3 * TC_MAX_STAGES;
     uint64_t* accum_full = bars + 4 * TC_MAX_STAGES;
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 4 * TC_MAX_STAGES + 1);
+    uint64_t* full_a = bars + 4 * TC_MAX_STAGES + 1;      // packed tile landed
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 4 * TC_MAX_STAGES + 2);
 
     const int o0 = static_cast<int>(blockIdx.x % static_cast<unsigned>(g.tiles_o)) * g.TN;   // filter tile fastest
     const TcTile tile = tc_decode_tile(g, static_cast<int>(blockIdx.x / static_cast<unsigned>(g.tiles_o)));
@@ -327,6 +376,7 @@ __global__ void __launch_bounds__(TC_THREADS) bitserial_conv_tc_kernel(const __g
             mbar_init(&empty_e[s], 1);
         }
         mbar_init(accum_full, 1);
+        mbar_init(full_a, 1);
         fence_barrier_init();
         fence_proxy_async();
     }
@@ -347,16 +397,13 @@ __global__ void __launch_bounds__(TC_THREADS) bitserial_conv_tc_kernel(const __g
     if (warp == 4) {
         // ------------------------------------------------------------------ producer
         if (lane == 0) {
+            tc_load_tile(g, tc_smem + g.off_p, full_a, tile);
             for (int c = 0; c < g.nchunks; ++c) {
                 const int s = c % g.nsp, k = c / g.nsp;
                 if (k >= 1 && !mbar_wait_bounded(&empty_p[s], (k - 1) & 1)) { atomicOr(g.status, STATUS_TIMEOUT); break; }
-                unsigned char* pa = tc_smem + s * stage_p_bytes;
-                unsigned char* pb = pa + g.pa_bytes;
-                mbar_expect_tx(&full_p[s], static_cast<unsigned>(g.pa_tx_bytes + g.b_bytes));
-                if (g.flat) tma_load_2d(pa, &g.tmA, &full_p[s], c * g.CWC * A, tile.q0);
-                else tma_load_4d(pa, &g.tmA, &full_p[s], c * g.CWC * A, tile.q0 * g.stride - g.pad, tile.p0 * g.stride - g.pad, tile.n0);
+                mbar_expect_tx(&full_p[s], static_cast<unsigned>(g.b_bytes));
                 const size_t src = (static_cast<size_t>(c) * g.opad8 + (o0 >> 3)) * RS * (g.CK >> 4) * 128;
-                bulk_load(pb, g.wgt + src, static_cast<unsigned>(g.b_bytes), &full_p[s]);
+                bulk_load(tc_smem + s * stage_p_bytes, g.wgt + src, static_cast<unsigned>(g.b_bytes), &full_p[s]);
             }
         }
         __syncwarp();
@@ -364,6 +411,7 @@ __global__ void __launch_bounds__(TC_THREADS) bitserial_conv_tc_kernel(const __g
         // ------------------------------------------------------------------ MMA issuer
         if (lane == 0) {
             const uint32_t e_base = smem_u32(tc_smem + g.off_e);
+            const TcIssue is = tc_make_issue(g);
             for (int c = 0; c < g.nchunks; ++c) {
                 const int s = c % g.nsp, e = c % g.nse;
                 if (!(mbar_wait_bounded(&full_p[s], (c / g.nsp) & 1) && mbar_wait_bounded(&full_e[e], (c / g.nse) & 1))) {
@@ -371,7 +419,7 @@ __global__ void __launch_bounds__(TC_THREADS) bitserial_conv_tc_kernel(const __g
                     break;
                 }
                 tc_fence_after();
-                tc_issue_chunk(g, e_base + static_cast<uint32_t>(e) * g.e_bytes, smem_u32(tc_smem + s * stage_p_bytes + g.pa_bytes),
+                tc_issue_chunk(g, is, e_base + static_cast<uint32_t>(e) * g.e_bytes, smem_u32(tc_smem + s * stage_p_bytes),
                                tmem_base, c == 0);
                 umma_commit(&empty_e[e]);
                 umma_commit(&empty_p[s]);
@@ -381,13 +429,12 @@ __global__ void __launch_bounds__(TC_THREADS) bitserial_conv_tc_kernel(const __g
         __syncwarp();
     } else {
         // ------------------------------------------------------------------ expanders (warps 0-3), then epilogue
-        bool ok = true;
+        bool ok = mbar_wait_bounded(full_a, 0);
         for (int c = 0; c < g.nchunks; ++c) {
-            const int s = c % g.nsp, e = c % g.nse, k = c / g.nse;
-            if (ok) ok = mbar_wait_bounded(&full_p[s], (c / g.nsp) & 1);
+            const int e = c % g.nse, k = c / g.nse;
             if (ok && k >= 1) ok = mbar_wait_bounded(&empty_e[e], (k - 1) & 1);
             if (!ok) atomicOr(g.status, STATUS_TIMEOUT);
-            tc_expand_chunk<A>(g, reinterpret_cast<const uint32_t*>(tc_smem + s * stage_p_bytes), tc_smem + g.off_e + e * g.e_bytes, tid);
+            tc_expand_chunk<A>(g, reinterpret_cast<const uint32_t*>(tc_smem + g.off_p), tc_smem + g.off_e + e * g.e_bytes, tid, c);
             fence_proxy_async();          // make the generic-proxy writes visible to the tensor core's reads
             mbar_arrive(&full_e[e]);
         }
@@ -412,7 +459,7 @@ __global__ void __launch_bounds__(TC_THREADS) bitserial_conv_tc_kernel(const __g
 // epilogue of tile i overlap the MMAs of tile i + 1.
 
 constexpr int TCP_THREADS = 320;
-constexpr int TCP_NSP = 4;            // packed-chunk ring
+constexpr int TCP_NSP = 3;            // packed-tile ring (at most)
 constexpr int TCP_NSE = 3;            // expanded-chunk ring (at most)
 
 template <int A>
@@ -422,7 +469,7 @@ __global__ void __launch_bounds__(TCP_THREADS) bitserial_conv_tc_persistent_kern
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int RS = g.R * g.S;
     unsigned char* s_w = tc_smem;                                              // [nchunks][b_bytes]
-    unsigned char* s_p = tc_smem + g.off_p;                                    // [TCP_NSP][pa_bytes]
+    unsigned char* s_p = tc_smem + g.off_p;                                    // [nsp][pa_bytes] packed tiles
     unsigned char* s_e = tc_smem + g.off_e;                                    // [nse][e_bytes]
     float2* s_sb = reinterpret_cast<float2*>(tc_smem + g.off_sb);
     float4* s_bounds = reinterpret_cast<float4*>(tc_smem + g.off_sb + g.TN * 8);
@@ -471,18 +518,12 @@ __global__ void __launch_bounds__(TCP_THREADS) bitserial_conv_tc_persistent_kern
                 const size_t src = (static_cast<size_t>(c) * g.opad8 + (o0 >> 3)) * RS * (g.CK >> 4) * 128;
                 bulk_load(s_w + static_cast<size_t>(c) * g.b_bytes, g.wgt + src, static_cast<unsigned>(g.b_bytes), wgt_full);
             }
-            int it = 0;
+            int i = 0;
             bool ok = true;
-            for (int mt = first_tile; mt < tiles_m && ok; mt += tile_step) {
-                const TcTile tile = tc_decode_tile(g, mt);
-                for (int c = 0; c < g.nchunks; ++c, ++it) {
-                    const int s = it % TCP_NSP, k = it / TCP_NSP;
-                    if (k >= 1 && !mbar_wait_bounded(&empty_p[s], (k - 1) & 1)) { ok = false; break; }
-                    unsigned char* pa = s_p + s * g.pa_bytes;
-                    mbar_expect_tx(&full_p[s], static_cast<unsigned>(g.pa_tx_bytes));
-                    if (g.flat) tma_load_2d(pa, &g.tmA, &full_p[s], c * g.CWC * A, tile.q0);
-                    else tma_load_4d(pa, &g.tmA, &full_p[s], c * g.CWC * A, tile.q0 * g.stride - g.pad, tile.p0 * g.stride - g.pad, tile.n0);
-                }
+            for (int mt = first_tile; mt < tiles_m && ok; mt += tile_step, ++i) {
+                const int s = i % g.nsp, k = i / g.nsp;
+                if (k >= 1 && !mbar_wait_bounded(&empty_p[s], (k - 1) & 1)) { ok = false; break; }
+                tc_load_tile(g, s_p + s * g.pa_bytes, &full_p[s], tc_decode_tile(g, mt));
             }
             if (!ok) atomicOr(g.status, STATUS_TIMEOUT);
         }
@@ -490,6 +531,7 @@ __global__ void __launch_bounds__(TCP_THREADS) bitserial_conv_tc_persistent_kern
     } else if (warp == 9) {
         // ------------------------------------------------------------------ MMA issuer
         if (lane == 0) {
+            const TcIssue is = tc_make_issue(g);
             bool ok = mbar_wait_bounded(wgt_full, 0);       // also keeps the CTA alive until the filter copy has landed
             int it = 0, i = 0;
             for (int mt = first_tile; mt < tiles_m && ok; mt += tile_step, ++i) {
@@ -502,7 +544,7 @@ __global__ void __launch_bounds__(TCP_THREADS) bitserial_conv_tc_persistent_kern
                     const int e = it % g.nse;
                     if (!mbar_wait_bounded(&full_e[e], (it / g.nse) & 1)) { ok = false; break; }
                     tc_fence_after();
-                    tc_issue_chunk(g, smem_u32(s_e + e * g.e_bytes), smem_u32(s_w + static_cast<size_t>(c) * g.b_bytes), tmem_acc, c == 0);
+                    tc_issue_chunk(g, is, smem_u32(s_e + e * g.e_bytes), smem_u32(s_w + static_cast<size_t>(c) * g.b_bytes), tmem_acc, c == 0);
                     umma_commit(&empty_e[e]);
                 }
                 if (ok) umma_commit(&full_acc[buf]);
@@ -513,19 +555,20 @@ __global__ void __launch_bounds__(TCP_THREADS) bitserial_conv_tc_persistent_kern
     } else if (warp >= 4) {
         // ------------------------------------------------------------------ expanders (warps 4-7)
         const int et = tid - 128;
-        int it = 0;
+        int it = 0, i = 0;
         bool ok = true;
-        for (int mt = first_tile; mt < tiles_m && ok; mt += tile_step) {
-            for (int c = 0; c < g.nchunks; ++c, ++it) {
-                const int s = it % TCP_NSP, e = it % g.nse, k = it / g.nse;
-                ok = mbar_wait_bounded(&full_p[s], (it / TCP_NSP) & 1);
-                if (ok && k >= 1) ok = mbar_wait_bounded(&empty_e[e], (k - 1) & 1);
+        for (int mt = first_tile; mt < tiles_m && ok; mt += tile_step, ++i) {
+            const int s = i % g.nsp;
+            ok = mbar_wait_bounded(&full_p[s], (i / g.nsp) & 1);
+            for (int c = 0; c < g.nchunks && ok; ++c, ++it) {
+                const int e = it % g.nse, k = it / g.nse;
+                if (k >= 1) ok = mbar_wait_bounded(&empty_e[e], (k - 1) & 1);
                 if (!ok) break;
-                tc_expand_chunk<A>(g, reinterpret_cast<const uint32_t*>(s_p + s * g.pa_bytes), s_e + e * g.e_bytes, et);
+                tc_expand_chunk<A>(g, reinterpret_cast<const uint32_t*>(s_p + s * g.pa_bytes), s_e + e * g.e_bytes, et, c);
                 fence_proxy_async();
                 mbar_arrive(&full_e[e]);
-                mbar_arrive(&empty_p[s]);
             }
+            if (ok) mbar_arrive(&empty_p[s]);
         }
         if (!ok) atomicOr(g.status, STATUS_TIMEOUT);
     } else {
@@ -583,12 +626,11 @@ __global__ void tc_prepare_weights_kernel(const uint32_t* __restrict__ packed, i
 
 static int round_up_i(int v, int m) { return (v + m - 1) / m * m; }
 
-// Channel chunk per pipeline stage: the smallest of 32/64/128 whose packed record (CK/32 * A words) is a
-// 16-byte multiple (a TMA box requirement); 0 if C does not allow it.
-static int tc_chunk_channels(int C, int A)
+// Channels per pipeline chunk (and per block of the prepared filter layout): 64 when C allows, else 32.
+static int tc_chunk_channels(int C, int /*a_bits*/)
 {
-    for (int ck = 32; ck <= 128; ck *= 2)
-        if (((ck / 32) * A) % 4 == 0 && C % ck == 0) return ck;
+    if (C % 64 == 0) return 64;
+    if (C % 32 == 0) return 32;
     return 0;
 }
 
@@ -678,6 +720,8 @@ static int tc_conv_impl(const uint32_t* act, const int8_t* wgt, const bs_conv_pa
 
     g.CK = tc_chunk_channels(p->C, A);
     g.CWC = g.CK / 32;
+    g.fullA = Cw * A;
+    g.act = act;
     g.nchunks = p->C / g.CK;
     g.nsp = g.nse = g.nchunks < TC_MAX_STAGES ? g.nchunks : TC_MAX_STAGES;
     g.opad8 = round_up_i(p->O, 128) / 8;
@@ -688,7 +732,8 @@ static int tc_conv_impl(const uint32_t* act, const int8_t* wgt, const bs_conv_pa
         if (npix > 0x7fffffffLL) return BS_ERR_UNSUPPORTED;
         g.tiles_q = static_cast<int>(ceil_div_ll(npix, TC_M)); g.tiles_p = 1; g.tiles_n = 1;
         g.TNI = 1; g.GI = 16; g.hh = 1; g.hw = TC_M; g.HWP = TC_M; g.HWH = 0; g.HPE = TC_M;
-        g.pa_tx_bytes = TC_M * g.CWC * A * 4;
+        g.pa_tx_bytes = TC_M * g.fullA * 4;
+        g.pmode = 0;
         tiles_m = g.tiles_q;
     } else {
         g.hw = 7 * p->stride + p->S;
@@ -710,7 +755,9 @@ static int tc_conv_impl(const uint32_t* act, const int8_t* wgt, const bs_conv_pa
         const int rows_box = g.TNI * g.hh;
         const int rows_read = 15 * p->stride + p->R;
         g.HPE = (rows_box > rows_read ? rows_box : rows_read) * g.HWP;
-        g.pa_tx_bytes = g.TNI * g.hh * g.hw * g.CWC * A * 4;
+        g.pa_tx_bytes = g.TNI * g.hh * g.hw * g.fullA * 4;
+        g.pmode = (g.hw * g.fullA <= 256) ? 1 : 2;
+        if (g.pmode == 2 && g.fullA > 256) return BS_ERR_UNSUPPORTED;
         tiles_m = static_cast<long long>(g.tiles_q) * g.tiles_p * g.tiles_n;
     }
     g.pa_bytes = round_up_i(g.pa_tx_bytes, 128);
@@ -726,13 +773,15 @@ static int tc_conv_impl(const uint32_t* act, const int8_t* wgt, const bs_conv_pa
         const long long pairs = tiles_m * ceil_div(p->O, TN);
         if (TN > 32 && pairs < sms) continue;
         const size_t wbytes = static_cast<size_t>(g.nchunks) * TN * RS * g.CK;
-        for (int nse = TCP_NSE; nse >= 2; --nse) {
-            const size_t total = wbytes + static_cast<size_t>(TCP_NSP) * g.pa_bytes + static_cast<size_t>(nse) * g.e_bytes +
+        const int shapes[4][2] = {{3, 3}, {2, 3}, {2, 2}, {1, 2}};      // (packed-tile stages, expanded-chunk stages)
+        for (const auto& sh : shapes) {
+            const int nsp = sh[0], nse = sh[1];
+            const size_t total = wbytes + static_cast<size_t>(nsp) * g.pa_bytes + static_cast<size_t>(nse) * g.e_bytes +
                                  static_cast<size_t>(TN) * 8 + 256 + bar_bytes + 128;
             if (total <= 220 * 1024) {
-                g.persistent = 1; g.TN = TN; g.b_bytes = TN * RS * g.CK; g.nse = nse; g.nsp = TCP_NSP;
+                g.persistent = 1; g.TN = TN; g.b_bytes = TN * RS * g.CK; g.nse = nse; g.nsp = nsp;
                 g.off_p = static_cast<int>(wbytes);
-                g.off_e = g.off_p + TCP_NSP * g.pa_bytes;
+                g.off_e = g.off_p + nsp * g.pa_bytes;
                 g.off_sb = g.off_e + nse * g.e_bytes;
                 g.off_bar = round_up_i(g.off_sb + TN * 8 + 256, 16);
                 smem = static_cast<size_t>(g.off_bar) + bar_bytes;
@@ -748,14 +797,15 @@ static int tc_conv_impl(const uint32_t* act, const int8_t* wgt, const bs_conv_pa
         for (;; TN /= 2) {
             g.TN = TN;
             g.b_bytes = TN * RS * g.CK;
-            const size_t total = static_cast<size_t>(g.nsp) * (g.pa_bytes + g.b_bytes) + static_cast<size_t>(g.nse) * g.e_bytes +
-                                 2 * TN * 4 + 256 + (4 * TC_MAX_STAGES + 2) * 8 + 128;
+            const size_t total = static_cast<size_t>(g.nsp) * g.b_bytes + g.pa_bytes + static_cast<size_t>(g.nse) * g.e_bytes +
+                                 2 * TN * 4 + 256 + (4 * TC_MAX_STAGES + 3) * 8 + 128;
             if (total <= 200 * 1024 || TN == 32) break;
         }
-        g.off_e = g.nsp * (g.pa_bytes + g.b_bytes);
+        g.off_p = g.nsp * g.b_bytes;
+        g.off_e = g.off_p + g.pa_bytes;
         g.off_sb = g.off_e + g.nse * g.e_bytes;
         g.off_bar = round_up_i(g.off_sb + 2 * g.TN * 4 + 256, 16);
-        smem = static_cast<size_t>(g.off_bar) + (4 * TC_MAX_STAGES + 2) * 8;
+        smem = static_cast<size_t>(g.off_bar) + (4 * TC_MAX_STAGES + 3) * 8;
         if (smem > 220 * 1024) return BS_ERR_UNSUPPORTED;
     }
     g.tiles_o = ceil_div(p->O, g.TN);
@@ -774,18 +824,18 @@ static int tc_conv_impl(const uint32_t* act, const int8_t* wgt, const bs_conv_pa
     if (!enc) return BS_ERR_CUDA;
     const cuuint64_t fullA = static_cast<cuuint64_t>(Cw) * A;
     cuuint32_t estr[4] = {1, 1, 1, 1};
-    CUresult cr;
-    if (g.flat) {
-        cuuint64_t dims[2] = {fullA, static_cast<cuuint64_t>(p->N) * p->H * p->W};
-        cuuint64_t strides[1] = {fullA * 4};
-        cuuint32_t box[2] = {static_cast<cuuint32_t>(g.CWC * A), static_cast<cuuint32_t>(TC_M)};
-        cr = enc(&g.tmA, CU_TENSOR_MAP_DATA_TYPE_UINT32, 2, const_cast<uint32_t*>(act), dims, strides, box, estr,
+    CUresult cr = CUDA_SUCCESS;
+    if (g.pmode == 1) {
+        cuuint64_t dims[3] = {fullA * p->W, static_cast<cuuint64_t>(p->H), static_cast<cuuint64_t>(p->N)};
+        cuuint64_t strides[2] = {fullA * 4 * p->W, fullA * 4 * p->W * p->H};
+        cuuint32_t box[3] = {static_cast<cuuint32_t>(g.hw * g.fullA), static_cast<cuuint32_t>(g.hh), static_cast<cuuint32_t>(g.TNI)};
+        cr = enc(&g.tmA, CU_TENSOR_MAP_DATA_TYPE_UINT32, 3, const_cast<uint32_t*>(act), dims, strides, box, estr,
                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-    } else {
+    } else if (g.pmode == 2) {
         cuuint64_t dims[4] = {fullA, static_cast<cuuint64_t>(p->W), static_cast<cuuint64_t>(p->H), static_cast<cuuint64_t>(p->N)};
         cuuint64_t strides[3] = {fullA * 4, fullA * 4 * p->W, fullA * 4 * p->W * p->H};
-        cuuint32_t box[4] = {static_cast<cuuint32_t>(g.CWC * A), static_cast<cuuint32_t>(g.hw), static_cast<cuuint32_t>(g.hh),
+        cuuint32_t box[4] = {static_cast<cuuint32_t>(g.fullA), static_cast<cuuint32_t>(g.hw), static_cast<cuuint32_t>(g.hh),
                              static_cast<cuuint32_t>(g.TNI)};
         cr = enc(&g.tmA, CU_TENSOR_MAP_DATA_TYPE_UINT32, 4, const_cast<uint32_t*>(act), dims, strides, box, estr,
                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
