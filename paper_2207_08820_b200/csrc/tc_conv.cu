@@ -50,7 +50,7 @@ struct TcArgs {
     int tiles_o, tiles_q, tiles_p, tiles_n;
     int opad8;                        // padded filter count / 8 in the prepared weights
     int pa_bytes, pa_tx_bytes, b_bytes, e_bytes;   // per stage (pa_tx_bytes: bytes the activation box delivers)
-    int off_p, off_e, off_sb, off_bar;   // shared-memory offsets (bytes)
+    int off_p, off_e, off_sb, off_bar, off_tab;   // shared-memory offsets (bytes)
     int persistent;
     int tmem_cols;
     unsigned idesc;
@@ -64,6 +64,44 @@ struct TcArgs {
 __device__ __forceinline__ void mbar_arrive(uint64_t* bar)
 {
     asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+// Barrier among the 128 threads of one warp group (expanders or epilogue); ids 1 and 2, id 0 is __syncthreads.
+__device__ __forceinline__ void group_sync(int id) { asm volatile("bar.sync %0, 128;" ::"r"(id) : "memory"); }
+// Low-latency bounded wait for the tensor-core pipeline: non-blocking test_wait in a spin loop (try_wait may park the
+// thread and wake it late, which costs microseconds per hand-off between the roles).  About a second at most.
+__device__ __forceinline__ bool mbar_spin_bounded(uint64_t* bar, unsigned parity)
+{
+    const uint32_t addr = smem_u32(bar);
+    for (unsigned it = 0; it < (1u << 26); ++it) {
+        unsigned ok;
+        asm volatile(
+            "{\n\t.reg .pred p;\n\t"
+            "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+            "selp.u32 %0, 1, 0, p;\n\t}"
+            : "=r"(ok) : "r"(addr), "r"(parity) : "memory");
+        if (ok) return true;
+    }
+    return false;
+}
+// Group-wide AND of a per-thread flag (also a barrier): every thread of the group gets the same answer, so a wait
+// that ran out makes the whole group leave its loop together and nobody is left behind at a later group_sync.
+__device__ __forceinline__ bool group_all(int id, bool ok)
+{
+    unsigned r;
+    asm volatile(
+        "{\n\t.reg .pred p, q;\n\t"
+        "setp.ne.u32 q, %1, 0;\n\t"
+        "bar.red.and.pred p, %2, 128, q;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(r) : "r"(ok ? 1u : 0u), "r"(id) : "memory");
+    return r != 0;
+}
+// One lane polls the mbarrier for its warp (128 threads hammering one shared-memory word is slow); result is broadcast.
+__device__ __forceinline__ bool mbar_wait_warp(uint64_t* bar, unsigned parity, int lane)
+{
+    unsigned ok = 1;
+    if (lane == 0) ok = mbar_spin_bounded(bar, parity) ? 1u : 0u;
+    return __shfl_sync(0xffffffffu, ok, 0) != 0;
 }
 __device__ __forceinline__ void tmem_alloc(uint32_t* slot, unsigned ncols)
 {
@@ -189,48 +227,66 @@ __device__ __forceinline__ void tc_expand_chunk(const TcArgs& g, const uint32_t*
 }
 
 // All MMAs of one chunk: R*S taps x CK/32 steps of K = 32; a tap only moves the descriptor start address.
-// The loop is issued by a single thread, so it is kept to a few 32-bit adds per MMA: the constant descriptor halves
-// are prepared once (TcIssue) and the start-address fields advance in 16-byte units.
+// One thread issues them, and a lone thread retires only an instruction every few cycles, so the per-MMA work is cut
+// to a table look-up and two adds: the start-address offsets of every (tap, K step) are tabulated once per CTA in
+// shared memory (in 16-byte units, relative to the stage base) and the constant descriptor words live in registers.
+constexpr int TC_MAX_MMA_PER_CHUNK = 128;       // R*S * CK/32 <= 49 * 2
+
 struct TcIssue {
-    uint64_t a_hi, b_hi;      // descriptor bits above the start-address field
-    uint32_t lbo16;           // A: distance between the two K halves, in 16-byte units
-    uint32_t k16;             // 16-channel groups per chunk
+    uint32_t a_lo, a_hi, b_lo, b_hi;   // descriptor words with a zero start-address field
     uint32_t idesc;
+    int n;                             // MMAs per chunk
 };
 
-__device__ __forceinline__ TcIssue tc_make_issue(const TcArgs& g)
+__device__ __forceinline__ TcIssue tc_make_issue(const TcArgs& g, uint2* tab)
 {
     TcIssue is;
     const uint32_t lbo_a = static_cast<uint32_t>(g.HPE) * 16u;
     const uint32_t sbo_a = g.flat ? 128u : static_cast<uint32_t>(g.stride * g.HWP) * 16u;
-    is.k16 = static_cast<uint32_t>(g.CK >> 4);
-    const uint32_t sbo_b = static_cast<uint32_t>(g.R * g.S) * is.k16 * 128u;
-    is.a_hi = umma_desc(0, lbo_a, sbo_a);
-    is.b_hi = umma_desc(0, 128u, sbo_b);
-    is.lbo16 = lbo_a >> 4;
+    const uint32_t k16 = static_cast<uint32_t>(g.CK >> 4);
+    const uint32_t sbo_b = static_cast<uint32_t>(g.R * g.S) * k16 * 128u;
+    const uint64_t ad = umma_desc(0, lbo_a, sbo_a), bd = umma_desc(0, 128u, sbo_b);
+    is.a_lo = static_cast<uint32_t>(ad); is.a_hi = static_cast<uint32_t>(ad >> 32);
+    is.b_lo = static_cast<uint32_t>(bd); is.b_hi = static_cast<uint32_t>(bd >> 32);
     is.idesc = g.idesc;
+    int n = 0;
+    uint32_t b16 = 0;
+    for (int r = 0; r < g.R; ++r)
+        for (int sx = 0; sx < g.S; ++sx) {
+            const uint32_t a16 = static_cast<uint32_t>(r * g.HWP + (g.stride == 2 ? (sx & 1) * g.HWH + (sx >> 1) : sx));
+            for (uint32_t kp = 0; kp < k16 / 2; ++kp) tab[n++] = make_uint2(a16 + 2 * kp * (lbo_a >> 4), b16 + 16 * kp);
+            b16 += k16 * 8;
+        }
+    is.n = n;
     return is;
 }
 
-__device__ __forceinline__ void tc_issue_chunk(const TcArgs& g, const TcIssue& is, uint32_t ea, uint32_t ba, uint32_t tmem_acc,
+__device__ __forceinline__ void umma_i8_words(uint32_t d_tmem, uint32_t a_lo, uint32_t a_hi, uint32_t b_lo, uint32_t b_hi,
+                                              uint32_t idesc, uint32_t accumulate)
+{
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t.reg .b64 da, db;\n\t"
+        "mov.b64 da, {%1, %2};\n\t"
+        "mov.b64 db, {%3, %4};\n\t"
+        "setp.ne.b32 p, %6, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::i8 [%0], da, db, %5, p;\n\t}"
+        ::"r"(d_tmem), "r"(a_lo), "r"(a_hi), "r"(b_lo), "r"(b_hi), "r"(idesc), "r"(accumulate) : "memory");
+}
+
+__device__ __forceinline__ void tc_issue_chunk(const TcIssue& is, const uint2* tab, uint32_t ea, uint32_t ba, uint32_t tmem_acc,
                                                bool first_chunk)
 {
-    const uint32_t ea16 = ea >> 4;
-    uint32_t b16 = ba >> 4;
-    uint32_t accumulate = first_chunk ? 0u : 1u;
-    const uint32_t kpn = is.k16 >> 1;
-    for (int r = 0; r < g.R; ++r) {
-        const uint32_t row16 = ea16 + static_cast<uint32_t>(r * g.HWP);
-        for (int sx = 0; sx < g.S; ++sx) {
-            const uint32_t a16 = row16 + static_cast<uint32_t>(g.stride == 2 ? (sx & 1) * g.HWH + (sx >> 1) : sx);
-            for (uint32_t kp = 0; kp < kpn; ++kp) {
-                const uint64_t ad = is.a_hi | static_cast<uint64_t>((a16 + 2 * kp * is.lbo16) & 0x3FFFu);
-                const uint64_t bd = is.b_hi | static_cast<uint64_t>((b16 + 16 * kp) & 0x3FFFu);
-                umma_i8(tmem_acc, ad, bd, is.idesc, accumulate);
-                accumulate = 1u;
-            }
-            b16 += is.k16 * 8;
-        }
+    const uint32_t ea16 = ea >> 4, ba16 = ba >> 4;
+    int m = 0;
+    if (first_chunk) {          // the first MMA of a tile overwrites the accumulator
+        const uint2 d = tab[0];
+        umma_i8_words(tmem_acc, is.a_lo | ((ea16 + d.x) & 0x3FFFu), is.a_hi, is.b_lo | ((ba16 + d.y) & 0x3FFFu), is.b_hi, is.idesc, 0u);
+        m = 1;
+    }
+#pragma unroll 4
+    for (; m < is.n; ++m) {
+        const uint2 d = tab[m];
+        umma_i8_words(tmem_acc, is.a_lo | ((ea16 + d.x) & 0x3FFFu), is.a_hi, is.b_lo | ((ba16 + d.y) & 0x3FFFu), is.b_hi, is.idesc, 1u);
     }
 }
 
@@ -372,7 +428,7 @@ __global__ void __launch_bounds__(TC_THREADS) bitserial_conv_tc_kernel(const __g
         for (int s = 0; s < TC_MAX_STAGES; ++s) {
             mbar_init(&full_p[s], 1);
             mbar_init(&empty_p[s], 1);
-            mbar_init(&full_e[s], 128);
+            mbar_init(&full_e[s], 1);
             mbar_init(&empty_e[s], 1);
         }
         mbar_init(accum_full, 1);
@@ -400,7 +456,7 @@ __global__ void __launch_bounds__(TC_THREADS) bitserial_conv_tc_kernel(const __g
             tc_load_tile(g, tc_smem + g.off_p, full_a, tile);
             for (int c = 0; c < g.nchunks; ++c) {
                 const int s = c % g.nsp, k = c / g.nsp;
-                if (k >= 1 && !mbar_wait_bounded(&empty_p[s], (k - 1) & 1)) { atomicOr(g.status, STATUS_TIMEOUT); break; }
+                if (k >= 1 && !mbar_spin_bounded(&empty_p[s], (k - 1) & 1)) { atomicOr(g.status, STATUS_TIMEOUT); break; }
                 mbar_expect_tx(&full_p[s], static_cast<unsigned>(g.b_bytes));
                 const size_t src = (static_cast<size_t>(c) * g.opad8 + (o0 >> 3)) * RS * (g.CK >> 4) * 128;
                 bulk_load(tc_smem + s * stage_p_bytes, g.wgt + src, static_cast<unsigned>(g.b_bytes), &full_p[s]);
@@ -411,15 +467,16 @@ __global__ void __launch_bounds__(TC_THREADS) bitserial_conv_tc_kernel(const __g
         // ------------------------------------------------------------------ MMA issuer
         if (lane == 0) {
             const uint32_t e_base = smem_u32(tc_smem + g.off_e);
-            const TcIssue is = tc_make_issue(g);
+            uint2* tab = reinterpret_cast<uint2*>(tc_smem + g.off_tab);
+            const TcIssue is = tc_make_issue(g, tab);
             for (int c = 0; c < g.nchunks; ++c) {
                 const int s = c % g.nsp, e = c % g.nse;
-                if (!(mbar_wait_bounded(&full_p[s], (c / g.nsp) & 1) && mbar_wait_bounded(&full_e[e], (c / g.nse) & 1))) {
+                if (!(mbar_spin_bounded(&full_p[s], (c / g.nsp) & 1) && mbar_spin_bounded(&full_e[e], (c / g.nse) & 1))) {
                     atomicOr(g.status, STATUS_TIMEOUT);
                     break;
                 }
                 tc_fence_after();
-                tc_issue_chunk(g, is, e_base + static_cast<uint32_t>(e) * g.e_bytes, smem_u32(tc_smem + s * stage_p_bytes),
+                tc_issue_chunk(is, tab, e_base + static_cast<uint32_t>(e) * g.e_bytes, smem_u32(tc_smem + s * stage_p_bytes),
                                tmem_base, c == 0);
                 umma_commit(&empty_e[e]);
                 umma_commit(&empty_p[s]);
@@ -429,16 +486,17 @@ __global__ void __launch_bounds__(TC_THREADS) bitserial_conv_tc_kernel(const __g
         __syncwarp();
     } else {
         // ------------------------------------------------------------------ expanders (warps 0-3), then epilogue
-        bool ok = mbar_wait_bounded(full_a, 0);
+        bool ok = mbar_wait_warp(full_a, 0, lane);
         for (int c = 0; c < g.nchunks; ++c) {
             const int e = c % g.nse, k = c / g.nse;
-            if (ok && k >= 1) ok = mbar_wait_bounded(&empty_e[e], (k - 1) & 1);
+            if (ok && k >= 1) ok = mbar_wait_warp(&empty_e[e], (k - 1) & 1, lane);
             if (!ok) atomicOr(g.status, STATUS_TIMEOUT);
             tc_expand_chunk<A>(g, reinterpret_cast<const uint32_t*>(tc_smem + g.off_p), tc_smem + g.off_e + e * g.e_bytes, tid, c);
             fence_proxy_async();          // make the generic-proxy writes visible to the tensor core's reads
-            mbar_arrive(&full_e[e]);
+            group_sync(1);
+            if (tid == 0) mbar_arrive(&full_e[e]);
         }
-        if (ok) ok = mbar_wait_bounded(accum_full, 0);
+        if (ok) ok = mbar_wait_warp(accum_full, 0, lane);
         if (!ok) atomicOr(g.status, STATUS_TIMEOUT);
         tc_fence_after();
         tc_epilogue_tile(g, tmem_base, tid, warp, tile, o0, s_sb, s_bounds);
@@ -489,9 +547,9 @@ __global__ void __launch_bounds__(TCP_THREADS) bitserial_conv_tc_persistent_kern
     const int tiles_m = g.tiles_q * g.tiles_p * g.tiles_n;
 
     if (tid == 0) {
-        for (int s = 0; s < TCP_NSP; ++s) { mbar_init(&full_p[s], 1); mbar_init(&empty_p[s], 128); }
-        for (int s = 0; s < TCP_NSE; ++s) { mbar_init(&full_e[s], 128); mbar_init(&empty_e[s], 1); }
-        for (int s = 0; s < 2; ++s) { mbar_init(&full_acc[s], 1); mbar_init(&empty_acc[s], 128); }
+        for (int s = 0; s < TCP_NSP; ++s) { mbar_init(&full_p[s], 1); mbar_init(&empty_p[s], 1); }
+        for (int s = 0; s < TCP_NSE; ++s) { mbar_init(&full_e[s], 1); mbar_init(&empty_e[s], 1); }
+        for (int s = 0; s < 2; ++s) { mbar_init(&full_acc[s], 1); mbar_init(&empty_acc[s], 1); }
         mbar_init(wgt_full, 1);
         fence_barrier_init();
         fence_proxy_async();
@@ -522,7 +580,7 @@ __global__ void __launch_bounds__(TCP_THREADS) bitserial_conv_tc_persistent_kern
             bool ok = true;
             for (int mt = first_tile; mt < tiles_m && ok; mt += tile_step, ++i) {
                 const int s = i % g.nsp, k = i / g.nsp;
-                if (k >= 1 && !mbar_wait_bounded(&empty_p[s], (k - 1) & 1)) { ok = false; break; }
+                if (k >= 1 && !mbar_spin_bounded(&empty_p[s], (k - 1) & 1)) { ok = false; break; }
                 tc_load_tile(g, s_p + s * g.pa_bytes, &full_p[s], tc_decode_tile(g, mt));
             }
             if (!ok) atomicOr(g.status, STATUS_TIMEOUT);
@@ -531,20 +589,21 @@ __global__ void __launch_bounds__(TCP_THREADS) bitserial_conv_tc_persistent_kern
     } else if (warp == 9) {
         // ------------------------------------------------------------------ MMA issuer
         if (lane == 0) {
-            const TcIssue is = tc_make_issue(g);
-            bool ok = mbar_wait_bounded(wgt_full, 0);       // also keeps the CTA alive until the filter copy has landed
+            uint2* tab = reinterpret_cast<uint2*>(tc_smem + g.off_tab);
+            const TcIssue is = tc_make_issue(g, tab);
+            bool ok = mbar_spin_bounded(wgt_full, 0);       // also keeps the CTA alive until the filter copy has landed
             int it = 0, i = 0;
             for (int mt = first_tile; mt < tiles_m && ok; mt += tile_step, ++i) {
                 const int buf = i & 1, use = i >> 1;
-                if (use >= 1) ok = mbar_wait_bounded(&empty_acc[buf], (use - 1) & 1);
+                if (use >= 1) ok = mbar_spin_bounded(&empty_acc[buf], (use - 1) & 1);
                 if (!ok) break;
                 tc_fence_after();
                 const uint32_t tmem_acc = tmem_base + static_cast<uint32_t>(buf * g.TN);
                 for (int c = 0; c < g.nchunks; ++c, ++it) {
                     const int e = it % g.nse;
-                    if (!mbar_wait_bounded(&full_e[e], (it / g.nse) & 1)) { ok = false; break; }
+                    if (!mbar_spin_bounded(&full_e[e], (it / g.nse) & 1)) { ok = false; break; }
                     tc_fence_after();
-                    tc_issue_chunk(g, is, smem_u32(s_e + e * g.e_bytes), smem_u32(s_w + static_cast<size_t>(c) * g.b_bytes), tmem_acc, c == 0);
+                    tc_issue_chunk(is, tab, smem_u32(s_e + e * g.e_bytes), smem_u32(s_w + static_cast<size_t>(c) * g.b_bytes), tmem_acc, c == 0);
                     umma_commit(&empty_e[e]);
                 }
                 if (ok) umma_commit(&full_acc[buf]);
@@ -559,16 +618,18 @@ __global__ void __launch_bounds__(TCP_THREADS) bitserial_conv_tc_persistent_kern
         bool ok = true;
         for (int mt = first_tile; mt < tiles_m && ok; mt += tile_step, ++i) {
             const int s = i % g.nsp;
-            ok = mbar_wait_bounded(&full_p[s], (i / g.nsp) & 1);
-            for (int c = 0; c < g.nchunks && ok; ++c, ++it) {
+            ok = mbar_wait_warp(&full_p[s], (i / g.nsp) & 1, lane);
+            for (int c = 0; c < g.nchunks; ++c, ++it) {
                 const int e = it % g.nse, k = it / g.nse;
-                if (k >= 1) ok = mbar_wait_bounded(&empty_e[e], (k - 1) & 1);
+                if (ok && k >= 1) ok = mbar_wait_warp(&empty_e[e], (k - 1) & 1, lane);
+                ok = group_all(1, ok);
                 if (!ok) break;
                 tc_expand_chunk<A>(g, reinterpret_cast<const uint32_t*>(s_p + s * g.pa_bytes), s_e + e * g.e_bytes, et, c);
                 fence_proxy_async();
-                mbar_arrive(&full_e[e]);
+                group_sync(1);                       // all 128 expander threads have written and fenced
+                if (et == 0) mbar_arrive(&full_e[e]);
             }
-            if (ok) mbar_arrive(&empty_p[s]);
+            if (ok && et == 0) mbar_arrive(&empty_p[s]);   // ordered after the last group_sync: every thread is done reading
         }
         if (!ok) atomicOr(g.status, STATUS_TIMEOUT);
     } else {
@@ -577,13 +638,14 @@ __global__ void __launch_bounds__(TCP_THREADS) bitserial_conv_tc_persistent_kern
         bool ok = true;
         for (int mt = first_tile; mt < tiles_m && ok; mt += tile_step, ++i) {
             const int buf = i & 1, use = i >> 1;
-            ok = mbar_wait_bounded(&full_acc[buf], use & 1);
+            ok = group_all(2, mbar_wait_warp(&full_acc[buf], use & 1, lane));
             if (!ok) break;
             tc_fence_after();
             const TcTile tile = tc_decode_tile(g, mt);
             tc_epilogue_tile(g, tmem_base + static_cast<uint32_t>(buf * g.TN), tid, warp, tile, o0, s_sb, s_bounds);
             tc_fence_before();
-            mbar_arrive(&empty_acc[buf]);
+            group_sync(2);                           // all four warps have read their accumulator rows
+            if (tid == 0) mbar_arrive(&empty_acc[buf]);
         }
         if (!ok) atomicOr(g.status, STATUS_TIMEOUT);
     }
@@ -777,14 +839,15 @@ static int tc_conv_impl(const uint32_t* act, const int8_t* wgt, const bs_conv_pa
         for (const auto& sh : shapes) {
             const int nsp = sh[0], nse = sh[1];
             const size_t total = wbytes + static_cast<size_t>(nsp) * g.pa_bytes + static_cast<size_t>(nse) * g.e_bytes +
-                                 static_cast<size_t>(TN) * 8 + 256 + bar_bytes + 128;
+                                 static_cast<size_t>(TN) * 8 + 256 + bar_bytes + 128 + TC_MAX_MMA_PER_CHUNK * 8 + 16;
             if (total <= 220 * 1024) {
                 g.persistent = 1; g.TN = TN; g.b_bytes = TN * RS * g.CK; g.nse = nse; g.nsp = nsp;
                 g.off_p = static_cast<int>(wbytes);
                 g.off_e = g.off_p + nsp * g.pa_bytes;
                 g.off_sb = g.off_e + nse * g.e_bytes;
                 g.off_bar = round_up_i(g.off_sb + TN * 8 + 256, 16);
-                smem = static_cast<size_t>(g.off_bar) + bar_bytes;
+                g.off_tab = round_up_i(g.off_bar + bar_bytes, 16);
+                smem = static_cast<size_t>(g.off_tab) + TC_MAX_MMA_PER_CHUNK * 8;
                 break;
             }
         }
@@ -798,14 +861,15 @@ static int tc_conv_impl(const uint32_t* act, const int8_t* wgt, const bs_conv_pa
             g.TN = TN;
             g.b_bytes = TN * RS * g.CK;
             const size_t total = static_cast<size_t>(g.nsp) * g.b_bytes + g.pa_bytes + static_cast<size_t>(g.nse) * g.e_bytes +
-                                 2 * TN * 4 + 256 + (4 * TC_MAX_STAGES + 3) * 8 + 128;
+                                 2 * TN * 4 + 256 + (4 * TC_MAX_STAGES + 3) * 8 + 128 + TC_MAX_MMA_PER_CHUNK * 8 + 16;
             if (total <= 200 * 1024 || TN == 32) break;
         }
         g.off_p = g.nsp * g.b_bytes;
         g.off_e = g.off_p + g.pa_bytes;
         g.off_sb = g.off_e + g.nse * g.e_bytes;
         g.off_bar = round_up_i(g.off_sb + 2 * g.TN * 4 + 256, 16);
-        smem = static_cast<size_t>(g.off_bar) + (4 * TC_MAX_STAGES + 3) * 8;
+        g.off_tab = round_up_i(g.off_bar + (4 * TC_MAX_STAGES + 3) * 8, 16);
+        smem = static_cast<size_t>(g.off_tab) + TC_MAX_MMA_PER_CHUNK * 8;
         if (smem > 220 * 1024) return BS_ERR_UNSUPPORTED;
     }
     g.tiles_o = ceil_div(p->O, g.TN);
