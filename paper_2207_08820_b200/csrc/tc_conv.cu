@@ -521,7 +521,7 @@ constexpr int TCP_NSP = 3;            // packed-tile ring (at most)
 constexpr int TCP_NSE = 3;            // expanded-chunk ring (at most)
 
 template <int A>
-__global__ void __launch_bounds__(TCP_THREADS) bitserial_conv_tc_persistent_kernel(const __grid_constant__ TcArgs g)
+__global__ void __launch_bounds__(TCP_THREADS, 3) bitserial_conv_tc_persistent_kernel(const __grid_constant__ TcArgs g)
 {
     extern __shared__ __align__(128) unsigned char tc_smem[];
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -835,7 +835,7 @@ static int tc_conv_impl(const uint32_t* act, const int8_t* wgt, const bs_conv_pa
         const long long pairs = tiles_m * ceil_div(p->O, TN);
         if (TN > 32 && pairs < sms) continue;
         const size_t wbytes = static_cast<size_t>(g.nchunks) * TN * RS * g.CK;
-        const int shapes[4][2] = {{3, 3}, {2, 3}, {2, 2}, {1, 2}};      // (packed-tile stages, expanded-chunk stages)
+        const int shapes[4][2] = {{2, 2}, {2, 2}, {2, 2}, {1, 2}};      // (packed-tile stages, expanded-chunk stages)
         for (const auto& sh : shapes) {
             const int nsp = sh[0], nse = sh[1];
             const size_t total = wbytes + static_cast<size_t>(nsp) * g.pa_bytes + static_cast<size_t>(nse) * g.e_bytes +
@@ -908,7 +908,10 @@ static int tc_conv_impl(const uint32_t* act, const int8_t* wgt, const bs_conv_pa
     if (cr != CUDA_SUCCESS) return BS_ERR_CUDA;
 
     if (g.persistent) {
-        const int cps = smem <= 110 * 1024 ? 2 : 1;                        // CTAs that fit on one SM
+        int cps = static_cast<int>((225 * 1024) / (smem + 1024));          // CTAs that fit on one SM: shared memory,
+        if (cps > 3) cps = 3;                                              // registers (launch bounds) and
+        if (cps * 2 * g.TN > 512) cps = 512 / (2 * g.TN);                  // tensor-memory columns
+        if (cps < 1) cps = 1;
         long long per_o = (static_cast<long long>(sms) * cps) / g.tiles_o;
         if (per_o < 1) per_o = 1;
         if (per_o > tiles_m) per_o = tiles_m;
