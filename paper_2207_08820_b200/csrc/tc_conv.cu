@@ -853,10 +853,14 @@ static int tc_conv_impl(const uint32_t* act, const int8_t* wgt, const bs_conv_pa
         }
         if (g.persistent) break;
     }
+    // A resident plan that had to shrink the filter tile to 32 wastes the tensor core (an N = 32 MMA costs as many
+    // cycles as N = 64): stream the filters instead when a 128-wide tile leaves enough (pixel tile, filter tile) pairs.
+    if (g.persistent && g.TN == 32 && p->O >= 128 && tiles_m * ceil_div(p->O, 128) >= sms / 2) g.persistent = 0;
     if (!g.persistent) {
-        // one tile per CTA, filters streamed with every chunk: as many filters as keep the grid at two or more waves
+        // one tile per CTA, filters streamed with every chunk: the widest filter tile that keeps about one pair per SM
+        g.nsp = g.nse = g.nchunks < TC_MAX_STAGES ? g.nchunks : TC_MAX_STAGES;
         int TN = 128;
-        while (TN > 32 && (TN / 2 >= round_up_i(p->O, 32) || tiles_m * ceil_div(p->O, TN) < 2LL * sms)) TN /= 2;
+        while (TN > 32 && (TN / 2 >= round_up_i(p->O, 32) || tiles_m * ceil_div(p->O, TN) < sms / 2)) TN /= 2;
         for (;; TN /= 2) {
             g.TN = TN;
             g.b_bytes = TN * RS * g.CK;
