@@ -50,7 +50,7 @@ struct TcArgs {
     int tiles_o, tiles_q, tiles_p, tiles_n;
     int opad8;                        // padded filter count / 8 in the prepared weights
     int pa_bytes, pa_tx_bytes, b_bytes, e_bytes;   // per stage (pa_tx_bytes: bytes the activation box delivers)
-    int off_p, off_e, off_sb, off_bar, off_tab;   // shared-memory offsets (bytes)
+    int off_p, off_e, off_sb, off_bar, off_tab, off_lut;   // shared-memory offsets (bytes)
     int persistent;
     int tmem_cols;
     unsigned idesc;
@@ -72,13 +72,13 @@ __device__ __forceinline__ void group_sync(int id) { asm volatile("bar.sync %0, 
 __device__ __forceinline__ bool mbar_spin_bounded(uint64_t* bar, unsigned parity)
 {
     const uint32_t addr = smem_u32(bar);
-    for (unsigned it = 0; it < (1u << 26); ++it) {
+    for (unsigned it = 0; it < (1u << 24); ++it) {
         unsigned ok;
         asm volatile(
             "{\n\t.reg .pred p;\n\t"
-            "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+            "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
             "selp.u32 %0, 1, 0, p;\n\t}"
-            : "=r"(ok) : "r"(addr), "r"(parity) : "memory");
+            : "=r"(ok) : "r"(addr), "r"(parity), "r"(2000u) : "memory");     // park for at most ~2 us per attempt
         if (ok) return true;
     }
     return false;
@@ -193,31 +193,52 @@ __device__ __forceinline__ void tc_load_tile(const TcArgs& g, void* dst, uint64_
     }
 }
 
-// Expansion of channel chunk c of the staged tile: bitplanes of (pixel, 32-channel word) -> 32 int8 values, written as two 16-byte rows
-// of the K-major core-matrix layout [16-channel group][halo pixel][16 bytes].  `et` = 0..127 within the expander group.
-template <int A>
-__device__ __forceinline__ void tc_expand_chunk(const TcArgs& g, const uint32_t* pa, unsigned char* eb, int et, int c)
+// Byte look-up table of the expansion: entry [j][b] holds, for the eight bits of byte b of plane j, eight int8 lanes
+// with value mul[j] where the bit is set (two 32-bit words).  Adding the entries of all planes gives eight codes at once.
+constexpr int TC_LUT_BYTES_PER_PLANE = 256 * 8;
+
+__device__ __forceinline__ void tc_build_lut(const TcArgs& g, uint2* lut, int tid, int nthreads)
 {
-    const int items = g.flat ? TC_M * g.CWC : g.TNI * g.hh * g.hw * g.CWC;
+    for (int e = tid; e < g.A * 256; e += nthreads) {
+        const unsigned b = e & 255u, m = g.mul[e >> 8];
+        const unsigned lo = (((b & 0xFu) * 0x00204081u) & 0x01010101u) * m;
+        const unsigned hi = (((b >> 4) * 0x00204081u) & 0x01010101u) * m;
+        lut[e] = make_uint2(lo, hi);
+    }
+}
+
+// Expansion of channel chunk c of the staged tile: bitplanes of (pixel, 32-channel word) -> 32 int8 values, written as
+// two 16-byte rows of the K-major core-matrix layout [16-channel group][halo pixel][16 bytes].  `et` = 0..127 within
+// the expander group.  A 1x1 stride-2 layer only ever reads even halo rows and columns, so only those are expanded.
+template <int A>
+__device__ __forceinline__ void tc_expand_chunk(const TcArgs& g, const uint32_t* pa, unsigned char* eb, const uint2* lut, int et, int c)
+{
+    const int step = (!g.flat && g.R == 1 && g.stride == 2) ? 2 : 1;
+    const int nx = g.flat ? TC_M : (g.hw + step - 1) / step;
+    const int ny = g.flat ? 1 : (g.TNI * g.hh + step - 1) / step;      // hh is even for stride 2, so rows of all images keep their parity
+    const int items = nx * ny * g.CWC;
     for (int it = et; it < items; it += 128) {
-        const int cw = it % g.CWC, hp = it / g.CWC;
-        int ep = hp;
+        const int cw = it % g.CWC, pp = it / g.CWC;
+        int hp = pp, ep = pp;
         if (!g.flat) {
-            const int hy = hp / g.hw, hx = hp - hy * g.hw;
+            const int y2 = pp / nx, x2 = pp - y2 * nx;
+            const int hy = y2 * step, hx = x2 * step;
+            hp = hy * g.hw + hx;
             ep = hy * g.HWP + (g.stride == 2 ? (hx & 1) * g.HWH + (hx >> 1) : hx);
         }
         uint32_t w[A];
         load_planes<A>(pa + static_cast<size_t>(hp) * g.fullA + (c * g.CWC + cw) * A, w);
         uint32_t out[8];
 #pragma unroll
-        for (int nb = 0; nb < 8; ++nb) {
-            uint32_t acc = 0;
+        for (int q = 0; q < 4; ++q) {
+            uint2 acc = lut[(w[0] >> (8 * q)) & 0xFFu];
 #pragma unroll
-            for (int j = 0; j < A; ++j) {
-                const uint32_t sp = (((w[j] >> (4 * nb)) & 0xFu) * 0x00204081u) & 0x01010101u;
-                acc += sp * g.mul[j];
+            for (int j = 1; j < A; ++j) {
+                const uint2 t = lut[j * 256 + ((w[j] >> (8 * q)) & 0xFFu)];
+                acc.x += t.x; acc.y += t.y;
             }
-            out[nb] = acc ^ g.xormask;
+            out[2 * q] = acc.x ^ g.xormask;
+            out[2 * q + 1] = acc.y ^ g.xormask;
         }
         uint4* d0 = reinterpret_cast<uint4*>(eb + static_cast<size_t>(2 * cw) * g.HPE * 16 + static_cast<size_t>(ep) * 16);
         uint4* d1 = reinterpret_cast<uint4*>(eb + static_cast<size_t>(2 * cw + 1) * g.HPE * 16 + static_cast<size_t>(ep) * 16);
@@ -290,6 +311,32 @@ __device__ __forceinline__ void tc_issue_chunk(const TcIssue& is, const uint2* t
     }
 }
 
+// Comparison-form epilogue of 32 accumulators of one pixel: plane bits of the 1- or 2-bit code into ow[0], ow[1].
+template <bool SMALL, bool HAS_RES>
+__device__ __forceinline__ void tc_compare_block(const uint32_t (&v)[32], const float2* sb32, const float4* s_bounds, const float4 bnd0,
+                                                 const uint32_t (&rw)[4], int res_bits, uint32_t (&ow)[4])
+{
+    uint32_t w0 = 0, w1 = 0;
+#pragma unroll
+    for (int f = 0; f < 32; ++f) {
+        const int acc = static_cast<int>(v[f]);
+        const float2 sb = sb32[f];
+        const float t = fmaf(SMALL ? int_to_float_exact(acc) : static_cast<float>(acc), sb.x, sb.y);
+        float b0 = bnd0.x, b1 = bnd0.y, b2 = bnd0.z;
+        if (HAS_RES) {
+            unsigned rpat = ((rw[0] >> f) & 1u) | (((rw[1] >> f) & 1u) << 1);
+            if (res_bits > 2) rpat |= (((rw[2] >> f) & 1u) << 2) | (((rw[3] >> f) & 1u) << 3);
+            const float4 bb = s_bounds[rpat];
+            b0 = bb.x; b1 = bb.y; b2 = bb.z;
+        }
+        const uint32_t m1 = t >= b0 ? 0xffffffffu : 0u, m2 = t >= b1 ? 0xffffffffu : 0u, m3 = t >= b2 ? 0xffffffffu : 0u;
+        w0 |= (m1 ^ m2 ^ m3) & (1u << f);      // count = c1 + c2 + c3 with c1 >= c2 >= c3: bit 0 is the parity
+        w1 |= m2 & (1u << f);                  // bit 1 is c2
+    }
+    ow[0] = w0;
+    ow[1] = w1;
+}
+
 // Epilogue of one tile: thread `tid` (0..127, warp = TMEM lane quadrant) owns accumulator row tid = one output pixel.
 __device__ __forceinline__ void tc_epilogue_tile(const TcArgs& g, uint32_t tmem_acc, int tid, int warp, const TcTile& tile, int o0,
                                                  const float2* s_sb, const float4* s_bounds)
@@ -342,27 +389,16 @@ __device__ __forceinline__ void tc_epilogue_tile(const TcArgs& g, uint32_t tmem_
             }
             uint32_t ow[4] = {0, 0, 0, 0};
             if (g.rb.enabled) {
-                // comparison form: t = fmaf(acc, scale, bias) against the bounds of the residual pattern
+                // comparison form: t = fmaf(acc, scale, bias) against the bounds of the residual pattern.  The
+                // uniform switches are resolved once per 32 outputs, so the unrolled body is straight-line code.
                 const unsigned valid_mask = (g.O - ob >= 32) ? 0xffffffffu : ((1u << (g.O - ob)) - 1u);
-#pragma unroll
-                for (int f = 0; f < 32; ++f) {
-                    const int acc = static_cast<int>(v[f]);
-                    const float2 sb = s_sb[cc * 32 + f];
-                    const float t = fmaf(g.acc_small ? int_to_float_exact(acc) : static_cast<float>(acc), sb.x, sb.y);
-                    float b0, b1, b2;
-                    if (g.residual) {
-                        unsigned rpat = 0;
-#pragma unroll
-                        for (int j = 0; j < 4; ++j)
-                            if (j < g.res_bits) rpat |= ((rw[j] >> f) & 1u) << j;
-                        const float4 bb = s_bounds[rpat];
-                        b0 = bb.x; b1 = bb.y; b2 = bb.z;
-                    } else {
-                        b0 = bnd0.x; b1 = bnd0.y; b2 = bnd0.z;
-                    }
-                    const bool c1 = t >= b0, c2 = t >= b1, c3 = t >= b2;
-                    if ((c1 != c2) != c3) ow[0] |= 1u << f;
-                    if (c2) ow[1] |= 1u << f;
+                const float2* sb32 = s_sb + cc * 32;
+                if (g.residual) {
+                    if (g.acc_small) tc_compare_block<true, true>(v, sb32, s_bounds, bnd0, rw, g.res_bits, ow);
+                    else tc_compare_block<false, true>(v, sb32, s_bounds, bnd0, rw, g.res_bits, ow);
+                } else {
+                    if (g.acc_small) tc_compare_block<true, false>(v, sb32, s_bounds, bnd0, rw, g.res_bits, ow);
+                    else tc_compare_block<false, false>(v, sb32, s_bounds, bnd0, rw, g.res_bits, ow);
                 }
                 ow[0] = (ow[0] ^ ((g.rb.flip & 1u) ? 0xffffffffu : 0u)) & valid_mask;
                 ow[1] = (ow[1] ^ ((g.rb.flip & 2u) ? 0xffffffffu : 0u)) & valid_mask;
@@ -412,6 +448,7 @@ __global__ void __launch_bounds__(TC_THREADS) bitserial_conv_tc_kernel(const __g
     const int stage_p_bytes = g.b_bytes;                                    // filter ring; the packed tile sits at off_p
     float2* s_sb = reinterpret_cast<float2*>(tc_smem + g.off_sb);           // (scale, bias) per filter of the tile
     float4* s_bounds = reinterpret_cast<float4*>(tc_smem + g.off_sb + g.TN * 8);   // comparison bounds per residual pattern
+    uint2* s_lut = reinterpret_cast<uint2*>(tc_smem + g.off_lut);
     uint64_t* bars = reinterpret_cast<uint64_t*>(tc_smem + g.off_bar);
     uint64_t* full_p = bars;                       // [TC_MAX_STAGES]
     uint64_t* empty_p = bars + TC_MAX_STAGES;
@@ -445,6 +482,7 @@ __global__ void __launch_bounds__(TC_THREADS) bitserial_conv_tc_kernel(const __g
         s_sb[tid] = (g.out_packed && o < g.O) ? make_float2(g.scale[o], g.bias[o]) : make_float2(0.f, 0.f);
     }
     if (tid < 16) s_bounds[tid] = make_float4(g.rb.bound[tid][0], g.rb.bound[tid][1], g.rb.bound[tid][2], 0.f);
+    tc_build_lut(g, s_lut, tid, blockDim.x);
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
@@ -491,7 +529,7 @@ __global__ void __launch_bounds__(TC_THREADS) bitserial_conv_tc_kernel(const __g
             const int e = c % g.nse, k = c / g.nse;
             if (ok && k >= 1) ok = mbar_wait_warp(&empty_e[e], (k - 1) & 1, lane);
             if (!ok) atomicOr(g.status, STATUS_TIMEOUT);
-            tc_expand_chunk<A>(g, reinterpret_cast<const uint32_t*>(tc_smem + g.off_p), tc_smem + g.off_e + e * g.e_bytes, tid, c);
+            tc_expand_chunk<A>(g, reinterpret_cast<const uint32_t*>(tc_smem + g.off_p), tc_smem + g.off_e + e * g.e_bytes, s_lut, tid, c);
             fence_proxy_async();          // make the generic-proxy writes visible to the tensor core's reads
             group_sync(1);
             if (tid == 0) mbar_arrive(&full_e[e]);
@@ -531,6 +569,7 @@ __global__ void __launch_bounds__(TCP_THREADS, 3) bitserial_conv_tc_persistent_k
     unsigned char* s_e = tc_smem + g.off_e;                                    // [nse][e_bytes]
     float2* s_sb = reinterpret_cast<float2*>(tc_smem + g.off_sb);
     float4* s_bounds = reinterpret_cast<float4*>(tc_smem + g.off_sb + g.TN * 8);
+    uint2* s_lut = reinterpret_cast<uint2*>(tc_smem + g.off_lut);
     uint64_t* bars = reinterpret_cast<uint64_t*>(tc_smem + g.off_bar);
     uint64_t* full_p = bars;                        // [TCP_NSP]
     uint64_t* empty_p = bars + TCP_NSP;             // [TCP_NSP]
@@ -563,6 +602,7 @@ __global__ void __launch_bounds__(TCP_THREADS, 3) bitserial_conv_tc_persistent_k
         s_sb[tid] = (g.out_packed && o < g.O) ? make_float2(g.scale[o], g.bias[o]) : make_float2(0.f, 0.f);
     }
     if (tid < 16) s_bounds[tid] = make_float4(g.rb.bound[tid][0], g.rb.bound[tid][1], g.rb.bound[tid][2], 0.f);
+    tc_build_lut(g, s_lut, tid, blockDim.x);
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
@@ -624,7 +664,7 @@ __global__ void __launch_bounds__(TCP_THREADS, 3) bitserial_conv_tc_persistent_k
                 if (ok && k >= 1) ok = mbar_wait_warp(&empty_e[e], (k - 1) & 1, lane);
                 ok = group_all(1, ok);
                 if (!ok) break;
-                tc_expand_chunk<A>(g, reinterpret_cast<const uint32_t*>(s_p + s * g.pa_bytes), s_e + e * g.e_bytes, et, c);
+                tc_expand_chunk<A>(g, reinterpret_cast<const uint32_t*>(s_p + s * g.pa_bytes), s_e + e * g.e_bytes, s_lut, et, c);
                 fence_proxy_async();
                 group_sync(1);                       // all 128 expander threads have written and fenced
                 if (et == 0) mbar_arrive(&full_e[e]);
@@ -839,7 +879,7 @@ static int tc_conv_impl(const uint32_t* act, const int8_t* wgt, const bs_conv_pa
         for (const auto& sh : shapes) {
             const int nsp = sh[0], nse = sh[1];
             const size_t total = wbytes + static_cast<size_t>(nsp) * g.pa_bytes + static_cast<size_t>(nse) * g.e_bytes +
-                                 static_cast<size_t>(TN) * 8 + 256 + bar_bytes + 128 + TC_MAX_MMA_PER_CHUNK * 8 + 16;
+                                 static_cast<size_t>(TN) * 8 + 256 + bar_bytes + 128 + TC_MAX_MMA_PER_CHUNK * 8 + 16 + static_cast<size_t>(A) * TC_LUT_BYTES_PER_PLANE;
             if (total <= 220 * 1024) {
                 g.persistent = 1; g.TN = TN; g.b_bytes = TN * RS * g.CK; g.nse = nse; g.nsp = nsp;
                 g.off_p = static_cast<int>(wbytes);
@@ -847,7 +887,8 @@ static int tc_conv_impl(const uint32_t* act, const int8_t* wgt, const bs_conv_pa
                 g.off_sb = g.off_e + nse * g.e_bytes;
                 g.off_bar = round_up_i(g.off_sb + TN * 8 + 256, 16);
                 g.off_tab = round_up_i(g.off_bar + bar_bytes, 16);
-                smem = static_cast<size_t>(g.off_tab) + TC_MAX_MMA_PER_CHUNK * 8;
+                g.off_lut = g.off_tab + TC_MAX_MMA_PER_CHUNK * 8;
+                smem = static_cast<size_t>(g.off_lut) + static_cast<size_t>(A) * TC_LUT_BYTES_PER_PLANE;
                 break;
             }
         }
@@ -865,7 +906,7 @@ static int tc_conv_impl(const uint32_t* act, const int8_t* wgt, const bs_conv_pa
             g.TN = TN;
             g.b_bytes = TN * RS * g.CK;
             const size_t total = static_cast<size_t>(g.nsp) * g.b_bytes + g.pa_bytes + static_cast<size_t>(g.nse) * g.e_bytes +
-                                 2 * TN * 4 + 256 + (4 * TC_MAX_STAGES + 3) * 8 + 128 + TC_MAX_MMA_PER_CHUNK * 8 + 16;
+                                 2 * TN * 4 + 256 + (4 * TC_MAX_STAGES + 3) * 8 + 128 + TC_MAX_MMA_PER_CHUNK * 8 + 16 + static_cast<size_t>(A) * TC_LUT_BYTES_PER_PLANE;
             if (total <= 200 * 1024 || TN == 32) break;
         }
         g.off_p = g.nsp * g.b_bytes;
@@ -873,7 +914,8 @@ static int tc_conv_impl(const uint32_t* act, const int8_t* wgt, const bs_conv_pa
         g.off_sb = g.off_e + g.nse * g.e_bytes;
         g.off_bar = round_up_i(g.off_sb + 2 * g.TN * 4 + 256, 16);
         g.off_tab = round_up_i(g.off_bar + (4 * TC_MAX_STAGES + 3) * 8, 16);
-        smem = static_cast<size_t>(g.off_tab) + TC_MAX_MMA_PER_CHUNK * 8;
+        g.off_lut = g.off_tab + TC_MAX_MMA_PER_CHUNK * 8;
+        smem = static_cast<size_t>(g.off_lut) + static_cast<size_t>(A) * TC_LUT_BYTES_PER_PLANE;
         if (smem > 220 * 1024) return BS_ERR_UNSUPPORTED;
     }
     g.tiles_o = ceil_div(p->O, g.TN);
