@@ -210,21 +210,25 @@ __device__ __forceinline__ void tc_build_lut(const TcArgs& g, uint2* lut, int ti
 // Expansion of channel chunk c of the staged tile: bitplanes of (pixel, 32-channel word) -> 32 int8 values, written as
 // two 16-byte rows of the K-major core-matrix layout [16-channel group][halo pixel][16 bytes].  `et` = 0..127 within
 // the expander group.  A 1x1 stride-2 layer only ever reads even halo rows and columns, so only those are expanded.
-template <int A>
-__device__ __forceinline__ void tc_expand_chunk(const TcArgs& g, const uint32_t* pa, unsigned char* eb, const uint2* lut, int et, int c)
+// MODE: 0 flat tile, 1 2-D tile stride 1, 2 2-D tile stride 2, 3 2-D tile 1x1 stride 2 (even rows and columns only).
+// The mode is a template parameter so that the per-item body is straight-line code.
+template <int A, int MODE>
+__device__ __forceinline__ void tc_expand_items(const TcArgs& g, const uint32_t* pa, unsigned char* eb, const uint2* lut, int et, int c)
 {
-    const int step = (!g.flat && g.R == 1 && g.stride == 2) ? 2 : 1;
-    const int nx = g.flat ? TC_M : (g.hw + step - 1) / step;
-    const int ny = g.flat ? 1 : (g.TNI * g.hh + step - 1) / step;      // hh is even for stride 2, so rows of all images keep their parity
+    constexpr int step = MODE == 3 ? 2 : 1;
+    const int nx = MODE == 0 ? TC_M : (g.hw + step - 1) / step;
+    const int ny = MODE == 0 ? 1 : (g.TNI * g.hh + step - 1) / step;   // hh is even for stride 2: rows of all images keep their parity
     const int items = nx * ny * g.CWC;
+    const uint32_t xormask = g.xormask;
+    const int plane_bytes = g.HPE * 16;
     for (int it = et; it < items; it += 128) {
         const int cw = it % g.CWC, pp = it / g.CWC;
         int hp = pp, ep = pp;
-        if (!g.flat) {
+        if (MODE != 0) {
             const int y2 = pp / nx, x2 = pp - y2 * nx;
             const int hy = y2 * step, hx = x2 * step;
             hp = hy * g.hw + hx;
-            ep = hy * g.HWP + (g.stride == 2 ? (hx & 1) * g.HWH + (hx >> 1) : hx);
+            ep = hy * g.HWP + (MODE == 1 ? hx : (hx & 1) * g.HWH + (hx >> 1));
         }
         uint32_t w[A];
         load_planes<A>(pa + static_cast<size_t>(hp) * g.fullA + (c * g.CWC + cw) * A, w);
@@ -237,14 +241,22 @@ __device__ __forceinline__ void tc_expand_chunk(const TcArgs& g, const uint32_t*
                 const uint2 t = lut[j * 256 + ((w[j] >> (8 * q)) & 0xFFu)];
                 acc.x += t.x; acc.y += t.y;
             }
-            out[2 * q] = acc.x ^ g.xormask;
-            out[2 * q + 1] = acc.y ^ g.xormask;
+            out[2 * q] = acc.x ^ xormask;
+            out[2 * q + 1] = acc.y ^ xormask;
         }
-        uint4* d0 = reinterpret_cast<uint4*>(eb + static_cast<size_t>(2 * cw) * g.HPE * 16 + static_cast<size_t>(ep) * 16);
-        uint4* d1 = reinterpret_cast<uint4*>(eb + static_cast<size_t>(2 * cw + 1) * g.HPE * 16 + static_cast<size_t>(ep) * 16);
-        *d0 = make_uint4(out[0], out[1], out[2], out[3]);
-        *d1 = make_uint4(out[4], out[5], out[6], out[7]);
+        unsigned char* d = eb + static_cast<size_t>(2 * cw) * plane_bytes + static_cast<size_t>(ep) * 16;
+        *reinterpret_cast<uint4*>(d) = make_uint4(out[0], out[1], out[2], out[3]);
+        *reinterpret_cast<uint4*>(d + plane_bytes) = make_uint4(out[4], out[5], out[6], out[7]);
     }
+}
+
+template <int A>
+__device__ __forceinline__ void tc_expand_chunk(const TcArgs& g, const uint32_t* pa, unsigned char* eb, const uint2* lut, int et, int c)
+{
+    if (g.flat) tc_expand_items<A, 0>(g, pa, eb, lut, et, c);
+    else if (g.stride == 1) tc_expand_items<A, 1>(g, pa, eb, lut, et, c);
+    else if (g.R == 1) tc_expand_items<A, 3>(g, pa, eb, lut, et, c);
+    else tc_expand_items<A, 2>(g, pa, eb, lut, et, c);
 }
 
 // All MMAs of one chunk: R*S taps x CK/32 steps of K = 32; a tap only moves the descriptor start address.
@@ -312,9 +324,9 @@ __device__ __forceinline__ void tc_issue_chunk(const TcIssue& is, const uint2* t
 }
 
 // Comparison-form epilogue of 32 accumulators of one pixel: plane bits of the 1- or 2-bit code into ow[0], ow[1].
-template <bool SMALL, bool HAS_RES>
+template <bool SMALL, int RES>      // RES: 0 no residual, 1 residual of 1-2 bits, 2 residual of 3-4 bits
 __device__ __forceinline__ void tc_compare_block(const uint32_t (&v)[32], const float2* sb32, const float4* s_bounds, const float4 bnd0,
-                                                 const uint32_t (&rw)[4], int res_bits, uint32_t (&ow)[4])
+                                                 const uint32_t (&rw)[4], uint32_t (&ow)[4])
 {
     uint32_t w0 = 0, w1 = 0;
 #pragma unroll
@@ -323,9 +335,9 @@ __device__ __forceinline__ void tc_compare_block(const uint32_t (&v)[32], const 
         const float2 sb = sb32[f];
         const float t = fmaf(SMALL ? int_to_float_exact(acc) : static_cast<float>(acc), sb.x, sb.y);
         float b0 = bnd0.x, b1 = bnd0.y, b2 = bnd0.z;
-        if (HAS_RES) {
-            unsigned rpat = ((rw[0] >> f) & 1u) | (((rw[1] >> f) & 1u) << 1);
-            if (res_bits > 2) rpat |= (((rw[2] >> f) & 1u) << 2) | (((rw[3] >> f) & 1u) << 3);
+        if (RES != 0) {
+            unsigned rpat = ((rw[0] >> f) & 1u) | (((rw[1] >> f) & 1u) << 1);      // planes beyond res_bits are zero
+            if (RES == 2) rpat |= (((rw[2] >> f) & 1u) << 2) | (((rw[3] >> f) & 1u) << 3);
             const float4 bb = s_bounds[rpat];
             b0 = bb.x; b1 = bb.y; b2 = bb.z;
         }
@@ -393,12 +405,15 @@ __device__ __forceinline__ void tc_epilogue_tile(const TcArgs& g, uint32_t tmem_
                 // uniform switches are resolved once per 32 outputs, so the unrolled body is straight-line code.
                 const unsigned valid_mask = (g.O - ob >= 32) ? 0xffffffffu : ((1u << (g.O - ob)) - 1u);
                 const float2* sb32 = s_sb + cc * 32;
-                if (g.residual) {
-                    if (g.acc_small) tc_compare_block<true, true>(v, sb32, s_bounds, bnd0, rw, g.res_bits, ow);
-                    else tc_compare_block<false, true>(v, sb32, s_bounds, bnd0, rw, g.res_bits, ow);
+                if (!g.residual) {
+                    if (g.acc_small) tc_compare_block<true, 0>(v, sb32, s_bounds, bnd0, rw, ow);
+                    else tc_compare_block<false, 0>(v, sb32, s_bounds, bnd0, rw, ow);
+                } else if (g.res_bits <= 2) {
+                    if (g.acc_small) tc_compare_block<true, 1>(v, sb32, s_bounds, bnd0, rw, ow);
+                    else tc_compare_block<false, 1>(v, sb32, s_bounds, bnd0, rw, ow);
                 } else {
-                    if (g.acc_small) tc_compare_block<true, false>(v, sb32, s_bounds, bnd0, rw, g.res_bits, ow);
-                    else tc_compare_block<false, false>(v, sb32, s_bounds, bnd0, rw, g.res_bits, ow);
+                    if (g.acc_small) tc_compare_block<true, 2>(v, sb32, s_bounds, bnd0, rw, ow);
+                    else tc_compare_block<false, 2>(v, sb32, s_bounds, bnd0, rw, ow);
                 }
                 ow[0] = (ow[0] ^ ((g.rb.flip & 1u) ? 0xffffffffu : 0u)) & valid_mask;
                 ow[1] = (ow[1] ^ ((g.rb.flip & 2u) ? 0xffffffffu : 0u)) & valid_mask;
