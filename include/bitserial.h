@@ -203,8 +203,8 @@ int bitserial_gemm_noalloc(const uint32_t* a_packed, const uint32_t* w_packed, i
  * once by bs_tc_prepare_weights.  Results (accumulators and requantised codes) are bit-identical to
  * bitserial_conv2d / bitserial_gemm; the epilogue is the one documented at bs_conv_params.
  *   Supported subset (bs_tc_supported returns 1): C a multiple of 32 whose packed pixel record (C/32 * a_bits words)
- *   is a 16-byte multiple (a_bits 4: any such C; a_bits 2: C % 64 == 0; a_bits 1 or 3: C % 128 == 0), res_c_offset
- *   a multiple of 32; everything else as bitserial_conv2d.  Unsupported shapes return BS_ERR_UNSUPPORTED: use the
+ *   is a 16-byte multiple, or an 8-byte multiple when a packed image row (W records) is a 16-byte multiple and, for
+ *   1x1 stride-1 layers, N*H*W is even; res_c_offset a multiple of 32; everything else as bitserial_conv2d.  Unsupported shapes return BS_ERR_UNSUPPORTED: use the
  *   popcount entry points.
  *   bs_tc_weights_bytes    bytes of the prepared int8 filter tensor (0 on bad input).
  *   bs_tc_prepare_weights  packed weights [O][R][S][Cw][w_bits] -> int8 tiles [C/CK][ceil(O/128)*16][R*S][CK/16][8][16];

@@ -45,7 +45,9 @@ struct TcArgs {
     int TN, CK, CWC, nchunks, nsp, nse;
     int fullA;                        // words of one packed pixel record (Cw * A)
     int pmode;                        // how a tile's packed halo is fetched: 0 flat bulk copy, 1 rows merged with W, 2 4-D box
-    int TNI, GI, hh, hw;              // packed box: TNI images x hh rows x hw columns; GI row groups per image
+    int TNI, GI, hh, hw;              // packed halo: TNI images x hh rows x hw columns; GI row groups per image
+    int hwb, xsh;                     // row pitch of the staged halo in pixels, and pixels skipped at the start of a row
+                                      // (8-byte records: the box starts one pixel early to stay 16-byte aligned)
     int HWP, HWH, HPE;                // expanded layout: row pitch, half-row offset (stride 2), pixels per 16-channel plane
     int tiles_o, tiles_q, tiles_p, tiles_n;
     int opad8;                        // padded filter count / 8 in the prepared weights
@@ -188,7 +190,7 @@ __device__ __forceinline__ void tc_load_tile(const TcArgs& g, void* dst, uint64_
     } else {
         mbar_expect_tx(bar, static_cast<unsigned>(g.pa_tx_bytes));
         const int x0 = tile.q0 * g.stride - g.pad, y0 = tile.p0 * g.stride - g.pad;
-        if (g.pmode == 1) tma_load_3d(dst, &g.tmA, bar, x0 * g.fullA, y0, tile.n0);
+        if (g.pmode == 1) tma_load_3d(dst, &g.tmA, bar, (x0 - g.xsh) * g.fullA, y0, tile.n0);
         else tma_load_4d(dst, &g.tmA, bar, 0, x0, y0, tile.n0);
     }
 }
@@ -227,7 +229,7 @@ __device__ __forceinline__ void tc_expand_items(const TcArgs& g, const uint32_t*
         if (MODE != 0) {
             const int y2 = pp / nx, x2 = pp - y2 * nx;
             const int hy = y2 * step, hx = x2 * step;
-            hp = hy * g.hw + hx;
+            hp = hy * g.hwb + hx + g.xsh;
             ep = hy * g.HWP + (MODE == 1 ? hx : (hx & 1) * g.HWH + (hx >> 1));
         }
         uint32_t w[A];
@@ -791,7 +793,15 @@ static int tc_validate(const bs_conv_params* p)
     if (p->a_sign == BS_BIPOLAR && p->pad != 0) return BS_ERR_UNSUPPORTED;
     if (p->H + 2 * p->pad < p->R || p->W + 2 * p->pad < p->S) return BS_ERR_INVALID_ARG;
     if (p->C % 32 != 0 || tc_chunk_channels(p->C, p->a_bits) == 0) return BS_ERR_UNSUPPORTED;
-    if ((ceil_div(p->C, 32) * p->a_bits) % 4 != 0) return BS_ERR_UNSUPPORTED;
+    {
+        // packed pixel records must be 16-byte multiples, or 8-byte multiples on rows that are 16-byte multiples
+        const int fullA = ceil_div(p->C, 32) * p->a_bits;
+        const bool flat = p->R == 1 && p->stride == 1 && p->pad == 0;
+        if (fullA % 4 != 0) {
+            if (fullA % 2 != 0 || (p->W * fullA) % 4 != 0) return BS_ERR_UNSUPPORTED;
+            if (flat && (static_cast<long long>(p->N) * p->H * p->W) % 2 != 0) return BS_ERR_UNSUPPORTED;
+        }
+    }
     const long long kred = static_cast<long long>(p->C) * p->R * p->S;
     if (kred * tc_max_abs(p->a_bits, p->a_sign) * tc_max_abs(p->w_bits, p->w_sign) >= (1LL << 31)) return BS_ERR_UNSUPPORTED;
     return BS_OK;
@@ -848,12 +858,14 @@ static int tc_conv_impl(const uint32_t* act, const int8_t* wgt, const bs_conv_pa
         const long long npix = static_cast<long long>(p->N) * p->H * p->W;
         if (npix > 0x7fffffffLL) return BS_ERR_UNSUPPORTED;
         g.tiles_q = static_cast<int>(ceil_div_ll(npix, TC_M)); g.tiles_p = 1; g.tiles_n = 1;
-        g.TNI = 1; g.GI = 16; g.hh = 1; g.hw = TC_M; g.HWP = TC_M; g.HWH = 0; g.HPE = TC_M;
+        g.TNI = 1; g.GI = 16; g.hh = 1; g.hw = TC_M; g.hwb = TC_M; g.xsh = 0; g.HWP = TC_M; g.HWH = 0; g.HPE = TC_M;
         g.pa_tx_bytes = TC_M * g.fullA * 4;
         g.pmode = 0;
         tiles_m = g.tiles_q;
     } else {
         g.hw = 7 * p->stride + p->S;
+        g.xsh = (g.fullA % 4 != 0 && (p->pad & 1)) ? 1 : 0;
+        g.hwb = g.fullA % 4 != 0 ? round_up_i(g.hw + g.xsh, 2) : g.hw;
         g.HWH = (g.hw + 1) / 2;
         g.HWP = p->stride == 2 ? 2 * g.HWH : g.hw;
         if (g.P <= 16) {        // whole image height in one tile; stack as many images as fit in the 16 row groups
@@ -872,9 +884,9 @@ static int tc_conv_impl(const uint32_t* act, const int8_t* wgt, const bs_conv_pa
         const int rows_box = g.TNI * g.hh;
         const int rows_read = 15 * p->stride + p->R;
         g.HPE = (rows_box > rows_read ? rows_box : rows_read) * g.HWP;
-        g.pa_tx_bytes = g.TNI * g.hh * g.hw * g.fullA * 4;
-        g.pmode = (g.hw * g.fullA <= 256) ? 1 : 2;
-        if (g.pmode == 2 && g.fullA > 256) return BS_ERR_UNSUPPORTED;
+        g.pa_tx_bytes = g.TNI * g.hh * g.hwb * g.fullA * 4;
+        g.pmode = (g.hwb * g.fullA <= 256) ? 1 : 2;
+        if (g.pmode == 2 && (g.fullA > 256 || g.fullA % 4 != 0)) return BS_ERR_UNSUPPORTED;
         tiles_m = static_cast<long long>(g.tiles_q) * g.tiles_p * g.tiles_n;
     }
     g.pa_bytes = round_up_i(g.pa_tx_bytes, 128);
@@ -953,7 +965,7 @@ static int tc_conv_impl(const uint32_t* act, const int8_t* wgt, const bs_conv_pa
     if (g.pmode == 1) {
         cuuint64_t dims[3] = {fullA * p->W, static_cast<cuuint64_t>(p->H), static_cast<cuuint64_t>(p->N)};
         cuuint64_t strides[2] = {fullA * 4 * p->W, fullA * 4 * p->W * p->H};
-        cuuint32_t box[3] = {static_cast<cuuint32_t>(g.hw * g.fullA), static_cast<cuuint32_t>(g.hh), static_cast<cuuint32_t>(g.TNI)};
+        cuuint32_t box[3] = {static_cast<cuuint32_t>(g.hwb * g.fullA), static_cast<cuuint32_t>(g.hh), static_cast<cuuint32_t>(g.TNI)};
         cr = enc(&g.tmA, CU_TENSOR_MAP_DATA_TYPE_UINT32, 3, const_cast<uint32_t*>(act), dims, strides, box, estr,
                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);

@@ -67,6 +67,17 @@ def test_tc_channel_counts_multi_chunk(C, O):
     assert np.array_equal(packed, oracle.pack_activations(codes, 2, 0))
 
 
+@pytest.mark.parametrize("k,stride,pad", [(1, 1, 0), (3, 1, 1), (3, 2, 1), (1, 2, 0), (3, 1, 0)])
+def test_tc_eight_byte_records(k, stride, pad):
+    """C = 32 with 2-bit activations: 8-byte pixel records (detection-stack first stage)."""
+    c = wl.single_conv_case(seed=40 + k + stride, N=2, C=32, H=20, W=22, O=64, k=k, stride=stride, pad=pad, calibrated=True)
+    acc, packed = run_tc(c)
+    want = oracle.conv2d_i32(c["x"], c["w"], stride, pad)
+    assert np.array_equal(acc, want)
+    codes = oracle.requantize(want, c["scale"], c["bias"], True, 2, 0)
+    assert np.array_equal(packed, oracle.pack_activations(codes, 2, 0))
+
+
 def test_tc_residual_matches_oracle_and_popcount_path():
     c = wl.single_conv_case(seed=9, N=2, C=64, H=12, W=12, O=64, calibrated=True)
     rng = np.random.default_rng(4)
@@ -90,6 +101,8 @@ def test_tc_gemm(M, N, K):
 
 
 def test_tc_unsupported_shape_is_refused():
-    assert not api.tc_supported(1, 32, 8, 8, 32, 3, 1, 1, 2, 0, 2, 1)       # 8-byte pixel records cannot be a TMA box
+    assert api.tc_supported(1, 32, 8, 8, 32, 3, 1, 1, 2, 0, 2, 1)           # 8-byte records on 16-byte rows are fine
+    assert not api.tc_supported(1, 32, 8, 7, 32, 3, 1, 1, 2, 0, 2, 1)       # ... but not on odd-width images
+    assert not api.tc_supported(1, 32, 8, 8, 32, 3, 1, 1, 1, 0, 2, 1)       # 4-byte records cannot be fetched in bulk
     assert not api.tc_supported(1, 40, 8, 8, 32, 3, 1, 1, 4, 0, 2, 1)       # C not a multiple of 32
     assert api.tc_supported(1, 64, 8, 8, 32, 3, 1, 1, 2, 0, 2, 1)
