@@ -216,6 +216,17 @@ int bs_tc_prepare_weights(const uint32_t* wgt_packed, int O, int C, int R, int S
 int bs_tc_supported(const bs_conv_params* p);
 int bitserial_conv2d_tc(const uint32_t* act_packed, const int8_t* wgt_tc, const bs_conv_params* p, int32_t* out_i32,
                         uint32_t* out_packed, void* stream);
+/*
+ * bitserial_conv2d_tc_chained -- bitserial_conv2d_tc for a layer inside a chain of layers on one stream (the paper
+ * runs a network layer by layer, Section V; overlapping consecutive layers is this library's addition).  The kernel
+ * is launched so that its set-up (barriers, tensor memory, filter fetch, scale/bias fetch) may run while the
+ * preceding kernel of `stream` is still finishing; activations and the residual are read, and outputs written,
+ * only after that kernel has completed.  The CALLER PROMISES that wgt_tc, p->scale and p->bias were final before
+ * the preceding kernel of the stream was launched (e.g. prepared at model load time, followed by a
+ * synchronisation).  Results are identical to bitserial_conv2d_tc; errors likewise.  Works under stream capture.
+ */
+int bitserial_conv2d_tc_chained(const uint32_t* act_packed, const int8_t* wgt_tc, const bs_conv_params* p,
+                                int32_t* out_i32, uint32_t* out_packed, void* stream);
 int bitserial_gemm_tc(const uint32_t* a_packed, const int8_t* w_tc, int M, int N, int K, int a_bits, bs_sign_t a_sign,
                       int w_bits, bs_sign_t w_sign, const float* scale, const float* bias, int relu, int out_bits,
                       bs_sign_t out_sign, int32_t* out_i32, uint32_t* out_packed, void* stream);

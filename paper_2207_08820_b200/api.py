@@ -113,11 +113,14 @@ def bitserial_conv2d(act_packed: torch.Tensor, wgt_packed: torch.Tensor, *, C: i
                      res_bits: int = 0, res_sign: int = UNSIGNED, res_c_offset: int = 0, res_c_total: int = 0,
                      out_i32: Optional[torch.Tensor] = None, want_i32: bool = False, i32_layout: int = NCHW,
                      out_packed: Optional[torch.Tensor] = None, out_c_offset: int = 0, out_c_total: int = 0,
-                     workspace: Optional[torch.Tensor] = None, wgt_tc: Optional[torch.Tensor] = None, stream=None):
+                     workspace: Optional[torch.Tensor] = None, wgt_tc: Optional[torch.Tensor] = None, chained: bool = False,
+                     stream=None):
     """act_packed [N,H,W,Cw,a_bits], wgt_packed [O,R,S,Cw,w_bits].  Returns (out_i32 or None, out_packed or None).
     A packed output is produced when ``out_bits`` > 0 (allocated here unless ``out_packed`` is given).
     ``workspace`` (zeroed device tensor, see :func:`conv_workspace`) enables the reduction split (``bitserial_conv2d_ws``).
-    ``wgt_tc`` (from :func:`tc_prepare_weights`) selects the tensor-core entry point ``bitserial_conv2d_tc``."""
+    ``wgt_tc`` (from :func:`tc_prepare_weights`) selects the tensor-core entry point ``bitserial_conv2d_tc``;
+    with ``chained`` it is ``bitserial_conv2d_tc_chained`` (set-up overlaps the preceding kernel of the stream: filters,
+    scale and bias must have been final before that kernel was launched)."""
     N, H, W, Cw, a_bits = act_packed.shape
     O, R, S, Cw2, w_bits = wgt_packed.shape
     if Cw != Cw2 or Cw != (C + 31) // 32:
@@ -140,8 +143,9 @@ def bitserial_conv2d(act_packed: torch.Tensor, wgt_packed: torch.Tensor, *, C: i
                    res_c_total=res_c_total if res_c_total else res_c_offset + O,
                    out_c_offset=out_c_offset, out_c_total=out_c_total, i32_layout=i32_layout)
     if wgt_tc is not None:
-        st = lib().bitserial_conv2d_tc(_ptr(act_packed), _ptr(wgt_tc), ctypes.byref(p), _ptr(out_i32),
-                                       _ptr(out_packed) if out_bits > 0 else None, _stream_ptr(stream))
+        entry = lib().bitserial_conv2d_tc_chained if chained else lib().bitserial_conv2d_tc
+        st = entry(_ptr(act_packed), _ptr(wgt_tc), ctypes.byref(p), _ptr(out_i32),
+                   _ptr(out_packed) if out_bits > 0 else None, _stream_ptr(stream))
     elif workspace is not None:
         st = lib().bitserial_conv2d_ws(_ptr(act_packed), _ptr(wgt_packed), ctypes.byref(p), _ptr(out_i32),
                                        _ptr(out_packed) if out_bits > 0 else None, _ptr(workspace),

@@ -105,6 +105,12 @@ __device__ __forceinline__ bool mbar_wait_warp(uint64_t* bar, unsigned parity, i
     if (lane == 0) ok = mbar_spin_bounded(bar, parity) ? 1u : 0u;
     return __shfl_sync(0xffffffffu, ok, 0) != 0;
 }
+// Programmatic dependent launch: `pdl_release` lets the next kernel of the stream start its prologue once every CTA of
+// this grid has passed it; `pdl_acquire` returns when the preceding grid has completed and its writes are visible.
+// Both are no-ops when the launches involved do not carry the programmatic-serialisation attribute.
+__device__ __forceinline__ void pdl_release() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void pdl_acquire() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
 __device__ __forceinline__ void tmem_alloc(uint32_t* slot, unsigned ncols)
 {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(slot)), "r"(ncols) : "memory");
@@ -478,6 +484,7 @@ __global__ void __launch_bounds__(TC_THREADS) bitserial_conv_tc_kernel(const __g
     const int o0 = static_cast<int>(blockIdx.x % static_cast<unsigned>(g.tiles_o)) * g.TN;   // filter tile fastest
     const TcTile tile = tc_decode_tile(g, static_cast<int>(blockIdx.x / static_cast<unsigned>(g.tiles_o)));
 
+    pdl_release();
     if (tid == 0) {
         for (int s = 0; s < TC_MAX_STAGES; ++s) {
             mbar_init(&full_p[s], 1);
@@ -508,14 +515,17 @@ __global__ void __launch_bounds__(TC_THREADS) bitserial_conv_tc_kernel(const __g
     if (warp == 4) {
         // ------------------------------------------------------------------ producer
         if (lane == 0) {
-            tc_load_tile(g, tc_smem + g.off_p, full_a, tile);
+            // the first ring of filter chunks does not depend on the preceding kernel: fetch it before waiting for it
+            const int early = g.nchunks < g.nsp ? g.nchunks : g.nsp;
             for (int c = 0; c < g.nchunks; ++c) {
                 const int s = c % g.nsp, k = c / g.nsp;
+                if (c == early) { pdl_acquire(); tc_load_tile(g, tc_smem + g.off_p, full_a, tile); }
                 if (k >= 1 && !mbar_spin_bounded(&empty_p[s], (k - 1) & 1)) { atomicOr(g.status, STATUS_TIMEOUT); break; }
                 mbar_expect_tx(&full_p[s], static_cast<unsigned>(g.b_bytes));
                 const size_t src = (static_cast<size_t>(c) * g.opad8 + (o0 >> 3)) * RS * (g.CK >> 4) * 128;
                 bulk_load(tc_smem + s * stage_p_bytes, g.wgt + src, static_cast<unsigned>(g.b_bytes), &full_p[s]);
             }
+            if (early == g.nchunks) { pdl_acquire(); tc_load_tile(g, tc_smem + g.off_p, full_a, tile); }
         }
         __syncwarp();
     } else if (warp == 5) {
@@ -541,6 +551,7 @@ __global__ void __launch_bounds__(TC_THREADS) bitserial_conv_tc_kernel(const __g
         __syncwarp();
     } else {
         // ------------------------------------------------------------------ expanders (warps 0-3), then epilogue
+        pdl_acquire();                    // the epilogue reads the residual and overwrites buffers the preceding kernel may use
         bool ok = mbar_wait_warp(full_a, 0, lane);
         for (int c = 0; c < g.nchunks; ++c) {
             const int e = c % g.nse, k = c / g.nse;
@@ -602,6 +613,7 @@ __global__ void __launch_bounds__(TCP_THREADS, 3) bitserial_conv_tc_persistent_k
     const int tile_step = static_cast<int>(gridDim.x / static_cast<unsigned>(g.tiles_o));
     const int tiles_m = g.tiles_q * g.tiles_p * g.tiles_n;
 
+    pdl_release();
     if (tid == 0) {
         for (int s = 0; s < TCP_NSP; ++s) { mbar_init(&full_p[s], 1); mbar_init(&empty_p[s], 1); }
         for (int s = 0; s < TCP_NSE; ++s) { mbar_init(&full_e[s], 1); mbar_init(&empty_e[s], 1); }
@@ -633,6 +645,7 @@ __global__ void __launch_bounds__(TCP_THREADS, 3) bitserial_conv_tc_persistent_k
                 const size_t src = (static_cast<size_t>(c) * g.opad8 + (o0 >> 3)) * RS * (g.CK >> 4) * 128;
                 bulk_load(s_w + static_cast<size_t>(c) * g.b_bytes, g.wgt + src, static_cast<unsigned>(g.b_bytes), wgt_full);
             }
+            pdl_acquire();                // activations come from the preceding kernel; the filters above do not
             int i = 0;
             bool ok = true;
             for (int mt = first_tile; mt < tiles_m && ok; mt += tile_step, ++i) {
@@ -691,6 +704,7 @@ __global__ void __launch_bounds__(TCP_THREADS, 3) bitserial_conv_tc_persistent_k
         if (!ok) atomicOr(g.status, STATUS_TIMEOUT);
     } else {
         // ------------------------------------------------------------------ epilogue (warps 0-3)
+        pdl_acquire();                    // the epilogue reads the residual and overwrites buffers the preceding kernel may use
         int i = 0;
         bool ok = true;
         for (int mt = first_tile; mt < tiles_m && ok; mt += tile_step, ++i) {
@@ -807,8 +821,27 @@ static int tc_validate(const bs_conv_params* p)
     return BS_OK;
 }
 
+// Launch with or without the programmatic-serialisation attribute.  With it, the grid may begin (barrier and TMEM
+// set-up, byte table, filter fetch) while the preceding kernel of the stream drains; everything it reads before
+// pdl_acquire() must therefore have been final before that preceding kernel was launched.
+static cudaError_t tc_launch(void (*kern)(TcArgs), unsigned grid, unsigned block, size_t smem, cudaStream_t st, bool chained,
+                             const TcArgs& g)
+{
+    cudaLaunchConfig_t cfg{};
+    cfg.gridDim = dim3(grid);
+    cfg.blockDim = dim3(block);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = chained ? 1 : 0;
+    return cudaLaunchKernelEx(&cfg, kern, g);
+}
+
 static int tc_conv_impl(const uint32_t* act, const int8_t* wgt, const bs_conv_params* p, int32_t* out_i32, uint32_t* out_packed,
-                        cudaStream_t st)
+                        cudaStream_t st, bool chained = false)
 {
     int rc = tc_validate(p);
     if (rc != BS_OK) return rc;
@@ -1001,8 +1034,11 @@ static int tc_conv_impl(const uint32_t* act, const int8_t* wgt, const bs_conv_pa
             cudaGetLastError();
             return BS_ERR_CUDA;
         }
-        kern<<<static_cast<unsigned>(grid), TCP_THREADS, smem, st>>>(g);
-        return cudaGetLastError() == cudaSuccess ? BS_OK : BS_ERR_CUDA;
+        if (tc_launch(kern, static_cast<unsigned>(grid), TCP_THREADS, smem, st, chained, g) != cudaSuccess) {
+            cudaGetLastError();
+            return BS_ERR_CUDA;
+        }
+        return BS_OK;
     }
     const long long grid = tiles_m * g.tiles_o;
     if (grid > 0x7fffffffLL) return BS_ERR_UNSUPPORTED;
@@ -1018,8 +1054,11 @@ static int tc_conv_impl(const uint32_t* act, const int8_t* wgt, const bs_conv_pa
         cudaGetLastError();
         return BS_ERR_CUDA;
     }
-    kern<<<static_cast<unsigned>(grid), TC_THREADS, smem, st>>>(g);
-    return cudaGetLastError() == cudaSuccess ? BS_OK : BS_ERR_CUDA;
+    if (tc_launch(kern, static_cast<unsigned>(grid), TC_THREADS, smem, st, chained, g) != cudaSuccess) {
+        cudaGetLastError();
+        return BS_ERR_CUDA;
+    }
+    return BS_OK;
 }
 
 }  // namespace bs
@@ -1053,6 +1092,12 @@ extern "C" int bitserial_conv2d_tc(const uint32_t* act_packed, const int8_t* wgt
                                    uint32_t* out_packed, void* stream)
 {
     return bs::tc_conv_impl(act_packed, wgt_tc, p, out_i32, out_packed, static_cast<cudaStream_t>(stream));
+}
+
+extern "C" int bitserial_conv2d_tc_chained(const uint32_t* act_packed, const int8_t* wgt_tc, const bs_conv_params* p,
+                                           int32_t* out_i32, uint32_t* out_packed, void* stream)
+{
+    return bs::tc_conv_impl(act_packed, wgt_tc, p, out_i32, out_packed, static_cast<cudaStream_t>(stream), true);
 }
 
 extern "C" int bitserial_gemm_tc(const uint32_t* a_packed, const int8_t* w_tc, int M, int N, int K, int a_bits, bs_sign_t a_sign,

@@ -43,6 +43,7 @@ class BitserialNet:
         self.bufs: Dict[str, torch.Tensor] = {}
         for name, (C, H, W) in self.shapes.items():
             self.bufs[name] = torch.zeros(self.batch, H, W, (C + 31) // 32, net.a_bits, dtype=torch.int32, device=self.device)
+        torch.cuda.synchronize(self.device)   # chained layers fetch filters, scale and bias ahead of stream order
         self.graph = None
         self.static_in = None
         self.launches_per_forward = 1 + len(self.layers)
@@ -59,7 +60,7 @@ class BitserialNet:
                 out_sign=api.UNSIGNED, residual=res, res_scale=L.res_scale, res_bits=net.a_bits if L.res else 0,
                 res_sign=api.UNSIGNED, res_c_offset=0, res_c_total=self.shapes[L.res][0] if L.res else 0,
                 out_packed=self.bufs[L.dst], out_c_offset=L.dst_c_offset, out_c_total=self.shapes[L.dst][0],
-                wgt_tc=item["w_tc"])
+                wgt_tc=item["w_tc"], chained=item["w_tc"] is not None)
         return self.bufs[net.out_name]
 
     def forward(self, x: torch.Tensor) -> torch.Tensor:

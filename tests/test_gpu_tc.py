@@ -78,6 +78,34 @@ def test_tc_eight_byte_records(k, stride, pad):
     assert np.array_equal(packed, oracle.pack_activations(codes, 2, 0))
 
 
+def test_tc_chained_layers_match_oracle():
+    """Three dependent layers launched back to back through the chained entry point (set-up overlapping the
+    preceding kernel) give the oracle's codes, residual from the first tensor included."""
+    rng = np.random.default_rng(77)
+    N, C, H, W = 8, 64, 28, 28
+    codes0 = wl.rand_codes(rng, (N, C, H, W), 2, wl.UNSIGNED)
+    ws = [wl.rand_weights_zero_mean(rng, (C, C, 3, 3), 2, wl.SIGNED) for _ in range(3)]
+    sb = [wl.calibrated_scale_bias(w, 2, 0, 2, res_scale=0.5 if i == 2 else 0.0, res_bits=2 if i == 2 else 0)
+          for i, w in enumerate(ws)]
+    x0 = api.bitpack_activations(dev(codes0), 1.0, 2, api.UNSIGNED, api.NCHW)
+    wp = [api.pack_weights(dev(w), 2, api.SIGNED) for w in ws]
+    wt = [api.tc_prepare_weights(p, C, api.SIGNED, 2) for p in wp]
+    sc = [(dev(s), dev(b)) for s, b in sb]
+    torch.cuda.synchronize()
+    for rep in range(3):
+        cur = x0
+        for i in range(3):
+            _, cur = api.bitserial_conv2d(cur, wp[i], C=C, stride=1, pad=1, w_sign=api.SIGNED, scale=sc[i][0], bias=sc[i][1],
+                                          relu=True, out_bits=2, residual=x0 if i == 2 else None, res_scale=0.5 if i == 2 else 0.0,
+                                          res_bits=2 if i == 2 else 0, res_c_total=C, wgt_tc=wt[i], chained=True)
+    api.bs_check_status()
+    ref = codes0
+    for i in range(3):
+        acc = oracle.conv2d_i32(ref, ws[i], 1, 1)
+        ref = oracle.requantize(acc, sb[i][0], sb[i][1], True, 2, 0, res=codes0 if i == 2 else None, res_scale=0.5 if i == 2 else 0.0)
+    assert np.array_equal(cur.cpu().numpy().view(np.uint32), oracle.pack_activations(ref, 2, 0))
+
+
 def test_tc_residual_matches_oracle_and_popcount_path():
     c = wl.single_conv_case(seed=9, N=2, C=64, H=12, W=12, O=64, calibrated=True)
     rng = np.random.default_rng(4)
