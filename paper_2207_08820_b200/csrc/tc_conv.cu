@@ -11,6 +11,7 @@
 //   - four warps read the accumulator rows back with tcgen05.ld (one pixel per thread), apply the same fused
 //     requantisation epilogue as the popcount kernel and build the output plane words thread-locally.
 // Every wait on an mbarrier is bounded; a wait that runs out sets the device status word and the CTA drains.
+#include <cstdlib>
 #include <array>
 #include <map>
 #include <mutex>
@@ -201,12 +202,24 @@ __device__ __forceinline__ void tc_load_tile(const TcArgs& g, void* dst, uint64_
     }
 }
 
-// Byte look-up table of the expansion: entry [j][b] holds, for the eight bits of byte b of plane j, eight int8 lanes
-// with value mul[j] where the bit is set (two 32-bit words).  Adding the entries of all planes gives eight codes at once.
+// Look-up tables of the expansion, built once per CTA.
+// A == 2 (the 2-bit activations of the headline networks): one table of 256 words indexed by a nibble of plane 0
+// (low four index bits) and the same nibble of plane 1 (high four): the entry is the four finished int8 codes.
+// Other widths: entry [j][b] holds, for the eight bits of byte b of plane j, eight int8 lanes with value mul[j] where
+// the bit is set (two 32-bit words); adding the entries of all planes gives eight codes at once.
 constexpr int TC_LUT_BYTES_PER_PLANE = 256 * 8;
 
 __device__ __forceinline__ void tc_build_lut(const TcArgs& g, uint2* lut, int tid, int nthreads)
 {
+    if (g.A == 2) {
+        uint32_t* lut4 = reinterpret_cast<uint32_t*>(lut);
+        for (int e = tid; e < 256; e += nthreads) {
+            const unsigned n0 = e & 15u, n1 = static_cast<unsigned>(e) >> 4;
+            const unsigned s0 = (n0 * 0x00204081u) & 0x01010101u, s1 = (n1 * 0x00204081u) & 0x01010101u;
+            lut4[e] = s0 * g.mul[0] + s1 * g.mul[1];      // per byte: at most 1 + 254, no carry between lanes
+        }
+        return;
+    }
     for (int e = tid; e < g.A * 256; e += nthreads) {
         const unsigned b = e & 255u, m = g.mul[e >> 8];
         const unsigned lo = (((b & 0xFu) * 0x00204081u) & 0x01010101u) * m;
@@ -215,56 +228,101 @@ __device__ __forceinline__ void tc_build_lut(const TcArgs& g, uint2* lut, int ti
     }
 }
 
+// Where an expander thread starts in the item grid of a chunk, and how 128 items further move it: found once per
+// kernel so that the per-item loop has no division.  Items are (pixel, channel word) pairs, channel word fastest;
+// a chunk has one or two channel words.
+struct TcExpand {
+    int cw;            // channel word of this thread's items (the item stride 128 is a multiple of the words per chunk)
+    int x2, y2;        // first item's position in the (possibly subsampled) halo grid
+    int dx, dy;        // movement of 128 items
+    int nx, items;
+};
+
+__device__ __forceinline__ TcExpand tc_expand_init(const TcArgs& g, int et)
+{
+    TcExpand x;
+    const int sub = (!g.flat && g.stride == 2 && g.R == 1) ? 2 : 1;
+    x.nx = g.flat ? TC_M : (g.hw + sub - 1) / sub;
+    const int ny = g.flat ? 1 : (g.TNI * g.hh + sub - 1) / sub;   // hh is even for stride 2: rows of all images keep their parity
+    x.items = x.nx * ny * g.CWC;
+    const int sh = g.CWC >> 1;                                     // CWC is 1 or 2
+    x.cw = et & (g.CWC - 1);
+    const int pp = et >> sh, pstep = 128 >> sh;
+    x.y2 = pp / x.nx; x.x2 = pp - x.y2 * x.nx;
+    x.dy = pstep / x.nx; x.dx = pstep - x.dy * x.nx;
+    return x;
+}
+
 // Expansion of channel chunk c of the staged tile: bitplanes of (pixel, 32-channel word) -> 32 int8 values, written as
 // two 16-byte rows of the K-major core-matrix layout [16-channel group][halo pixel][16 bytes].  `et` = 0..127 within
 // the expander group.  A 1x1 stride-2 layer only ever reads even halo rows and columns, so only those are expanded.
 // MODE: 0 flat tile, 1 2-D tile stride 1, 2 2-D tile stride 2, 3 2-D tile 1x1 stride 2 (even rows and columns only).
 // The mode is a template parameter so that the per-item body is straight-line code.
 template <int A, int MODE>
-__device__ __forceinline__ void tc_expand_items(const TcArgs& g, const uint32_t* pa, unsigned char* eb, const uint2* lut, int et, int c)
+__device__ __forceinline__ void tc_expand_items(const TcArgs& g, const TcExpand& x, const uint32_t* pa, unsigned char* eb,
+                                                const uint2* lut, int et, int c)
 {
     constexpr int step = MODE == 3 ? 2 : 1;
-    const int nx = MODE == 0 ? TC_M : (g.hw + step - 1) / step;
-    const int ny = MODE == 0 ? 1 : (g.TNI * g.hh + step - 1) / step;   // hh is even for stride 2: rows of all images keep their parity
-    const int items = nx * ny * g.CWC;
     const uint32_t xormask = g.xormask;
     const int plane_bytes = g.HPE * 16;
-    for (int it = et; it < items; it += 128) {
-        const int cw = it % g.CWC, pp = it / g.CWC;
-        int hp = pp, ep = pp;
-        if (MODE != 0) {
-            const int y2 = pp / nx, x2 = pp - y2 * nx;
+    const int cw = x.cw;
+    int x2 = x.x2, y2 = x.y2;
+    const uint32_t* src_c = pa + (c * g.CWC + cw) * A;
+    unsigned char* dst_c = eb + static_cast<size_t>(2 * cw) * plane_bytes;
+    for (int it = et; it < x.items; it += 128) {
+        int hp, ep;
+        if (MODE == 0) {
+            hp = ep = x2;
+        } else {
             const int hy = y2 * step, hx = x2 * step;
             hp = hy * g.hwb + hx + g.xsh;
             ep = hy * g.HWP + (MODE == 1 ? hx : (hx & 1) * g.HWH + (hx >> 1));
         }
         uint32_t w[A];
-        load_planes<A>(pa + static_cast<size_t>(hp) * g.fullA + (c * g.CWC + cw) * A, w);
+        load_planes<A>(src_c + static_cast<size_t>(hp) * g.fullA, w);
         uint32_t out[8];
+        if (A == 2) {
+            // byte j of t / u: table index of nibble 2j / 2j+1 (plane 0 in the low four bits, plane 1 in the high four)
+            const char* lut4 = reinterpret_cast<const char*>(lut);
+            const uint32_t t = (w[0] & 0x0F0F0F0Fu) | ((w[A - 1] << 4) & 0xF0F0F0F0u);
+            const uint32_t u = ((w[0] >> 4) & 0x0F0F0F0Fu) | (w[A - 1] & 0xF0F0F0F0u);
+            out[0] = *reinterpret_cast<const uint32_t*>(lut4 + ((t << 2) & 0x3FCu));
+            out[1] = *reinterpret_cast<const uint32_t*>(lut4 + ((u << 2) & 0x3FCu));
+            out[2] = *reinterpret_cast<const uint32_t*>(lut4 + ((t >> 6) & 0x3FCu));
+            out[3] = *reinterpret_cast<const uint32_t*>(lut4 + ((u >> 6) & 0x3FCu));
+            out[4] = *reinterpret_cast<const uint32_t*>(lut4 + ((t >> 14) & 0x3FCu));
+            out[5] = *reinterpret_cast<const uint32_t*>(lut4 + ((u >> 14) & 0x3FCu));
+            out[6] = *reinterpret_cast<const uint32_t*>(lut4 + ((t >> 22) & 0x3FCu));
+            out[7] = *reinterpret_cast<const uint32_t*>(lut4 + ((u >> 22) & 0x3FCu));
+        } else {
 #pragma unroll
-        for (int q = 0; q < 4; ++q) {
-            uint2 acc = lut[(w[0] >> (8 * q)) & 0xFFu];
+            for (int q = 0; q < 4; ++q) {
+                uint2 acc = lut[(w[0] >> (8 * q)) & 0xFFu];
 #pragma unroll
-            for (int j = 1; j < A; ++j) {
-                const uint2 t = lut[j * 256 + ((w[j] >> (8 * q)) & 0xFFu)];
-                acc.x += t.x; acc.y += t.y;
+                for (int j = 1; j < A; ++j) {
+                    const uint2 tt = lut[j * 256 + ((w[j] >> (8 * q)) & 0xFFu)];
+                    acc.x += tt.x; acc.y += tt.y;
+                }
+                out[2 * q] = acc.x ^ xormask;
+                out[2 * q + 1] = acc.y ^ xormask;
             }
-            out[2 * q] = acc.x ^ xormask;
-            out[2 * q + 1] = acc.y ^ xormask;
         }
-        unsigned char* d = eb + static_cast<size_t>(2 * cw) * plane_bytes + static_cast<size_t>(ep) * 16;
+        unsigned char* d = dst_c + static_cast<size_t>(ep) * 16;
         *reinterpret_cast<uint4*>(d) = make_uint4(out[0], out[1], out[2], out[3]);
         *reinterpret_cast<uint4*>(d + plane_bytes) = make_uint4(out[4], out[5], out[6], out[7]);
+        x2 += x.dx; y2 += x.dy;
+        if (x2 >= x.nx) { x2 -= x.nx; ++y2; }
     }
 }
 
 template <int A>
-__device__ __forceinline__ void tc_expand_chunk(const TcArgs& g, const uint32_t* pa, unsigned char* eb, const uint2* lut, int et, int c)
+__device__ __forceinline__ void tc_expand_chunk(const TcArgs& g, const TcExpand& x, const uint32_t* pa, unsigned char* eb,
+                                                const uint2* lut, int et, int c)
 {
-    if (g.flat) tc_expand_items<A, 0>(g, pa, eb, lut, et, c);
-    else if (g.stride == 1) tc_expand_items<A, 1>(g, pa, eb, lut, et, c);
-    else if (g.R == 1) tc_expand_items<A, 3>(g, pa, eb, lut, et, c);
-    else tc_expand_items<A, 2>(g, pa, eb, lut, et, c);
+    if (g.flat) tc_expand_items<A, 0>(g, x, pa, eb, lut, et, c);
+    else if (g.stride == 1) tc_expand_items<A, 1>(g, x, pa, eb, lut, et, c);
+    else if (g.R == 1) tc_expand_items<A, 3>(g, x, pa, eb, lut, et, c);
+    else tc_expand_items<A, 2>(g, x, pa, eb, lut, et, c);
 }
 
 // All MMAs of one chunk: R*S taps x CK/32 steps of K = 32; a tap only moves the descriptor start address.
@@ -552,12 +610,13 @@ __global__ void __launch_bounds__(TC_THREADS) bitserial_conv_tc_kernel(const __g
     } else {
         // ------------------------------------------------------------------ expanders (warps 0-3), then epilogue
         pdl_acquire();                    // the epilogue reads the residual and overwrites buffers the preceding kernel may use
+        const TcExpand xp = tc_expand_init(g, tid);
         bool ok = mbar_wait_warp(full_a, 0, lane);
         for (int c = 0; c < g.nchunks; ++c) {
             const int e = c % g.nse, k = c / g.nse;
             if (ok && k >= 1) ok = mbar_wait_warp(&empty_e[e], (k - 1) & 1, lane);
             if (!ok) atomicOr(g.status, STATUS_TIMEOUT);
-            tc_expand_chunk<A>(g, reinterpret_cast<const uint32_t*>(tc_smem + g.off_p), tc_smem + g.off_e + e * g.e_bytes, s_lut, tid, c);
+            tc_expand_chunk<A>(g, xp, reinterpret_cast<const uint32_t*>(tc_smem + g.off_p), tc_smem + g.off_e + e * g.e_bytes, s_lut, tid, c);
             fence_proxy_async();          // make the generic-proxy writes visible to the tensor core's reads
             group_sync(1);
             if (tid == 0) mbar_arrive(&full_e[e]);
@@ -684,6 +743,7 @@ __global__ void __launch_bounds__(TCP_THREADS, 3) bitserial_conv_tc_persistent_k
     } else if (warp >= 4) {
         // ------------------------------------------------------------------ expanders (warps 4-7)
         const int et = tid - 128;
+        const TcExpand xp = tc_expand_init(g, et);
         int it = 0, i = 0;
         bool ok = true;
         for (int mt = first_tile; mt < tiles_m && ok; mt += tile_step, ++i) {
@@ -694,7 +754,7 @@ __global__ void __launch_bounds__(TCP_THREADS, 3) bitserial_conv_tc_persistent_k
                 if (ok && k >= 1) ok = mbar_wait_warp(&empty_e[e], (k - 1) & 1, lane);
                 ok = group_all(1, ok);
                 if (!ok) break;
-                tc_expand_chunk<A>(g, reinterpret_cast<const uint32_t*>(s_p + s * g.pa_bytes), s_e + e * g.e_bytes, s_lut, et, c);
+                tc_expand_chunk<A>(g, xp, reinterpret_cast<const uint32_t*>(s_p + s * g.pa_bytes), s_e + e * g.e_bytes, s_lut, et, c);
                 fence_proxy_async();
                 group_sync(1);                       // all 128 expander threads have written and fenced
                 if (et == 0) mbar_arrive(&full_e[e]);
@@ -930,7 +990,16 @@ static int tc_conv_impl(const uint32_t* act, const int8_t* wgt, const bs_conv_pa
     size_t smem = 0;
     g.persistent = 0;
     const int bar_bytes = (2 * TCP_NSP + 2 * TCP_NSE + 5) * 8 + 16;
+    int tn_max = 128;
+    bool force_stream = false, keep_narrow = false;
+#ifdef BS_TUNING
+    // plan overrides for tuning runs (not compiled into the library by default)
+    if (const char* e = getenv("BS_TC_TNMAX")) tn_max = atoi(e);
+    force_stream = getenv("BS_TC_STREAM") != nullptr;
+    keep_narrow = getenv("BS_TC_KEEP_NARROW") != nullptr;
+#endif
     for (int TN = 128; TN >= 32; TN /= 2) {
+        if (TN > tn_max) continue;
         if (TN / 2 >= round_up_i(p->O, 32)) continue;                      // tile twice as wide as the filter bank
         const long long pairs = tiles_m * ceil_div(p->O, TN);
         if (TN > 32 && pairs < sms) continue;
@@ -956,7 +1025,8 @@ static int tc_conv_impl(const uint32_t* act, const int8_t* wgt, const bs_conv_pa
     }
     // A resident plan that had to shrink the filter tile to 32 wastes the tensor core (an N = 32 MMA costs as many
     // cycles as N = 64): stream the filters instead when a 128-wide tile leaves enough (pixel tile, filter tile) pairs.
-    if (g.persistent && g.TN == 32 && p->O >= 128 && tiles_m * ceil_div(p->O, 128) >= sms / 2) g.persistent = 0;
+    if (!keep_narrow && g.persistent && g.TN == 32 && p->O >= 128 && tiles_m * ceil_div(p->O, 128) >= sms / 2) g.persistent = 0;
+    if (force_stream) g.persistent = 0;
     if (!g.persistent) {
         // one tile per CTA, filters streamed with every chunk: the widest filter tile that keeps about one pair per SM
         g.nsp = g.nse = g.nchunks < TC_MAX_STAGES ? g.nchunks : TC_MAX_STAGES;
