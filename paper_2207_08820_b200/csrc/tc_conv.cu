@@ -53,8 +53,9 @@ struct TcArgs {
     int tiles_o, tiles_q, tiles_p, tiles_n;
     int opad8;                        // padded filter count / 8 in the prepared weights
     int pa_bytes, pa_tx_bytes, b_bytes, e_bytes;   // per stage (pa_tx_bytes: bytes the activation box delivers)
-    int off_p, off_e, off_sb, off_bar, off_tab, off_lut;   // shared-memory offsets (bytes)
+    int off_p, off_e, off_sb, off_bar, off_lut;   // shared-memory offsets (bytes)
     int persistent;
+    int PT;                           // streaming kernel: pixel tiles per CTA (they share every streamed filter chunk)
     int tmem_cols;
     unsigned idesc;
     unsigned mul[4];                  // byte value of plane j (2^j, or 256 - 2^(A-1) for a two's-complement top plane)
@@ -326,18 +327,19 @@ __device__ __forceinline__ void tc_expand_chunk(const TcArgs& g, const TcExpand&
 }
 
 // All MMAs of one chunk: R*S taps x CK/32 steps of K = 32; a tap only moves the descriptor start address.
-// One thread issues them, and a lone thread retires only an instruction every few cycles, so the per-MMA work is cut
-// to a table look-up and two adds: the start-address offsets of every (tap, K step) are tabulated once per CTA in
-// shared memory (in 16-byte units, relative to the stage base) and the constant descriptor words live in registers.
-constexpr int TC_MAX_MMA_PER_CHUNK = 128;       // R*S * CK/32 <= 49 * 2
-
+// One thread issues them.  A lone thread cannot hide the latency of a load in front of every MMA (a tabulated
+// offset per MMA measured 120-160 cycles per MMA against 64 for the MMA itself), so the start addresses are produced
+// by register arithmetic alone: the filter operand advances by a constant per MMA, the activation operand by the
+// tap's column, row and K-half offsets (16-byte units; shared-memory addresses fit the 14-bit field without a mask).
 struct TcIssue {
     uint32_t a_lo, a_hi, b_lo, b_hi;   // descriptor words with a zero start-address field
     uint32_t idesc;
-    int n;                             // MMAs per chunk
+    uint32_t row16, half16, kstep16;   // halo row, odd-column plane (stride 2) and second K half, in 16-byte units
+    int R, S;
+    bool stride2, two;                 // even/odd column split; two K = 32 steps per tap (64-channel chunks)
 };
 
-__device__ __forceinline__ TcIssue tc_make_issue(const TcArgs& g, uint2* tab)
+__device__ __forceinline__ TcIssue tc_make_issue(const TcArgs& g)
 {
     TcIssue is;
     const uint32_t lbo_a = static_cast<uint32_t>(g.HPE) * 16u;
@@ -348,15 +350,12 @@ __device__ __forceinline__ TcIssue tc_make_issue(const TcArgs& g, uint2* tab)
     is.a_lo = static_cast<uint32_t>(ad); is.a_hi = static_cast<uint32_t>(ad >> 32);
     is.b_lo = static_cast<uint32_t>(bd); is.b_hi = static_cast<uint32_t>(bd >> 32);
     is.idesc = g.idesc;
-    int n = 0;
-    uint32_t b16 = 0;
-    for (int r = 0; r < g.R; ++r)
-        for (int sx = 0; sx < g.S; ++sx) {
-            const uint32_t a16 = static_cast<uint32_t>(r * g.HWP + (g.stride == 2 ? (sx & 1) * g.HWH + (sx >> 1) : sx));
-            for (uint32_t kp = 0; kp < k16 / 2; ++kp) tab[n++] = make_uint2(a16 + 2 * kp * (lbo_a >> 4), b16 + 16 * kp);
-            b16 += k16 * 8;
-        }
-    is.n = n;
+    is.row16 = static_cast<uint32_t>(g.HWP);
+    is.half16 = static_cast<uint32_t>(g.HWH);
+    is.kstep16 = 2u * (lbo_a >> 4);
+    is.R = g.R; is.S = g.S;
+    is.stride2 = !g.flat && g.stride == 2;
+    is.two = g.CK == 64;
     return is;
 }
 
@@ -372,20 +371,24 @@ __device__ __forceinline__ void umma_i8_words(uint32_t d_tmem, uint32_t a_lo, ui
         ::"r"(d_tmem), "r"(a_lo), "r"(a_hi), "r"(b_lo), "r"(b_hi), "r"(idesc), "r"(accumulate) : "memory");
 }
 
-__device__ __forceinline__ void tc_issue_chunk(const TcIssue& is, const uint2* tab, uint32_t ea, uint32_t ba, uint32_t tmem_acc,
-                                               bool first_chunk)
+__device__ __forceinline__ void tc_issue_chunk(const TcIssue& is, uint32_t ea, uint32_t ba, uint32_t tmem_acc, bool first_chunk)
 {
-    const uint32_t ea16 = ea >> 4, ba16 = ba >> 4;
-    int m = 0;
-    if (first_chunk) {          // the first MMA of a tile overwrites the accumulator
-        const uint2 d = tab[0];
-        umma_i8_words(tmem_acc, is.a_lo | ((ea16 + d.x) & 0x3FFFu), is.a_hi, is.b_lo | ((ba16 + d.y) & 0x3FFFu), is.b_hi, is.idesc, 0u);
-        m = 1;
-    }
-#pragma unroll 4
-    for (; m < is.n; ++m) {
-        const uint2 d = tab[m];
-        umma_i8_words(tmem_acc, is.a_lo | ((ea16 + d.x) & 0x3FFFu), is.a_hi, is.b_lo | ((ba16 + d.y) & 0x3FFFu), is.b_hi, is.idesc, 1u);
+    uint32_t arow = is.a_lo + (ea >> 4);
+    uint32_t b = is.b_lo + (ba >> 4);              // filters: [tap][K half] tiles of 16 x 16 bytes, one after the other
+    uint32_t acc = first_chunk ? 0u : 1u;          // the first MMA of a tile overwrites the accumulator
+    for (int r = 0; r < is.R; ++r) {
+        for (int sx = 0; sx < is.S; ++sx) {
+            const uint32_t a = arow + (is.stride2 ? static_cast<uint32_t>(sx & 1) * is.half16 + static_cast<uint32_t>(sx >> 1)
+                                                  : static_cast<uint32_t>(sx));
+            umma_i8_words(tmem_acc, a, is.a_hi, b, is.b_hi, is.idesc, acc);
+            acc = 1u;
+            b += 16;
+            if (is.two) {
+                umma_i8_words(tmem_acc, a + is.kstep16, is.a_hi, b, is.b_hi, is.idesc, 1u);
+                b += 16;
+            }
+        }
+        arow += is.row16;
     }
 }
 
@@ -540,7 +543,10 @@ __global__ void __launch_bounds__(TC_THREADS) bitserial_conv_tc_kernel(const __g
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 4 * TC_MAX_STAGES + 2);
 
     const int o0 = static_cast<int>(blockIdx.x % static_cast<unsigned>(g.tiles_o)) * g.TN;   // filter tile fastest
-    const TcTile tile = tc_decode_tile(g, static_cast<int>(blockIdx.x / static_cast<unsigned>(g.tiles_o)));
+    const int tiles_m = g.tiles_q * g.tiles_p * g.tiles_n;
+    const int mt0 = static_cast<int>(blockIdx.x / static_cast<unsigned>(g.tiles_o)) * g.PT;      // first pixel tile of this CTA
+    const int nt = tiles_m - mt0 < g.PT ? tiles_m - mt0 : g.PT;                                   // 1..PT pixel tiles
+    const int e_stage = g.PT * g.e_bytes;
 
     pdl_release();
     if (tid == 0) {
@@ -551,7 +557,7 @@ __global__ void __launch_bounds__(TC_THREADS) bitserial_conv_tc_kernel(const __g
             mbar_init(&empty_e[s], 1);
         }
         mbar_init(accum_full, 1);
-        mbar_init(full_a, 1);
+        mbar_init(full_a, static_cast<unsigned>(nt));
         fence_barrier_init();
         fence_proxy_async();
     }
@@ -577,21 +583,26 @@ __global__ void __launch_bounds__(TC_THREADS) bitserial_conv_tc_kernel(const __g
             const int early = g.nchunks < g.nsp ? g.nchunks : g.nsp;
             for (int c = 0; c < g.nchunks; ++c) {
                 const int s = c % g.nsp, k = c / g.nsp;
-                if (c == early) { pdl_acquire(); tc_load_tile(g, tc_smem + g.off_p, full_a, tile); }
+                if (c == early) {
+                    pdl_acquire();
+                    for (int t = 0; t < nt; ++t) tc_load_tile(g, tc_smem + g.off_p + t * g.pa_bytes, full_a, tc_decode_tile(g, mt0 + t));
+                }
                 if (k >= 1 && !mbar_spin_bounded(&empty_p[s], (k - 1) & 1)) { atomicOr(g.status, STATUS_TIMEOUT); break; }
                 mbar_expect_tx(&full_p[s], static_cast<unsigned>(g.b_bytes));
                 const size_t src = (static_cast<size_t>(c) * g.opad8 + (o0 >> 3)) * RS * (g.CK >> 4) * 128;
                 bulk_load(tc_smem + s * stage_p_bytes, g.wgt + src, static_cast<unsigned>(g.b_bytes), &full_p[s]);
             }
-            if (early == g.nchunks) { pdl_acquire(); tc_load_tile(g, tc_smem + g.off_p, full_a, tile); }
+            if (early == g.nchunks) {
+                pdl_acquire();
+                for (int t = 0; t < nt; ++t) tc_load_tile(g, tc_smem + g.off_p + t * g.pa_bytes, full_a, tc_decode_tile(g, mt0 + t));
+            }
         }
         __syncwarp();
     } else if (warp == 5) {
         // ------------------------------------------------------------------ MMA issuer
         if (lane == 0) {
             const uint32_t e_base = smem_u32(tc_smem + g.off_e);
-            uint2* tab = reinterpret_cast<uint2*>(tc_smem + g.off_tab);
-            const TcIssue is = tc_make_issue(g, tab);
+            const TcIssue is = tc_make_issue(g);
             for (int c = 0; c < g.nchunks; ++c) {
                 const int s = c % g.nsp, e = c % g.nse;
                 if (!(mbar_spin_bounded(&full_p[s], (c / g.nsp) & 1) && mbar_spin_bounded(&full_e[e], (c / g.nse) & 1))) {
@@ -599,8 +610,9 @@ __global__ void __launch_bounds__(TC_THREADS) bitserial_conv_tc_kernel(const __g
                     break;
                 }
                 tc_fence_after();
-                tc_issue_chunk(is, tab, e_base + static_cast<uint32_t>(e) * g.e_bytes, smem_u32(tc_smem + s * stage_p_bytes),
-                               tmem_base, c == 0);
+                for (int t = 0; t < nt; ++t)
+                    tc_issue_chunk(is, e_base + static_cast<uint32_t>(e * e_stage + t * g.e_bytes), smem_u32(tc_smem + s * stage_p_bytes),
+                                   tmem_base + static_cast<uint32_t>(t * g.TN), c == 0);
                 umma_commit(&empty_e[e]);
                 umma_commit(&empty_p[s]);
             }
@@ -616,7 +628,9 @@ __global__ void __launch_bounds__(TC_THREADS) bitserial_conv_tc_kernel(const __g
             const int e = c % g.nse, k = c / g.nse;
             if (ok && k >= 1) ok = mbar_wait_warp(&empty_e[e], (k - 1) & 1, lane);
             if (!ok) atomicOr(g.status, STATUS_TIMEOUT);
-            tc_expand_chunk<A>(g, xp, reinterpret_cast<const uint32_t*>(tc_smem + g.off_p), tc_smem + g.off_e + e * g.e_bytes, s_lut, tid, c);
+            for (int t = 0; t < nt; ++t)
+                tc_expand_chunk<A>(g, xp, reinterpret_cast<const uint32_t*>(tc_smem + g.off_p + t * g.pa_bytes),
+                                   tc_smem + g.off_e + e * e_stage + t * g.e_bytes, s_lut, tid, c);
             fence_proxy_async();          // make the generic-proxy writes visible to the tensor core's reads
             group_sync(1);
             if (tid == 0) mbar_arrive(&full_e[e]);
@@ -624,7 +638,8 @@ __global__ void __launch_bounds__(TC_THREADS) bitserial_conv_tc_kernel(const __g
         if (ok) ok = mbar_wait_warp(accum_full, 0, lane);
         if (!ok) atomicOr(g.status, STATUS_TIMEOUT);
         tc_fence_after();
-        tc_epilogue_tile(g, tmem_base, tid, warp, tile, o0, s_sb, s_bounds);
+        for (int t = 0; t < nt; ++t)
+            tc_epilogue_tile(g, tmem_base + static_cast<uint32_t>(t * g.TN), tid, warp, tc_decode_tile(g, mt0 + t), o0, s_sb, s_bounds);
         tc_fence_before();
     }
     __syncthreads();
@@ -718,8 +733,7 @@ __global__ void __launch_bounds__(TCP_THREADS, 3) bitserial_conv_tc_persistent_k
     } else if (warp == 9) {
         // ------------------------------------------------------------------ MMA issuer
         if (lane == 0) {
-            uint2* tab = reinterpret_cast<uint2*>(tc_smem + g.off_tab);
-            const TcIssue is = tc_make_issue(g, tab);
+            const TcIssue is = tc_make_issue(g);
             bool ok = mbar_spin_bounded(wgt_full, 0);       // also keeps the CTA alive until the filter copy has landed
             int it = 0, i = 0;
             for (int mt = first_tile; mt < tiles_m && ok; mt += tile_step, ++i) {
@@ -732,7 +746,7 @@ __global__ void __launch_bounds__(TCP_THREADS, 3) bitserial_conv_tc_persistent_k
                     const int e = it % g.nse;
                     if (!mbar_spin_bounded(&full_e[e], (it / g.nse) & 1)) { ok = false; break; }
                     tc_fence_after();
-                    tc_issue_chunk(is, tab, smem_u32(s_e + e * g.e_bytes), smem_u32(s_w + static_cast<size_t>(c) * g.b_bytes), tmem_acc, c == 0);
+                    tc_issue_chunk(is, smem_u32(s_e + e * g.e_bytes), smem_u32(s_w + static_cast<size_t>(c) * g.b_bytes), tmem_acc, c == 0);
                     umma_commit(&empty_e[e]);
                 }
                 if (ok) umma_commit(&full_acc[buf]);
@@ -992,11 +1006,14 @@ static int tc_conv_impl(const uint32_t* act, const int8_t* wgt, const bs_conv_pa
     const int bar_bytes = (2 * TCP_NSP + 2 * TCP_NSE + 5) * 8 + 16;
     int tn_max = 128;
     bool force_stream = false, keep_narrow = false;
+    int stream_pt = 1, stream_tn = 0;
 #ifdef BS_TUNING
     // plan overrides for tuning runs (not compiled into the library by default)
     if (const char* e = getenv("BS_TC_TNMAX")) tn_max = atoi(e);
     force_stream = getenv("BS_TC_STREAM") != nullptr;
     keep_narrow = getenv("BS_TC_KEEP_NARROW") != nullptr;
+    if (const char* e = getenv("BS_TC_PT")) stream_pt = atoi(e);
+    if (const char* e = getenv("BS_TC_STN")) stream_tn = atoi(e);
 #endif
     for (int TN = 128; TN >= 32; TN /= 2) {
         if (TN > tn_max) continue;
@@ -1008,15 +1025,14 @@ static int tc_conv_impl(const uint32_t* act, const int8_t* wgt, const bs_conv_pa
         for (const auto& sh : shapes) {
             const int nsp = sh[0], nse = sh[1];
             const size_t total = wbytes + static_cast<size_t>(nsp) * g.pa_bytes + static_cast<size_t>(nse) * g.e_bytes +
-                                 static_cast<size_t>(TN) * 8 + 256 + bar_bytes + 128 + TC_MAX_MMA_PER_CHUNK * 8 + 16 + static_cast<size_t>(A) * TC_LUT_BYTES_PER_PLANE;
+                                 static_cast<size_t>(TN) * 8 + 256 + bar_bytes + 128 + 16 + static_cast<size_t>(A) * TC_LUT_BYTES_PER_PLANE;
             if (total <= 220 * 1024) {
                 g.persistent = 1; g.TN = TN; g.b_bytes = TN * RS * g.CK; g.nse = nse; g.nsp = nsp;
                 g.off_p = static_cast<int>(wbytes);
                 g.off_e = g.off_p + nsp * g.pa_bytes;
                 g.off_sb = g.off_e + nse * g.e_bytes;
                 g.off_bar = round_up_i(g.off_sb + TN * 8 + 256, 16);
-                g.off_tab = round_up_i(g.off_bar + bar_bytes, 16);
-                g.off_lut = g.off_tab + TC_MAX_MMA_PER_CHUNK * 8;
+                g.off_lut = round_up_i(g.off_bar + bar_bytes, 16);
                 smem = static_cast<size_t>(g.off_lut) + static_cast<size_t>(A) * TC_LUT_BYTES_PER_PLANE;
                 break;
             }
@@ -1027,29 +1043,35 @@ static int tc_conv_impl(const uint32_t* act, const int8_t* wgt, const bs_conv_pa
     // cycles as N = 64): stream the filters instead when a 128-wide tile leaves enough (pixel tile, filter tile) pairs.
     if (!keep_narrow && g.persistent && g.TN == 32 && p->O >= 128 && tiles_m * ceil_div(p->O, 128) >= sms / 2) g.persistent = 0;
     if (force_stream) g.persistent = 0;
+    g.PT = 1;
     if (!g.persistent) {
-        // one tile per CTA, filters streamed with every chunk: the widest filter tile that keeps about one pair per SM
+        // Filters streamed chunk by chunk; a CTA takes PT pixel tiles (PT accumulators in tensor memory) so that every
+        // filter chunk fetched from L2 serves PT tiles.  Widest filter tile that keeps about one CTA per SM.
         g.nsp = g.nse = g.nchunks < TC_MAX_STAGES ? g.nchunks : TC_MAX_STAGES;
         int TN = 128;
         while (TN > 32 && (TN / 2 >= round_up_i(p->O, 32) || tiles_m * ceil_div(p->O, TN) < sms / 2)) TN /= 2;
-        for (;; TN /= 2) {
-            g.TN = TN;
-            g.b_bytes = TN * RS * g.CK;
-            const size_t total = static_cast<size_t>(g.nsp) * g.b_bytes + g.pa_bytes + static_cast<size_t>(g.nse) * g.e_bytes +
-                                 2 * TN * 4 + 256 + (4 * TC_MAX_STAGES + 3) * 8 + 128 + TC_MAX_MMA_PER_CHUNK * 8 + 16 + static_cast<size_t>(A) * TC_LUT_BYTES_PER_PLANE;
-            if (total <= 200 * 1024 || TN == 32) break;
-        }
+        int PT = stream_pt;
+        auto stream_bytes = [&](int tn, int pt) {
+            return static_cast<size_t>(g.nsp) * tn * RS * g.CK + static_cast<size_t>(pt) * g.pa_bytes +
+                   static_cast<size_t>(g.nse) * pt * g.e_bytes + 2 * tn * 4 + 256 + (4 * TC_MAX_STAGES + 3) * 8 + 128 +
+                   16 + static_cast<size_t>(A) * TC_LUT_BYTES_PER_PLANE;
+        };
+        if (stream_tn) TN = stream_tn;
+        while (PT > 1 && (PT * TN > 512 || stream_bytes(TN, PT) > 220 * 1024)) PT /= 2;
+        while (TN > 32 && stream_bytes(TN, PT) > 200 * 1024) TN /= 2;
+        g.TN = TN;
+        g.PT = PT;
+        g.b_bytes = TN * RS * g.CK;
         g.off_p = g.nsp * g.b_bytes;
-        g.off_e = g.off_p + g.pa_bytes;
-        g.off_sb = g.off_e + g.nse * g.e_bytes;
+        g.off_e = g.off_p + PT * g.pa_bytes;
+        g.off_sb = g.off_e + g.nse * PT * g.e_bytes;
         g.off_bar = round_up_i(g.off_sb + 2 * g.TN * 4 + 256, 16);
-        g.off_tab = round_up_i(g.off_bar + (4 * TC_MAX_STAGES + 3) * 8, 16);
-        g.off_lut = g.off_tab + TC_MAX_MMA_PER_CHUNK * 8;
+        g.off_lut = round_up_i(g.off_bar + (4 * TC_MAX_STAGES + 3) * 8, 16);
         smem = static_cast<size_t>(g.off_lut) + static_cast<size_t>(A) * TC_LUT_BYTES_PER_PLANE;
         if (smem > 220 * 1024) return BS_ERR_UNSUPPORTED;
     }
     g.tiles_o = ceil_div(p->O, g.TN);
-    g.tmem_cols = g.persistent ? 2 * g.TN : g.TN;      // TN is 32, 64 or 128: powers of two, at least 32 columns
+    g.tmem_cols = g.persistent ? 2 * g.TN : g.PT * g.TN;      // TN is 32, 64 or 128, PT 1, 2 or 4: powers of two, 32..512 columns
     g.idesc = (2u << 4) | (1u << 7) | (1u << 10) | (static_cast<unsigned>(g.TN >> 3) << 17) | (static_cast<unsigned>(TC_M >> 4) << 24);
     for (int j = 0; j < 4; ++j) g.mul[j] = 1u << j;
     g.xormask = 0;
@@ -1110,7 +1132,7 @@ static int tc_conv_impl(const uint32_t* act, const int8_t* wgt, const bs_conv_pa
         }
         return BS_OK;
     }
-    const long long grid = tiles_m * g.tiles_o;
+    const long long grid = ceil_div_ll(tiles_m, g.PT) * g.tiles_o;
     if (grid > 0x7fffffffLL) return BS_ERR_UNSUPPORTED;
     void (*kern)(TcArgs) = nullptr;
     switch (A) {
