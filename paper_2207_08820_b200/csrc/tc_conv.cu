@@ -53,7 +53,8 @@ struct TcArgs {
     int tiles_o, tiles_q, tiles_p, tiles_n;
     int opad8;                        // padded filter count / 8 in the prepared weights
     int pa_bytes, pa_tx_bytes, b_bytes, e_bytes;   // per stage (pa_tx_bytes: bytes the activation box delivers)
-    int off_p, off_e, off_sb, off_bar, off_lut;   // shared-memory offsets (bytes)
+    int off_p, off_e, off_sb, off_bar, off_lut;
+    int off_thr, thr_pats;            // integer thresholds of the epilogue: offset (0 = not used) and residual patterns (1 or 4)   // shared-memory offsets (bytes)
     int persistent;
     int PT;                           // streaming kernel: pixel tiles per CTA (they share every streamed filter chunk)
     int tmem_cols;
@@ -418,9 +419,103 @@ __device__ __forceinline__ void tc_compare_block(const uint32_t (&v)[32], const 
     ow[1] = w1;
 }
 
+// Integer form of the comparison epilogue.  t = fmaf((float)acc, scale, bias) is monotone in the integer accumulator
+// when scale > 0, so "t >= bound" is "acc >= T" for the smallest accumulator T that satisfies it.  The thresholds are
+// found per (residual pattern, filter) once per CTA: an estimate (bound - bias) / scale, corrected by evaluating the
+// very fmaf of the formula at T - 1 and T until  f(T - 1) < bound <= f(T)  holds, which pins T exactly.  Accumulators
+// and thresholds stay within +-2^29, so differences cannot overflow.  Anything unusual (scale <= 0, non-finite
+// numbers, no convergence) clears *ok and the CTA keeps the floating-point comparison.
+constexpr int TC_THR_LIM = 1 << 29;
+
+__device__ __forceinline__ int tc_threshold(float s, float b, float bound, int* ok)
+{
+    if (!(bound == bound)) { *ok = 0; return TC_THR_LIM; }
+    float x = (bound - b) / s;
+    x = fminf(fmaxf(x, -6.0e8f), 6.0e8f);             // NaN cannot occur: s > 0 and b finite are checked by the caller
+    int T = static_cast<int>(ceilf(x));
+    T = T < -TC_THR_LIM ? -TC_THR_LIM : (T > TC_THR_LIM ? TC_THR_LIM : T);
+    int it = 0;
+    while (T > -TC_THR_LIM && fmaf(static_cast<float>(T - 1), s, b) >= bound && it < 8) { --T; ++it; }
+    if (it == 8) *ok = 0;
+    it = 0;
+    while (T < TC_THR_LIM && !(fmaf(static_cast<float>(T), s, b) >= bound) && it < 8) { ++T; ++it; }
+    if (it == 8) *ok = 0;
+    return T;
+}
+
+// thr[filter * patterns + pattern] = (T1, T2, T3, -) for the filters of this CTA (the patterns of one filter share a
+// 64-byte line, so lanes with different residuals do not collide on banks); called by `nthreads` threads (index `t`).
+__device__ __forceinline__ void tc_build_thresholds(const TcArgs& g, int4* thr, int* ok, const float2* s_sb, const float4* s_bounds,
+                                                    int o0, int t, int nthreads)
+{
+    for (int e = t; e < g.thr_pats * g.TN; e += nthreads) {
+        const int f = e % g.TN, pat = e / g.TN;
+        int4 T = make_int4(TC_THR_LIM, TC_THR_LIM, TC_THR_LIM, 0);         // filters past O: never reached, masked anyway
+        if (o0 + f < g.O) {
+            const float2 sb = s_sb[f];
+            if (!(sb.x > 0.0f) || !(sb.x < 3.0e38f) || !(fabsf(sb.y) < 3.0e38f)) {
+                *ok = 0;
+            } else {
+                const float4 bb = s_bounds[pat];
+                T.x = tc_threshold(sb.x, sb.y, bb.x, ok);
+                T.y = tc_threshold(sb.x, sb.y, bb.y, ok);
+                T.z = tc_threshold(sb.x, sb.y, bb.z, ok);
+            }
+        }
+        thr[f * g.thr_pats + pat] = T;
+    }
+}
+
+__device__ __forceinline__ int4 lds_int4(uint32_t addr)
+{
+    int4 r;
+    asm volatile("ld.shared.v4.s32 {%0, %1, %2, %3}, [%4];" : "=r"(r.x), "=r"(r.y), "=r"(r.z), "=r"(r.w) : "r"(addr));
+    return r;
+}
+// Bits of the low half of x moved to the even bit positions.
+__device__ __forceinline__ uint32_t spread16(uint32_t x)
+{
+    x &= 0xFFFFu;
+    x = (x | (x << 8)) & 0x00FF00FFu;
+    x = (x | (x << 4)) & 0x0F0F0F0Fu;
+    x = (x | (x << 2)) & 0x33333333u;
+    x = (x | (x << 1)) & 0x55555555u;
+    return x;
+}
+
+// 32 accumulators of one pixel against their integer thresholds.  The sign bit of acc - T_k says "below level k";
+// a funnel shift collects it, so an output costs three subtractions, one three-way xor and two shifts.
+// thr_addr: shared-memory address of the thresholds of filter 0 of this group of 32.
+template <int RES>      // 0: no residual, 1: residual of 1-2 bits selects one of four threshold sets
+__device__ __forceinline__ void tc_compare_int(const uint32_t (&v)[32], uint32_t thr_addr, const uint32_t (&rw)[4], uint32_t (&ow)[4])
+{
+    uint32_t w0 = 0, w1 = 0;
+    // residual pattern of filter f at bits 2f, 2f+1 of (z_hi : z_lo)
+    const uint32_t z_lo = RES ? (spread16(rw[0]) | (spread16(rw[1]) << 1)) : 0u;
+    const uint32_t z_hi = RES ? (spread16(rw[0] >> 16) | (spread16(rw[1] >> 16) << 1)) : 0u;
+#pragma unroll
+    for (int f = 31; f >= 0; --f) {
+        const uint32_t acc = v[f];
+        int4 T;
+        if (RES == 0) {
+            T = lds_int4(thr_addr + f * 16);
+        } else {
+            const uint32_t z = f < 16 ? z_lo : z_hi;
+            const int sh = 2 * (f & 15) - 4;                                  // pattern * 16 bytes
+            const uint32_t off = (sh >= 0 ? (z >> sh) : (z << -sh)) & 0x30u;
+            T = lds_int4(thr_addr + f * 64 + off);
+        }
+        const uint32_t d1 = acc - static_cast<uint32_t>(T.x), d2 = acc - static_cast<uint32_t>(T.y), d3 = acc - static_cast<uint32_t>(T.z);
+        w1 = __funnelshift_l(d2, w1, 1);                 // (w1 << 1) | sign(d2)
+        w0 = __funnelshift_l(d1 ^ d2 ^ d3, w0, 1);
+    }
+    ow[0] = ~w0;        // levels reached = 3 - (number of set signs): bit 0 is the complemented parity,
+    ow[1] = ~w1;        // bit 1 is "level 2 reached"
+}
+
 // Epilogue of one tile: thread `tid` (0..127, warp = TMEM lane quadrant) owns accumulator row tid = one output pixel.
 __device__ __forceinline__ void tc_epilogue_tile(const TcArgs& g, uint32_t tmem_acc, int tid, int warp, const TcTile& tile, int o0,
-                                                 const float2* s_sb, const float4* s_bounds)
+                                                 const float2* s_sb, const float4* s_bounds, uint32_t thr_addr)
 {
     const int n0 = tile.n0, p0 = tile.p0, q0 = tile.q0;
     const int m = tid;                               // TMEM lane = tile pixel
@@ -474,7 +569,10 @@ __device__ __forceinline__ void tc_epilogue_tile(const TcArgs& g, uint32_t tmem_
                 // uniform switches are resolved once per 32 outputs, so the unrolled body is straight-line code.
                 const unsigned valid_mask = (g.O - ob >= 32) ? 0xffffffffu : ((1u << (g.O - ob)) - 1u);
                 const float2* sb32 = s_sb + cc * 32;
-                if (!g.residual) {
+                if (thr_addr) {
+                    if (!g.residual) tc_compare_int<0>(v, thr_addr + cc * 512, rw, ow);
+                    else tc_compare_int<1>(v, thr_addr + cc * 2048, rw, ow);
+                } else if (!g.residual) {
                     if (g.acc_small) tc_compare_block<true, 0>(v, sb32, s_bounds, bnd0, rw, ow);
                     else tc_compare_block<false, 0>(v, sb32, s_bounds, bnd0, rw, ow);
                 } else if (g.res_bits <= 2) {
@@ -570,6 +668,7 @@ __global__ void __launch_bounds__(TC_THREADS) bitserial_conv_tc_kernel(const __g
         s_sb[tid] = (g.out_packed && o < g.O) ? make_float2(g.scale[o], g.bias[o]) : make_float2(0.f, 0.f);
     }
     if (tid < 16) s_bounds[tid] = make_float4(g.rb.bound[tid][0], g.rb.bound[tid][1], g.rb.bound[tid][2], 0.f);
+    if (tid == 32 && g.off_thr) *reinterpret_cast<int*>(tc_smem + g.off_thr + g.thr_pats * g.TN * 16) = 1;
     tc_build_lut(g, s_lut, tid, blockDim.x);
     tc_fence_before();
     __syncthreads();
@@ -635,11 +734,20 @@ __global__ void __launch_bounds__(TC_THREADS) bitserial_conv_tc_kernel(const __g
             group_sync(1);
             if (tid == 0) mbar_arrive(&full_e[e]);
         }
+        // the last chunks are still in the tensor core: time to turn the comparison bounds into integer thresholds
+        uint32_t thr = 0;                 // shared-memory address of the thresholds, 0: floating-point comparison
+        if (g.off_thr) {
+            int4* s_thr = reinterpret_cast<int4*>(tc_smem + g.off_thr);
+            int* thr_ok = reinterpret_cast<int*>(s_thr + g.thr_pats * g.TN);
+            tc_build_thresholds(g, s_thr, thr_ok, s_sb, s_bounds, o0, tid, 128);
+            group_sync(1);
+            if (*thr_ok) thr = smem_u32(s_thr);
+        }
         if (ok) ok = mbar_wait_warp(accum_full, 0, lane);
         if (!ok) atomicOr(g.status, STATUS_TIMEOUT);
         tc_fence_after();
         for (int t = 0; t < nt; ++t)
-            tc_epilogue_tile(g, tmem_base + static_cast<uint32_t>(t * g.TN), tid, warp, tc_decode_tile(g, mt0 + t), o0, s_sb, s_bounds);
+            tc_epilogue_tile(g, tmem_base + static_cast<uint32_t>(t * g.TN), tid, warp, tc_decode_tile(g, mt0 + t), o0, s_sb, s_bounds, thr);
         tc_fence_before();
     }
     __syncthreads();
@@ -705,6 +813,7 @@ __global__ void __launch_bounds__(TCP_THREADS, 3) bitserial_conv_tc_persistent_k
         s_sb[tid] = (g.out_packed && o < g.O) ? make_float2(g.scale[o], g.bias[o]) : make_float2(0.f, 0.f);
     }
     if (tid < 16) s_bounds[tid] = make_float4(g.rb.bound[tid][0], g.rb.bound[tid][1], g.rb.bound[tid][2], 0.f);
+    if (tid == 32 && g.off_thr) *reinterpret_cast<int*>(tc_smem + g.off_thr + g.thr_pats * g.TN * 16) = 1;
     tc_build_lut(g, s_lut, tid, blockDim.x);
     tc_fence_before();
     __syncthreads();
@@ -778,6 +887,14 @@ __global__ void __launch_bounds__(TCP_THREADS, 3) bitserial_conv_tc_persistent_k
         if (!ok) atomicOr(g.status, STATUS_TIMEOUT);
     } else {
         // ------------------------------------------------------------------ epilogue (warps 0-3)
+        uint32_t thr = 0;                 // shared-memory address of the thresholds, 0: floating-point comparison
+        if (g.off_thr) {                  // while the pipeline fills: comparison bounds -> integer thresholds
+            int4* s_thr = reinterpret_cast<int4*>(tc_smem + g.off_thr);
+            int* thr_ok = reinterpret_cast<int*>(s_thr + g.thr_pats * g.TN);
+            tc_build_thresholds(g, s_thr, thr_ok, s_sb, s_bounds, o0, tid, 128);
+            group_sync(2);
+            if (*thr_ok) thr = smem_u32(s_thr);
+        }
         pdl_acquire();                    // the epilogue reads the residual and overwrites buffers the preceding kernel may use
         int i = 0;
         bool ok = true;
@@ -787,7 +904,7 @@ __global__ void __launch_bounds__(TCP_THREADS, 3) bitserial_conv_tc_persistent_k
             if (!ok) break;
             tc_fence_after();
             const TcTile tile = tc_decode_tile(g, mt);
-            tc_epilogue_tile(g, tmem_base + static_cast<uint32_t>(buf * g.TN), tid, warp, tile, o0, s_sb, s_bounds);
+            tc_epilogue_tile(g, tmem_base + static_cast<uint32_t>(buf * g.TN), tid, warp, tile, o0, s_sb, s_bounds, thr);
             tc_fence_before();
             group_sync(2);                           // all four warps have read their accumulator rows
             if (tid == 0) mbar_arrive(&empty_acc[buf]);
@@ -1082,6 +1199,23 @@ static int tc_conv_impl(const uint32_t* act, const int8_t* wgt, const bs_conv_pa
                                out_packed ? p->out_bits : 0, p->out_sign);
     if (!out_packed) g.rb.enabled = 0;
 
+    // Integer thresholds for the comparison epilogue, when they fit without costing a resident CTA.  With 2-bit
+    // activations the nibble-pair table fills only the first 1 KB of the 4 KB table region; the rest is reused.
+    auto ctas_per_sm = [](size_t bytes) { return static_cast<int>((225 * 1024) / (bytes + 1024)); };
+    g.off_thr = 0;
+    g.thr_pats = g.residual ? 4 : 1;
+    if (g.rb.enabled && (!g.residual || p->res_bits <= 2) &&
+        static_cast<long long>(p->C) * RS * tc_max_abs(p->a_bits, p->a_sign) * tc_max_abs(p->w_bits, p->w_sign) < TC_THR_LIM) {
+        const size_t bytes = static_cast<size_t>(g.thr_pats) * g.TN * 16 + 16;
+        const size_t off = A == 2 ? static_cast<size_t>(g.off_lut) + 1024 : smem;
+        const size_t grown = off + bytes > smem ? off + bytes : smem;
+        const bool same_occupancy = !g.persistent || ctas_per_sm(grown) >= (ctas_per_sm(smem) < 3 ? ctas_per_sm(smem) : 3);
+        if (grown <= 220 * 1024 && same_occupancy) {
+            g.off_thr = static_cast<int>(off);
+            smem = grown;
+        }
+    }
+
     auto enc = tc_encode_fn();
     if (!enc) return BS_ERR_CUDA;
     const cuuint64_t fullA = static_cast<cuuint64_t>(Cw) * A;
@@ -1106,7 +1240,7 @@ static int tc_conv_impl(const uint32_t* act, const int8_t* wgt, const bs_conv_pa
     if (cr != CUDA_SUCCESS) return BS_ERR_CUDA;
 
     if (g.persistent) {
-        int cps = static_cast<int>((225 * 1024) / (smem + 1024));          // CTAs that fit on one SM: shared memory,
+        int cps = ctas_per_sm(smem);                                       // CTAs that fit on one SM: shared memory,
         if (cps > 3) cps = 3;                                              // registers (launch bounds) and
         if (cps * 2 * g.TN > 512) cps = 512 / (2 * g.TN);                  // tensor-memory columns
         if (cps < 1) cps = 1;

@@ -117,6 +117,37 @@ def test_tc_residual_matches_oracle_and_popcount_path():
     assert np.array_equal(packed, oracle.pack_activations(codes, 2, 0))
 
 
+@pytest.mark.parametrize("kind", ["extreme_positive", "mixed_sign"])
+@pytest.mark.parametrize("with_res", [False, True])
+@pytest.mark.parametrize("out", [(2, 0), (2, 1), (1, 0), (1, 2)])
+def test_tc_epilogue_scale_bias_corner_cases(kind, with_res, out):
+    """Per-filter scales and biases at the corners of the comparison epilogue: tiny and huge positive scales with
+    biases that push every threshold out of the accumulator range (integer thresholds saturate), and filters with
+    zero or negative scale (the kernel must fall back to the floating-point comparison)."""
+    out_bits, out_sign = out
+    c = wl.single_conv_case(seed=31, N=2, C=64, H=13, W=13, O=96, calibrated=True)
+    rng = np.random.default_rng(5)
+    scale, bias = c["scale"].copy(), c["bias"].copy()
+    O = scale.shape[0]
+    scale[0::7] = 1e-6; scale[1::7] = 3e5; scale[2::7] = 1e-30
+    bias[0::5] = 1e6; bias[1::5] = -1e6; bias[2::5] = 0.5; bias[3::5] = 2.5
+    if kind == "mixed_sign":
+        scale[3::11] *= -1.0
+        scale[4::11] = 0.0
+    res = wl.rand_codes(rng, (2, O, 13, 13), 2, 0) if with_res else None
+    xa = api.bitpack_activations(dev(c["x"]), 1.0, 2, 0, api.NCHW)
+    wp = api.pack_weights(dev(c["w"]), 2, c["w_sign"], api.NCHW)
+    wt = api.tc_prepare_weights(wp, 64, c["w_sign"], 2)
+    res_t = api.bitpack_activations(dev(res), 1.0, 2, 0, api.NCHW) if with_res else None
+    _, packed = api.bitserial_conv2d(xa, wp, C=64, stride=1, pad=1, w_sign=c["w_sign"], scale=dev(scale), bias=dev(bias), relu=True,
+                                     out_bits=out_bits, out_sign=out_sign, residual=res_t, res_scale=0.75 if with_res else 0.0,
+                                     res_bits=2 if with_res else 0, res_c_total=O if with_res else 0, wgt_tc=wt)
+    api.bs_check_status()
+    want = oracle.conv2d_i32(c["x"], c["w"], 1, 1)
+    codes = oracle.requantize(want, scale, bias, True, out_bits, out_sign, res=res, res_scale=0.75 if with_res else 0.0)
+    assert np.array_equal(words(packed), oracle.pack_activations(codes, out_bits, out_sign))
+
+
 @pytest.mark.parametrize("M,N,K", [(1, 8, 64), (130, 40, 128), (300, 72, 1024), (1031, 96, 64), (256, 256, 576), (1024, 1024, 2304)])
 def test_tc_gemm(M, N, K):
     c = wl.gemm_case(M, N, K, seed=M + N + K)
