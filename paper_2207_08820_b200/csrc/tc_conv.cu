@@ -21,7 +21,8 @@
 
 namespace bs {
 
-constexpr int TC_THREADS = 192;       // warps 0-3: expand + epilogue, warp 4: TMA producer, warp 5: MMA issuer
+constexpr int TC_THREADS = 320;       // warps 0-3 and 6-9: expand + epilogue, warp 4: TMA producer, warp 5: MMA issuer
+constexpr int TC_WORKERS = 256;       // threads of the eight expand + epilogue warps
 constexpr int TC_M = 128;             // pixels per tile = 16 row groups x 8 columns (or 128 flat pixels)
 constexpr int TC_MAX_STAGES = 2;
 
@@ -70,8 +71,8 @@ __device__ __forceinline__ void mbar_arrive(uint64_t* bar)
 {
     asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
 }
-// Barrier among the 128 threads of one warp group (expanders or epilogue); ids 1 and 2, id 0 is __syncthreads.
-__device__ __forceinline__ void group_sync(int id) { asm volatile("bar.sync %0, 128;" ::"r"(id) : "memory"); }
+// Barrier among the threads of one warp group (expanders or epilogue); ids 1 and 2, id 0 is __syncthreads.
+__device__ __forceinline__ void group_sync(int id, int nthreads = 128) { asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(nthreads) : "memory"); }
 // Low-latency bounded wait for the tensor-core pipeline: non-blocking test_wait in a spin loop (try_wait may park the
 // thread and wake it late, which costs microseconds per hand-off between the roles).  About a second at most.
 __device__ __forceinline__ bool mbar_spin_bounded(uint64_t* bar, unsigned parity)
@@ -234,22 +235,24 @@ __device__ __forceinline__ void tc_build_lut(const TcArgs& g, uint2* lut, int ti
 // kernel so that the per-item loop has no division.  Items are (pixel, channel word) pairs, channel word fastest;
 // a chunk has one or two channel words.
 struct TcExpand {
-    int cw;            // channel word of this thread's items (the item stride 128 is a multiple of the words per chunk)
+    int cw;            // channel word of this thread's items (the item stride is a multiple of the words per chunk)
     int x2, y2;        // first item's position in the (possibly subsampled) halo grid
-    int dx, dy;        // movement of 128 items
+    int dx, dy;        // movement of `step` items
     int nx, items;
+    int step;          // threads of the expander group
 };
 
-__device__ __forceinline__ TcExpand tc_expand_init(const TcArgs& g, int et)
+__device__ __forceinline__ TcExpand tc_expand_init(const TcArgs& g, int et, int nthreads)
 {
     TcExpand x;
+    x.step = nthreads;
     const int sub = (!g.flat && g.stride == 2 && g.R == 1) ? 2 : 1;
     x.nx = g.flat ? TC_M : (g.hw + sub - 1) / sub;
     const int ny = g.flat ? 1 : (g.TNI * g.hh + sub - 1) / sub;   // hh is even for stride 2: rows of all images keep their parity
     x.items = x.nx * ny * g.CWC;
     const int sh = g.CWC >> 1;                                     // CWC is 1 or 2
     x.cw = et & (g.CWC - 1);
-    const int pp = et >> sh, pstep = 128 >> sh;
+    const int pp = et >> sh, pstep = nthreads >> sh;
     x.y2 = pp / x.nx; x.x2 = pp - x.y2 * x.nx;
     x.dy = pstep / x.nx; x.dx = pstep - x.dy * x.nx;
     return x;
@@ -271,7 +274,7 @@ __device__ __forceinline__ void tc_expand_items(const TcArgs& g, const TcExpand&
     int x2 = x.x2, y2 = x.y2;
     const uint32_t* src_c = pa + (c * g.CWC + cw) * A;
     unsigned char* dst_c = eb + static_cast<size_t>(2 * cw) * plane_bytes;
-    for (int it = et; it < x.items; it += 128) {
+    for (int it = et; it < x.items; it += x.step) {
         int hp, ep;
         if (MODE == 0) {
             hp = ep = x2;
@@ -515,7 +518,7 @@ __device__ __forceinline__ void tc_compare_int(const uint32_t (&v)[32], uint32_t
 
 // Epilogue of one tile: thread `tid` (0..127, warp = TMEM lane quadrant) owns accumulator row tid = one output pixel.
 __device__ __forceinline__ void tc_epilogue_tile(const TcArgs& g, uint32_t tmem_acc, int tid, int warp, const TcTile& tile, int o0,
-                                                 const float2* s_sb, const float4* s_bounds, uint32_t thr_addr)
+                                                 const float2* s_sb, const float4* s_bounds, uint32_t thr_addr, int cc0 = 0, int ccstep = 1)
 {
     const int n0 = tile.n0, p0 = tile.p0, q0 = tile.q0;
     const int m = tid;                               // TMEM lane = tile pixel
@@ -539,7 +542,7 @@ __device__ __forceinline__ void tc_epilogue_tile(const TcArgs& g, uint32_t tmem_
     code_limits(g.out_bits > 0 ? g.out_bits : 1, g.out_sign, qmin, qmax);
     const float fqmin = static_cast<float>(qmin), fqmax = static_cast<float>(qmax);
     const float4 bnd0 = s_bounds[0];
-    for (int cc = 0; cc < g.TN / 32; ++cc) {
+    for (int cc = cc0; cc < g.TN / 32; cc += ccstep) {       // groups of 32 filters; two warps may share a lane quadrant
         uint32_t v[32];
         tmem_ld32(tmem_acc + (static_cast<uint32_t>(warp * 32) << 16) + static_cast<uint32_t>(cc * 32), v);
         tmem_ld_wait();
@@ -719,9 +722,10 @@ __global__ void __launch_bounds__(TC_THREADS) bitserial_conv_tc_kernel(const __g
         }
         __syncwarp();
     } else {
-        // ------------------------------------------------------------------ expanders (warps 0-3), then epilogue
+        // ------------------------------------------------------------------ expanders (warps 0-3, 6-9), then epilogue
         pdl_acquire();                    // the epilogue reads the residual and overwrites buffers the preceding kernel may use
-        const TcExpand xp = tc_expand_init(g, tid);
+        const int ct = warp < 4 ? tid : tid - 64;          // 0..255 among the workers
+        const TcExpand xp = tc_expand_init(g, ct, TC_WORKERS);
         bool ok = mbar_wait_warp(full_a, 0, lane);
         for (int c = 0; c < g.nchunks; ++c) {
             const int e = c % g.nse, k = c / g.nse;
@@ -729,9 +733,9 @@ __global__ void __launch_bounds__(TC_THREADS) bitserial_conv_tc_kernel(const __g
             if (!ok) atomicOr(g.status, STATUS_TIMEOUT);
             for (int t = 0; t < nt; ++t)
                 tc_expand_chunk<A>(g, xp, reinterpret_cast<const uint32_t*>(tc_smem + g.off_p + t * g.pa_bytes),
-                                   tc_smem + g.off_e + e * e_stage + t * g.e_bytes, s_lut, tid, c);
+                                   tc_smem + g.off_e + e * e_stage + t * g.e_bytes, s_lut, ct, c);
             fence_proxy_async();          // make the generic-proxy writes visible to the tensor core's reads
-            group_sync(1);
+            group_sync(1, TC_WORKERS);
             if (tid == 0) mbar_arrive(&full_e[e]);
         }
         // the last chunks are still in the tensor core: time to turn the comparison bounds into integer thresholds
@@ -739,15 +743,18 @@ __global__ void __launch_bounds__(TC_THREADS) bitserial_conv_tc_kernel(const __g
         if (g.off_thr) {
             int4* s_thr = reinterpret_cast<int4*>(tc_smem + g.off_thr);
             int* thr_ok = reinterpret_cast<int*>(s_thr + g.thr_pats * g.TN);
-            tc_build_thresholds(g, s_thr, thr_ok, s_sb, s_bounds, o0, tid, 128);
-            group_sync(1);
+            tc_build_thresholds(g, s_thr, thr_ok, s_sb, s_bounds, o0, ct, TC_WORKERS);
+            group_sync(1, TC_WORKERS);
             if (*thr_ok) thr = smem_u32(s_thr);
         }
         if (ok) ok = mbar_wait_warp(accum_full, 0, lane);
         if (!ok) atomicOr(g.status, STATUS_TIMEOUT);
         tc_fence_after();
         for (int t = 0; t < nt; ++t)
-            tc_epilogue_tile(g, tmem_base + static_cast<uint32_t>(t * g.TN), tid, warp, tc_decode_tile(g, mt0 + t), o0, s_sb, s_bounds, thr);
+            // a warp reads the tensor-memory lanes of quadrant (warp % 4): warps 0-3 take the even groups of 32 filters,
+            // warps 6-9 (quadrants 2, 3, 0, 1) the odd ones
+            tc_epilogue_tile(g, tmem_base + static_cast<uint32_t>(t * g.TN), (warp & 3) * 32 + lane, warp & 3, tc_decode_tile(g, mt0 + t), o0,
+                             s_sb, s_bounds, thr, warp < 4 ? 0 : 1, 2);
         tc_fence_before();
     }
     __syncthreads();
@@ -866,7 +873,7 @@ __global__ void __launch_bounds__(TCP_THREADS, 3) bitserial_conv_tc_persistent_k
     } else if (warp >= 4) {
         // ------------------------------------------------------------------ expanders (warps 4-7)
         const int et = tid - 128;
-        const TcExpand xp = tc_expand_init(g, et);
+        const TcExpand xp = tc_expand_init(g, et, 128);
         int it = 0, i = 0;
         bool ok = true;
         for (int mt = first_tile; mt < tiles_m && ok; mt += tile_step, ++i) {
@@ -1156,9 +1163,12 @@ static int tc_conv_impl(const uint32_t* act, const int8_t* wgt, const bs_conv_pa
         }
         if (g.persistent) break;
     }
-    // A resident plan that had to shrink the filter tile to 32 wastes the tensor core (an N = 32 MMA costs as many
-    // cycles as N = 64): stream the filters instead when a 128-wide tile leaves enough (pixel tile, filter tile) pairs.
-    if (!keep_narrow && g.persistent && g.TN == 32 && p->O >= 128 && tiles_m * ceil_div(p->O, 128) >= sms / 2) g.persistent = 0;
+    // A resident plan that had to shrink the filter tile wastes the tensor core (an N = 32 MMA costs as many cycles
+    // as N = 64, and N = 64 only a fifth less than N = 128): stream the filters instead when a 128-wide tile leaves
+    // enough (pixel tile, filter tile) pairs -- always for N = 32, for N = 64 when the reduction is deep (measured).
+    if (!keep_narrow && g.persistent && (g.TN == 32 || (g.TN == 64 && g.nchunks >= 4)) && p->O >= 128 &&
+        tiles_m * ceil_div(p->O, 128) >= sms / 2)
+        g.persistent = 0;
     if (force_stream) g.persistent = 0;
     g.PT = 1;
     if (!g.persistent) {
