@@ -289,6 +289,11 @@ __global__ void __launch_bounds__(256, (PB * FB <= 32) ? 3 : 1) bitserial_conv_k
     for (int i = 0; i < WB; ++i)
 #pragma unroll
         for (int j = 0; j < A; ++j) coef[i][j] = g.coef[i][j];
+    int coef2[WB][A];
+#pragma unroll
+    for (int i = 0; i < WB; ++i)
+#pragma unroll
+        for (int j = 0; j < A; ++j) coef2[i][j] = 2 * g.coef[i][j];
 
     // window sums for the bipolar corrections: thread tid covers tile pixels tid, tid + nthreads, ...
     int rs_acc[4] = {0, 0, 0, 0};
@@ -308,18 +313,47 @@ __global__ void __launch_bounds__(256, (PB * FB <= 32) ? 3 : 1) bitserial_conv_k
         }
         if (any_cp) __syncthreads();
 
-        // ---- plane-pair popcount MACs over all taps and words of this chunk (idle pixel groups skip them)
+        // ---- plane-pair popcount MACs over all taps and words of this chunk (idle pixel groups skip them).
+        // Within a filter row the reduction words (tap column, channel word) are contiguous for both operands.  They
+        // are taken three at a time through a carry-save adder: with x_q = a_q & w_q,
+        //     popc(x0) + popc(x1) + popc(x2) = popc(x0 ^ x1 ^ x2) + 2 * popc(maj(x0, x1, x2)),
+        // i.e. two population counts (the scarce pipe: 16 lanes per clock per SM) and two 3-input logic operations
+        // instead of three counts.  A remainder of one or two words takes the plain form.
         if (pg_used)
-        for (int tap = 0; tap < RS; ++tap) {
-            const int r = tap / g.S, sx = tap - r * g.S;
-            const uint32_t* pa = sA + a_off0 + (r * g.hw + sx) * recA;
-            const uint32_t* pw = sW + w_off0 + tap * recW;
-            for (int cw = 0; cw < g.CWC; ++cw) {
+        for (int r = 0; r < g.R; ++r) {
+            const uint32_t* par = sA + a_off0 + r * g.hw * recA;
+            const uint32_t* pwr = sW + w_off0 + r * g.S * recW;
+            const int M = g.S * g.CWC;
+            int m = 0;
+            for (; m + 3 <= M; m += 3) {
+                uint32_t w[3][FB][WB];
+#pragma unroll
+                for (int q = 0; q < 3; ++q)
+#pragma unroll
+                    for (int u = 0; u < FB; ++u) load_planes<WB>(pwr + u * w_fstep + (m + q) * WB, w[q][u]);
+#pragma unroll
+                for (int v = 0; v < PB; ++v) {
+                    uint32_t a[3][A];
+#pragma unroll
+                    for (int q = 0; q < 3; ++q) load_planes<A>(par + v * a_pstep + (m + q) * A, a[q]);
+#pragma unroll
+                    for (int u = 0; u < FB; ++u)
+#pragma unroll
+                        for (int i = 0; i < WB; ++i)
+#pragma unroll
+                            for (int j = 0; j < A; ++j) {
+                                const uint32_t x0 = a[0][j] & w[0][u][i], x1 = a[1][j] & w[1][u][i], x2 = a[2][j] & w[2][u][i];
+                                const uint32_t sum = x0 ^ x1 ^ x2, carry = (x0 & x1) | (x2 & (x0 ^ x1));
+                                acc[v][u] += coef[i][j] * __popc(sum) + coef2[i][j] * __popc(carry);
+                            }
+                }
+            }
+            for (; m < M; ++m) {
                 uint32_t a[PB][A], w[FB][WB];
 #pragma unroll
-                for (int v = 0; v < PB; ++v) load_planes<A>(pa + v * a_pstep + cw * A, a[v]);
+                for (int v = 0; v < PB; ++v) load_planes<A>(par + v * a_pstep + m * A, a[v]);
 #pragma unroll
-                for (int u = 0; u < FB; ++u) load_planes<WB>(pw + u * w_fstep + cw * WB, w[u]);
+                for (int u = 0; u < FB; ++u) load_planes<WB>(pwr + u * w_fstep + m * WB, w[u]);
 #pragma unroll
                 for (int v = 0; v < PB; ++v)
 #pragma unroll

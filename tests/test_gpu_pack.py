@@ -25,6 +25,28 @@ def test_bitpack_fp32_nchw_matches_oracle(bits, sign, shape):
     assert np.array_equal(got, want)
 
 
+@pytest.mark.parametrize("bits,sign", [(1, 0), (2, 0), (2, 1), (1, 2), (3, 0)])
+@pytest.mark.parametrize("s", [0.37, 1.0, 2.5e-3, 1e-38])
+def test_bitpack_special_values(bits, sign, s):
+    """NaN, infinities, signed zeros, denormals and the neighbours of every rounding tie: the sign-bit form of the
+    quantiser must take the decision of the Section IV formula on all of them."""
+    lo, hi = wl.code_range(bits, sign)
+    s32 = np.float32(s)
+    ties = (np.arange(lo - 1, hi + 2, dtype=np.float32) + np.float32(0.5)) * s32
+    near = np.concatenate([ties, np.nextafter(ties, np.float32(np.inf)), np.nextafter(ties, np.float32(-np.inf)),
+                           np.arange(lo - 1, hi + 2, dtype=np.float32) * s32])
+    special = np.array([np.nan, np.inf, -np.inf, 0.0, -0.0, 1e-45, -1e-45, 1e-39, -1e-39, 3e38, -3e38, 1.0, -1.0], dtype=np.float32)
+    vals = np.concatenate([near, special]).astype(np.float32)
+    rng = np.random.default_rng(3)
+    x = rng.choice(vals, size=(2, 64, 6, 17)).astype(np.float32)
+    with np.errstate(all="ignore"):
+        want = oracle.pack_activations(oracle.quantize(x, s, bits, sign), bits, sign)
+    got = words(api.bitpack_activations(dev(x), s, bits, sign, api.NCHW))
+    assert np.array_equal(got, want)
+    got = words(api.bitpack_activations(dev(np.ascontiguousarray(x.transpose(0, 2, 3, 1))), s, bits, sign, api.NHWC))
+    assert np.array_equal(got, want)
+
+
 @pytest.mark.parametrize("bits,sign", [(2, 0), (3, 1), (1, 2)])
 @pytest.mark.parametrize("shape", [(2, 64, 9, 11), (1, 70, 6, 50)])
 def test_bitpack_nhwc_and_int8_inputs(bits, sign, shape):
