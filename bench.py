@@ -31,7 +31,7 @@ ACT_SCALE = 0.25
 METRIC = "bitserial_conv_effective_gops"
 UNIT = "GOPS"
 POPC_PER_CLK_PER_SM = 16          # population count throughput per SM per clock (CUDA programming guide, arithmetic table)
-WORDS_PER_POPC = 1.5              # the kernel's 3:2 carry-save adder: three popc32(AND) word operations cost two counts
+POPC_PER_WORDOP = 2.0 / 3.0       # executed by the kernel's 3:2 carry-save adder: three popc32(AND) word operations cost two counts
 
 
 def make_net(name: str, batch: int):
@@ -272,7 +272,7 @@ def run_ours(args):
         gops = 2.0 * macs * world / (t_step * 1e-3) / 1e9
         peaks, peak_kind = measured_peaks()
         sms = torch.cuda.get_device_properties(local).multi_processor_count
-        popc_peak = WORDS_PER_POPC * POPC_PER_CLK_PER_SM * sms * peaks["sm_max_mhz"] * 1e6   # word-ops/s at the maximum SM clock
+        popc_peak = POPC_PER_CLK_PER_SM * sms * peaks["sm_max_mhz"] * 1e6          # counts/s at the maximum SM clock
         popc_measured = api.bs_popc_rate(4096)
         int8_peak_tops = 2.0 * peaks.get("bf16_tflops_sustained", peaks["bf16_tflops"])   # dense int8 = 2 x bf16 (nominal ratio)
 
@@ -280,8 +280,10 @@ def run_ours(args):
             a = wops / (t_ms * 1e-3)
             return {"bound": "alu", "kernel": "bitserial_conv_kernel", "achieved": a / 1e12, "peak": popc_peak / 1e12,
                     "unit": "Tword-op/s", "frac": a / popc_peak, "traffic": None,
-                    "peak_source": f"{WORDS_PER_POPC} words per popc (3:2 carry-save) x {POPC_PER_CLK_PER_SM} popc/clk/SM x {sms} SMs x "
-                                   f"{peaks['sm_max_mhz']:.0f} MHz ({peak_kind} clock)",
+                    "peak_source": f"{POPC_PER_CLK_PER_SM} popc/clk/SM x {sms} SMs x {peaks['sm_max_mhz']:.0f} MHz ({peak_kind} clock); "
+                                   "achieved counts ALGORITHMIC word operations, the kernel's 3:2 carry-save adder executes 2/3 "
+                                   "as many population counts, so frac can exceed 1 (frac_executed is on the executed counts)",
+                    "frac_executed": a * POPC_PER_WORDOP / popc_peak,
                     "popc_pipe_measured": popc_measured / 1e12, "launches_per_step": len(net.layers),
                     "avg_launch_ms": t_ms / len(net.layers)}
 
