@@ -39,6 +39,10 @@ def make_net(name: str, batch: int):
         return wl.resnet18_body(batch), 3000
     if name == "detection_backbone":
         return wl.detection_backbone(batch), 4000
+    if name == "resnet50_body":
+        return wl.resnet50_body(batch), 6000
+    if name == "vgg16_ssd_body":
+        return wl.vgg16_ssd_body(batch), 7000
     raise SystemExit(f"unknown workload {name}")
 
 
@@ -358,8 +362,8 @@ def main():
     ap.add_argument("--steps", type=int, default=50)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="resnet18_body", choices=["resnet18_body", "detection_backbone"])
-    ap.add_argument("--batch", type=int, default=0, help="images per GPU (default: 64 / 16 as the workload defines)")
+    ap.add_argument("--workload", default="resnet18_body", choices=["resnet18_body", "detection_backbone", "resnet50_body", "vgg16_ssd_body"])
+    ap.add_argument("--batch", type=int, default=0, help="images per GPU (default: 64 / 16 / 32 / 8 as the workload defines)")
     ap.add_argument("--ref-images", type=int, default=2, help="images per step of the reference arm (bounded CPU sample)")
     ap.add_argument("--cpu-baseline-images", type=int, default=64, help="images of the one oracle pass timed beside the GPU run")
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -368,7 +372,7 @@ def main():
     ap.add_argument("--eager", action="store_true", help="plain stream launches instead of CUDA graphs (for per-launch profiling)")
     args = ap.parse_args()
     if args.batch == 0:
-        args.batch = 64 if args.workload == "resnet18_body" else 16
+        args.batch = {"resnet18_body": 64, "detection_backbone": 16, "resnet50_body": 32, "vgg16_ssd_body": 8}[args.workload]
     if args.warmup < 3 and args.impl == "ours":
         args.warmup = 3
     if args.impl == "reference":

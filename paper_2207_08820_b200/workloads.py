@@ -233,6 +233,47 @@ def resnet18_body(batch: int = 64, hw: int = 56) -> NetSpec:
     return net
 
 
+def resnet50_body(batch: int = 32, hw: int = 56) -> NetSpec:
+    """conv2_x .. conv5_x of a 50-layer residual network at 224 px input: stages of 3/4/6/3 bottleneck blocks
+    (1x1 c_in -> c, 3x3 c -> c carrying the stride, 1x1 c -> 4c + shortcut; c = 64/128/256/512), a 1x1 projection
+    shortcut in the first block of every stage.  The first packed tensor is the 64-channel output of the
+    floating-point stem; stem and classifier are not part of the stack."""
+    net = NetSpec(name="resnet50_body", batch=batch, in_name="x0", in_shape=(64, hw, hw))
+    cur, c_in = "x0", 64
+    for si, (c, nblocks) in enumerate(((64, 3), (128, 4), (256, 6), (512, 3))):
+        for b in range(nblocks):
+            stride = 2 if (si > 0 and b == 0) else 1
+            tag = f"s{si + 2}b{b}"
+            shortcut = cur
+            if b == 0:
+                shortcut = f"{tag}_sc"
+                net.layers.append(ConvSpec(f"{tag}_down", cur, shortcut, c_in, 4 * c, 1, stride, 0, relu=False))
+            net.layers.append(ConvSpec(f"{tag}_1x1a", cur, f"{tag}_a", c_in, c, 1, 1, 0))
+            net.layers.append(ConvSpec(f"{tag}_3x3", f"{tag}_a", f"{tag}_b", c, c, 3, stride, 1))
+            net.layers.append(ConvSpec(f"{tag}_1x1b", f"{tag}_b", f"{tag}_out", c, 4 * c, 1, 1, 0, res=shortcut, res_scale=RES_SCALE))
+            cur, c_in = f"{tag}_out", 4 * c
+    net.out_name = cur
+    return net
+
+
+def vgg16_ssd_body(batch: int = 8, hw: int = 300) -> NetSpec:
+    """The 3x3 conv layers of a 16-layer plain network at 300 px (single-shot-detector sized input) after its first,
+    floating-point layer: conv1_2 (64 -> 64 at 300 px), then 2 x 128 at 150 px, 3 x 256 at 75 px, 3 x 512 at 38 px and
+    3 x 512 at 19 px.  The 2x2 poolings between the groups are written as the stride of the next group's first
+    conv (a pooling kernel is not part of the hot path; the layer shapes and MAC counts of the groups are kept)."""
+    net = NetSpec(name="vgg16_ssd_body", batch=batch, in_name="x0", in_shape=(64, hw, hw))
+    cur, c_in = "x0", 64
+    groups = ((64, 1), (128, 2), (256, 3), (512, 3), (512, 3))
+    for gi, (c, n) in enumerate(groups):
+        for k in range(n):
+            stride = 2 if (gi > 0 and k == 0) else 1
+            name = f"g{gi + 1}_{k + 1}"
+            net.layers.append(ConvSpec(name, cur, name + "_out", c_in, c, 3, stride, 1))
+            cur, c_in = name + "_out", c
+    net.out_name = cur
+    return net
+
+
 def detection_backbone(batch: int = 16, hw: int = 320) -> NetSpec:
     """Detection-backbone-shaped stack at 640 px input (first packed tensor 32 x 320 x 320): four
     stages, each a 3x3 stride-2 conv c/2 -> c followed by a cross-stage block with n bottlenecks:

@@ -72,3 +72,20 @@ def test_resnet18_body_tensor_core_full_batch_graph_sampled():
 
 def test_detection_backbone_tensor_core_full_size_sampled():
     compare_stack(wl.detection_backbone(16), 16, seed=4000, sample=[0, 15], graph=True, engine="tc")
+
+
+@pytest.mark.parametrize("engine", ["popc", "tc"])
+def test_resnet50_body_small(engine):
+    """Bottleneck stack (1x1 / 3x3 / 1x1 with 4x widening, projection shortcuts) at a reduced resolution."""
+    compare_stack(wl.resnet50_body(2, hw=16), 2, seed=6000, engine=engine)
+
+
+@pytest.mark.parametrize("engine", ["popc", "tc"])
+def test_vgg16_ssd_body_small(engine):
+    """Plain 3x3 stack with odd intermediate widths (40 -> 20 -> 10 -> 5 -> 3) at a reduced resolution."""
+    compare_stack(wl.vgg16_ssd_body(1, hw=40), 1, seed=7000, engine=engine)
+
+
+def test_vgg16_ssd_body_full_resolution_sampled():
+    """300 px: widths 300/150/75/38/19 (odd and even) through the tensor-core engine, one image checked."""
+    compare_stack(wl.vgg16_ssd_body(2), 2, seed=7000, sample=[1], graph=True, engine="tc")
