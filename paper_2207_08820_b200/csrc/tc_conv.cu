@@ -44,7 +44,7 @@ struct TcArgs {
     int i32_nhwc, acc_small;
     // tiling
     int flat;                         // 1: 128 consecutive pixels of the flattened image (1x1, stride 1)
-    int TN, CK, CWC, nchunks, nsp, nse;
+    int TN, CK, MB, CWC, nchunks, nsp, nse;   // CK: channels per filter-layout block, MB: blocks per pipeline chunk, CWC: words per chunk
     int fullA;                        // words of one packed pixel record (Cw * A)
     int pmode;                        // how a tile's packed halo is fetched: 0 flat bulk copy, 1 rows merged with W, 2 4-D box
     int TNI, GI, hh, hw;              // packed halo: TNI images x hh rows x hw columns; GI row groups per image
@@ -250,7 +250,7 @@ __device__ __forceinline__ TcExpand tc_expand_init(const TcArgs& g, int et, int 
     x.nx = g.flat ? TC_M : (g.hw + sub - 1) / sub;
     const int ny = g.flat ? 1 : (g.TNI * g.hh + sub - 1) / sub;   // hh is even for stride 2: rows of all images keep their parity
     x.items = x.nx * ny * g.CWC;
-    const int sh = g.CWC >> 1;                                     // CWC is 1 or 2
+    const int sh = __ffs(g.CWC) - 1;                               // CWC is a power of two (1 .. 8)
     x.cw = et & (g.CWC - 1);
     const int pp = et >> sh, pstep = nthreads >> sh;
     x.y2 = pp / x.nx; x.x2 = pp - x.y2 * x.nx;
@@ -340,7 +340,10 @@ struct TcIssue {
     uint32_t idesc;
     uint32_t row16, half16, kstep16;   // halo row, odd-column plane (stride 2) and second K half, in 16-byte units
     int R, S;
-    bool stride2, two;                 // even/odd column split; two K = 32 steps per tap (64-channel chunks)
+    bool stride2;                      // even/odd column split
+    int ksteps;                        // K = 32 steps per tap and layout block (block channels / 32)
+    int blocks;                        // layout blocks per chunk
+    uint32_t blk_b16;                  // filter tile of one layout block, in 16-byte units
 };
 
 __device__ __forceinline__ TcIssue tc_make_issue(const TcArgs& g)
@@ -359,7 +362,9 @@ __device__ __forceinline__ TcIssue tc_make_issue(const TcArgs& g)
     is.kstep16 = 2u * (lbo_a >> 4);
     is.R = g.R; is.S = g.S;
     is.stride2 = !g.flat && g.stride == 2;
-    is.two = g.CK == 64;
+    is.ksteps = g.CK >> 5;
+    is.blocks = g.MB;
+    is.blk_b16 = static_cast<uint32_t>(g.b_bytes / g.MB) >> 4;
     return is;
 }
 
@@ -377,22 +382,28 @@ __device__ __forceinline__ void umma_i8_words(uint32_t d_tmem, uint32_t a_lo, ui
 
 __device__ __forceinline__ void tc_issue_chunk(const TcIssue& is, uint32_t ea, uint32_t ba, uint32_t tmem_acc, bool first_chunk)
 {
-    uint32_t arow = is.a_lo + (ea >> 4);
-    uint32_t b = is.b_lo + (ba >> 4);              // filters: [tap][K half] tiles of 16 x 16 bytes, one after the other
     uint32_t acc = first_chunk ? 0u : 1u;          // the first MMA of a tile overwrites the accumulator
-    for (int r = 0; r < is.R; ++r) {
-        for (int sx = 0; sx < is.S; ++sx) {
-            const uint32_t a = arow + (is.stride2 ? static_cast<uint32_t>(sx & 1) * is.half16 + static_cast<uint32_t>(sx >> 1)
-                                                  : static_cast<uint32_t>(sx));
-            umma_i8_words(tmem_acc, a, is.a_hi, b, is.b_hi, is.idesc, acc);
-            acc = 1u;
-            b += 16;
-            if (is.two) {
-                umma_i8_words(tmem_acc, a + is.kstep16, is.a_hi, b, is.b_hi, is.idesc, 1u);
-                b += 16;
+    uint32_t ablk = is.a_lo + (ea >> 4);
+    uint32_t bblk = is.b_lo + (ba >> 4);
+    for (int blk = 0; blk < is.blocks; ++blk) {
+        uint32_t arow = ablk;
+        uint32_t b = bblk;                         // filters of a block: [tap][K half] tiles of 16 x 16 bytes, one after the other
+        for (int r = 0; r < is.R; ++r) {
+            for (int sx = 0; sx < is.S; ++sx) {
+                const uint32_t a = arow + (is.stride2 ? static_cast<uint32_t>(sx & 1) * is.half16 + static_cast<uint32_t>(sx >> 1)
+                                                      : static_cast<uint32_t>(sx));
+                uint32_t ak = a;
+                for (int kp = 0; kp < is.ksteps; ++kp) {
+                    umma_i8_words(tmem_acc, ak, is.a_hi, b, is.b_hi, is.idesc, acc);
+                    acc = 1u;
+                    ak += is.kstep16;
+                    b += 16;
+                }
             }
+            arow += is.row16;
         }
-        arow += is.row16;
+        ablk += static_cast<uint32_t>(is.ksteps) * is.kstep16;     // the block's 16-channel groups follow each other
+        bblk += is.blk_b16;
     }
 }
 
@@ -691,8 +702,11 @@ __global__ void __launch_bounds__(TC_THREADS) bitserial_conv_tc_kernel(const __g
                 }
                 if (k >= 1 && !mbar_spin_bounded(&empty_p[s], (k - 1) & 1)) { atomicOr(g.status, STATUS_TIMEOUT); break; }
                 mbar_expect_tx(&full_p[s], static_cast<unsigned>(g.b_bytes));
-                const size_t src = (static_cast<size_t>(c) * g.opad8 + (o0 >> 3)) * RS * (g.CK >> 4) * 128;
-                bulk_load(tc_smem + s * stage_p_bytes, g.wgt + src, static_cast<unsigned>(g.b_bytes), &full_p[s]);
+                const int blk_bytes = g.b_bytes / g.MB;
+                for (int j = 0; j < g.MB; ++j) {
+                    const size_t src = (static_cast<size_t>(c * g.MB + j) * g.opad8 + (o0 >> 3)) * RS * (g.CK >> 4) * 128;
+                    bulk_load(tc_smem + s * stage_p_bytes + j * blk_bytes, g.wgt + src, static_cast<unsigned>(blk_bytes), &full_p[s]);
+                }
             }
             if (early == g.nchunks) {
                 pdl_acquire();
@@ -831,9 +845,10 @@ __global__ void __launch_bounds__(TCP_THREADS, 3) bitserial_conv_tc_persistent_k
         // ------------------------------------------------------------------ producer: filters once, then packed chunks
         if (lane == 0) {
             mbar_expect_tx(wgt_full, static_cast<unsigned>(g.nchunks * g.b_bytes));
-            for (int c = 0; c < g.nchunks; ++c) {
+            const int blk_bytes = g.b_bytes / g.MB;
+            for (int c = 0; c < g.nchunks * g.MB; ++c) {       // layout blocks, consecutive in shared memory
                 const size_t src = (static_cast<size_t>(c) * g.opad8 + (o0 >> 3)) * RS * (g.CK >> 4) * 128;
-                bulk_load(s_w + static_cast<size_t>(c) * g.b_bytes, g.wgt + src, static_cast<unsigned>(g.b_bytes), wgt_full);
+                bulk_load(s_w + static_cast<size_t>(c) * blk_bytes, g.wgt + src, static_cast<unsigned>(blk_bytes), wgt_full);
             }
             pdl_acquire();                // activations come from the preceding kernel; the filters above do not
             int i = 0;
@@ -957,7 +972,8 @@ __global__ void tc_prepare_weights_kernel(const uint32_t* __restrict__ packed, i
 
 static int round_up_i(int v, int m) { return (v + m - 1) / m * m; }
 
-// Channels per pipeline chunk (and per block of the prepared filter layout): 64 when C allows, else 32.
+// Channels per block of the prepared filter layout: 64 when C allows, else 32.  A pipeline chunk is one block, or
+// several consecutive blocks for 1x1 stride-1 layers (one tap per block is only two MMAs per hand-off otherwise).
 static int tc_chunk_channels(int C, int /*a_bits*/)
 {
     if (C % 64 == 0) return 64;
@@ -1077,10 +1093,23 @@ static int tc_conv_impl(const uint32_t* act, const int8_t* wgt, const bs_conv_pa
     g.acc_small = kred * tc_max_abs(p->a_bits, p->a_sign) * tc_max_abs(p->w_bits, p->w_sign) < (1LL << 22);
 
     g.CK = tc_chunk_channels(p->C, A);
-    g.CWC = g.CK / 32;
+    g.MB = 1;
+    {
+        // 1x1 stride-1 layers: two 64-channel blocks per pipeline chunk (the expanded tile is 128 pixels x 128 channels =
+        // 16 KB per stage); four measured no better than two on the bottleneck and detection stacks
+        int wide = 2;
+#ifdef BS_TUNING
+        if (const char* e = getenv("BS_TC_MB")) wide = atoi(e);
+#endif
+        if (RS == 1 && p->stride == 1 && p->pad == 0 && g.CK == 64)
+            for (int mb = wide; mb > 1; mb /= 2)
+                if (p->C % (g.CK * mb) == 0) { g.MB = mb; break; }
+    }
+    const int CKP = g.CK * g.MB;                  // channels per pipeline chunk
+    g.CWC = CKP / 32;
     g.fullA = Cw * A;
     g.act = act;
-    g.nchunks = p->C / g.CK;
+    g.nchunks = p->C / CKP;
     g.nsp = g.nse = g.nchunks < TC_MAX_STAGES ? g.nchunks : TC_MAX_STAGES;
     g.opad8 = round_up_i(p->O, 128) / 8;
     g.flat = (p->R == 1 && p->stride == 1 && p->pad == 0);
@@ -1121,7 +1150,7 @@ static int tc_conv_impl(const uint32_t* act, const int8_t* wgt, const bs_conv_pa
         tiles_m = static_cast<long long>(g.tiles_q) * g.tiles_p * g.tiles_n;
     }
     g.pa_bytes = round_up_i(g.pa_tx_bytes, 128);
-    g.e_bytes = round_up_i((g.CK / 16) * g.HPE * 16, 128);
+    g.e_bytes = round_up_i((CKP / 16) * g.HPE * 16, 128);
     const int sms = 148;
     // Persistent plan: the filters of a tile (all channel chunks) stay resident in shared memory.  Largest filter tile
     // that fits and still leaves one (pixel tile, filter tile) pair per SM.
@@ -1144,14 +1173,14 @@ static int tc_conv_impl(const uint32_t* act, const int8_t* wgt, const bs_conv_pa
         if (TN / 2 >= round_up_i(p->O, 32)) continue;                      // tile twice as wide as the filter bank
         const long long pairs = tiles_m * ceil_div(p->O, TN);
         if (TN > 32 && pairs < sms) continue;
-        const size_t wbytes = static_cast<size_t>(g.nchunks) * TN * RS * g.CK;
+        const size_t wbytes = static_cast<size_t>(g.nchunks) * TN * RS * CKP;
         const int shapes[4][2] = {{2, 2}, {2, 2}, {2, 2}, {1, 2}};      // (packed-tile stages, expanded-chunk stages)
         for (const auto& sh : shapes) {
             const int nsp = sh[0], nse = sh[1];
             const size_t total = wbytes + static_cast<size_t>(nsp) * g.pa_bytes + static_cast<size_t>(nse) * g.e_bytes +
                                  static_cast<size_t>(TN) * 8 + 256 + bar_bytes + 128 + 16 + static_cast<size_t>(A) * TC_LUT_BYTES_PER_PLANE;
             if (total <= 220 * 1024) {
-                g.persistent = 1; g.TN = TN; g.b_bytes = TN * RS * g.CK; g.nse = nse; g.nsp = nsp;
+                g.persistent = 1; g.TN = TN; g.b_bytes = TN * RS * CKP; g.nse = nse; g.nsp = nsp;
                 g.off_p = static_cast<int>(wbytes);
                 g.off_e = g.off_p + nsp * g.pa_bytes;
                 g.off_sb = g.off_e + nse * g.e_bytes;
@@ -1179,7 +1208,7 @@ static int tc_conv_impl(const uint32_t* act, const int8_t* wgt, const bs_conv_pa
         while (TN > 32 && (TN / 2 >= round_up_i(p->O, 32) || tiles_m * ceil_div(p->O, TN) < sms / 2)) TN /= 2;
         int PT = stream_pt;
         auto stream_bytes = [&](int tn, int pt) {
-            return static_cast<size_t>(g.nsp) * tn * RS * g.CK + static_cast<size_t>(pt) * g.pa_bytes +
+            return static_cast<size_t>(g.nsp) * tn * RS * CKP + static_cast<size_t>(pt) * g.pa_bytes +
                    static_cast<size_t>(g.nse) * pt * g.e_bytes + 2 * tn * 4 + 256 + (4 * TC_MAX_STAGES + 3) * 8 + 128 +
                    16 + static_cast<size_t>(A) * TC_LUT_BYTES_PER_PLANE;
         };
@@ -1188,7 +1217,7 @@ static int tc_conv_impl(const uint32_t* act, const int8_t* wgt, const bs_conv_pa
         while (TN > 32 && stream_bytes(TN, PT) > 200 * 1024) TN /= 2;
         g.TN = TN;
         g.PT = PT;
-        g.b_bytes = TN * RS * g.CK;
+        g.b_bytes = TN * RS * CKP;
         g.off_p = g.nsp * g.b_bytes;
         g.off_e = g.off_p + PT * g.pa_bytes;
         g.off_sb = g.off_e + g.nse * PT * g.e_bytes;
