@@ -392,11 +392,12 @@ __device__ __forceinline__ void tc_issue_chunk(const TcIssue& is, uint32_t ea, u
             for (int sx = 0; sx < is.S; ++sx) {
                 const uint32_t a = arow + (is.stride2 ? static_cast<uint32_t>(sx & 1) * is.half16 + static_cast<uint32_t>(sx >> 1)
                                                       : static_cast<uint32_t>(sx));
-                uint32_t ak = a;
-                for (int kp = 0; kp < is.ksteps; ++kp) {
-                    umma_i8_words(tmem_acc, ak, is.a_hi, b, is.b_hi, is.idesc, acc);
-                    acc = 1u;
-                    ak += is.kstep16;
+                // straight-line per tap: a loop over the K steps costs the lone issuing thread tens of cycles per MMA
+                umma_i8_words(tmem_acc, a, is.a_hi, b, is.b_hi, is.idesc, acc);
+                acc = 1u;
+                b += 16;
+                if (is.ksteps == 2) {
+                    umma_i8_words(tmem_acc, a + is.kstep16, is.a_hi, b, is.b_hi, is.idesc, 1u);
                     b += 16;
                 }
             }
@@ -1110,7 +1111,7 @@ static int tc_conv_impl(const uint32_t* act, const int8_t* wgt, const bs_conv_pa
     g.fullA = Cw * A;
     g.act = act;
     g.nchunks = p->C / CKP;
-    g.nsp = g.nse = g.nchunks < TC_MAX_STAGES ? g.nchunks : TC_MAX_STAGES;
+    g.nsp = g.nse = g.nchunks < 2 ? g.nchunks : 2;
     g.opad8 = round_up_i(p->O, 128) / 8;
     g.flat = (p->R == 1 && p->stride == 1 && p->pad == 0);
     long long tiles_m;
@@ -1203,7 +1204,7 @@ static int tc_conv_impl(const uint32_t* act, const int8_t* wgt, const bs_conv_pa
     if (!g.persistent) {
         // Filters streamed chunk by chunk; a CTA takes PT pixel tiles (PT accumulators in tensor memory) so that every
         // filter chunk fetched from L2 serves PT tiles.  Widest filter tile that keeps about one CTA per SM.
-        g.nsp = g.nse = g.nchunks < TC_MAX_STAGES ? g.nchunks : TC_MAX_STAGES;
+        g.nsp = g.nse = g.nchunks < 2 ? g.nchunks : 2;
         int TN = 128;
         while (TN > 32 && (TN / 2 >= round_up_i(p->O, 32) || tiles_m * ceil_div(p->O, TN) < sms / 2)) TN /= 2;
         int PT = stream_pt;
