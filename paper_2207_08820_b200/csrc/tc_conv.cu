@@ -380,8 +380,38 @@ __device__ __forceinline__ void umma_i8_words(uint32_t d_tmem, uint32_t a_lo, ui
         ::"r"(d_tmem), "r"(a_lo), "r"(a_hi), "r"(b_lo), "r"(b_hi), "r"(idesc), "r"(accumulate) : "memory");
 }
 
+// Fully unrolled issue of one layout block for the commonest shape classes (stride 1, two K steps per tap): no loop
+// counters or branches between the MMAs of the lone issuing thread.
+template <int R, int S, bool STRIDE2>
+__device__ __forceinline__ void tc_issue_block_unrolled(const TcIssue& is, uint32_t arow, uint32_t b, uint32_t tmem_acc, uint32_t acc)
+{
+#pragma unroll
+    for (int r = 0; r < R; ++r) {
+#pragma unroll
+        for (int sx = 0; sx < S; ++sx) {
+            const uint32_t a = arow + (STRIDE2 ? static_cast<uint32_t>(sx & 1) * is.half16 + static_cast<uint32_t>(sx >> 1) : static_cast<uint32_t>(sx));
+            umma_i8_words(tmem_acc, a, is.a_hi, b, is.b_hi, is.idesc, (r == 0 && sx == 0) ? acc : 1u);
+            umma_i8_words(tmem_acc, a + is.kstep16, is.a_hi, b + 16, is.b_hi, is.idesc, 1u);
+            b += 32;
+        }
+        arow += is.row16;
+    }
+}
+
 __device__ __forceinline__ void tc_issue_chunk(const TcIssue& is, uint32_t ea, uint32_t ba, uint32_t tmem_acc, bool first_chunk)
 {
+    if (is.ksteps == 2 && is.R == is.S && (is.R == 3 || is.R == 1)) {
+        uint32_t arow0 = is.a_lo + (ea >> 4), b0 = is.b_lo + (ba >> 4), acc0 = first_chunk ? 0u : 1u;
+        for (int blk = 0; blk < is.blocks; ++blk) {
+            if (is.R == 1) tc_issue_block_unrolled<1, 1, false>(is, arow0, b0, tmem_acc, acc0);     // a lone tap has no column offset
+            else if (is.stride2) tc_issue_block_unrolled<3, 3, true>(is, arow0, b0, tmem_acc, acc0);
+            else tc_issue_block_unrolled<3, 3, false>(is, arow0, b0, tmem_acc, acc0);
+            acc0 = 1u;
+            arow0 += 2u * is.kstep16;
+            b0 += is.blk_b16;
+        }
+        return;
+    }
     uint32_t acc = first_chunk ? 0u : 1u;          // the first MMA of a tile overwrites the accumulator
     uint32_t ablk = is.a_lo + (ea >> 4);
     uint32_t bblk = is.b_lo + (ba >> 4);
