@@ -173,6 +173,7 @@ def run_ours(args):
         runner.forward(x_dev)
         api.bs_check_status(stream)
         def run_pack():
+            runner.prefetch_filters()
             api.bitpack_activations(x_dev, ACT_SCALE, net.a_bits, api.UNSIGNED, api.NCHW, out=in_buf.view(-1))
 
         def run_convs():

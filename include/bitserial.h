@@ -239,6 +239,16 @@ int bitserial_gemm_tc(const uint32_t* a_packed, const int8_t* w_tc, int M, int N
 int bs_check_status(void* stream);
 
 /*
+ * bs_l2_prefetch -- asks the memory system to bring `count` device buffers into the L2 cache (bulk prefetches; the
+ * kernel that issues them ends at once and the transfers overlap whatever runs next on `stream`).  Used at the start
+ * of a forward pass for the prepared filters of all layers, which a layer otherwise fetches from HBM chunk by chunk
+ * on its critical path (the paper keeps its weights in the CPU caches implicitly; it has no counterpart of this call).
+ *   buffers  HOST array of `count` device pointers, 16-byte aligned;  bytes  HOST array of sizes (rounded down to 16).
+ * Nothing is modified; a hint only.  Errors: BS_ERR_INVALID_ARG, BS_ERR_ALIGNMENT, BS_ERR_CUDA.
+ */
+int bs_l2_prefetch(const void* const* buffers, const size_t* bytes, int count, void* stream);
+
+/*
  * bs_popc_rate -- register-only micro-benchmark of the SM population-count pipe: every thread runs
  * `iters` rounds of independent  acc += popc(x & y)  chains.  Writes the measured rate in
  * popc32(AND) word-operations per second to *wordops_per_s (HOST pointer).  Synchronises the device.

@@ -83,6 +83,8 @@ def lib() -> ctypes.CDLL:
     L.bs_tc_supported.argtypes = [ctypes.POINTER(ConvParams)]
     L.bitserial_conv2d_tc.restype = i
     L.bitserial_conv2d_tc.argtypes = [vp, vp, ctypes.POINTER(ConvParams), vp, vp, vp]
+    L.bs_l2_prefetch.restype = i
+    L.bs_l2_prefetch.argtypes = [ctypes.POINTER(ctypes.c_void_p), ctypes.POINTER(ctypes.c_size_t), ctypes.c_int, vp]
     L.bitserial_conv2d_tc_chained.restype = i
     L.bitserial_conv2d_tc_chained.argtypes = [vp, vp, ctypes.POINTER(ConvParams), vp, vp, vp]
     L.bitserial_gemm_tc.restype = i
@@ -101,5 +103,5 @@ EXPORTED = ("bs_packed_act_bytes", "bs_packed_wgt_bytes", "bs_packed_rows_bytes"
             "bitunpack_activations", "pack_weights", "bs_pack_rows", "bitserial_conv2d", "bitserial_gemm",
             "bitserial_conv2d_ws", "bitserial_gemm_ws", "bs_conv_workspace_bytes", "bs_gemm_workspace_bytes",
             "bitserial_gemm_noalloc", "bs_gemm_noalloc_max_scratch_bytes",
-            "bs_tc_weights_bytes", "bs_tc_prepare_weights", "bs_tc_supported", "bitserial_conv2d_tc", "bitserial_conv2d_tc_chained", "bitserial_gemm_tc",
+            "bs_tc_weights_bytes", "bs_tc_prepare_weights", "bs_tc_supported", "bitserial_conv2d_tc", "bitserial_conv2d_tc_chained", "bitserial_gemm_tc", "bs_l2_prefetch",
             "bs_check_status", "bs_popc_rate", "bs_status_string")

@@ -239,6 +239,16 @@ def bs_check_status(stream=None) -> None:
         raise BitserialError(st, "bs_check_status")
 
 
+def l2_prefetch(tensors, stream=None) -> None:
+    """Hint: bring the given device tensors into L2 while the following kernels of the stream run (``bs_l2_prefetch``)."""
+    ts = [t for t in tensors if t is not None and t.numel() > 0]
+    if not ts:
+        return
+    ptrs = (ctypes.c_void_p * len(ts))(*[t.data_ptr() for t in ts])
+    sizes = (ctypes.c_size_t * len(ts))(*[t.numel() * t.element_size() for t in ts])
+    _check(lib().bs_l2_prefetch(ptrs, sizes, len(ts), _stream_ptr(stream)), "bs_l2_prefetch")
+
+
 def bs_popc_rate(iters: int = 4096) -> float:
     out = ctypes.c_double(0.0)
     st = lib().bs_popc_rate(iters, ctypes.byref(out))

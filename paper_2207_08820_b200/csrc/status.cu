@@ -33,7 +33,50 @@ __global__ void __launch_bounds__(256) popc_rate_kernel(int iters, unsigned seed
     if (total == 0xFFFFFFFFu) atomicOr(sink, 0);   // never true in practice; keeps the chains alive
 }
 
+// L2 prefetch of up to 64 buffers: one thread per 4 KB piece issues a bulk prefetch, which returns at once; the copy
+// into L2 proceeds while the following kernels of the stream run.
+struct PrefetchList {
+    const unsigned char* ptr[64];
+    unsigned long long bytes[64];      // multiples of 16
+};
+
+__global__ void l2_prefetch_kernel(const __grid_constant__ PrefetchList list)
+{
+    const unsigned char* base = list.ptr[blockIdx.y];
+    const unsigned long long total = list.bytes[blockIdx.y];
+    const unsigned long long piece = 4096;
+    for (unsigned long long off = (static_cast<unsigned long long>(blockIdx.x) * blockDim.x + threadIdx.x) * piece; off < total;
+         off += static_cast<unsigned long long>(gridDim.x) * blockDim.x * piece) {
+        const unsigned long long left = total - off;
+        const unsigned n = static_cast<unsigned>(left < piece ? left : piece);
+        asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(base + off), "r"(n) : "memory");
+    }
+}
+
 }  // namespace bs
+
+extern "C" int bs_l2_prefetch(const void* const* buffers, const size_t* bytes, int count, void* stream)
+{
+    if (count < 0 || (count > 0 && (!buffers || !bytes))) return BS_ERR_INVALID_ARG;
+    for (int i = 0; i < count; ++i)
+        if (!buffers[i] || !bs::aligned16(buffers[i])) return buffers[i] ? BS_ERR_ALIGNMENT : BS_ERR_INVALID_ARG;
+    for (int first = 0; first < count; first += 64) {
+        bs::PrefetchList list{};
+        const int n = count - first < 64 ? count - first : 64;
+        size_t largest = 0;
+        for (int i = 0; i < n; ++i) {
+            list.ptr[i] = static_cast<const unsigned char*>(buffers[first + i]);
+            list.bytes[i] = bytes[first + i] & ~static_cast<size_t>(15);
+            if (bytes[first + i] > largest) largest = bytes[first + i];
+        }
+        if (largest < 16) continue;
+        size_t bx = (largest + 4096ull * 128 - 1) / (4096ull * 128);
+        if (bx > 64) bx = 64;
+        bs::l2_prefetch_kernel<<<dim3(static_cast<unsigned>(bx), static_cast<unsigned>(n)), 128, 0, static_cast<cudaStream_t>(stream)>>>(list);
+        if (cudaGetLastError() != cudaSuccess) return BS_ERR_CUDA;
+    }
+    return BS_OK;
+}
 
 extern "C" int bs_popc_rate(int iters, double* wordops_per_s)
 {

@@ -46,10 +46,11 @@ class BitserialNet:
         torch.cuda.synchronize(self.device)   # chained layers fetch filters, scale and bias ahead of stream order
         self.graph = None
         self.static_in = None
-        self.launches_per_forward = 1 + len(self.layers)
+        self.launches_per_forward = 2 + len(self.layers)
 
     def _run(self, x: torch.Tensor) -> torch.Tensor:
         net = self.net
+        self.prefetch_filters()
         api.bitpack_activations(x, self.act_scale, net.a_bits, api.UNSIGNED, api.NCHW, out=self.bufs[net.in_name].view(-1))
         for item in self.layers:
             L = item["spec"]
@@ -62,6 +63,10 @@ class BitserialNet:
                 out_packed=self.bufs[L.dst], out_c_offset=L.dst_c_offset, out_c_total=self.shapes[L.dst][0],
                 wgt_tc=item["w_tc"], chained=item["w_tc"] is not None)
         return self.bufs[net.out_name]
+
+    def prefetch_filters(self) -> None:
+        """The filters of every layer start on their way into L2 while the pack kernel and the first layers run."""
+        api.l2_prefetch([item["w_tc"] if item["w_tc"] is not None else item["w"] for item in self.layers])
 
     def forward(self, x: torch.Tensor) -> torch.Tensor:
         """x: float32 [batch, C, H, W] on the device.  Returns the packed output tensor of the stack."""
