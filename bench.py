@@ -228,20 +228,57 @@ def run_ours(args):
         t_step = sum(e[0].elapsed_time(e[2]) for e in events) / args.steps
         api.bs_check_status(stream)
 
-        # end to end through the public API: pinned host input -> device, path, packed result -> host
-        e2e_events = [[torch.cuda.Event(enable_timing=True) for _ in range(2)] for _ in range(args.steps)]
+        # end to end through the public API: pinned host input -> device, path, packed result -> host, every step.
+        # Two device input buffers: the host -> device copy of step k+1 (copy stream) runs beside the kernels of step
+        # k (compute stream), the device -> host read of the result on a third stream; the L2 flush stays inside the
+        # timed region on the compute stream.  Timed with CUDA events on the compute stream around all steps.
+        x_dev_b = [x_dev, torch.empty_like(x_dev)]
+        if args.eager:
+            packs = [run_pack, None]
+        else:
+            g_pack_b = torch.cuda.CUDAGraph()
+            def run_pack_b():
+                runner.prefetch_filters()
+                api.bitpack_activations(x_dev_b[1], ACT_SCALE, net.a_bits, api.UNSIGNED, api.NCHW, out=in_buf.view(-1))
+            run_pack_b()
+            stream.synchronize()
+            with torch.cuda.graph(g_pack_b, stream=stream):
+                run_pack_b()
+            packs = [replay_pack, g_pack_b.replay]
+        h2d_stream, d2h_stream = torch.cuda.Stream(), torch.cuda.Stream()
+        ev_h2d = [torch.cuda.Event() for _ in range(2)]
+        ev_read = [torch.cuda.Event() for _ in range(2)]       # the pack kernel has consumed input buffer b
+        ev_out, ev_d2h = torch.cuda.Event(), torch.cuda.Event()
+        e2e_ev = [torch.cuda.Event(enable_timing=True) for _ in range(2)]
+        for b_ in range(2):
+            ev_read[b_].record(stream)
+        ev_d2h.record(stream)
+        stream.synchronize()
         for k in range(args.warmup + args.steps):
+            bi = k % 2 if packs[1] is not None else 0
+            if k == args.warmup:
+                stream.wait_event(ev_d2h)                      # the warm-up steps have drained
+                e2e_ev[0].record(stream)
+                h2d_stream.wait_event(e2e_ev[0])               # no timed copy starts before the start mark
+            h2d_stream.wait_event(ev_read[bi])
+            with torch.cuda.stream(h2d_stream):
+                x_dev_b[bi].copy_(x_host, non_blocking=True)
+                ev_h2d[bi].record(h2d_stream)
             flush.zero_()
-            timed = k >= args.warmup
-            if timed:
-                e2e_events[k - args.warmup][0].record(stream)
-            x_dev.copy_(x_host, non_blocking=True)
-            step()
-            out_host.copy_(out_packed, non_blocking=True)
-            if timed:
-                e2e_events[k - args.warmup][1].record(stream)
+            stream.wait_event(ev_h2d[bi])
+            packs[bi]()
+            ev_read[bi].record(stream)
+            stream.wait_event(ev_d2h)                          # the previous result has left the output buffer
+            replay_conv()
+            ev_out.record(stream)
+            d2h_stream.wait_event(ev_out)
+            with torch.cuda.stream(d2h_stream):
+                out_host.copy_(out_packed, non_blocking=True)
+                ev_d2h.record(d2h_stream)
+        stream.wait_event(ev_d2h)
+        e2e_ev[1].record(stream)
         barrier()
-        t_e2e = sum(e[0].elapsed_time(e[1]) for e in e2e_events) / args.steps
+        t_e2e = e2e_ev[0].elapsed_time(e2e_ev[1]) / args.steps
 
         # the other engine on the same inputs, conv layers only (reported beside the headline, not part of it)
         other = "popc" if args.engine == "tc" else "tc"
@@ -317,7 +354,7 @@ def run_ours(args):
             "roofline": roof,
             "pack": {"bound": "hbm", "ms": t_pack, "achieved": pack_bytes / (t_pack * 1e-3) / 1e9, "peak": peaks["hbm_gbs"],
                      "unit": "GB/s", "frac": pack_bytes / (t_pack * 1e-3) / 1e9 / peaks["hbm_gbs"]},
-            "e2e": {"value": 2.0 * macs * world / (t_e2e * 1e-3) / 1e9, "unit": UNIT, "ms_per_step": t_e2e,
+            "e2e": {"value": 2.0 * macs * world / (t_e2e * 1e-3) / 1e9, "unit": UNIT, "ms_per_step": t_e2e, "overlap": "h2d of step k+1 beside the kernels of step k (two input buffers); L2 flush inside",
                     "h2d_bytes_per_step": in_bytes, "d2h_bytes_per_step": out_host.numel() * 4},
             "gpu_launches": runner.launches_per_forward * args.steps,
             "clocks": clocks.summary(),
