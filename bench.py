@@ -177,8 +177,7 @@ def run_ours(args):
             api.bitpack_activations(x_dev, ACT_SCALE, net.a_bits, api.UNSIGNED, api.NCHW, out=in_buf.view(-1))
 
         def run_convs():
-            for item in runner.layers:
-                runner_conv(runner, item)
+            runner.run_layers()
 
         if args.eager:
             replay_pack, replay_conv = run_pack, run_convs
@@ -286,13 +285,11 @@ def run_ours(args):
         if world == 1 and not args.eager:
             runner2 = BitserialNet(net, params, ACT_SCALE, batch=net.batch, engine=other)
             runner2.bufs[net.in_name].copy_(in_buf)
-            for item in runner2.layers:
-                runner_conv(runner2, item)
+            runner2.run_layers()
             stream.synchronize()
             g2 = torch.cuda.CUDAGraph()
             with torch.cuda.graph(g2, stream=stream):
-                for item in runner2.layers:
-                    runner_conv(runner2, item)
+                runner2.run_layers()
             n2 = min(args.steps, 10)
             ev2 = [[torch.cuda.Event(enable_timing=True) for _ in range(2)] for _ in range(n2)]
             for k in range(3 + n2):
@@ -349,7 +346,8 @@ def run_ours(args):
             "dtype": "int32", "data": "synthetic",
             "config": {"workload": f"{net.name}_batch{net.batch}_w{net.w_bits}a{net.a_bits}",
                        "global_batch": net.batch * world, "parallelism": f"replicas{world}", "layers": len(net.layers),
-                       "l2": "flushed between timed iterations (256 MB write)", "launch": "eager stream launches" if args.eager else "CUDA graphs (pack, convs)"},
+                       "l2": "flushed between timed iterations (256 MB write)", "launch": ("eager stream launches" if args.eager else "CUDA graphs (pack, convs)") +
+                                 "; layers chained (programmatic dependent launch), independent neighbours on two streams"},
             "images_per_s": net.batch * world / (t_step * 1e-3),
             "roofline": roof,
             "pack": {"bound": "hbm", "ms": t_pack, "achieved": pack_bytes / (t_pack * 1e-3) / 1e9, "peak": peaks["hbm_gbs"],
@@ -370,19 +368,6 @@ def run_ours(args):
         print(json.dumps(line))
     if world > 1:
         dist.destroy_process_group()
-
-
-def runner_conv(runner, item):
-    """One conv layer of the stack through the C ABI (same call BitserialNet.forward makes)."""
-    from paper_2207_08820_b200 import api
-    net, L = runner.net, item["spec"]
-    res = runner.bufs[L.res] if L.res else None
-    api.bitserial_conv2d(
-        runner.bufs[L.src], item["w"], C=L.C, stride=L.stride, pad=L.pad, a_sign=api.UNSIGNED, w_sign=item["w_sign"],
-        scale=item["scale"], bias=item["bias"], relu=L.relu, out_bits=net.a_bits, out_sign=api.UNSIGNED, residual=res,
-        res_scale=L.res_scale, res_bits=net.a_bits if L.res else 0, res_sign=api.UNSIGNED, res_c_offset=0,
-        res_c_total=runner.shapes[L.res][0] if L.res else 0, out_packed=runner.bufs[L.dst],
-        out_c_offset=L.dst_c_offset, out_c_total=runner.shapes[L.dst][0], wgt_tc=item["w_tc"])
 
 
 def cpu_baseline(net, params, seed, sample):

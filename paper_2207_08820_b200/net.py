@@ -16,9 +16,10 @@ from .workloads import NetSpec
 
 class BitserialNet:
     def __init__(self, net: NetSpec, params: Dict[str, Dict], act_scale: float, device="cuda", batch: Optional[int] = None,
-                 engine: str = "popc"):
+                 engine: str = "popc", concurrent: bool = True):
         """engine: "popc" = popcount kernels on the integer pipes; "tc" = tensor-core entry point for every layer it
-        supports (others fall back to the popcount kernel)."""
+        supports (others fall back to the popcount kernel).  concurrent: launch independent neighbouring layers on
+        two streams (see :meth:`run_layers`)."""
         self.net = net
         self.engine = engine
         self.act_scale = float(act_scale)
@@ -44,6 +45,8 @@ class BitserialNet:
         for name, (C, H, W) in self.shapes.items():
             self.bufs[name] = torch.zeros(self.batch, H, W, (C + 31) // 32, net.a_bits, dtype=torch.int32, device=self.device)
         torch.cuda.synchronize(self.device)   # chained layers fetch filters, scale and bias ahead of stream order
+        self.concurrent = concurrent
+        self.side = torch.cuda.Stream(device=self.device)
         self.graph = None
         self.static_in = None
         self.launches_per_forward = 2 + len(self.layers)
@@ -52,17 +55,52 @@ class BitserialNet:
         net = self.net
         self.prefetch_filters()
         api.bitpack_activations(x, self.act_scale, net.a_bits, api.UNSIGNED, api.NCHW, out=self.bufs[net.in_name].view(-1))
-        for item in self.layers:
-            L = item["spec"]
-            res = self.bufs[L.res] if L.res else None
-            api.bitserial_conv2d(
-                self.bufs[L.src], item["w"], C=L.C, stride=L.stride, pad=L.pad, a_sign=api.UNSIGNED,
-                w_sign=item["w_sign"], scale=item["scale"], bias=item["bias"], relu=L.relu, out_bits=net.a_bits,
-                out_sign=api.UNSIGNED, residual=res, res_scale=L.res_scale, res_bits=net.a_bits if L.res else 0,
-                res_sign=api.UNSIGNED, res_c_offset=0, res_c_total=self.shapes[L.res][0] if L.res else 0,
-                out_packed=self.bufs[L.dst], out_c_offset=L.dst_c_offset, out_c_total=self.shapes[L.dst][0],
-                wgt_tc=item["w_tc"], chained=item["w_tc"] is not None)
+        self.run_layers()
         return self.bufs[net.out_name]
+
+    def run_layer(self, item, chained: bool = True) -> None:
+        """One conv layer through the C ABI on the current stream."""
+        net, L = self.net, item["spec"]
+        res = self.bufs[L.res] if L.res else None
+        api.bitserial_conv2d(
+            self.bufs[L.src], item["w"], C=L.C, stride=L.stride, pad=L.pad, a_sign=api.UNSIGNED,
+            w_sign=item["w_sign"], scale=item["scale"], bias=item["bias"], relu=L.relu, out_bits=net.a_bits,
+            out_sign=api.UNSIGNED, residual=res, res_scale=L.res_scale, res_bits=net.a_bits if L.res else 0,
+            res_sign=api.UNSIGNED, res_c_offset=0, res_c_total=self.shapes[L.res][0] if L.res else 0,
+            out_packed=self.bufs[L.dst], out_c_offset=L.dst_c_offset, out_c_total=self.shapes[L.dst][0],
+            wgt_tc=item["w_tc"], chained=chained and item["w_tc"] is not None)
+
+    def run_layers(self) -> None:
+        """All conv layers in order.  With ``concurrent`` a layer whose successor in the list neither reads nor
+        overwrites its output (a projection shortcut beside the first conv of its block, the two 1x1 branches of a
+        cross-stage block) is launched on a side stream, so the two kernels share the GPU; events carry the
+        dependencies, and under stream capture they become the edges of the graph."""
+        main = torch.cuda.current_stream(self.device)
+        pending: Dict[str, torch.cuda.Event] = {}
+        n = len(self.layers)
+        for i, item in enumerate(self.layers):
+            L = item["spec"]
+            nxt = self.layers[i + 1]["spec"] if i + 1 < n else None
+            aside = (self.concurrent and nxt is not None and L.dst not in (nxt.src, nxt.res)
+                     and nxt.dst not in (L.src, L.res)
+                     and (nxt.dst != L.dst or nxt.dst_c_offset != L.dst_c_offset) and L.src not in pending
+                     and (L.res is None or L.res not in pending))
+            if aside:
+                fork = torch.cuda.Event()
+                fork.record(main)
+                self.side.wait_event(fork)
+                with torch.cuda.stream(self.side):
+                    self.run_layer(item, chained=False)
+                    done = torch.cuda.Event()
+                    done.record(self.side)
+                pending[L.dst] = done
+                continue
+            for t in (L.src, L.res, L.dst):
+                if t is not None and t in pending:
+                    main.wait_event(pending.pop(t))
+            self.run_layer(item)
+        for ev in pending.values():
+            main.wait_event(ev)
 
     def prefetch_filters(self) -> None:
         """The filters of every layer start on their way into L2 while the pack kernel and the first layers run."""
