@@ -820,8 +820,10 @@ constexpr int TCP_THREADS = 320;
 constexpr int TCP_NSP = 3;            // packed-tile ring (at most)
 constexpr int TCP_NSE = 3;            // expanded-chunk ring (at most)
 
-template <int A>
-__global__ void __launch_bounds__(TCP_THREADS, 3) bitserial_conv_tc_persistent_kernel(const __grid_constant__ TcArgs g)
+// CPS: CTAs per SM the registers are budgeted for (3: 64 registers per thread; 1: no cap, for plans whose shared memory
+// leaves room for one or two CTAs anyway).
+template <int A, int CPS>
+__global__ void __launch_bounds__(TCP_THREADS, CPS) bitserial_conv_tc_persistent_kernel(const __grid_constant__ TcArgs g)
 {
     extern __shared__ __align__(128) unsigned char tc_smem[];
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -1320,10 +1322,13 @@ static int tc_conv_impl(const uint32_t* act, const int8_t* wgt, const bs_conv_pa
         const long long grid = per_o * g.tiles_o;
         void (*kern)(TcArgs) = nullptr;
         switch (A) {
-            case 1: kern = bitserial_conv_tc_persistent_kernel<1>; break;
-            case 2: kern = bitserial_conv_tc_persistent_kernel<2>; break;
-            case 3: kern = bitserial_conv_tc_persistent_kernel<3>; break;
-            default: kern = bitserial_conv_tc_persistent_kernel<4>; break;
+#define BS_TCP_PICK(ABITS) (cps >= 3 ? bitserial_conv_tc_persistent_kernel<ABITS, 3> \
+                          : cps == 2 ? bitserial_conv_tc_persistent_kernel<ABITS, 2> : bitserial_conv_tc_persistent_kernel<ABITS, 1>)
+            case 1: kern = BS_TCP_PICK(1); break;
+            case 2: kern = BS_TCP_PICK(2); break;
+            case 3: kern = BS_TCP_PICK(3); break;
+            default: kern = BS_TCP_PICK(4); break;
+#undef BS_TCP_PICK
         }
         if (smem > 48 * 1024 &&
             cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)) != cudaSuccess) {
