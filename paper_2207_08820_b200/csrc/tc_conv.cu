@@ -1315,6 +1315,9 @@ static int tc_conv_impl(const uint32_t* act, const int8_t* wgt, const bs_conv_pa
         int cps = ctas_per_sm(smem);                                       // CTAs that fit on one SM: shared memory,
         if (cps > 3) cps = 3;                                              // registers (launch bounds) and
         if (cps * 2 * g.TN > 512) cps = 512 / (2 * g.TN);                  // tensor-memory columns
+#ifdef BS_TUNING
+        if (const char* e = getenv("BS_TC_CPSMAX")) { const int m = atoi(e); if (cps > m) cps = m; }
+#endif
         if (cps < 1) cps = 1;
         long long per_o = (static_cast<long long>(sms) * cps) / g.tiles_o;
         if (per_o < 1) per_o = 1;
