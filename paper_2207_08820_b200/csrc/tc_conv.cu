@@ -1231,6 +1231,20 @@ static int tc_conv_impl(const uint32_t* act, const int8_t* wgt, const bs_conv_pa
     if (!keep_narrow && g.persistent && (g.TN == 32 || (g.TN == 64 && g.nchunks >= 4)) && p->O >= 128 &&
         tiles_m * ceil_div(p->O, 128) >= sms / 2)
         g.persistent = 0;
+    // A resident plan also loses when its CTAs see hardly more than one pixel tile each: nothing amortises the filter
+    // fetch, and the streaming kernel has twice the expand/epilogue warps.  Measured on the bottleneck stack for
+    // reductions of 512 and more (shallower ones are epilogue-bound and stay resident).
+    if (!keep_narrow && g.persistent && kred >= 512) {
+        int cps_est = static_cast<int>((225 * 1024) / (smem + 1024));
+        if (cps_est > 3) cps_est = 3;
+        if (cps_est * 2 * g.TN > 512) cps_est = 512 / (2 * g.TN);
+        if (cps_est < 1) cps_est = 1;
+        const int tiles_o = ceil_div(p->O, g.TN);
+        long long per_o = static_cast<long long>(sms) * cps_est / tiles_o;
+        if (per_o < 1) per_o = 1;
+        if (per_o > tiles_m) per_o = tiles_m;
+        if (2 * tiles_m <= 3 * per_o) g.persistent = 0;       // at most 1.5 pixel tiles per CTA
+    }
     if (force_stream) g.persistent = 0;
     g.PT = 1;
     if (!g.persistent) {
