@@ -91,15 +91,15 @@ __device__ __forceinline__ bool mbar_spin_bounded(uint64_t* bar, unsigned parity
 }
 // Group-wide AND of a per-thread flag (also a barrier): every thread of the group gets the same answer, so a wait
 // that ran out makes the whole group leave its loop together and nobody is left behind at a later group_sync.
-__device__ __forceinline__ bool group_all(int id, bool ok)
+__device__ __forceinline__ bool group_all(int id, bool ok, int nthreads = 128)
 {
     unsigned r;
     asm volatile(
         "{\n\t.reg .pred p, q;\n\t"
         "setp.ne.u32 q, %1, 0;\n\t"
-        "bar.red.and.pred p, %2, 128, q;\n\t"
+        "bar.red.and.pred p, %2, %3, q;\n\t"
         "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(r) : "r"(ok ? 1u : 0u), "r"(id) : "memory");
+        : "=r"(r) : "r"(ok ? 1u : 0u), "r"(id), "r"(nthreads) : "memory");
     return r != 0;
 }
 // One lane polls the mbarrier for its warp (128 threads hammering one shared-memory word is slow); result is broadcast.
@@ -817,13 +817,16 @@ __global__ void __launch_bounds__(TC_THREADS) bitserial_conv_tc_kernel(const __g
 // epilogue of tile i overlap the MMAs of tile i + 1.
 
 constexpr int TCP_THREADS = 320;
+constexpr int TCP_THREADS_WIDE = 448;   // with a second set of four epilogue warps (10-13)
 constexpr int TCP_NSP = 3;            // packed-tile ring (at most)
 constexpr int TCP_NSE = 3;            // expanded-chunk ring (at most)
 
 // CPS: CTAs per SM the registers are budgeted for (3: 64 registers per thread; 1: no cap, for plans whose shared memory
 // leaves room for one or two CTAs anyway).
-template <int A, int CPS>
-__global__ void __launch_bounds__(TCP_THREADS, CPS) bitserial_conv_tc_persistent_kernel(const __grid_constant__ TcArgs g)
+// WIDE: eight epilogue warps (0-3 and 10-13, two per tensor-memory lane quadrant, sharing the groups of 32 filters).
+template <int A, int CPS, bool WIDE = false>
+__global__ void __launch_bounds__(WIDE ? TCP_THREADS_WIDE : TCP_THREADS, CPS)
+bitserial_conv_tc_persistent_kernel(const __grid_constant__ TcArgs g)
 {
     extern __shared__ __align__(128) unsigned char tc_smem[];
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -918,7 +921,7 @@ __global__ void __launch_bounds__(TCP_THREADS, CPS) bitserial_conv_tc_persistent
             if (!ok) atomicOr(g.status, STATUS_TIMEOUT);
         }
         __syncwarp();
-    } else if (warp >= 4) {
+    } else if (warp >= 4 && warp < 8) {
         // ------------------------------------------------------------------ expanders (warps 4-7)
         const int et = tid - 128;
         const TcExpand xp = tc_expand_init(g, et, 128);
@@ -941,13 +944,16 @@ __global__ void __launch_bounds__(TCP_THREADS, CPS) bitserial_conv_tc_persistent
         }
         if (!ok) atomicOr(g.status, STATUS_TIMEOUT);
     } else {
-        // ------------------------------------------------------------------ epilogue (warps 0-3)
+        // ------------------------------------------------------------------ epilogue (warps 0-3, and 10-13 when WIDE)
+        constexpr int EPI_THREADS = WIDE ? 256 : 128;
+        const int second = warp >= 10 ? 1 : 0;                 // second set: the odd groups of 32 filters
+        const int ei = second ? tid - 192 : tid;               // 0 .. EPI_THREADS-1
         uint32_t thr = 0;                 // shared-memory address of the thresholds, 0: floating-point comparison
         if (g.off_thr) {                  // while the pipeline fills: comparison bounds -> integer thresholds
             int4* s_thr = reinterpret_cast<int4*>(tc_smem + g.off_thr);
             int* thr_ok = reinterpret_cast<int*>(s_thr + g.thr_pats * g.TN);
-            tc_build_thresholds(g, s_thr, thr_ok, s_sb, s_bounds, o0, tid, 128);
-            group_sync(2);
+            tc_build_thresholds(g, s_thr, thr_ok, s_sb, s_bounds, o0, ei, EPI_THREADS);
+            group_sync(2, EPI_THREADS);
             if (*thr_ok) thr = smem_u32(s_thr);
         }
         pdl_acquire();                    // the epilogue reads the residual and overwrites buffers the preceding kernel may use
@@ -955,13 +961,14 @@ __global__ void __launch_bounds__(TCP_THREADS, CPS) bitserial_conv_tc_persistent
         bool ok = true;
         for (int mt = first_tile; mt < tiles_m && ok; mt += tile_step, ++i) {
             const int buf = i & 1, use = i >> 1;
-            ok = group_all(2, mbar_wait_warp(&full_acc[buf], use & 1, lane));
+            ok = group_all(2, mbar_wait_warp(&full_acc[buf], use & 1, lane), EPI_THREADS);
             if (!ok) break;
             tc_fence_after();
             const TcTile tile = tc_decode_tile(g, mt);
-            tc_epilogue_tile(g, tmem_base + static_cast<uint32_t>(buf * g.TN), tid, warp, tile, o0, s_sb, s_bounds, thr);
+            tc_epilogue_tile(g, tmem_base + static_cast<uint32_t>(buf * g.TN), (warp & 3) * 32 + lane, warp & 3, tile, o0, s_sb, s_bounds, thr,
+                             WIDE ? second : 0, WIDE ? 2 : 1);
             tc_fence_before();
-            group_sync(2);                           // all four warps have read their accumulator rows
+            group_sync(2, EPI_THREADS);              // every epilogue warp has read its accumulator rows
             if (tid == 0) mbar_arrive(&empty_acc[buf]);
         }
         if (!ok) atomicOr(g.status, STATUS_TIMEOUT);
@@ -1337,10 +1344,16 @@ static int tc_conv_impl(const uint32_t* act, const int8_t* wgt, const bs_conv_pa
         if (per_o < 1) per_o = 1;
         if (per_o > tiles_m) per_o = tiles_m;
         const long long grid = per_o * g.tiles_o;
+        // eight epilogue warps when registers allow (one or two CTAs per SM) and the tile has at least two groups of 32 filters
+        bool wide = cps <= 2 && g.TN >= 64;
+#ifdef BS_TUNING
+        if (const char* e = getenv("BS_TC_WIDE")) wide = wide && atoi(e) != 0;
+#endif
         void (*kern)(TcArgs) = nullptr;
         switch (A) {
 #define BS_TCP_PICK(ABITS) (cps >= 3 ? bitserial_conv_tc_persistent_kernel<ABITS, 3> \
-                          : cps == 2 ? bitserial_conv_tc_persistent_kernel<ABITS, 2> : bitserial_conv_tc_persistent_kernel<ABITS, 1>)
+                          : cps == 2 ? (wide ? bitserial_conv_tc_persistent_kernel<ABITS, 2, true> : bitserial_conv_tc_persistent_kernel<ABITS, 2>) \
+                                     : (wide ? bitserial_conv_tc_persistent_kernel<ABITS, 1, true> : bitserial_conv_tc_persistent_kernel<ABITS, 1>))
             case 1: kern = BS_TCP_PICK(1); break;
             case 2: kern = BS_TCP_PICK(2); break;
             case 3: kern = BS_TCP_PICK(3); break;
@@ -1352,7 +1365,7 @@ static int tc_conv_impl(const uint32_t* act, const int8_t* wgt, const bs_conv_pa
             cudaGetLastError();
             return BS_ERR_CUDA;
         }
-        if (tc_launch(kern, static_cast<unsigned>(grid), TCP_THREADS, smem, st, chained, g) != cudaSuccess) {
+        if (tc_launch(kern, static_cast<unsigned>(grid), wide ? TCP_THREADS_WIDE : TCP_THREADS, smem, st, chained, g) != cudaSuccess) {
             cudaGetLastError();
             return BS_ERR_CUDA;
         }
