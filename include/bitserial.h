@@ -207,8 +207,8 @@ int bitserial_gemm_noalloc(const uint32_t* a_packed, const uint32_t* w_packed, i
  *   1x1 stride-1 layers, N*H*W is even; res_c_offset a multiple of 32; everything else as bitserial_conv2d.  Unsupported shapes return BS_ERR_UNSUPPORTED: use the
  *   popcount entry points.
  *   bs_tc_weights_bytes    bytes of the prepared int8 filter tensor (0 on bad input).
- *   bs_tc_prepare_weights  packed weights [O][R][S][Cw][w_bits] -> int8 tiles [C/CK][ceil(O/128)*16][R*S][CK/16][8][16];
- *                          CK = 64 when C % 64 == 0, else 32 (a_bits is accepted for forward compatibility).
+ *   bs_tc_prepare_weights  packed weights [O][R][S][Cw][w_bits] -> int8 tiles [C/32][ceil(O/128)*16][R*S][2][8][16]
+ *                          (blocks of 32 channels; a_bits is accepted for forward compatibility).
  */
 size_t bs_tc_weights_bytes(int O, int C, int R, int S);
 int bs_tc_prepare_weights(const uint32_t* wgt_packed, int O, int C, int R, int S, int w_bits, bs_sign_t w_sign,

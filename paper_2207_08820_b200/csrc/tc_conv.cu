@@ -24,7 +24,7 @@ namespace bs {
 constexpr int TC_THREADS = 320;       // warps 0-3 and 6-9: expand + epilogue, warp 4: TMA producer, warp 5: MMA issuer
 constexpr int TC_WORKERS = 256;       // threads of the eight expand + epilogue warps
 constexpr int TC_M = 128;             // pixels per tile = 16 row groups x 8 columns (or 128 flat pixels)
-constexpr int TC_MAX_STAGES = 2;
+constexpr int TC_MAX_STAGES = 4;
 
 struct TcArgs {
     CUtensorMap tmA;                  // packed activations: (W*Cw*A, H, N) words when a halo row fits one box row, else (Cw*A, W, H, N)
@@ -382,7 +382,7 @@ __device__ __forceinline__ void umma_i8_words(uint32_t d_tmem, uint32_t a_lo, ui
 
 // Fully unrolled issue of one layout block for the commonest shape classes (stride 1, two K steps per tap): no loop
 // counters or branches between the MMAs of the lone issuing thread.
-template <int R, int S, bool STRIDE2>
+template <int R, int S, bool STRIDE2, int KS>
 __device__ __forceinline__ void tc_issue_block_unrolled(const TcIssue& is, uint32_t arow, uint32_t b, uint32_t tmem_acc, uint32_t acc)
 {
 #pragma unroll
@@ -391,8 +391,8 @@ __device__ __forceinline__ void tc_issue_block_unrolled(const TcIssue& is, uint3
         for (int sx = 0; sx < S; ++sx) {
             const uint32_t a = arow + (STRIDE2 ? static_cast<uint32_t>(sx & 1) * is.half16 + static_cast<uint32_t>(sx >> 1) : static_cast<uint32_t>(sx));
             umma_i8_words(tmem_acc, a, is.a_hi, b, is.b_hi, is.idesc, (r == 0 && sx == 0) ? acc : 1u);
-            umma_i8_words(tmem_acc, a + is.kstep16, is.a_hi, b + 16, is.b_hi, is.idesc, 1u);
-            b += 32;
+            if (KS == 2) umma_i8_words(tmem_acc, a + is.kstep16, is.a_hi, b + 16, is.b_hi, is.idesc, 1u);
+            b += 16 * KS;
         }
         arow += is.row16;
     }
@@ -400,14 +400,20 @@ __device__ __forceinline__ void tc_issue_block_unrolled(const TcIssue& is, uint3
 
 __device__ __forceinline__ void tc_issue_chunk(const TcIssue& is, uint32_t ea, uint32_t ba, uint32_t tmem_acc, bool first_chunk)
 {
-    if (is.ksteps == 2 && is.R == is.S && (is.R == 3 || is.R == 1)) {
+    if (is.ksteps <= 2 && is.R == is.S && (is.R == 3 || is.R == 1)) {
         uint32_t arow0 = is.a_lo + (ea >> 4), b0 = is.b_lo + (ba >> 4), acc0 = first_chunk ? 0u : 1u;
         for (int blk = 0; blk < is.blocks; ++blk) {
-            if (is.R == 1) tc_issue_block_unrolled<1, 1, false>(is, arow0, b0, tmem_acc, acc0);     // a lone tap has no column offset
-            else if (is.stride2) tc_issue_block_unrolled<3, 3, true>(is, arow0, b0, tmem_acc, acc0);
-            else tc_issue_block_unrolled<3, 3, false>(is, arow0, b0, tmem_acc, acc0);
+            if (is.ksteps == 2) {
+                if (is.R == 1) tc_issue_block_unrolled<1, 1, false, 2>(is, arow0, b0, tmem_acc, acc0);     // a lone tap has no column offset
+                else if (is.stride2) tc_issue_block_unrolled<3, 3, true, 2>(is, arow0, b0, tmem_acc, acc0);
+                else tc_issue_block_unrolled<3, 3, false, 2>(is, arow0, b0, tmem_acc, acc0);
+            } else {
+                if (is.R == 1) tc_issue_block_unrolled<1, 1, false, 1>(is, arow0, b0, tmem_acc, acc0);
+                else if (is.stride2) tc_issue_block_unrolled<3, 3, true, 1>(is, arow0, b0, tmem_acc, acc0);
+                else tc_issue_block_unrolled<3, 3, false, 1>(is, arow0, b0, tmem_acc, acc0);
+            }
             acc0 = 1u;
-            arow0 += 2u * is.kstep16;
+            arow0 += static_cast<uint32_t>(is.ksteps) * is.kstep16;
             b0 += is.blk_b16;
         }
         return;
@@ -1012,13 +1018,11 @@ __global__ void tc_prepare_weights_kernel(const uint32_t* __restrict__ packed, i
 
 static int round_up_i(int v, int m) { return (v + m - 1) / m * m; }
 
-// Channels per block of the prepared filter layout: 64 when C allows, else 32.  A pipeline chunk is one block, or
-// several consecutive blocks for 1x1 stride-1 layers (one tap per block is only two MMAs per hand-off otherwise).
+// Channels per block of the prepared filter layout.  A pipeline chunk is one or several consecutive blocks, chosen per
+// layer by the plan (which knows stride and batch; the prepared filters do not depend on them).
 static int tc_chunk_channels(int C, int /*a_bits*/)
 {
-    if (C % 64 == 0) return 64;
-    if (C % 32 == 0) return 32;
-    return 0;
+    return C % 32 == 0 ? 32 : 0;
 }
 
 static typename std::add_pointer<CUresult(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
@@ -1133,19 +1137,24 @@ static int tc_conv_impl(const uint32_t* act, const int8_t* wgt, const bs_conv_pa
     g.acc_small = kred * tc_max_abs(p->a_bits, p->a_sign) * tc_max_abs(p->w_bits, p->w_sign) < (1LL << 22);
 
     g.CK = tc_chunk_channels(p->C, A);
-    g.MB = 1;
+    // Blocks per pipeline chunk: 64 channels when C allows (two MMAs per tap and hand-off), 128 for 1x1 stride-1 layers
+    // (one tap per block is too little work per hand-off), a single 32-channel block for stride-2 3x3 layers, whose
+    // expanded halo is four times larger per output and would otherwise push the plan to a narrower filter tile.
+    g.MB = p->C % 64 == 0 ? 2 : 1;
     {
-        // 1x1 stride-1 layers: two 64-channel blocks per pipeline chunk (the expanded tile is 128 pixels x 128 channels =
-        // 16 KB per stage); four measured no better than two on the bottleneck and detection stacks
-        int wide = 2;
+        int wide = 4;
 #ifdef BS_TUNING
         if (const char* e = getenv("BS_TC_MB")) wide = atoi(e);
 #endif
-        if (RS == 1 && p->stride == 1 && p->pad == 0 && g.CK == 64)
+        if (RS == 1 && p->stride == 1 && p->pad == 0)
             for (int mb = wide; mb > 1; mb /= 2)
                 if (p->C % (g.CK * mb) == 0) { g.MB = mb; break; }
+        if (RS > 1 && p->stride == 2) g.MB = 1;
+#ifdef BS_TUNING
+        if (const char* e = getenv("BS_TC_MBALL")) { const int mb = atoi(e); if (p->C % (g.CK * mb) == 0) g.MB = mb; }
+#endif
     }
-    const int CKP = g.CK * g.MB;                  // channels per pipeline chunk
+    int CKP = g.CK * g.MB;                        // channels per pipeline chunk
     g.CWC = CKP / 32;
     g.fullA = Cw * A;
     g.act = act;
@@ -1258,6 +1267,9 @@ static int tc_conv_impl(const uint32_t* act, const int8_t* wgt, const bs_conv_pa
         // Filters streamed chunk by chunk; a CTA takes PT pixel tiles (PT accumulators in tensor memory) so that every
         // filter chunk fetched from L2 serves PT tiles.  Widest filter tile that keeps about one CTA per SM.
         g.nsp = g.nse = g.nchunks < 2 ? g.nchunks : 2;
+#ifdef BS_TUNING
+        if (const char* e = getenv("BS_TC_NSP")) { const int n = atoi(e); g.nsp = g.nchunks < n ? g.nchunks : n; }
+#endif
         int TN = 128;
         while (TN > 32 && (TN / 2 >= round_up_i(p->O, 32) || tiles_m * ceil_div(p->O, TN) < sms / 2)) TN /= 2;
         int PT = stream_pt;
@@ -1269,6 +1281,17 @@ static int tc_conv_impl(const uint32_t* act, const int8_t* wgt, const bs_conv_pa
         if (stream_tn) TN = stream_tn;
         while (PT > 1 && (PT * TN > 512 || stream_bytes(TN, PT) > 220 * 1024)) PT /= 2;
         while (TN > 32 && stream_bytes(TN, PT) > 200 * 1024) TN /= 2;
+        // More CTAs than SMs: halve the chunk if that lets two CTAs share an SM (one wave instead of two)
+        if (g.MB == 2 && RS > 1 && ceil_div_ll(tiles_m, PT) * ceil_div(p->O, TN) > sms) {
+            const int e_keep = g.e_bytes, n_keep = g.nchunks;
+            g.MB = 1; CKP = g.CK; g.CWC = CKP / 32; g.nchunks = p->C / CKP;
+            g.e_bytes = round_up_i((CKP / 16) * g.HPE * 16, 128);
+            g.nsp = g.nse = g.nchunks < 2 ? g.nchunks : 2;
+            if (stream_bytes(TN, PT) + 5 * 1024 > 112 * 1024) {
+                g.MB = 2; CKP = 2 * g.CK; g.CWC = CKP / 32; g.nchunks = n_keep; g.e_bytes = e_keep;
+                g.nsp = g.nse = g.nchunks < 2 ? g.nchunks : 2;
+            }
+        }
         g.TN = TN;
         g.PT = PT;
         g.b_bytes = TN * RS * CKP;
