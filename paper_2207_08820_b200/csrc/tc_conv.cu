@@ -1138,7 +1138,7 @@ static int tc_conv_impl(const uint32_t* act, const int8_t* wgt, const bs_conv_pa
 
     g.CK = tc_chunk_channels(p->C, A);
     // Blocks per pipeline chunk: 64 channels when C allows (two MMAs per tap and hand-off), 128 for 1x1 stride-1 layers
-    // (one tap per block is too little work per hand-off), a single 32-channel block for stride-2 3x3 layers, whose
+    // (one tap per block is too little work per hand-off), a single 32-channel block for stride-2 3x3 layers of 128 and more channels, whose
     // expanded halo is four times larger per output and would otherwise push the plan to a narrower filter tile.
     g.MB = p->C % 64 == 0 ? 2 : 1;
     {
@@ -1149,7 +1149,7 @@ static int tc_conv_impl(const uint32_t* act, const int8_t* wgt, const bs_conv_pa
         if (RS == 1 && p->stride == 1 && p->pad == 0)
             for (int mb = wide; mb > 1; mb /= 2)
                 if (p->C % (g.CK * mb) == 0) { g.MB = mb; break; }
-        if (RS > 1 && p->stride == 2) g.MB = 1;
+        if (RS > 1 && p->stride == 2 && p->C >= 128) g.MB = 1;
 #ifdef BS_TUNING
         if (const char* e = getenv("BS_TC_MBALL")) { const int mb = atoi(e); if (p->C % (g.CK * mb) == 0) g.MB = mb; }
 #endif
