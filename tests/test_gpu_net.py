@@ -89,3 +89,9 @@ def test_vgg16_ssd_body_small(engine):
 def test_vgg16_ssd_body_full_resolution_sampled():
     """300 px: widths 300/150/75/38/19 (odd and even) through the tensor-core engine, one image checked."""
     compare_stack(wl.vgg16_ssd_body(2), 2, seed=7000, sample=[1], graph=True, engine="tc")
+
+
+def test_resnet50_body_full_batch_sampled():
+    """Batch 32 at 56 px (the configuration `bench.py --workload resnet50_body` times): wide 1x1 chunks, streamed deep
+    reductions and projection shortcuts on the second stream, two images checked against the oracle."""
+    compare_stack(wl.resnet50_body(32), 32, seed=6000, sample=[0, 31], graph=True, engine="tc")
