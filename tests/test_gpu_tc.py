@@ -148,6 +148,29 @@ def test_tc_epilogue_scale_bias_corner_cases(kind, with_res, out):
     assert np.array_equal(words(packed), oracle.pack_activations(codes, out_bits, out_sign))
 
 
+@pytest.mark.parametrize("out_bits,out_sign", [(3, 0), (4, 0), (3, 1), (4, 1)])
+@pytest.mark.parametrize("with_res", [False, True])
+def test_tc_wide_output_codes(out_bits, out_sign, with_res):
+    """3- and 4-bit outputs take the formula epilogue (no comparison form); with a 3-bit signed residual on top."""
+    c = wl.single_conv_case(seed=77, N=2, C=64, H=11, W=13, O=72, calibrated=True)
+    rng = np.random.default_rng(9)
+    scale = (c["scale"] * (2 ** (out_bits - 2))).astype(np.float32)
+    bias = (c["bias"] * (2 ** (out_bits - 2)) - (2 ** (out_bits - 1) if out_sign else 0)).astype(np.float32)
+    res = wl.rand_codes(rng, (2, 72, 11, 13), 3, 1) if with_res else None
+    xa = api.bitpack_activations(dev(c["x"]), 1.0, 2, 0, api.NCHW)
+    wp = api.pack_weights(dev(c["w"]), 2, c["w_sign"], api.NCHW)
+    wt = api.tc_prepare_weights(wp, 64, c["w_sign"], 2)
+    res_t = api.bitpack_activations(dev(res), 1.0, 3, 1, api.NCHW) if with_res else None
+    _, packed = api.bitserial_conv2d(xa, wp, C=64, stride=1, pad=1, w_sign=c["w_sign"], scale=dev(scale), bias=dev(bias), relu=False,
+                                     out_bits=out_bits, out_sign=out_sign, residual=res_t, res_scale=0.3 if with_res else 0.0,
+                                     res_bits=3 if with_res else 0, res_sign=1, res_c_total=72 if with_res else 0, wgt_tc=wt)
+    api.bs_check_status()
+    want = oracle.conv2d_i32(c["x"], c["w"], 1, 1)
+    codes = oracle.requantize(want, scale, bias, False, out_bits, out_sign, res=res, res_scale=0.3 if with_res else 0.0)
+    assert len(np.unique(codes)) >= 4
+    assert np.array_equal(words(packed), oracle.pack_activations(codes, out_bits, out_sign))
+
+
 @pytest.mark.parametrize("M,N,K", [(1, 8, 64), (130, 40, 128), (300, 72, 1024), (1031, 96, 64), (256, 256, 576), (1024, 1024, 2304)])
 def test_tc_gemm(M, N, K):
     c = wl.gemm_case(M, N, K, seed=M + N + K)
