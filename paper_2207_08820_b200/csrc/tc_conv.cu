@@ -564,6 +564,19 @@ __device__ __forceinline__ void tc_compare_int(const uint32_t (&v)[32], uint32_t
     ow[1] = ~w1;        // bit 1 is "level 2 reached"
 }
 
+// (scale, bias) of the CTA's filters, the comparison bounds and the "thresholds are valid" flag, written by the
+// `nthreads` threads that run the epilogue (index t); the caller synchronises them afterwards.
+__device__ __forceinline__ void tc_epilogue_tables(const TcArgs& g, unsigned char* tc_smem, float2* s_sb, float4* s_bounds, int o0,
+                                                   int t, int nthreads)
+{
+    for (int f = t; f < g.TN; f += nthreads) {
+        const int o = o0 + f;
+        s_sb[f] = (g.out_packed && o < g.O) ? make_float2(g.scale[o], g.bias[o]) : make_float2(0.f, 0.f);
+    }
+    if (t < 16) s_bounds[t] = make_float4(g.rb.bound[t][0], g.rb.bound[t][1], g.rb.bound[t][2], 0.f);
+    if (t == 32 && g.off_thr) *reinterpret_cast<int*>(tc_smem + g.off_thr + g.thr_pats * g.TN * 16) = 1;
+}
+
 // Epilogue of one tile: thread `tid` (0..127, warp = TMEM lane quadrant) owns accumulator row tid = one output pixel.
 __device__ __forceinline__ void tc_epilogue_tile(const TcArgs& g, uint32_t tmem_acc, int tid, int warp, const TcTile& tile, int o0,
                                                  const float2* s_sb, const float4* s_bounds, uint32_t thr_addr, int cc0 = 0, int ccstep = 1)
@@ -714,13 +727,8 @@ __global__ void __launch_bounds__(TC_THREADS) bitserial_conv_tc_kernel(const __g
         tmem_alloc(tmem_slot, static_cast<unsigned>(g.tmem_cols));
         tmem_relinquish();
     }
-    if (tid < g.TN) {
-        const int o = o0 + tid;
-        s_sb[tid] = (g.out_packed && o < g.O) ? make_float2(g.scale[o], g.bias[o]) : make_float2(0.f, 0.f);
-    }
-    if (tid < 16) s_bounds[tid] = make_float4(g.rb.bound[tid][0], g.rb.bound[tid][1], g.rb.bound[tid][2], 0.f);
-    if (tid == 32 && g.off_thr) *reinterpret_cast<int*>(tc_smem + g.off_thr + g.thr_pats * g.TN * 16) = 1;
-    tc_build_lut(g, s_lut, tid, blockDim.x);
+    // Only the barriers and the tensor-memory address are needed by every role: the producer starts fetching right
+    // after this barrier; the byte table and the scale/bias/bounds tables are set up by the warps that use them.
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
@@ -776,6 +784,9 @@ __global__ void __launch_bounds__(TC_THREADS) bitserial_conv_tc_kernel(const __g
         // ------------------------------------------------------------------ expanders (warps 0-3, 6-9), then epilogue
         pdl_acquire();                    // the epilogue reads the residual and overwrites buffers the preceding kernel may use
         const int ct = warp < 4 ? tid : tid - 64;          // 0..255 among the workers
+        tc_build_lut(g, s_lut, ct, TC_WORKERS);
+        tc_epilogue_tables(g, tc_smem, s_sb, s_bounds, o0, ct, TC_WORKERS);
+        group_sync(1, TC_WORKERS);
         const TcExpand xp = tc_expand_init(g, ct, TC_WORKERS);
         bool ok = mbar_wait_warp(full_a, 0, lane);
         for (int c = 0; c < g.nchunks; ++c) {
@@ -871,13 +882,8 @@ bitserial_conv_tc_persistent_kernel(const __grid_constant__ TcArgs g)
         tmem_alloc(tmem_slot, static_cast<unsigned>(g.tmem_cols));
         tmem_relinquish();
     }
-    if (tid < g.TN) {
-        const int o = o0 + tid;
-        s_sb[tid] = (g.out_packed && o < g.O) ? make_float2(g.scale[o], g.bias[o]) : make_float2(0.f, 0.f);
-    }
-    if (tid < 16) s_bounds[tid] = make_float4(g.rb.bound[tid][0], g.rb.bound[tid][1], g.rb.bound[tid][2], 0.f);
-    if (tid == 32 && g.off_thr) *reinterpret_cast<int*>(tc_smem + g.off_thr + g.thr_pats * g.TN * 16) = 1;
-    tc_build_lut(g, s_lut, tid, blockDim.x);
+    // Only the barriers and the tensor-memory address are needed by every role: the producer starts fetching right
+    // after this barrier; the byte table and the scale/bias/bounds tables are set up by the warps that use them.
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
@@ -930,6 +936,8 @@ bitserial_conv_tc_persistent_kernel(const __grid_constant__ TcArgs g)
     } else if (warp >= 4 && warp < 8) {
         // ------------------------------------------------------------------ expanders (warps 4-7)
         const int et = tid - 128;
+        tc_build_lut(g, s_lut, et, 128);
+        group_sync(1);
         const TcExpand xp = tc_expand_init(g, et, 128);
         int it = 0, i = 0;
         bool ok = true;
@@ -954,6 +962,8 @@ bitserial_conv_tc_persistent_kernel(const __grid_constant__ TcArgs g)
         constexpr int EPI_THREADS = WIDE ? 256 : 128;
         const int second = warp >= 10 ? 1 : 0;                 // second set: the odd groups of 32 filters
         const int ei = second ? tid - 192 : tid;               // 0 .. EPI_THREADS-1
+        tc_epilogue_tables(g, tc_smem, s_sb, s_bounds, o0, ei, EPI_THREADS);
+        group_sync(2, EPI_THREADS);
         uint32_t thr = 0;                 // shared-memory address of the thresholds, 0: floating-point comparison
         if (g.off_thr) {                  // while the pipeline fills: comparison bounds -> integer thresholds
             int4* s_thr = reinterpret_cast<int4*>(tc_smem + g.off_thr);
