@@ -42,6 +42,8 @@ struct TcArgs {
     int relu, out_bits, out_sign, out_cw_off, out_cw_total;
     int res_bits, res_sign, res_c_off, res_cw_total;
     int i32_nhwc, acc_small;
+    int acc_bound;                    // |accumulator| <= acc_bound
+    int thr_packed;                   // thresholds stored for two filters per entry (16-bit lanes), see tc_compare_pairs
     // tiling
     int flat;                         // 1: 128 consecutive pixels of the flattened image (1x1, stride 1)
     int TN, CK, MB, CWC, nchunks, nsp, nse;   // CK: channels per filter-layout block, MB: blocks per pipeline chunk, CWC: words per chunk
@@ -499,6 +501,37 @@ __device__ __forceinline__ int tc_threshold(float s, float b, float bound, int* 
 __device__ __forceinline__ void tc_build_thresholds(const TcArgs& g, int4* thr, int* ok, const float2* s_sb, const float4* s_bounds,
                                                     int o0, int t, int nthreads)
 {
+    if (g.thr_packed) {
+        // entry (group of 32 filters, j = 0..15) serves filters j and j + 16 of the group: per level the word
+        // (2^15 - T[j + 16]) << 16 | (2^15 - T[j]).  Thresholds are clamped to +-(acc_bound + 1), which decides the same
+        // for every possible accumulator and keeps each 16-bit lane of  acc + 2^15 - T  inside (0, 2^16).
+        const int lim = g.acc_bound + 1;
+        for (int e = t; e < g.TN / 2; e += nthreads) {
+            const int grp = e >> 4, j = e & 15;
+            unsigned d[3] = {0u, 0u, 0u};
+            for (int half = 0; half < 2; ++half) {
+                const int f = grp * 32 + half * 16 + j;
+                int T[3] = {lim, lim, lim};                                      // filters past O: never reached, masked anyway
+                if (o0 + f < g.O) {
+                    const float2 sb = s_sb[f];
+                    if (!(sb.x > 0.0f) || !(sb.x < 3.0e38f) || !(fabsf(sb.y) < 3.0e38f)) {
+                        *ok = 0;
+                    } else {
+                        const float4 bb = s_bounds[0];
+                        T[0] = tc_threshold(sb.x, sb.y, bb.x, ok);
+                        T[1] = tc_threshold(sb.x, sb.y, bb.y, ok);
+                        T[2] = tc_threshold(sb.x, sb.y, bb.z, ok);
+                    }
+                }
+                for (int k = 0; k < 3; ++k) {
+                    const int Tc = T[k] < -lim ? -lim : (T[k] > lim ? lim : T[k]);
+                    d[k] |= static_cast<unsigned>(32768 - Tc) << (16 * half);
+                }
+            }
+            thr[e] = make_int4(static_cast<int>(d[0]), static_cast<int>(d[1]), static_cast<int>(d[2]), 0);
+        }
+        return;
+    }
     for (int e = t; e < g.thr_pats * g.TN; e += nthreads) {
         const int f = e % g.TN, pat = e / g.TN;
         int4 T = make_int4(TC_THR_LIM, TC_THR_LIM, TC_THR_LIM, 0);         // filters past O: never reached, masked anyway
@@ -532,6 +565,24 @@ __device__ __forceinline__ uint32_t spread16(uint32_t x)
     x = (x | (x << 2)) & 0x33333333u;
     x = (x | (x << 1)) & 0x55555555u;
     return x;
+}
+
+// 32 accumulators of one pixel, two per 32-bit word (filters j and j + 16 in the 16-bit lanes), against packed thresholds:
+// lane value acc + 2^15 - T_k has bit 15 set exactly when level k is reached, and no carry crosses the lanes.  Three
+// additions, one xor and four shift/merge operations per PAIR of outputs, and half the threshold loads.
+__device__ __forceinline__ void tc_compare_pairs(const uint32_t (&v)[32], uint32_t thr_addr, uint32_t (&ow)[4])
+{
+    uint32_t w0 = 0, w1 = 0;
+#pragma unroll
+    for (int j = 0; j < 16; ++j) {
+        const uint32_t q = v[j + 16] * 65536u + v[j];           // (acc_hi << 16) + acc_lo as one integer sum
+        const int4 D = lds_int4(thr_addr + j * 16);
+        const uint32_t x1 = q + static_cast<uint32_t>(D.x), x2 = q + static_cast<uint32_t>(D.y), x3 = q + static_cast<uint32_t>(D.z);
+        w1 = (w1 >> 1) | (x2 & 0x80008000u);                    // after 16 steps: filter j at bit j, filter j + 16 at bit 16 + j
+        w0 = (w0 >> 1) | ((x1 ^ x2 ^ x3) & 0x80008000u);
+    }
+    ow[0] = w0;         // parity of the levels reached
+    ow[1] = w1;         // level 2 reached
 }
 
 // 32 accumulators of one pixel against their integer thresholds.  The sign bit of acc - T_k says "below level k";
@@ -633,7 +684,9 @@ __device__ __forceinline__ void tc_epilogue_tile(const TcArgs& g, uint32_t tmem_
                 // uniform switches are resolved once per 32 outputs, so the unrolled body is straight-line code.
                 const unsigned valid_mask = (g.O - ob >= 32) ? 0xffffffffu : ((1u << (g.O - ob)) - 1u);
                 const float2* sb32 = s_sb + cc * 32;
-                if (thr_addr) {
+                if (thr_addr && g.thr_packed) {
+                    tc_compare_pairs(v, thr_addr + cc * 256, ow);
+                } else if (thr_addr) {
                     if (!g.residual) tc_compare_int<0>(v, thr_addr + cc * 512, rw, ow);
                     else tc_compare_int<1>(v, thr_addr + cc * 2048, rw, ow);
                 } else if (!g.residual) {
@@ -1145,6 +1198,11 @@ static int tc_conv_impl(const uint32_t* act, const int8_t* wgt, const bs_conv_pa
     g.i32_nhwc = p->i32_layout == BS_NHWC;
     const long long kred = static_cast<long long>(p->C) * RS;
     g.acc_small = kred * tc_max_abs(p->a_bits, p->a_sign) * tc_max_abs(p->w_bits, p->w_sign) < (1LL << 22);
+    {
+        const long long bound = kred * tc_max_abs(p->a_bits, p->a_sign) * tc_max_abs(p->w_bits, p->w_sign);
+        g.acc_bound = bound > 0x7fffffffLL ? 0x7fffffff : static_cast<int>(bound);
+    }
+    g.thr_packed = 0;
 
     g.CK = tc_chunk_channels(p->C, A);
     // Blocks per pipeline chunk: 64 channels when C allows (two MMAs per tap and hand-off), 128 for 1x1 stride-1 layers
@@ -1339,6 +1397,7 @@ static int tc_conv_impl(const uint32_t* act, const int8_t* wgt, const bs_conv_pa
         if (grown <= 220 * 1024 && same_occupancy) {
             g.off_thr = static_cast<int>(off);
             smem = grown;
+            g.thr_packed = (!g.residual && g.acc_bound <= 16383) ? 1 : 0;
         }
     }
 
