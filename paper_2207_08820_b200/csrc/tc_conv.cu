@@ -181,7 +181,8 @@ struct TcTile { int n0, p0, q0; };
 __device__ __forceinline__ TcTile tc_decode_tile(const TcArgs& g, int mt)
 {
     TcTile t;
-    t.q0 = (mt % g.tiles_q) * (g.flat ? TC_M : 8);   mt /= g.tiles_q;
+    if (g.flat) { t.q0 = mt * TC_M; t.p0 = 0; t.n0 = 0; return t; }      // tiles_p = tiles_n = 1
+    t.q0 = (mt % g.tiles_q) * 8;   mt /= g.tiles_q;
     t.p0 = (mt % g.tiles_p) * 16;                    mt /= g.tiles_p;
     t.n0 = mt * g.TNI;
     return t;
@@ -634,22 +635,30 @@ __device__ __forceinline__ void tc_epilogue_tile(const TcArgs& g, uint32_t tmem_
 {
     const int n0 = tile.n0, p0 = tile.p0, q0 = tile.q0;
     const int m = tid;                               // TMEM lane = tile pixel
-    int n, p, q;
+    int n = 0, p = 0, q = 0;
     bool valid;
+    size_t pix;
     if (g.flat) {
-        const long long pix = static_cast<long long>(q0) + m;
-        valid = pix < static_cast<long long>(g.N) * g.P * g.Q;
-        const int hwsz = g.P * g.Q;
-        n = static_cast<int>(pix / hwsz);
-        const int rem = static_cast<int>(pix - static_cast<long long>(n) * hwsz);
-        p = rem / g.Q; q = rem - p * g.Q;
+        // a flat tile is 128 consecutive pixels of the [N][P][Q] order: the pixel index is all the packed output and the
+        // NHWC accumulators need; (n, p, q) cost two divisions and are found only for NCHW accumulators
+        const unsigned upix = static_cast<unsigned>(q0) + static_cast<unsigned>(m);      // N*P*Q < 2^31 (checked on the host)
+        valid = upix < static_cast<unsigned>(g.N) * static_cast<unsigned>(g.P * g.Q);
+        pix = upix;
+        if (g.out_i32 && !g.i32_nhwc) {
+            const unsigned hwsz = static_cast<unsigned>(g.P * g.Q);
+            n = static_cast<int>(upix / hwsz);
+            const unsigned rem = upix - static_cast<unsigned>(n) * hwsz;
+            p = static_cast<int>(rem / static_cast<unsigned>(g.Q));
+            q = static_cast<int>(rem - static_cast<unsigned>(p) * static_cast<unsigned>(g.Q));
+        }
     } else {
         const int grp = m >> 3, tx = m & 7;
-        const int ni = grp / g.GI, ty = grp - ni * g.GI;
+        int ni = 0, ty = grp;
+        if (g.GI != 16) { ni = grp / g.GI; ty = grp - ni * g.GI; }          // stacked small images
         n = n0 + ni; p = p0 + ty; q = q0 + tx;
         valid = n < g.N && p < g.P && q < g.Q && ni < g.TNI && (g.GI == 16 || ty < g.P);
+        pix = (static_cast<size_t>(n) * g.P + p) * g.Q + q;
     }
-    const size_t pix = (static_cast<size_t>(n) * g.P + p) * g.Q + q;
     int qmin, qmax;
     code_limits(g.out_bits > 0 ? g.out_bits : 1, g.out_sign, qmin, qmax);
     const float fqmin = static_cast<float>(qmin), fqmax = static_cast<float>(qmax);
