@@ -34,15 +34,17 @@ POPC_PER_CLK_PER_SM = 16          # population count throughput per SM per clock
 POPC_PER_WORDOP = 2.0 / 3.0       # executed by the kernel's 3:2 carry-save adder: three popc32(AND) word operations cost two counts
 
 
-def make_net(name: str, batch: int):
+def make_net(name: str, batch: int, hw: int = 0):
+    """hw: side of the first packed tensor (0: the workload's own: 56 / 320 / 56 / 300)."""
+    kw = {"hw": hw} if hw else {}
     if name == "resnet18_body":
-        return wl.resnet18_body(batch), 3000
+        return wl.resnet18_body(batch, **kw), 3000
     if name == "detection_backbone":
-        return wl.detection_backbone(batch), 4000
+        return wl.detection_backbone(batch, **kw), 4000
     if name == "resnet50_body":
-        return wl.resnet50_body(batch), 6000
+        return wl.resnet50_body(batch, **kw), 6000
     if name == "vgg16_ssd_body":
-        return wl.vgg16_ssd_body(batch), 7000
+        return wl.vgg16_ssd_body(batch, **kw), 7000
     raise SystemExit(f"unknown workload {name}")
 
 
@@ -118,7 +120,7 @@ def run_reference(args):
         return
     import oracle
     from oracle import network as onet
-    net, seed = make_net(args.workload, args.batch)
+    net, seed = make_net(args.workload, args.batch, args.hw)
     params = wl.network_params(net, seed)
     sample = args.ref_images
     x = wl.network_input(net, seed, ACT_SCALE, batch=sample)
@@ -159,7 +161,7 @@ def run_ours(args):
     if world > 1:
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
 
-    net, seed = make_net(args.workload, args.batch)
+    net, seed = make_net(args.workload, args.batch, args.hw)
     params = wl.network_params(net, seed)
     x_host = torch.from_numpy(wl.network_input(net, replicas.rank_seed(seed, rank), ACT_SCALE)).pin_memory()
     x_dev = x_host.cuda()
@@ -344,7 +346,7 @@ def run_ours(args):
             "metric": METRIC, "value": gops, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
             "ms_per_step": t_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": "int32", "data": "synthetic",
-            "config": {"workload": f"{net.name}_batch{net.batch}_w{net.w_bits}a{net.a_bits}",
+            "config": {"workload": f"{net.name}_batch{net.batch}_w{net.w_bits}a{net.a_bits}" + (f"_hw{args.hw}" if args.hw else ""),
                        "global_batch": net.batch * world, "parallelism": f"replicas{world}", "layers": len(net.layers),
                        "l2": "flushed between timed iterations (256 MB write)", "launch": ("eager stream launches" if args.eager else "CUDA graphs (pack, convs)") +
                                  "; layers chained (programmatic dependent launch), independent neighbours on two streams"},
@@ -390,6 +392,8 @@ def main():
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="resnet18_body", choices=["resnet18_body", "detection_backbone", "resnet50_body", "vgg16_ssd_body"])
+    ap.add_argument("--hw", type=int, default=0, help="side of the first packed tensor (default: the workload's own; the paper's 320 / 352 px "
+                    "detection inputs are --workload detection_backbone --hw 160 / 176)")
     ap.add_argument("--batch", type=int, default=0, help="images per GPU (default: 64 / 16 / 32 / 8 as the workload defines)")
     ap.add_argument("--ref-images", type=int, default=2, help="images per step of the reference arm (bounded CPU sample)")
     ap.add_argument("--cpu-baseline-images", type=int, default=64, help="images of the one oracle pass timed beside the GPU run")

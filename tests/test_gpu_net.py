@@ -95,3 +95,8 @@ def test_resnet50_body_full_batch_sampled():
     """Batch 32 at 56 px (the configuration `bench.py --workload resnet50_body` times): wide 1x1 chunks, streamed deep
     reductions and projection shortcuts on the second stream, two images checked against the oracle."""
     compare_stack(wl.resnet50_body(32), 32, seed=6000, sample=[0, 31], graph=True, engine="tc")
+
+
+def test_detection_backbone_352px_input():
+    """The paper's 352 px detection input: first packed tensor 176 px, widths 176 / 88 / 44 / 22 / 11."""
+    compare_stack(wl.detection_backbone(1, hw=176), 1, seed=4000, engine="tc")
