@@ -88,6 +88,21 @@ def test_bad_arguments_are_rejected_on_the_host(L):
     assert L.bitserial_conv2d(addr, addr, ctypes.byref(p), addr, None, None) == UNSUPPORTED
     assert L.bitserial_gemm(addr, addr, 0, 4, 4, 2, 0, 2, 1, None, None, 0, 0, 0, addr, None, None) == INVALID
     assert L.bs_status_string(5) == b"BS_ERR_TIMEOUT"
+    # bs_l2_prefetch: nothing to do is fine; missing arrays, null or misaligned buffers are refused before any launch
+    assert L.bs_l2_prefetch(None, None, 0, None) == 0
+    assert L.bs_l2_prefetch(None, None, 1, None) == INVALID
+    ptrs = (ctypes.c_void_p * 2)(addr, None)
+    sizes = (ctypes.c_size_t * 2)(256, 256)
+    assert L.bs_l2_prefetch(ptrs, sizes, 2, None) == INVALID
+    ptrs[1] = addr + 8
+    assert L.bs_l2_prefetch(ptrs, sizes, 2, None) == ALIGN
+    # tensor-core entry points: channel counts and pixel records the tensor-core path cannot take
+    p2 = ConvParams(N=1, C=40, H=8, W=8, O=64, R=3, S=3, stride=1, pad=1, a_bits=2, a_sign=0, w_bits=2, w_sign=1, i32_layout=0)
+    assert L.bs_tc_supported(ctypes.byref(p2)) == 0
+    assert L.bitserial_conv2d_tc(addr, addr, ctypes.byref(p2), addr, None, None) == UNSUPPORTED
+    assert L.bitserial_conv2d_tc_chained(addr, addr, ctypes.byref(p2), addr, None, None) == UNSUPPORTED
+    assert L.bs_tc_weights_bytes(64, 40, 3, 3) == 0
+    assert L.bs_tc_weights_bytes(200, 64, 3, 3) == 256 * 9 * 64
 
 
 def test_binding_fails_loudly_without_library(tmp_path):
