@@ -19,6 +19,7 @@ constexpr int PACK_UNROLL = 8;      // NHWC: pixels in flight per warp
 // three compares instead of a division.  Wider codes evaluate the formula directly.
 struct QuantParams {
     float bound[3];
+    float below[3];     // largest binary32 value below bound[k] (never -0): x >= bound[k]  <=>  sign bit of (below[k] - x) is set
     float scale;
     int bits, sign, qmin, qmax;
     int by_bounds;      // 1: compare against bound[]; 0: evaluate the formula
@@ -58,6 +59,19 @@ struct PlaneBits {
 template <typename T> __device__ __forceinline__ T null_input(const QuantParams& q);
 template <> __device__ __forceinline__ float null_input<float>(const QuantParams& q) { return q.null_value; }
 template <> __device__ __forceinline__ int8_t null_input<int8_t>(const QuantParams& q) { return static_cast<int8_t>(q.null_value); }
+
+// A warp copies the contiguous packed records of its tile from shared to global memory, as 128-bit stores when the
+// tile starts on a 16-byte boundary.
+__device__ __forceinline__ void store_tile_records(const uint32_t* stage, uint32_t* dst, int nwords, bool vec, int lane)
+{
+    if (vec) {
+        const int nvec = nwords / 4;
+        for (int k = lane; k < nvec; k += 32) reinterpret_cast<uint4*>(dst)[k] = reinterpret_cast<const uint4*>(stage)[k];
+        for (int k = nvec * 4 + lane; k < nwords; k += 32) dst[k] = stage[k];
+    } else {
+        for (int k = lane; k < nwords; k += 32) dst[k] = stage[k];
+    }
+}
 
 // One warp packs 32 consecutive pixels (flattened y*W + x) of one image, all channels, with no block-wide barrier.
 //   NCHW: lane = pixel.  Every channel row is read with one coalesced 128-byte request per warp, a whole 32-channel
@@ -135,16 +149,78 @@ bitpack_kernel(const T* __restrict__ x, uint32_t* __restrict__ out, int C, int H
         }
     }
     __syncwarp();
-    // write-out: npix * rec contiguous words
-    uint32_t* dst = out + (static_cast<size_t>(n) * HW + hw0) * rec;
-    const int nwords = npix * rec;
-    if ((static_cast<size_t>(HW) * rec) % 4 == 0 && (32 * rec) % 4 == 0) {
-        const int nvec = nwords / 4;
-        for (int k = lane; k < nvec; k += 32) reinterpret_cast<uint4*>(dst)[k] = reinterpret_cast<const uint4*>(stage)[k];
-        for (int k = nvec * 4 + lane; k < nwords; k += 32) dst[k] = stage[k];
+    store_tile_records(stage, out + (static_cast<size_t>(n) * HW + hw0) * rec, npix * rec,
+                       (static_cast<size_t>(HW) * rec) % 4 == 0 && (32 * rec) % 4 == 0, lane);
+}
+
+// Sign-bit form of the comparison quantiser for fp32 NCHW input and 1- or 2-bit codes.
+//   With p the largest binary32 value below the bound b:  x >= b  <=>  x > p  <=>  the sign bit of p - x is set.
+//   An IEEE subtraction never rounds across zero and x == p gives +0; p is stored as +0 when it is a zero, so neither
+//   signed zero of x yields -0.  A NaN input gives the canonical NaN (sign clear): no level reached, the lowest
+//   code, which is what clip() makes of a NaN in the formula.  +-inf behave like the comparison.
+//   2-bit codes: plane 1 = (x >= b1); plane 0 = parity of the three comparisons = sign((p0-x) ^ (p1-x) ^ (p2-x)).
+// One funnel shift moves a sign bit into a plane word; channels are walked from 31 down to 0 so that channel c ends at
+// bit c.  Per element: one load, 1 or 3 subtractions, at most one three-input xor and BITS funnel shifts, which
+// leaves the kernel waiting on HBM rather than on the issue slots.
+// Work unit of a warp = 32 consecutive pixels of one image x one 32-channel word (lane = pixel): all 32 channel rows are
+// in flight at once (32 coalesced 128-byte requests per warp), and each lane stores the BITS plane words of its pixel
+// straight to the packed record (8-byte stores for 2-bit codes; the words of the other channel groups of the record
+// come from the neighbouring warps of the block, so the sectors fill up in L2).  Units are small and numerous, which
+// keeps the tail of the grid short; no shared memory, no barrier.
+constexpr int FAST_THREADS = 128;
+constexpr int FAST_WARPS = FAST_THREADS / 32;
+
+template <int BITS>
+__global__ void __launch_bounds__(FAST_THREADS, 8)
+bitpack_nchw_f32_kernel(const float* __restrict__ x, uint32_t* __restrict__ out, int C, int HW, int Cw, long long nunits,
+                        int units_per_img, const QuantParams q)
+{
+    static_assert(BITS == 1 || BITS == 2, "comparison form covers 1- and 2-bit codes");
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const long long unit = static_cast<long long>(blockIdx.x) * FAST_WARPS + warp;
+    if (unit >= nunits) return;
+    const long long n = unit / units_per_img;
+    const int rem = static_cast<int>(unit % units_per_img);
+    const int cw = rem % Cw;
+    const int hw0 = (rem / Cw) * 32;
+    const bool pvalid = lane < HW - hw0;
+    const float p0 = q.below[0], p1 = q.below[1], p2 = q.below[2];
+    // lanes beyond the image re-read the first pixel of the tile (always in bounds) and store nothing
+    const float* xin = x + (static_cast<size_t>(n) * C + cw * 32) * HW + hw0 + (pvalid ? lane : 0);
+    uint32_t w0 = 0u, w1 = 0u;
+    auto push = [&](float v) {
+        if constexpr (BITS == 1) {
+            w0 = __funnelshift_l(__float_as_uint(p0 - v), w0, 1);
+        } else {
+            const uint32_t d0 = __float_as_uint(p0 - v), d1 = __float_as_uint(p1 - v), d2 = __float_as_uint(p2 - v);
+            w1 = __funnelshift_l(d1, w1, 1);
+            w0 = __funnelshift_l(d0 ^ d1 ^ d2, w0, 1);
+        }
+    };
+    const int nvalid = min(32, C - cw * 32);
+    if (nvalid == 32) {
+        // a full channel word: unconditional loads, walking the channel rows downward from channel 31
+        const ptrdiff_t row = HW;
+        const float* pc = xin + 31 * row;
+        float v[32];
+#pragma unroll
+        for (int u = 0; u < 32; ++u) {
+            v[u] = __ldcs(pc);
+            pc -= row;
+        }
+#pragma unroll
+        for (int u = 0; u < 32; ++u) push(v[u]);
     } else {
-        for (int k = lane; k < nwords; k += 32) dst[k] = stage[k];
+        // the ragged last word: channels past C count as "no level reached"
+        for (int u = 31; u >= 0; --u) push(u < nvalid ? __ldcs(xin + static_cast<size_t>(u) * HW) : -INFINITY);
     }
+    if (!pvalid) return;
+    const unsigned fl = nvalid == 32 ? 0xffffffffu : ((1u << nvalid) - 1u);
+    if (q.flip & 1) w0 ^= fl;
+    if (q.flip & 2) w1 ^= fl;
+    uint32_t* dst = out + ((static_cast<size_t>(n) * HW + hw0 + lane) * Cw + cw) * BITS;
+    if constexpr (BITS == 2) *reinterpret_cast<uint2*>(dst) = make_uint2(w0, w1);
+    else *dst = w0;
 }
 
 __global__ void bitunpack_kernel(const uint32_t* __restrict__ packed, int8_t* __restrict__ codes, long long total,
@@ -230,6 +306,17 @@ static float key_float(uint32_t k)
     return f;
 }
 
+// below[k] = the binary32 value just under bound[k] (bounds are never -inf: -inf always quantises to the lowest code).
+static void set_below(QuantParams& q)
+{
+    for (int k = 0; k < 3; ++k) {
+        const float b = q.bound[k];
+        float p = b == 0.0f ? -1.401298464e-45f : key_float(float_key(b) - 1u);
+        if (p == 0.0f) p = 0.0f;          // drops the sign of a zero
+        q.below[k] = p;
+    }
+}
+
 static QuantParams make_quant_params(float s, int bits, int sign, bool quantise)
 {
     QuantParams q{};
@@ -243,6 +330,8 @@ static QuantParams make_quant_params(float s, int bits, int sign, bool quantise)
         q.null_value = -INFINITY;
         q.by_bounds = 1;
         q.bound[0] = 0.0f;
+        q.bound[1] = q.bound[2] = INFINITY;
+        set_below(q);
         return q;
     }
     if (bits <= 2) {
@@ -262,6 +351,7 @@ static QuantParams make_quant_params(float s, int bits, int sign, bool quantise)
         if (bits == 1) q.bound[1] = q.bound[2] = INFINITY;
         // pattern = (qmin + count) mod 2^bits; for two's-complement 2-bit codes qmin = -2 flips bit 1 only
         q.flip = (sign == BS_SIGNED) ? (static_cast<unsigned>(q.qmin) & ((1u << bits) - 1u)) : 0;
+        set_below(q);
     }
     return q;
 }
@@ -286,9 +376,28 @@ static int launch_bitpack_one(const void* x, uint32_t* out, int N, int C, int HW
     return cudaGetLastError() == cudaSuccess ? BS_OK : BS_ERR_CUDA;
 }
 
+template <int BITS>
+static int launch_bitpack_nchw_f32(const void* x, uint32_t* out, int N, int C, int HW, const QuantParams& q, cudaStream_t st)
+{
+    const int Cw = ceil_div(C, 32);
+    const long long units_per_img = static_cast<long long>(ceil_div(HW, 32)) * Cw;
+    const long long nunits = N * units_per_img;
+    const long long blocks = ceil_div_ll(nunits, FAST_WARPS);
+    if (units_per_img > 0x7fffffffLL || blocks > 0x7fffffffLL) return BS_ERR_UNSUPPORTED;
+    bitpack_nchw_f32_kernel<BITS><<<static_cast<unsigned>(blocks), FAST_THREADS, 0, st>>>(
+        static_cast<const float*>(x), out, C, HW, Cw, nunits, static_cast<int>(units_per_img), q);
+    return cudaGetLastError() == cudaSuccess ? BS_OK : BS_ERR_CUDA;
+}
+
 template <typename T, bool NHWC>
 static int launch_bitpack(const void* x, uint32_t* out, int N, int C, int HW, const QuantParams& q, cudaStream_t st)
 {
+    if constexpr (sizeof(T) == 4 && !NHWC) {
+        // comparison-form codes (1 and 2 bits) of an NCHW fp32 tensor take the sign-bit kernel
+        if (q.by_bounds)
+            return q.bits == 1 ? launch_bitpack_nchw_f32<1>(x, out, N, C, HW, q, st)
+                               : launch_bitpack_nchw_f32<2>(x, out, N, C, HW, q, st);
+    }
     switch (q.bits) {
         case 1: return launch_bitpack_one<T, NHWC, 1, true>(x, out, N, C, HW, q, st);
         case 2: return launch_bitpack_one<T, NHWC, 2, true>(x, out, N, C, HW, q, st);

@@ -52,11 +52,24 @@ class BitserialNet:
         self.launches_per_forward = 2 + len(self.layers)
 
     def _run(self, x: torch.Tensor) -> torch.Tensor:
-        net = self.net
-        self.prefetch_filters()
-        api.bitpack_activations(x, self.act_scale, net.a_bits, api.UNSIGNED, api.NCHW, out=self.bufs[net.in_name].view(-1))
+        self.pack_input(x)
         self.run_layers()
-        return self.bufs[net.out_name]
+        return self.bufs[self.net.out_name]
+
+    def pack_input(self, x: torch.Tensor) -> None:
+        """Quantise + bitplane-pack the fp32 input on the current stream; the filter prefetch runs beside it on the
+        side stream (a fork and a join: two parallel nodes under stream capture)."""
+        net = self.net
+        main = torch.cuda.current_stream(self.device)
+        fork = torch.cuda.Event()
+        fork.record(main)
+        self.side.wait_event(fork)
+        with torch.cuda.stream(self.side):
+            self.prefetch_filters()
+            done = torch.cuda.Event()
+            done.record(self.side)
+        api.bitpack_activations(x, self.act_scale, net.a_bits, api.UNSIGNED, api.NCHW, out=self.bufs[net.in_name].view(-1))
+        main.wait_event(done)
 
     def run_layer(self, item, chained: bool = True) -> None:
         """One conv layer through the C ABI on the current stream."""
