@@ -7,6 +7,9 @@ GPU, 2-bit weights and activations) with the fused requantisation epilogue.  Pri
 
   python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--workload NAME]
 
+`--workload bitwidth_sweep` / `gemm_sweep` time the single-layer sweeps (plane pairs W*A on a 3x3 conv; the im2col-form
+matrix products) case by case instead of a layer stack.
+
 N > 1 runs under torchrun, one rank per GPU, each rank its own batch (no data-path collective).
 `--impl reference` times the CPU oracle on a bounded sample of the same workload on the host cores.
 """
@@ -143,6 +146,107 @@ def run_reference(args):
         "cpu_baseline": {"value": gops, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": desc},
         "e2e": {"value": gops, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
     }))
+
+
+def run_sweep(args):
+    """Single-layer sweeps on one GPU, one JSON line with a table in "sweep":
+      bitwidth_sweep : 3x3 conv N=32, C=O=256, 28x28 for (W,A) in {(1,1),(1,2),(2,2),(2,3),(3,3)}, int32 accumulators +
+                       requantised output: time against the number of plane pairs W*A;
+      gemm_sweep     : bitserial_gemm, 1-bit bipolar weights x 2-bit activations, M=N in {256,1024,4096}, K in
+                       {576,2304,4608}, int32 outputs.
+    Every case is launched alone (CUDA events around each launch, L2 flushed before it) on the popcount kernels, the
+    conv cases on the tensor-core entry point as well."""
+    import torch
+
+    from paper_2207_08820_b200 import api
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the library has no CPU fallback")
+    if int(os.environ.get("RANK", "0")) != 0:
+        return
+    torch.cuda.set_device(0)
+    dev = lambda a: torch.from_numpy(np.ascontiguousarray(a)).cuda()
+    flush = torch.empty(256 * 1024 * 1024, dtype=torch.uint8, device="cuda")
+    flush_words = flush.view(torch.int32)
+    peaks, peak_kind = measured_peaks()
+    sms = torch.cuda.get_device_properties(0).multi_processor_count
+    popc_peak = POPC_PER_CLK_PER_SM * sms * peaks["sm_max_mhz"] * 1e6
+    int8_peak = 2.0 * peaks.get("bf16_tflops_sustained", peaks["bf16_tflops"]) * 1e12
+    hbm_peak = peaks["hbm_gbs"] * 1e9
+    steps = min(args.steps, 20)
+    launches = 0
+
+    def timed(fn):
+        nonlocal launches
+        ts = []
+        for k in range(args.warmup + steps):
+            flush.zero_()
+            torch.amax(flush_words)
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            fn()
+            e1.record()
+            e1.synchronize()
+            if k >= args.warmup:
+                ts.append(e0.elapsed_time(e1))
+                launches += 1
+        return float(np.mean(ts)), float(np.min(ts))
+
+    rows, tot_ops, tot_ms = [], 0.0, 0.0
+    with ClockSampler(0) as clocks:
+        if args.workload == "bitwidth_sweep":
+            for wb, ab in wl.BITWIDTH_SWEEP:
+                c = wl.bitwidth_sweep_case(wb, ab)
+                xp = api.bitpack_activations(dev(c["x"]), 1.0, ab, c["a_sign"], api.NCHW)
+                wp = api.pack_weights(dev(c["w"]), wb, c["w_sign"])
+                sc, bi = dev(c["scale"]), dev(c["bias"])
+                P = Q = c["H"]
+                acc = torch.empty(c["N"], c["O"], P, Q, dtype=torch.int32, device="cuda")
+                outp = torch.zeros(c["N"], P, Q, c["O"] // 32, ab, dtype=torch.int32, device="cuda")
+                kw = dict(C=c["C"], stride=1, pad=1, a_sign=c["a_sign"], w_sign=c["w_sign"], scale=sc, bias=bi, relu=True,
+                          out_bits=ab, out_sign=api.UNSIGNED, out_packed=outp)
+                macs = c["N"] * P * Q * c["O"] * c["C"] * 9
+                wops = macs // 32 * wb * ab
+                ms_acc, _ = timed(lambda: api.bitserial_conv2d(xp, wp, out_i32=acc, **kw))     # int32 + packed outputs
+                ms, best = timed(lambda: api.bitserial_conv2d(xp, wp, **kw))                   # packed output only
+                row = {"w_bits": wb, "a_bits": ab, "pairs": wb * ab, "ms": ms, "ms_best": best, "ms_with_int32_out": ms_acc,
+                       "gops": 2.0 * macs / ms / 1e6, "Tword_ops_per_s": wops / ms / 1e9, "frac_popc": wops / (ms * 1e-3) / popc_peak}
+                if api.tc_supported(c["N"], c["C"], c["H"], c["W"], c["O"], 3, 1, 1, ab, c["a_sign"], wb, c["w_sign"]):
+                    wt = api.tc_prepare_weights(wp, c["C"], c["w_sign"], ab)
+                    tms, _ = timed(lambda: api.bitserial_conv2d(xp, wp, wgt_tc=wt, **kw))
+                    row.update(tc_ms=tms, tc_gops=2.0 * macs / tms / 1e6, tc_frac_int8=2.0 * macs / (tms * 1e-3) / int8_peak)
+                rows.append(row)
+                tot_ops += 2.0 * macs
+                tot_ms += ms
+            name = "bitwidth_sweep_conv3x3_n32_c256_o256_hw28"
+        else:
+            for M in wl.GEMM_SWEEP_MN:
+                for K in wl.GEMM_SWEEP_K:
+                    c = wl.gemm_case(M, M, K, seed=wl.gemm_sweep_seed(M, K))
+                    a_p = api.bs_pack_rows(dev(c["a"]), c["a_bits"], c["a_sign"])
+                    w_p = api.bs_pack_rows(dev(c["w"]), c["w_bits"], c["w_sign"])
+                    out = torch.empty(M, M, dtype=torch.int32, device="cuda")
+                    ms, best = timed(lambda: api.bitserial_gemm(a_p, w_p, K, a_sign=c["a_sign"], w_sign=c["w_sign"], out_i32=out))
+                    macs = M * M * K
+                    wops = macs // 32 * c["a_bits"] * c["w_bits"]
+                    nbytes = (a_p.numel() + w_p.numel() + out.numel()) * 4
+                    t_popc, t_hbm = wops / popc_peak, nbytes / hbm_peak
+                    rows.append({"M": M, "N": M, "K": K, "ms": ms, "ms_best": best, "gops": 2.0 * macs / ms / 1e6,
+                                 "Tword_ops_per_s": wops / ms / 1e9, "GB_per_s": nbytes / ms / 1e6,
+                                 "bound": "alu" if t_popc >= t_hbm else "hbm",
+                                 "frac_roofline": max(t_popc, t_hbm) / (ms * 1e-3)})
+                    tot_ops += 2.0 * macs
+                    tot_ms += ms
+            name = "gemm_sweep_w1bipolar_a2_int32_out"
+    api.bs_check_status()
+    print(json.dumps({
+        "metric": METRIC, "value": tot_ops / tot_ms / 1e6, "unit": UNIT, "n_gpus": 1, "steps": steps, "warmup": args.warmup,
+        "ms_per_step": tot_ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "int32",
+        "data": "synthetic",
+        "config": {"workload": name, "engine": "popc", "l2": "flushed before every launch (256 MB write, then read back)",
+                   "launch": "one eager launch per case, CUDA events around it (launch latency included)"},
+        "sweep": rows,
+        "peaks": {"popc_word_ops_per_s": popc_peak, "int8_ops_per_s": int8_peak, "hbm_bytes_per_s": hbm_peak, "kind": peak_kind},
+        "gpu_launches": launches, "clocks": clocks.summary()}))
 
 
 def run_ours(args):
@@ -397,7 +501,7 @@ def main():
     ap.add_argument("--steps", type=int, default=50)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="resnet18_body", choices=["resnet18_body", "detection_backbone", "resnet50_body", "vgg16_ssd_body"])
+    ap.add_argument("--workload", default="resnet18_body", choices=["resnet18_body", "detection_backbone", "resnet50_body", "vgg16_ssd_body", "bitwidth_sweep", "gemm_sweep"])
     ap.add_argument("--hw", type=int, default=0, help="side of the first packed tensor (default: the workload's own; the paper's 320 / 352 px "
                     "detection inputs are --workload detection_backbone --hw 160 / 176)")
     ap.add_argument("--batch", type=int, default=0, help="images per GPU (default: 64 / 16 / 32 / 8 as the workload defines)")
@@ -408,6 +512,11 @@ def main():
                     help="popc: popcount kernels on the integer pipes; tc: exact int8 tensor-core formulation")
     ap.add_argument("--eager", action="store_true", help="plain stream launches instead of CUDA graphs (for per-launch profiling)")
     args = ap.parse_args()
+    if args.workload in ("bitwidth_sweep", "gemm_sweep"):
+        if args.impl == "reference":
+            raise SystemExit("the reference arm times the layer stacks only")
+        args.warmup = max(args.warmup, 3)
+        return run_sweep(args)
     if args.batch == 0:
         args.batch = {"resnet18_body": 64, "detection_backbone": 16, "resnet50_body": 32, "vgg16_ssd_body": 8}[args.workload]
     if args.warmup < 3 and args.impl == "ours":
