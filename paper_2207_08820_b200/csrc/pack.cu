@@ -223,6 +223,172 @@ bitpack_nchw_f32_kernel(const float* __restrict__ x, uint32_t* __restrict__ out,
     else *dst = w0;
 }
 
+// fp32 NHWC input, 1- or 2-bit codes in comparison form.  Work unit of a warp = 32 consecutive pixels x one 32-channel
+// word, lane = channel: the 32 channels of a pixel are one coalesced 128-byte request, all 32 pixels of the unit are in
+// flight at once, one __ballot_sync per plane turns the 32 comparisons of a pixel into its plane word, and lane p keeps
+// the words of pixel p, so the records leave as one store per lane like in the NCHW kernel.
+template <int BITS>
+__global__ void __launch_bounds__(FAST_THREADS, 8)
+bitpack_nhwc_f32_kernel(const float* __restrict__ x, uint32_t* __restrict__ out, int C, int HW, int Cw, long long nunits,
+                        int units_per_img, const QuantParams q)
+{
+    static_assert(BITS == 1 || BITS == 2, "comparison form covers 1- and 2-bit codes");
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const long long unit = static_cast<long long>(blockIdx.x) * FAST_WARPS + warp;
+    if (unit >= nunits) return;
+    const long long n = unit / units_per_img;
+    const int rem = static_cast<int>(unit % units_per_img);
+    const int cw = rem % Cw;
+    const int hw0 = (rem / Cw) * 32;
+    const int npix = min(32, HW - hw0);
+    const bool cvalid = cw * 32 + lane < C;
+    const unsigned valid_word = __ballot_sync(0xffffffffu, cvalid);
+    // lanes past the last channel re-read the first channel of the word (always in bounds) and vote "no level reached"
+    const float* xin = x + (static_cast<size_t>(n) * HW + hw0) * C + cw * 32 + (cvalid ? lane : 0);
+    const float b0 = q.bound[0], b1 = q.bound[1], b2 = q.bound[2];
+    uint32_t my0 = 0u, my1 = 0u;
+    auto vote = [&](float v, int u) {
+        const bool c1 = v >= b0;
+        if constexpr (BITS == 1) {
+            const uint32_t w0 = __ballot_sync(0xffffffffu, cvalid && c1);
+            if (lane == u) my0 = w0;
+        } else {
+            const bool c2 = v >= b1, c3 = v >= b2;      // count = c1 + c2 + c3: bit 0 is the parity, bit 1 is c2
+            const uint32_t w0 = __ballot_sync(0xffffffffu, cvalid && ((c1 != c2) != c3));
+            const uint32_t w1 = __ballot_sync(0xffffffffu, cvalid && c2);
+            if (lane == u) { my0 = w0; my1 = w1; }
+        }
+    };
+    if (npix == 32) {
+        const size_t row = C;
+        float v[32];
+#pragma unroll
+        for (int u = 0; u < 32; ++u) v[u] = __ldcs(xin + u * row);
+#pragma unroll
+        for (int u = 0; u < 32; ++u) vote(v[u], u);
+    } else {
+        for (int u = 0; u < npix; ++u) vote(__ldcs(xin + static_cast<size_t>(u) * C), u);
+    }
+    if (lane >= npix) return;
+    if (q.flip & 1) my0 ^= valid_word;
+    if (q.flip & 2) my1 ^= valid_word;
+    uint32_t* dst = out + ((static_cast<size_t>(n) * HW + hw0 + lane) * Cw + cw) * BITS;
+    if constexpr (BITS == 2) *reinterpret_cast<uint2*>(dst) = make_uint2(my0, my1);
+    else *dst = my0;
+}
+
+// Stores the BITS plane words of one (pixel, channel word) with the widest aligned store.
+template <int BITS>
+__device__ __forceinline__ void store_planes(uint32_t* dst, const uint32_t (&w)[BITS])
+{
+    if constexpr (BITS == 4) *reinterpret_cast<uint4*>(dst) = make_uint4(w[0], w[1], w[2], w[3]);
+    else if constexpr (BITS == 2) *reinterpret_cast<uint2*>(dst) = make_uint2(w[0], w[1]);
+    else {
+#pragma unroll
+        for (int j = 0; j < BITS; ++j) dst[j] = w[j];
+    }
+}
+
+// int8 codes, NCHW (unsigned or two's-complement codes: plane j is bit j of the byte).  At one byte per element the
+// HBM roofline leaves about five thread instructions per element, so the plane split works on four pixels at a time:
+// a lane owns four consecutive pixels and reads them as one 32-bit word per channel row (a warp = 128 pixels, 128-byte
+// requests); (r >> j) & 0x01010101 is bit j of the four codes, and a = 2 a + that, over eight channel rows from the
+// highest down, leaves in byte k of a the eight channel bits of pixel k.  A byte permute drops each finished byte into
+// the plane word of its pixel.  About 1.8 instructions per element for 2-bit codes.  Needs H*W to be a multiple of 4
+// (aligned 32-bit loads); work unit of a warp = 128 pixels x one 32-channel word.
+template <int BITS>
+__global__ void __launch_bounds__(FAST_THREADS, 8)
+bitpack_nchw_i8_kernel(const int8_t* __restrict__ x, uint32_t* __restrict__ out, int C, int HW, int Cw, long long nunits,
+                       int units_per_img)
+{
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const long long unit = static_cast<long long>(blockIdx.x) * FAST_WARPS + warp;
+    if (unit >= nunits) return;
+    const long long n = unit / units_per_img;
+    const int rem = static_cast<int>(unit % units_per_img);
+    const int cw = rem % Cw;
+    const int hw0 = (rem / Cw) * 128;
+    const int pix = hw0 + 4 * lane;
+    const bool pvalid = pix < HW;          // H*W is a multiple of 4: the four pixels of a lane are inside or outside together
+    const uint32_t* xin = reinterpret_cast<const uint32_t*>(x + (static_cast<size_t>(n) * C + cw * 32) * HW + (pvalid ? pix : hw0));
+    const int nvalid = min(32, C - cw * 32);
+    const size_t row = static_cast<size_t>(HW / 4);
+    uint32_t v[32];
+    if (nvalid == 32) {
+#pragma unroll
+        for (int u = 0; u < 32; ++u) v[u] = __ldcs(xin + u * row);
+    } else {
+#pragma unroll
+        for (int u = 0; u < 32; ++u) v[u] = u < nvalid ? __ldcs(xin + u * row) : 0u;
+    }
+    uint32_t w[4][BITS];
+#pragma unroll
+    for (int k = 0; k < 4; ++k)
+#pragma unroll
+        for (int j = 0; j < BITS; ++j) w[k][j] = 0u;
+#pragma unroll
+    for (int g = 0; g < 4; ++g) {
+        uint32_t a[BITS];
+#pragma unroll
+        for (int j = 0; j < BITS; ++j) a[j] = 0u;
+#pragma unroll
+        for (int i = 7; i >= 0; --i) {
+            const uint32_t r = v[8 * g + i];
+#pragma unroll
+            for (int j = 0; j < BITS; ++j) a[j] = a[j] * 2u + ((r >> j) & 0x01010101u);
+        }
+#pragma unroll
+        for (int k = 0; k < 4; ++k)
+#pragma unroll
+            for (int j = 0; j < BITS; ++j)      // byte k of a[j] becomes byte g of the plane word of pixel k
+                w[k][j] = __byte_perm(w[k][j], a[j], (0x3210u & ~(0xfu << (4 * g))) | ((4u + k) << (4 * g)));
+    }
+    if (!pvalid) return;
+#pragma unroll
+    for (int k = 0; k < 4; ++k)
+        store_planes<BITS>(out + ((static_cast<size_t>(n) * HW + pix + k) * Cw + cw) * BITS, w[k]);
+}
+
+// int8 codes, NHWC, C a multiple of 32: the 32 channels of a (pixel, channel word) are 32 contiguous, aligned bytes.
+// Lane = pixel; a warp takes 128 pixels x one channel word (four pixels per lane, eight 128-bit loads in flight).  For
+// each word of four codes, ((q >> j) & 0x01010101) * 0x01020408 gathers bit j of the four bytes in bits 24..27 (all
+// partial products fall on distinct bits, so nothing carries).  About 2.5 instructions per element for 2-bit codes.
+template <int BITS>
+__global__ void __launch_bounds__(FAST_THREADS, 8)
+bitpack_nhwc_i8_kernel(const int8_t* __restrict__ x, uint32_t* __restrict__ out, int C, int HW, int Cw, long long nunits,
+                       int units_per_img)
+{
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const long long unit = static_cast<long long>(blockIdx.x) * FAST_WARPS + warp;
+    if (unit >= nunits) return;
+    const long long n = unit / units_per_img;
+    const int rem = static_cast<int>(unit % units_per_img);
+    const int cw = rem % Cw;
+    const int hw0 = (rem / Cw) * 128;
+    uint4 q[4][2];
+#pragma unroll
+    for (int t = 0; t < 4; ++t) {
+        const int pix = min(hw0 + 32 * t + lane, HW - 1);       // clamped: always in bounds, stored only when inside
+        const uint4* src = reinterpret_cast<const uint4*>(x + (static_cast<size_t>(n) * HW + pix) * C + cw * 32);
+        q[t][0] = __ldcs(src);
+        q[t][1] = __ldcs(src + 1);
+    }
+#pragma unroll
+    for (int t = 0; t < 4; ++t) {
+        const uint32_t words[8] = {q[t][0].x, q[t][0].y, q[t][0].z, q[t][0].w, q[t][1].x, q[t][1].y, q[t][1].z, q[t][1].w};
+        uint32_t w[BITS];
+#pragma unroll
+        for (int j = 0; j < BITS; ++j) w[j] = 0u;
+#pragma unroll
+        for (int i = 0; i < 8; ++i)
+#pragma unroll
+            for (int j = 0; j < BITS; ++j)
+                w[j] |= ((((words[i] >> j) & 0x01010101u) * 0x01020408u) >> 24) << (4 * i);
+        const int pix = hw0 + 32 * t + lane;
+        if (pix < HW) store_planes<BITS>(out + ((static_cast<size_t>(n) * HW + pix) * Cw + cw) * BITS, w);
+    }
+}
+
 __global__ void bitunpack_kernel(const uint32_t* __restrict__ packed, int8_t* __restrict__ codes, long long total,
                                  int C, int HW, int Cw, int bits, int sign, int nhwc)
 {
@@ -376,27 +542,52 @@ static int launch_bitpack_one(const void* x, uint32_t* out, int N, int C, int HW
     return cudaGetLastError() == cudaSuccess ? BS_OK : BS_ERR_CUDA;
 }
 
-template <int BITS>
-static int launch_bitpack_nchw_f32(const void* x, uint32_t* out, int N, int C, int HW, const QuantParams& q, cudaStream_t st)
+template <typename P, typename... R> static P first_param(void (*)(P, R...));
+
+// Launch of a kernel whose warps each take `pix_per_unit` pixels x one channel word.
+template <typename K, typename... Extra>
+static int launch_units(K kern, const void* x, uint32_t* out, int N, int C, int HW, int pix_per_unit, cudaStream_t st, Extra... extra)
 {
     const int Cw = ceil_div(C, 32);
-    const long long units_per_img = static_cast<long long>(ceil_div(HW, 32)) * Cw;
+    const long long units_per_img = static_cast<long long>(ceil_div(HW, pix_per_unit)) * Cw;
     const long long nunits = N * units_per_img;
     const long long blocks = ceil_div_ll(nunits, FAST_WARPS);
     if (units_per_img > 0x7fffffffLL || blocks > 0x7fffffffLL) return BS_ERR_UNSUPPORTED;
-    bitpack_nchw_f32_kernel<BITS><<<static_cast<unsigned>(blocks), FAST_THREADS, 0, st>>>(
-        static_cast<const float*>(x), out, C, HW, Cw, nunits, static_cast<int>(units_per_img), q);
+    kern<<<static_cast<unsigned>(blocks), FAST_THREADS, 0, st>>>(
+        static_cast<decltype(first_param(kern))>(x), out, C, HW, Cw, nunits, static_cast<int>(units_per_img), extra...);
     return cudaGetLastError() == cudaSuccess ? BS_OK : BS_ERR_CUDA;
+}
+
+template <bool NHWC>
+static int launch_bitpack_i8(const void* x, uint32_t* out, int N, int C, int HW, int bits, cudaStream_t st)
+{
+    switch (bits) {
+        case 1: return NHWC ? launch_units(bitpack_nhwc_i8_kernel<1>, x, out, N, C, HW, 128, st)
+                            : launch_units(bitpack_nchw_i8_kernel<1>, x, out, N, C, HW, 128, st);
+        case 2: return NHWC ? launch_units(bitpack_nhwc_i8_kernel<2>, x, out, N, C, HW, 128, st)
+                            : launch_units(bitpack_nchw_i8_kernel<2>, x, out, N, C, HW, 128, st);
+        case 3: return NHWC ? launch_units(bitpack_nhwc_i8_kernel<3>, x, out, N, C, HW, 128, st)
+                            : launch_units(bitpack_nchw_i8_kernel<3>, x, out, N, C, HW, 128, st);
+        default: return NHWC ? launch_units(bitpack_nhwc_i8_kernel<4>, x, out, N, C, HW, 128, st)
+                             : launch_units(bitpack_nchw_i8_kernel<4>, x, out, N, C, HW, 128, st);
+    }
 }
 
 template <typename T, bool NHWC>
 static int launch_bitpack(const void* x, uint32_t* out, int N, int C, int HW, const QuantParams& q, cudaStream_t st)
 {
-    if constexpr (sizeof(T) == 4 && !NHWC) {
-        // comparison-form codes (1 and 2 bits) of an NCHW fp32 tensor take the sign-bit kernel
-        if (q.by_bounds)
-            return q.bits == 1 ? launch_bitpack_nchw_f32<1>(x, out, N, C, HW, q, st)
-                               : launch_bitpack_nchw_f32<2>(x, out, N, C, HW, q, st);
+    if constexpr (sizeof(T) == 4) {
+        // comparison-form codes (1 and 2 bits) of an fp32 tensor take the kernels with one (pixels, channel word) unit per warp
+        if (q.by_bounds) {
+            if (NHWC)
+                return q.bits == 1 ? launch_units(bitpack_nhwc_f32_kernel<1>, x, out, N, C, HW, 32, st, q)
+                                   : launch_units(bitpack_nhwc_f32_kernel<2>, x, out, N, C, HW, 32, st, q);
+            return q.bits == 1 ? launch_units(bitpack_nchw_f32_kernel<1>, x, out, N, C, HW, 32, st, q)
+                               : launch_units(bitpack_nchw_f32_kernel<2>, x, out, N, C, HW, 32, st, q);
+        }
+    } else {
+        // int8 codes whose planes are the low bits of the byte, in shapes that allow aligned vector loads
+        if (q.sign != BS_BIPOLAR && (NHWC ? C % 32 == 0 : HW % 4 == 0)) return launch_bitpack_i8<NHWC>(x, out, N, C, HW, q.bits, st);
     }
     switch (q.bits) {
         case 1: return launch_bitpack_one<T, NHWC, 1, true>(x, out, N, C, HW, q, st);

@@ -65,6 +65,24 @@ def test_bitpack_nhwc_and_int8_inputs(bits, sign, shape):
     assert np.array_equal(got, want)
 
 
+@pytest.mark.parametrize("bits,sign", [(1, 0), (2, 0), (3, 0), (4, 0), (1, 1), (2, 1), (3, 1), (4, 1), (1, 2)])
+@pytest.mark.parametrize("shape", [(2, 64, 8, 12), (1, 96, 7, 20), (3, 32, 6, 6), (1, 45, 4, 33), (2, 128, 13, 20), (1, 32, 1, 4)])
+def test_bitpack_vector_paths_all_layouts(bits, sign, shape):
+    """Shapes that reach the kernels with one (pixels, channel word) unit per warp: H*W a multiple of 4 (int8 NCHW reads
+    four pixels per word), C a multiple of 32 (int8 NHWC reads 32 channels per lane), ragged last tiles of 32 and of 128
+    pixels, a ragged last channel word; fp32 and int8 inputs in both layouts against the oracle, bit for bit."""
+    rng = np.random.default_rng(bits * 10 + sign + shape[1])
+    s = 0.61
+    lo, hi = wl.code_range(bits, sign)
+    x = rng.uniform((lo - 1.2) * s, (hi + 1.2) * s, size=shape).astype(np.float32)
+    codes = oracle.quantize(x, s, bits, sign)
+    want = oracle.pack_activations(codes, bits, sign)
+    assert np.array_equal(words(api.bitpack_activations(dev(x), s, bits, sign, api.NCHW)), want)
+    assert np.array_equal(words(api.bitpack_activations(dev(x.transpose(0, 2, 3, 1)), s, bits, sign, api.NHWC)), want)
+    assert np.array_equal(words(api.bitpack_activations(dev(codes), 1.0, bits, sign, api.NCHW)), want)
+    assert np.array_equal(words(api.bitpack_activations(dev(codes.transpose(0, 2, 3, 1)), 1.0, bits, sign, api.NHWC)), want)
+
+
 @pytest.mark.parametrize("bits,sign", [(1, 0), (2, 0), (4, 1), (1, 2)])
 def test_unpack_is_inverse(bits, sign):
     rng = np.random.default_rng(3)
