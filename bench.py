@@ -230,10 +230,17 @@ def run_sweep(args):
                     wops = macs // 32 * c["a_bits"] * c["w_bits"]
                     nbytes = (a_p.numel() + w_p.numel() + out.numel()) * 4
                     t_popc, t_hbm = wops / popc_peak, nbytes / hbm_peak
-                    rows.append({"M": M, "N": M, "K": K, "ms": ms, "ms_best": best, "gops": 2.0 * macs / ms / 1e6,
-                                 "Tword_ops_per_s": wops / ms / 1e9, "GB_per_s": nbytes / ms / 1e6,
-                                 "bound": "alu" if t_popc >= t_hbm else "hbm",
-                                 "frac_roofline": max(t_popc, t_hbm) / (ms * 1e-3)})
+                    row = {"M": M, "N": M, "K": K, "ms": ms, "ms_best": best, "gops": 2.0 * macs / ms / 1e6,
+                           "Tword_ops_per_s": wops / ms / 1e9, "GB_per_s": nbytes / ms / 1e6,
+                           "bound": "alu" if t_popc >= t_hbm else "hbm",
+                           "frac_roofline": max(t_popc, t_hbm) / (ms * 1e-3)}
+                    # the same product on the tensor-core entry point: bound by the int8 rate or by the int32 output
+                    wt = api.tc_prepare_weights(w_p.view(M, 1, 1, -1, c["w_bits"]), K, c["w_sign"], c["a_bits"])
+                    tms, _ = timed(lambda: api.bitserial_gemm_tc(a_p, wt, M, K, c["w_bits"], a_sign=c["a_sign"], w_sign=c["w_sign"]))
+                    t_tc, t_hbm_tc = 2.0 * macs / int8_peak, (a_p.numel() * 4 + wt.numel() + out.numel() * 4) / hbm_peak
+                    row.update(tc_ms=tms, tc_gops=2.0 * macs / tms / 1e6, tc_bound="tensor" if t_tc >= t_hbm_tc else "hbm",
+                               tc_frac_roofline=max(t_tc, t_hbm_tc) / (tms * 1e-3))
+                    rows.append(row)
                     tot_ops += 2.0 * macs
                     tot_ms += ms
             name = "gemm_sweep_w1bipolar_a2_int32_out"
