@@ -239,6 +239,16 @@ int bitserial_gemm_tc(const uint32_t* a_packed, const int8_t* w_tc, int M, int N
 int bs_check_status(void* stream);
 
 /*
+ * bs_selftest_wait_timeout -- exercises the failure path of the kernels' device-side waits without any fault (the paper
+ * has no counterpart; Section V only describes the computation).  Launches, on `stream`, a one-warp kernel that waits
+ * with the library's bounded wait on a barrier at which nothing ever arrives, gives up after `polls` polls (1..65536)
+ * and sets the device status word like a convolution kernel whose staged tile never arrived.  The kernel always
+ * returns; the next bs_check_status(stream) reports BS_ERR_TIMEOUT once and clears the word, and the device stays
+ * usable.  Returns BS_ERR_INVALID_ARG for a poll count outside the range, BS_ERR_CUDA if the launch failed.
+ */
+int bs_selftest_wait_timeout(int polls, void* stream);
+
+/*
  * bs_l2_prefetch -- asks the memory system to bring `count` device buffers into the L2 cache (bulk prefetches; the
  * kernel that issues them ends at once and the transfers overlap whatever runs next on `stream`).  Used at the start
  * of a forward pass for the prepared filters of all layers, which a layer otherwise fetches from HBM chunk by chunk

@@ -239,6 +239,12 @@ def bs_check_status(stream=None) -> None:
         raise BitserialError(st, "bs_check_status")
 
 
+def selftest_wait_timeout(polls: int = 256, stream=None) -> None:
+    """Launches the kernel whose bounded wait runs out (``bs_selftest_wait_timeout``); the next :func:`bs_check_status`
+    raises ``BitserialError`` with BS_ERR_TIMEOUT once."""
+    _check(lib().bs_selftest_wait_timeout(int(polls), _stream_ptr(stream)), "bs_selftest_wait_timeout")
+
+
 def l2_prefetch(tensors, stream=None) -> None:
     """Hint: bring the given device tensors into L2 while the following kernels of the stream run (``bs_l2_prefetch``)."""
     ts = [t for t in tensors if t is not None and t.numel() > 0]

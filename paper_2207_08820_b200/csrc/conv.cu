@@ -479,3 +479,28 @@ extern "C" int bitserial_gemm_noalloc(const uint32_t* a_packed, const uint32_t* 
     }
     return bs::conv_impl(a_packed, w_packed, &p, out_i32, out_packed, scratch, need, cs);
 }
+
+// ---- self-test of the failure path: a wait that runs out ------------------------------------------------------------
+namespace bs {
+// One warp; lane 0 waits, with the kernels' own bounded wait, on a barrier at which nothing ever arrives, gives up after
+// `polls` polls and reports through the status word exactly as the convolution kernels do.  Nothing traps or spins
+// without limit: the kernel always returns and the context stays usable.
+__global__ void wait_timeout_selftest_kernel(unsigned polls, int* status)
+{
+    __shared__ __align__(8) uint64_t bar;
+    if (threadIdx.x == 0) {
+        mbar_init(&bar, 1);
+        fence_barrier_init();
+        if (!mbar_wait_bounded(&bar, 0, polls)) atomicOr(status, STATUS_TIMEOUT);
+    }
+}
+}  // namespace bs
+
+extern "C" int bs_selftest_wait_timeout(int polls, void* stream)
+{
+    if (polls < 1 || polls > 65536) return BS_ERR_INVALID_ARG;
+    int* status = bs::status_device_ptr();
+    if (!status) return BS_ERR_CUDA;
+    bs::wait_timeout_selftest_kernel<<<1, 32, 0, static_cast<cudaStream_t>(stream)>>>(static_cast<unsigned>(polls), status);
+    return cudaGetLastError() == cudaSuccess ? BS_OK : BS_ERR_CUDA;
+}

@@ -82,9 +82,9 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, unsigned parity)
     return ok != 0;
 }
 // Bounded wait: returns false (and never blocks forever) if the phase does not complete.
-__device__ __forceinline__ bool mbar_wait_bounded(uint64_t* bar, unsigned parity)
+__device__ __forceinline__ bool mbar_wait_bounded(uint64_t* bar, unsigned parity, unsigned limit = WAIT_LIMIT)
 {
-    for (unsigned it = 0; it < WAIT_LIMIT; ++it)
+    for (unsigned it = 0; it < limit; ++it)
         if (mbar_try_wait(bar, parity)) return true;
     return false;
 }

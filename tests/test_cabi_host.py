@@ -88,6 +88,8 @@ def test_bad_arguments_are_rejected_on_the_host(L):
     assert L.bitserial_conv2d(addr, addr, ctypes.byref(p), addr, None, None) == UNSUPPORTED
     assert L.bitserial_gemm(addr, addr, 0, 4, 4, 2, 0, 2, 1, None, None, 0, 0, 0, addr, None, None) == INVALID
     assert L.bs_status_string(5) == b"BS_ERR_TIMEOUT"
+    assert L.bs_selftest_wait_timeout(0, None) == INVALID          # refused before any launch
+    assert L.bs_selftest_wait_timeout(1 << 20, None) == INVALID
     # bs_l2_prefetch: nothing to do is fine; missing arrays, null or misaligned buffers are refused before any launch
     assert L.bs_l2_prefetch(None, None, 0, None) == 0
     assert L.bs_l2_prefetch(None, None, 1, None) == INVALID
