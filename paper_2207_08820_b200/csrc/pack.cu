@@ -14,15 +14,17 @@ constexpr int PACK_UNROLL = 8;      // NHWC: pixels in flight per warp
 // Quantiser of Section IV prepared for the device.  For 1- and 2-bit codes the decision
 //     code = round_half_even(clip(x / s, qmin, qmax))
 // is monotone in x, so it equals qmin + #{k : x >= bound[k]} where bound[k] is the smallest binary32 value whose
-// code is >= qmin + k.  The host finds those bounds by bisection over the ordered float bit patterns using the very
+// code is >= qmin + k + 1.  The host finds those bounds by bisection over the ordered float bit patterns using the very
 // same IEEE division, clip and rint, so the comparison form takes exactly the decision of the formula while costing
-// three compares instead of a division.  Wider codes evaluate the formula directly.
+// a few compares instead of a division.  The NCHW kernel uses it for every width (a binary search over the bounds for
+// 3 and 4 bits); the generic kernel and the NHWC kernel use it for 1 and 2 bits and evaluate the formula otherwise.
 struct QuantParams {
-    float bound[3];
-    float below[3];     // largest binary32 value below bound[k] (never -0): x >= bound[k]  <=>  sign bit of (below[k] - x) is set
+    float bound[15];    // bound[k]: smallest input whose code is >= qmin + k + 1 (unused entries +inf)
+    float below[15];    // largest binary32 value below bound[k] (never -0): x >= bound[k]  <=>  sign bit of (below[k] - x) is set
     float scale;
     int bits, sign, qmin, qmax;
-    int by_bounds;      // 1: compare against bound[]; 0: evaluate the formula
+    int by_bounds;      // 1: the generic and NHWC kernels compare against bound[] (1-2 bits); 0: they evaluate the formula
+    int have_bounds;    // 1: bound[] and below[] are filled for every level (any width)
     int flip;           // plane bits to flip: pattern = (count ^ flip) for two's-complement codes
     float null_value;   // an input whose plane bits (before flipping) are all zero
 };
@@ -153,6 +155,18 @@ bitpack_kernel(const T* __restrict__ x, uint32_t* __restrict__ out, int C, int H
                        (static_cast<size_t>(HW) * rec) % 4 == 0 && (32 * rec) % 4 == 0, lane);
 }
 
+// Stores the BITS plane words of one (pixel, channel word) with the widest aligned store.
+template <int BITS>
+__device__ __forceinline__ void store_planes(uint32_t* dst, const uint32_t (&w)[BITS])
+{
+    if constexpr (BITS == 4) *reinterpret_cast<uint4*>(dst) = make_uint4(w[0], w[1], w[2], w[3]);
+    else if constexpr (BITS == 2) *reinterpret_cast<uint2*>(dst) = make_uint2(w[0], w[1]);
+    else {
+#pragma unroll
+        for (int j = 0; j < BITS; ++j) dst[j] = w[j];
+    }
+}
+
 // Sign-bit form of the comparison quantiser for fp32 NCHW input and 1- or 2-bit codes.
 //   With p the largest binary32 value below the bound b:  x >= b  <=>  x > p  <=>  the sign bit of p - x is set.
 //   An IEEE subtraction never rounds across zero and x == p gives +0; p is stored as +0 when it is a zero, so neither
@@ -161,7 +175,8 @@ bitpack_kernel(const T* __restrict__ x, uint32_t* __restrict__ out, int C, int H
 //   2-bit codes: plane 1 = (x >= b1); plane 0 = parity of the three comparisons = sign((p0-x) ^ (p1-x) ^ (p2-x)).
 // One funnel shift moves a sign bit into a plane word; channels are walked from 31 down to 0 so that channel c ends at
 // bit c.  Per element: one load, 1 or 3 subtractions, at most one three-input xor and BITS funnel shifts, which
-// leaves the kernel waiting on HBM rather than on the issue slots.
+// leaves the kernel waiting on HBM rather than on the issue slots.  3- and 4-bit codes search the 7 or 15 bounds
+// binarily, one subtraction, one sign test and one funnel shift per bit plus the selects that pick the next bound.
 // Work unit of a warp = 32 consecutive pixels of one image x one 32-channel word (lane = pixel): all 32 channel rows are
 // in flight at once (32 coalesced 128-byte requests per warp), and each lane stores the BITS plane words of its pixel
 // straight to the packed record (8-byte stores for 2-bit codes; the words of the other channel groups of the record
@@ -175,7 +190,6 @@ __global__ void __launch_bounds__(FAST_THREADS, 8)
 bitpack_nchw_f32_kernel(const float* __restrict__ x, uint32_t* __restrict__ out, int C, int HW, int Cw, long long nunits,
                         int units_per_img, const QuantParams q)
 {
-    static_assert(BITS == 1 || BITS == 2, "comparison form covers 1- and 2-bit codes");
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const long long unit = static_cast<long long>(blockIdx.x) * FAST_WARPS + warp;
     if (unit >= nunits) return;
@@ -184,17 +198,42 @@ bitpack_nchw_f32_kernel(const float* __restrict__ x, uint32_t* __restrict__ out,
     const int cw = rem % Cw;
     const int hw0 = (rem / Cw) * 32;
     const bool pvalid = lane < HW - hw0;
-    const float p0 = q.below[0], p1 = q.below[1], p2 = q.below[2];
     // lanes beyond the image re-read the first pixel of the tile (always in bounds) and store nothing
     const float* xin = x + (static_cast<size_t>(n) * C + cw * 32) * HW + hw0 + (pvalid ? lane : 0);
-    uint32_t w0 = 0u, w1 = 0u;
+    uint32_t w[BITS];
+#pragma unroll
+    for (int j = 0; j < BITS; ++j) w[j] = 0u;
     auto push = [&](float v) {
         if constexpr (BITS == 1) {
-            w0 = __funnelshift_l(__float_as_uint(p0 - v), w0, 1);
+            w[0] = __funnelshift_l(__float_as_uint(q.below[0] - v), w[0], 1);
+        } else if constexpr (BITS == 2) {
+            const uint32_t d0 = __float_as_uint(q.below[0] - v), d1 = __float_as_uint(q.below[1] - v),
+                           d2 = __float_as_uint(q.below[2] - v);
+            w[1] = __funnelshift_l(d1, w[1], 1);
+            w[0] = __funnelshift_l(d0 ^ d1 ^ d2, w[0], 1);
         } else {
-            const uint32_t d0 = __float_as_uint(p0 - v), d1 = __float_as_uint(p1 - v), d2 = __float_as_uint(p2 - v);
-            w1 = __funnelshift_l(d1, w1, 1);
-            w0 = __funnelshift_l(d0 ^ d1 ^ d2, w0, 1);
+            // binary search for the count of bounds reached, top bit first: with the higher bits m decided, bit L is
+            // "bound number m * 2^(L+1) + 2^L reached"; the candidates are folded with selects on the decided bits
+            bool c[BITS];
+#pragma unroll
+            for (int L = BITS - 1; L >= 0; --L) {
+                constexpr int MAXC = 1 << (BITS - 1);
+                float sel[MAXC];
+                const int nd = BITS - 1 - L;
+#pragma unroll
+                for (int m = 0; m < MAXC; ++m)
+                    if (m < (1 << nd)) sel[m] = q.below[m * (2 << L) + (1 << L) - 1];
+#pragma unroll
+                for (int d = 0; d < BITS - 1; ++d)
+                    if (d < nd) {
+#pragma unroll
+                        for (int m = 0; m < MAXC / 2; ++m)
+                            if (m < (1 << (nd - d - 1))) sel[m] = c[L + 1 + d] ? sel[2 * m + 1] : sel[2 * m];
+                    }
+                const uint32_t e = __float_as_uint(sel[0] - v);
+                c[L] = static_cast<int>(e) < 0;
+                w[L] = __funnelshift_l(e, w[L], 1);
+            }
         }
     };
     const int nvalid = min(32, C - cw * 32);
@@ -216,11 +255,9 @@ bitpack_nchw_f32_kernel(const float* __restrict__ x, uint32_t* __restrict__ out,
     }
     if (!pvalid) return;
     const unsigned fl = nvalid == 32 ? 0xffffffffu : ((1u << nvalid) - 1u);
-    if (q.flip & 1) w0 ^= fl;
-    if (q.flip & 2) w1 ^= fl;
-    uint32_t* dst = out + ((static_cast<size_t>(n) * HW + hw0 + lane) * Cw + cw) * BITS;
-    if constexpr (BITS == 2) *reinterpret_cast<uint2*>(dst) = make_uint2(w0, w1);
-    else *dst = w0;
+    // pattern = (qmin + count) mod 2^BITS: two's-complement codes (qmin = -2^(BITS-1)) flip the top plane only
+    if (q.sign == BS_SIGNED) w[BITS - 1] ^= fl;
+    store_planes<BITS>(out + ((static_cast<size_t>(n) * HW + hw0 + lane) * Cw + cw) * BITS, w);
 }
 
 // fp32 NHWC input, 1- or 2-bit codes in comparison form.  Work unit of a warp = 32 consecutive pixels x one 32-channel
@@ -275,18 +312,6 @@ bitpack_nhwc_f32_kernel(const float* __restrict__ x, uint32_t* __restrict__ out,
     uint32_t* dst = out + ((static_cast<size_t>(n) * HW + hw0 + lane) * Cw + cw) * BITS;
     if constexpr (BITS == 2) *reinterpret_cast<uint2*>(dst) = make_uint2(my0, my1);
     else *dst = my0;
-}
-
-// Stores the BITS plane words of one (pixel, channel word) with the widest aligned store.
-template <int BITS>
-__device__ __forceinline__ void store_planes(uint32_t* dst, const uint32_t (&w)[BITS])
-{
-    if constexpr (BITS == 4) *reinterpret_cast<uint4*>(dst) = make_uint4(w[0], w[1], w[2], w[3]);
-    else if constexpr (BITS == 2) *reinterpret_cast<uint2*>(dst) = make_uint2(w[0], w[1]);
-    else {
-#pragma unroll
-        for (int j = 0; j < BITS; ++j) dst[j] = w[j];
-    }
 }
 
 // int8 codes, NCHW (unsigned or two's-complement codes: plane j is bit j of the byte).  At one byte per element the
@@ -475,7 +500,7 @@ static float key_float(uint32_t k)
 // below[k] = the binary32 value just under bound[k] (bounds are never -inf: -inf always quantises to the lowest code).
 static void set_below(QuantParams& q)
 {
-    for (int k = 0; k < 3; ++k) {
+    for (int k = 0; k < 15; ++k) {
         const float b = q.bound[k];
         float p = b == 0.0f ? -1.401298464e-45f : key_float(float_key(b) - 1u);
         if (p == 0.0f) p = 0.0f;          // drops the sign of a zero
@@ -492,32 +517,32 @@ static QuantParams make_quant_params(float s, int bits, int sign, bool quantise)
     q.by_bounds = 0;
     q.null_value = (sign == BS_UNSIGNED) ? 0.0f : (sign == BS_BIPOLAR ? -1.0f : 0.0f);   // formula mode / int8 codes
     if (!quantise) return q;
+    for (int k = 0; k < 15; ++k) q.bound[k] = INFINITY;
+    q.have_bounds = 1;
     if (sign == BS_BIPOLAR) {                 // +1 iff x >= 0
         q.null_value = -INFINITY;
         q.by_bounds = 1;
         q.bound[0] = 0.0f;
-        q.bound[1] = q.bound[2] = INFINITY;
         set_below(q);
         return q;
     }
+    const uint32_t lo_key = float_key(-INFINITY), hi_key = float_key(INFINITY);
+    for (int k = 1; k <= q.qmax - q.qmin; ++k) {
+        // smallest x (in float order) with code >= qmin + k; the code is monotone in x and reaches qmax at +inf
+        uint32_t lo = lo_key, hi = hi_key;
+        while (lo < hi) {
+            const uint32_t mid = lo + (hi - lo) / 2;
+            if (host_quantize(key_float(mid), s, q.qmin, q.qmax) >= q.qmin + k) hi = mid;
+            else lo = mid + 1;
+        }
+        q.bound[k - 1] = key_float(lo);
+    }
+    set_below(q);
     if (bits <= 2) {
         q.by_bounds = 1;
         q.null_value = -INFINITY;
-        const uint32_t lo_key = float_key(-INFINITY), hi_key = float_key(INFINITY);
-        for (int k = 1; k <= q.qmax - q.qmin; ++k) {
-            // smallest x (in float order) with code >= qmin + k; the code is monotone in x and reaches qmax at +inf
-            uint32_t lo = lo_key, hi = hi_key;
-            while (lo < hi) {
-                const uint32_t mid = lo + (hi - lo) / 2;
-                if (host_quantize(key_float(mid), s, q.qmin, q.qmax) >= q.qmin + k) hi = mid;
-                else lo = mid + 1;
-            }
-            q.bound[k - 1] = key_float(lo);
-        }
-        if (bits == 1) q.bound[1] = q.bound[2] = INFINITY;
         // pattern = (qmin + count) mod 2^bits; for two's-complement 2-bit codes qmin = -2 flips bit 1 only
         q.flip = (sign == BS_SIGNED) ? (static_cast<unsigned>(q.qmin) & ((1u << bits) - 1u)) : 0;
-        set_below(q);
     }
     return q;
 }
@@ -577,14 +602,19 @@ template <typename T, bool NHWC>
 static int launch_bitpack(const void* x, uint32_t* out, int N, int C, int HW, const QuantParams& q, cudaStream_t st)
 {
     if constexpr (sizeof(T) == 4) {
-        // comparison-form codes (1 and 2 bits) of an fp32 tensor take the kernels with one (pixels, channel word) unit per warp
-        if (q.by_bounds) {
-            if (NHWC)
-                return q.bits == 1 ? launch_units(bitpack_nhwc_f32_kernel<1>, x, out, N, C, HW, 32, st, q)
-                                   : launch_units(bitpack_nhwc_f32_kernel<2>, x, out, N, C, HW, 32, st, q);
-            return q.bits == 1 ? launch_units(bitpack_nchw_f32_kernel<1>, x, out, N, C, HW, 32, st, q)
-                               : launch_units(bitpack_nchw_f32_kernel<2>, x, out, N, C, HW, 32, st, q);
+        // fp32 tensors take the kernels with one (pixels, channel word) unit per warp: NCHW at any width, NHWC for the
+        // 1- and 2-bit comparison form
+        if (!NHWC && q.have_bounds) {
+            switch (q.bits) {
+                case 1: return launch_units(bitpack_nchw_f32_kernel<1>, x, out, N, C, HW, 32, st, q);
+                case 2: return launch_units(bitpack_nchw_f32_kernel<2>, x, out, N, C, HW, 32, st, q);
+                case 3: return launch_units(bitpack_nchw_f32_kernel<3>, x, out, N, C, HW, 32, st, q);
+                default: return launch_units(bitpack_nchw_f32_kernel<4>, x, out, N, C, HW, 32, st, q);
+            }
         }
+        if (NHWC && q.by_bounds)
+            return q.bits == 1 ? launch_units(bitpack_nhwc_f32_kernel<1>, x, out, N, C, HW, 32, st, q)
+                               : launch_units(bitpack_nhwc_f32_kernel<2>, x, out, N, C, HW, 32, st, q);
     } else {
         // int8 codes whose planes are the low bits of the byte, in shapes that allow aligned vector loads
         if (q.sign != BS_BIPOLAR && (NHWC ? C % 32 == 0 : HW % 4 == 0)) return launch_bitpack_i8<NHWC>(x, out, N, C, HW, q.bits, st);
