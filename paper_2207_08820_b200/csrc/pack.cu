@@ -182,6 +182,56 @@ __device__ __forceinline__ void store_planes(uint32_t* dst, const uint32_t (&w)[
 // straight to the packed record (8-byte stores for 2-bit codes; the words of the other channel groups of the record
 // come from the neighbouring warps of the block, so the sectors fill up in L2).  Units are small and numerous, which
 // keeps the tail of the grid short; no shared memory, no barrier.
+// Shifts the BITS plane bits of one input into the plane words w (w = 2 w + bit), in the sign-bit comparison form.
+template <int BITS>
+__device__ __forceinline__ void quant_push(const QuantParams& q, float v, uint32_t (&w)[BITS])
+{
+    if constexpr (BITS == 1) {
+        w[0] = __funnelshift_l(__float_as_uint(q.below[0] - v), w[0], 1);
+    } else if constexpr (BITS == 2) {
+        const uint32_t d0 = __float_as_uint(q.below[0] - v), d1 = __float_as_uint(q.below[1] - v),
+                       d2 = __float_as_uint(q.below[2] - v);
+        w[1] = __funnelshift_l(d1, w[1], 1);
+        w[0] = __funnelshift_l(d0 ^ d1 ^ d2, w[0], 1);
+    } else {
+        // binary search for the count of bounds reached, top bit first: with the higher bits m decided, bit L is
+        // "bound number m * 2^(L+1) + 2^L reached"; the candidates are folded with selects on the decided bits
+        bool c[BITS];
+#pragma unroll
+        for (int L = BITS - 1; L >= 0; --L) {
+            constexpr int MAXC = 1 << (BITS - 1);
+            float sel[MAXC];
+            const int nd = BITS - 1 - L;
+#pragma unroll
+            for (int m = 0; m < MAXC; ++m)
+                if (m < (1 << nd)) sel[m] = q.below[m * (2 << L) + (1 << L) - 1];
+#pragma unroll
+            for (int d = 0; d < BITS - 1; ++d)
+                if (d < nd) {
+#pragma unroll
+                    for (int m = 0; m < MAXC / 2; ++m)
+                        if (m < (1 << (nd - d - 1))) sel[m] = c[L + 1 + d] ? sel[2 * m + 1] : sel[2 * m];
+                }
+            const uint32_t e = __float_as_uint(sel[0] - v);
+            c[L] = static_cast<int>(e) < 0;
+            w[L] = __funnelshift_l(e, w[L], 1);
+        }
+    }
+}
+
+// Transpose of the 32 x 32 bit matrix whose row r is the word held by lane r: afterwards lane r holds column r.  Five
+// butterfly stages; stage k swaps the off-diagonal k x k blocks between lanes r and r ^ k.
+__device__ __forceinline__ uint32_t warp_transpose32(uint32_t x, int lane)
+{
+#pragma unroll
+    for (int k = 16; k >= 1; k >>= 1) {
+        const uint32_t mask = k == 16 ? 0x0000FFFFu : k == 8 ? 0x00FF00FFu : k == 4 ? 0x0F0F0F0Fu : k == 2 ? 0x33333333u : 0x55555555u;
+        const uint32_t y = __shfl_xor_sync(0xffffffffu, x, k);
+        x = (lane & k) ? ((x & ~mask) | ((y & ~mask) >> k)) : ((x & mask) | ((y & mask) << k));
+    }
+    return x;
+}
+
 constexpr int FAST_THREADS = 128;
 constexpr int FAST_WARPS = FAST_THREADS / 32;
 
@@ -203,39 +253,7 @@ bitpack_nchw_f32_kernel(const float* __restrict__ x, uint32_t* __restrict__ out,
     uint32_t w[BITS];
 #pragma unroll
     for (int j = 0; j < BITS; ++j) w[j] = 0u;
-    auto push = [&](float v) {
-        if constexpr (BITS == 1) {
-            w[0] = __funnelshift_l(__float_as_uint(q.below[0] - v), w[0], 1);
-        } else if constexpr (BITS == 2) {
-            const uint32_t d0 = __float_as_uint(q.below[0] - v), d1 = __float_as_uint(q.below[1] - v),
-                           d2 = __float_as_uint(q.below[2] - v);
-            w[1] = __funnelshift_l(d1, w[1], 1);
-            w[0] = __funnelshift_l(d0 ^ d1 ^ d2, w[0], 1);
-        } else {
-            // binary search for the count of bounds reached, top bit first: with the higher bits m decided, bit L is
-            // "bound number m * 2^(L+1) + 2^L reached"; the candidates are folded with selects on the decided bits
-            bool c[BITS];
-#pragma unroll
-            for (int L = BITS - 1; L >= 0; --L) {
-                constexpr int MAXC = 1 << (BITS - 1);
-                float sel[MAXC];
-                const int nd = BITS - 1 - L;
-#pragma unroll
-                for (int m = 0; m < MAXC; ++m)
-                    if (m < (1 << nd)) sel[m] = q.below[m * (2 << L) + (1 << L) - 1];
-#pragma unroll
-                for (int d = 0; d < BITS - 1; ++d)
-                    if (d < nd) {
-#pragma unroll
-                        for (int m = 0; m < MAXC / 2; ++m)
-                            if (m < (1 << (nd - d - 1))) sel[m] = c[L + 1 + d] ? sel[2 * m + 1] : sel[2 * m];
-                    }
-                const uint32_t e = __float_as_uint(sel[0] - v);
-                c[L] = static_cast<int>(e) < 0;
-                w[L] = __funnelshift_l(e, w[L], 1);
-            }
-        }
-    };
+    auto push = [&](float v) { quant_push<BITS>(q, v, w); };
     const int nvalid = min(32, C - cw * 32);
     if (nvalid == 32) {
         // a full channel word: unconditional loads, walking the channel rows downward from channel 31
@@ -260,16 +278,16 @@ bitpack_nchw_f32_kernel(const float* __restrict__ x, uint32_t* __restrict__ out,
     store_planes<BITS>(out + ((static_cast<size_t>(n) * HW + hw0 + lane) * Cw + cw) * BITS, w);
 }
 
-// fp32 NHWC input, 1- or 2-bit codes in comparison form.  Work unit of a warp = 32 consecutive pixels x one 32-channel
-// word, lane = channel: the 32 channels of a pixel are one coalesced 128-byte request, all 32 pixels of the unit are in
-// flight at once, one __ballot_sync per plane turns the 32 comparisons of a pixel into its plane word, and lane p keeps
-// the words of pixel p, so the records leave as one store per lane like in the NCHW kernel.
+// fp32 NHWC input, comparison form at any width.  Work unit of a warp = 32 consecutive pixels x one 32-channel word, lane
+// = channel: the 32 channels of a pixel are one coalesced 128-byte request and all 32 pixels of the unit are in flight
+// at once.  A lane shifts the plane bits of its channel into words indexed by PIXEL (pixels walked from 31 down), a
+// 32 x 32 bit transpose across the warp (five shuffles per plane) turns them into words indexed by channel held by lane
+// = pixel, and the records leave as one store per lane like in the NCHW kernel.  No votes, no shared memory.
 template <int BITS>
 __global__ void __launch_bounds__(FAST_THREADS, 8)
 bitpack_nhwc_f32_kernel(const float* __restrict__ x, uint32_t* __restrict__ out, int C, int HW, int Cw, long long nunits,
                         int units_per_img, const QuantParams q)
 {
-    static_assert(BITS == 1 || BITS == 2, "comparison form covers 1- and 2-bit codes");
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const long long unit = static_cast<long long>(blockIdx.x) * FAST_WARPS + warp;
     if (unit >= nunits) return;
@@ -280,38 +298,31 @@ bitpack_nhwc_f32_kernel(const float* __restrict__ x, uint32_t* __restrict__ out,
     const int npix = min(32, HW - hw0);
     const bool cvalid = cw * 32 + lane < C;
     const unsigned valid_word = __ballot_sync(0xffffffffu, cvalid);
-    // lanes past the last channel re-read the first channel of the word (always in bounds) and vote "no level reached"
+    // lanes past the last channel re-read the first channel of the word (always in bounds); their words are cleared
     const float* xin = x + (static_cast<size_t>(n) * HW + hw0) * C + cw * 32 + (cvalid ? lane : 0);
-    const float b0 = q.bound[0], b1 = q.bound[1], b2 = q.bound[2];
-    uint32_t my0 = 0u, my1 = 0u;
-    auto vote = [&](float v, int u) {
-        const bool c1 = v >= b0;
-        if constexpr (BITS == 1) {
-            const uint32_t w0 = __ballot_sync(0xffffffffu, cvalid && c1);
-            if (lane == u) my0 = w0;
-        } else {
-            const bool c2 = v >= b1, c3 = v >= b2;      // count = c1 + c2 + c3: bit 0 is the parity, bit 1 is c2
-            const uint32_t w0 = __ballot_sync(0xffffffffu, cvalid && ((c1 != c2) != c3));
-            const uint32_t w1 = __ballot_sync(0xffffffffu, cvalid && c2);
-            if (lane == u) { my0 = w0; my1 = w1; }
-        }
-    };
+    uint32_t w[BITS];
+#pragma unroll
+    for (int j = 0; j < BITS; ++j) w[j] = 0u;
     if (npix == 32) {
-        const size_t row = C;
+        const ptrdiff_t row = C;
+        const float* pc = xin + 31 * row;
         float v[32];
 #pragma unroll
-        for (int u = 0; u < 32; ++u) v[u] = __ldcs(xin + u * row);
+        for (int u = 0; u < 32; ++u) {
+            v[u] = __ldcs(pc);
+            pc -= row;
+        }
 #pragma unroll
-        for (int u = 0; u < 32; ++u) vote(v[u], u);
+        for (int u = 0; u < 32; ++u) quant_push<BITS>(q, v[u], w);
     } else {
-        for (int u = 0; u < npix; ++u) vote(__ldcs(xin + static_cast<size_t>(u) * C), u);
+        // the ragged last tile of an image: pixels past the end count as "no level reached" and are not stored
+        for (int u = 31; u >= 0; --u) quant_push<BITS>(q, u < npix ? __ldcs(xin + static_cast<size_t>(u) * C) : -INFINITY, w);
     }
+#pragma unroll
+    for (int j = 0; j < BITS; ++j) w[j] = warp_transpose32(cvalid ? w[j] : 0u, lane);
     if (lane >= npix) return;
-    if (q.flip & 1) my0 ^= valid_word;
-    if (q.flip & 2) my1 ^= valid_word;
-    uint32_t* dst = out + ((static_cast<size_t>(n) * HW + hw0 + lane) * Cw + cw) * BITS;
-    if constexpr (BITS == 2) *reinterpret_cast<uint2*>(dst) = make_uint2(my0, my1);
-    else *dst = my0;
+    if (q.sign == BS_SIGNED) w[BITS - 1] ^= valid_word;
+    store_planes<BITS>(out + ((static_cast<size_t>(n) * HW + hw0 + lane) * Cw + cw) * BITS, w);
 }
 
 // int8 codes, NCHW (unsigned or two's-complement codes: plane j is bit j of the byte).  At one byte per element the
@@ -602,8 +613,7 @@ template <typename T, bool NHWC>
 static int launch_bitpack(const void* x, uint32_t* out, int N, int C, int HW, const QuantParams& q, cudaStream_t st)
 {
     if constexpr (sizeof(T) == 4) {
-        // fp32 tensors take the kernels with one (pixels, channel word) unit per warp: NCHW at any width, NHWC for the
-        // 1- and 2-bit comparison form
+        // fp32 tensors take the comparison-form kernels with one (pixels, channel word) unit per warp
         if (!NHWC && q.have_bounds) {
             switch (q.bits) {
                 case 1: return launch_units(bitpack_nchw_f32_kernel<1>, x, out, N, C, HW, 32, st, q);
@@ -612,9 +622,14 @@ static int launch_bitpack(const void* x, uint32_t* out, int N, int C, int HW, co
                 default: return launch_units(bitpack_nchw_f32_kernel<4>, x, out, N, C, HW, 32, st, q);
             }
         }
-        if (NHWC && q.by_bounds)
-            return q.bits == 1 ? launch_units(bitpack_nhwc_f32_kernel<1>, x, out, N, C, HW, 32, st, q)
-                               : launch_units(bitpack_nhwc_f32_kernel<2>, x, out, N, C, HW, 32, st, q);
+        if (NHWC && q.have_bounds) {
+            switch (q.bits) {
+                case 1: return launch_units(bitpack_nhwc_f32_kernel<1>, x, out, N, C, HW, 32, st, q);
+                case 2: return launch_units(bitpack_nhwc_f32_kernel<2>, x, out, N, C, HW, 32, st, q);
+                case 3: return launch_units(bitpack_nhwc_f32_kernel<3>, x, out, N, C, HW, 32, st, q);
+                default: return launch_units(bitpack_nhwc_f32_kernel<4>, x, out, N, C, HW, 32, st, q);
+            }
+        }
     } else {
         // int8 codes whose planes are the low bits of the byte, in shapes that allow aligned vector loads
         if (q.sign != BS_BIPOLAR && (NHWC ? C % 32 == 0 : HW % 4 == 0)) return launch_bitpack_i8<NHWC>(x, out, N, C, HW, q.bits, st);
