@@ -46,13 +46,4 @@ __host__ __device__ __forceinline__ void code_limits(int bits, int sign, int& qm
     else { qmin = 0; qmax = (1 << bits) - 1; }
 }
 
-// Section IV quantiser in IEEE binary32: round_half_even(clip(x / s, qmin, qmax)).
-__device__ __forceinline__ int quantize_code(float x, float s, int qmin, int qmax, int sign)
-{
-    if (sign == BS_BIPOLAR) return x >= 0.0f ? 1 : -1;
-    float t = __fdiv_rn(x, s);
-    t = fminf(fmaxf(t, static_cast<float>(qmin)), static_cast<float>(qmax));
-    return __float2int_rn(t);
-}
-
 }  // namespace bs

@@ -11,56 +11,24 @@ constexpr int PACK_THREADS = 256;
 constexpr int PACK_WARPS = PACK_THREADS / 32;
 constexpr int PACK_UNROLL = 8;      // NHWC: pixels in flight per warp
 
-// Quantiser of Section IV prepared for the device.  For 1- and 2-bit codes the decision
+// Quantiser of Section IV prepared for the device.  The decision
 //     code = round_half_even(clip(x / s, qmin, qmax))
 // is monotone in x, so it equals qmin + #{k : x >= bound[k]} where bound[k] is the smallest binary32 value whose
 // code is >= qmin + k + 1.  The host finds those bounds by bisection over the ordered float bit patterns using the very
 // same IEEE division, clip and rint, so the comparison form takes exactly the decision of the formula while costing
-// a few compares instead of a division.  The NCHW kernel uses it for every width (a binary search over the bounds for
-// 3 and 4 bits); the generic kernel and the NHWC kernel use it for 1 and 2 bits and evaluate the formula otherwise.
+// a few subtractions instead of a division (a binary search over the bounds for 3 and 4 bits).
 struct QuantParams {
-    float bound[15];    // bound[k]: smallest input whose code is >= qmin + k + 1 (unused entries +inf)
     float below[15];    // largest binary32 value below bound[k] (never -0): x >= bound[k]  <=>  sign bit of (below[k] - x) is set
-    float scale;
-    int bits, sign, qmin, qmax;
-    int by_bounds;      // 1: the generic and NHWC kernels compare against bound[] (1-2 bits); 0: they evaluate the formula
-    int have_bounds;    // 1: bound[] and below[] are filled for every level (any width)
-    int flip;           // plane bits to flip: pattern = (count ^ flip) for two's-complement codes
-    float null_value;   // an input whose plane bits (before flipping) are all zero
+    int bits, sign;
 };
 
-// Plane bits of one input element.  BITS is the code width; BOUNDS selects the comparison form of the quantiser.
-// Bits that a two's-complement offset flips (QuantParams::flip) are NOT applied here: the callers flip whole words.
-template <typename T, int BITS, bool BOUNDS>
-struct PlaneBits {
-    bool p[BITS];
-    __device__ __forceinline__ PlaneBits(T x, const QuantParams& q)
-    {
-        if constexpr (sizeof(T) == 1) {
-#pragma unroll
-            for (int j = 0; j < BITS; ++j) p[j] = (static_cast<int>(x) >> j) & 1;
-            if (q.sign == BS_BIPOLAR) p[0] = x > 0;
-        } else if constexpr (BOUNDS) {
-            const bool c1 = x >= q.bound[0];
-            if constexpr (BITS == 1) {
-                p[0] = c1;
-            } else {
-                const bool c2 = x >= q.bound[1], c3 = x >= q.bound[2];
-                p[0] = (c1 != c2) != c3;      // count = c1 + c2 + c3 with c1 >= c2 >= c3: bit 0 is the parity, bit 1 is c2
-                p[1] = c2;
-            }
-        } else {
-            const unsigned pat = stored_pattern(quantize_code(x, q.scale, q.qmin, q.qmax, q.sign), BITS, q.sign);
-#pragma unroll
-            for (int j = 0; j < BITS; ++j) p[j] = (pat >> j) & 1u;
-        }
-    }
-};
-
-// Input value that sets no plane bit (used for channels and pixels outside the tensor).
-template <typename T> __device__ __forceinline__ T null_input(const QuantParams& q);
-template <> __device__ __forceinline__ float null_input<float>(const QuantParams& q) { return q.null_value; }
-template <> __device__ __forceinline__ int8_t null_input<int8_t>(const QuantParams& q) { return static_cast<int8_t>(q.null_value); }
+// Stored pattern of an int8 code as plane bits (the two's-complement low bits; bipolar: bit 0 = code > 0).
+template <int BITS>
+__device__ __forceinline__ unsigned code_pattern(int8_t x, int sign)
+{
+    if (sign == BS_BIPOLAR) return x > 0 ? 1u : 0u;
+    return static_cast<unsigned>(static_cast<int>(x)) & ((1u << BITS) - 1u);
+}
 
 // A warp copies the contiguous packed records of its tile from shared to global memory, as 128-bit stores when the
 // tile starts on a 16-byte boundary.
@@ -75,49 +43,45 @@ __device__ __forceinline__ void store_tile_records(const uint32_t* stage, uint32
     }
 }
 
-// One warp packs 32 consecutive pixels (flattened y*W + x) of one image, all channels, with no block-wide barrier.
-//   NCHW: lane = pixel.  Every channel row is read with one coalesced 128-byte request per warp, a whole 32-channel
-//         word in flight; each lane sets bit c of its own plane words from the plane bits of channel c.
+// Fallback for int8 codes in shapes the vector kernels below refuse (H*W not a multiple of 4 in NCHW, C not a multiple
+// of 32 in NHWC, bipolar codes).  One warp packs 32 consecutive pixels (flattened y*W + x) of one image, all channels,
+// with no block-wide barrier.
+//   NCHW: lane = pixel.  Every channel row is read with one coalesced request per warp, a whole 32-channel word in
+//         flight; each lane sets bit c of its own plane words from the pattern of channel c.
 //   NHWC: lane = channel.  One coalesced request per (pixel, 32-channel word); __ballot_sync over the 32 channels
 //         yields one plane word per vote.
 // The packed records of the 32 pixels are contiguous in global memory; they are parked in the warp's slice of
 // shared memory and leave through coalesced 128-bit stores.
-template <typename T, bool NHWC, int BITS, bool BOUNDS>
+template <bool NHWC, int BITS>
 __global__ void __launch_bounds__(PACK_THREADS)
-bitpack_kernel(const T* __restrict__ x, uint32_t* __restrict__ out, int C, int HW, int Cw, long long ntiles,
-               int tiles_per_img, const QuantParams q)
+bitpack_codes_kernel(const int8_t* __restrict__ x, uint32_t* __restrict__ out, int C, int HW, int Cw, long long ntiles,
+                     int tiles_per_img, int sign)
 {
     extern __shared__ __align__(16) uint32_t pack_smem[];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const long long tile = static_cast<long long>(blockIdx.x) * PACK_WARPS + warp;
     if (tile >= ntiles) return;                       // whole warps leave; only __syncwarp is used below
-    constexpr int rec_bits = BITS;
-    const int rec = Cw * rec_bits;
+    const int rec = Cw * BITS;
     uint32_t* stage = pack_smem + static_cast<size_t>(warp) * 32 * rec;      // [32 pixels][rec]
     const long long n = tile / tiles_per_img;
     const int hw0 = static_cast<int>(tile % tiles_per_img) * 32;
     const int npix = min(32, HW - hw0);
-    const T nullv = null_input<T>(q);
 
     if (NHWC) {
-        const T* xin = x + (static_cast<size_t>(n) * HW + hw0) * C;
+        const int8_t* xin = x + (static_cast<size_t>(n) * HW + hw0) * C;
         for (int cw = 0; cw < Cw; ++cw) {
             const int c = cw * 32 + lane;
             const bool cvalid = c < C;
-            const unsigned valid_word = __ballot_sync(0xffffffffu, cvalid);
             for (int p0 = 0; p0 < 32; p0 += PACK_UNROLL) {
-                T v[PACK_UNROLL];
+                unsigned pat[PACK_UNROLL];
 #pragma unroll
                 for (int u = 0; u < PACK_UNROLL; ++u)
-                    v[u] = (cvalid && p0 + u < npix) ? xin[static_cast<size_t>(p0 + u) * C + c] : nullv;
+                    pat[u] = (cvalid && p0 + u < npix) ? code_pattern<BITS>(xin[static_cast<size_t>(p0 + u) * C + c], sign) : 0u;
 #pragma unroll
                 for (int u = 0; u < PACK_UNROLL; ++u) {
-                    const PlaneBits<T, BITS, BOUNDS> pb(v[u], q);
-                    const unsigned fl = (p0 + u < npix) ? valid_word : 0u;
 #pragma unroll
                     for (int j = 0; j < BITS; ++j) {
-                        unsigned word = __ballot_sync(0xffffffffu, pb.p[j]);
-                        if ((q.flip >> j) & 1) word ^= fl;
+                        const unsigned word = __ballot_sync(0xffffffffu, (pat[u] >> j) & 1u);
                         if (lane == j) stage[(p0 + u) * rec + cw * BITS + j] = word;
                     }
                 }
@@ -125,29 +89,23 @@ bitpack_kernel(const T* __restrict__ x, uint32_t* __restrict__ out, int C, int H
         }
     } else {
         const bool pvalid = lane < npix;
-        const T* xin = x + static_cast<size_t>(n) * C * HW + hw0 + lane;
+        const int8_t* xin = x + static_cast<size_t>(n) * C * HW + hw0 + lane;
         for (int cw = 0; cw < Cw; ++cw) {
             uint32_t words[BITS];
 #pragma unroll
             for (int j = 0; j < BITS; ++j) words[j] = 0u;
-            T v[32];
+            unsigned pat[32];
 #pragma unroll
             for (int u = 0; u < 32; ++u) {
                 const int c = cw * 32 + u;
-                v[u] = (pvalid && c < C) ? xin[static_cast<size_t>(c) * HW] : nullv;
+                pat[u] = (pvalid && c < C) ? code_pattern<BITS>(xin[static_cast<size_t>(c) * HW], sign) : 0u;
             }
 #pragma unroll
-            for (int u = 0; u < 32; ++u) {
-                const PlaneBits<T, BITS, BOUNDS> pb(v[u], q);
+            for (int u = 0; u < 32; ++u)
 #pragma unroll
-                for (int j = 0; j < BITS; ++j)
-                    if (pb.p[j]) words[j] |= 1u << u;
-            }
-            const int nvalid = min(32, C - cw * 32);
-            const unsigned fl = pvalid ? (nvalid == 32 ? 0xffffffffu : ((1u << nvalid) - 1u)) : 0u;
+                for (int j = 0; j < BITS; ++j) words[j] |= ((pat[u] >> j) & 1u) << u;
 #pragma unroll
-            for (int j = 0; j < BITS; ++j)
-                stage[lane * rec + cw * BITS + j] = ((q.flip >> j) & 1) ? (words[j] ^ fl) : words[j];
+            for (int j = 0; j < BITS; ++j) stage[lane * rec + cw * BITS + j] = words[j];
         }
     }
     __syncwarp();
@@ -167,21 +125,17 @@ __device__ __forceinline__ void store_planes(uint32_t* dst, const uint32_t (&w)[
     }
 }
 
-// Sign-bit form of the comparison quantiser for fp32 NCHW input and 1- or 2-bit codes.
+// Sign-bit form of the comparison quantiser for fp32 input.
 //   With p the largest binary32 value below the bound b:  x >= b  <=>  x > p  <=>  the sign bit of p - x is set.
 //   An IEEE subtraction never rounds across zero and x == p gives +0; p is stored as +0 when it is a zero, so neither
 //   signed zero of x yields -0.  A NaN input gives the canonical NaN (sign clear): no level reached, the lowest
 //   code, which is what clip() makes of a NaN in the formula.  +-inf behave like the comparison.
 //   2-bit codes: plane 1 = (x >= b1); plane 0 = parity of the three comparisons = sign((p0-x) ^ (p1-x) ^ (p2-x)).
-// One funnel shift moves a sign bit into a plane word; channels are walked from 31 down to 0 so that channel c ends at
-// bit c.  Per element: one load, 1 or 3 subtractions, at most one three-input xor and BITS funnel shifts, which
-// leaves the kernel waiting on HBM rather than on the issue slots.  3- and 4-bit codes search the 7 or 15 bounds
-// binarily, one subtraction, one sign test and one funnel shift per bit plus the selects that pick the next bound.
-// Work unit of a warp = 32 consecutive pixels of one image x one 32-channel word (lane = pixel): all 32 channel rows are
-// in flight at once (32 coalesced 128-byte requests per warp), and each lane stores the BITS plane words of its pixel
-// straight to the packed record (8-byte stores for 2-bit codes; the words of the other channel groups of the record
-// come from the neighbouring warps of the block, so the sectors fill up in L2).  Units are small and numerous, which
-// keeps the tail of the grid short; no shared memory, no barrier.
+//   3- and 4-bit codes search the 7 or 15 bounds binarily: one subtraction, one sign test and one funnel shift per bit
+//   plus the selects that pick the next bound.
+// One funnel shift moves a sign bit into a plane word (w = 2 w + bit); the inputs of a word are walked from position 31
+// down to 0 so that input i ends at bit i.  Per element of a 2-bit tensor: one load, three subtractions, one three-input
+// xor and two funnel shifts, which leaves the kernels waiting on HBM rather than on the issue slots.
 // Shifts the BITS plane bits of one input into the plane words w (w = 2 w + bit), in the sign-bit comparison form.
 template <int BITS>
 __device__ __forceinline__ void quant_push(const QuantParams& q, float v, uint32_t (&w)[BITS])
@@ -232,6 +186,11 @@ __device__ __forceinline__ uint32_t warp_transpose32(uint32_t x, int lane)
     return x;
 }
 
+// fp32 NCHW.  Work unit of a warp = 32 consecutive pixels of one image x one 32-channel word (lane = pixel): all 32
+// channel rows are in flight at once (32 coalesced 128-byte requests per warp), walked from channel 31 down, and each lane
+// stores the BITS plane words of its pixel straight to the packed record (8-byte stores for 2-bit codes; the words of
+// the other channel groups of the record come from the neighbouring warps of the block, so the sectors fill up in L2).
+// Units are small and numerous, which keeps the tail of the grid short; no shared memory, no barrier.
 constexpr int FAST_THREADS = 128;
 constexpr int FAST_WARPS = FAST_THREADS / 32;
 
@@ -508,64 +467,46 @@ static float key_float(uint32_t k)
     return f;
 }
 
-// below[k] = the binary32 value just under bound[k] (bounds are never -inf: -inf always quantises to the lowest code).
-static void set_below(QuantParams& q)
-{
-    for (int k = 0; k < 15; ++k) {
-        const float b = q.bound[k];
-        float p = b == 0.0f ? -1.401298464e-45f : key_float(float_key(b) - 1u);
-        if (p == 0.0f) p = 0.0f;          // drops the sign of a zero
-        q.below[k] = p;
-    }
-}
-
-static QuantParams make_quant_params(float s, int bits, int sign, bool quantise)
+// Comparison-form quantiser for scale s: below[k] = the binary32 value just under bound[k], the smallest input whose code
+// is >= qmin + k + 1 (bounds are never -inf: -inf always quantises to the lowest code; unreachable levels get +inf).
+static QuantParams make_quant_params(float s, int bits, int sign)
 {
     QuantParams q{};
-    q.scale = s; q.bits = bits; q.sign = sign;
-    code_limits(bits, sign, q.qmin, q.qmax);
-    q.flip = 0;
-    q.by_bounds = 0;
-    q.null_value = (sign == BS_UNSIGNED) ? 0.0f : (sign == BS_BIPOLAR ? -1.0f : 0.0f);   // formula mode / int8 codes
-    if (!quantise) return q;
-    for (int k = 0; k < 15; ++k) q.bound[k] = INFINITY;
-    q.have_bounds = 1;
+    q.bits = bits; q.sign = sign;
+    int qmin, qmax;
+    code_limits(bits, sign, qmin, qmax);
+    float bound[15];
+    for (int k = 0; k < 15; ++k) bound[k] = INFINITY;
     if (sign == BS_BIPOLAR) {                 // +1 iff x >= 0
-        q.null_value = -INFINITY;
-        q.by_bounds = 1;
-        q.bound[0] = 0.0f;
-        set_below(q);
-        return q;
-    }
-    const uint32_t lo_key = float_key(-INFINITY), hi_key = float_key(INFINITY);
-    for (int k = 1; k <= q.qmax - q.qmin; ++k) {
-        // smallest x (in float order) with code >= qmin + k; the code is monotone in x and reaches qmax at +inf
-        uint32_t lo = lo_key, hi = hi_key;
-        while (lo < hi) {
-            const uint32_t mid = lo + (hi - lo) / 2;
-            if (host_quantize(key_float(mid), s, q.qmin, q.qmax) >= q.qmin + k) hi = mid;
-            else lo = mid + 1;
+        bound[0] = 0.0f;
+    } else {
+        const uint32_t lo_key = float_key(-INFINITY), hi_key = float_key(INFINITY);
+        for (int k = 1; k <= qmax - qmin; ++k) {
+            // smallest x (in float order) with code >= qmin + k; the code is monotone in x and reaches qmax at +inf
+            uint32_t lo = lo_key, hi = hi_key;
+            while (lo < hi) {
+                const uint32_t mid = lo + (hi - lo) / 2;
+                if (host_quantize(key_float(mid), s, qmin, qmax) >= qmin + k) hi = mid;
+                else lo = mid + 1;
+            }
+            bound[k - 1] = key_float(lo);
         }
-        q.bound[k - 1] = key_float(lo);
     }
-    set_below(q);
-    if (bits <= 2) {
-        q.by_bounds = 1;
-        q.null_value = -INFINITY;
-        // pattern = (qmin + count) mod 2^bits; for two's-complement 2-bit codes qmin = -2 flips bit 1 only
-        q.flip = (sign == BS_SIGNED) ? (static_cast<unsigned>(q.qmin) & ((1u << bits) - 1u)) : 0;
+    for (int k = 0; k < 15; ++k) {
+        float p = bound[k] == 0.0f ? -1.401298464e-45f : key_float(float_key(bound[k]) - 1u);
+        if (p == 0.0f) p = fabsf(p);          // drops the sign of a zero
+        q.below[k] = p;
     }
     return q;
 }
 
-template <typename T, bool NHWC, int BITS, bool BOUNDS>
-static int launch_bitpack_one(const void* x, uint32_t* out, int N, int C, int HW, const QuantParams& q, cudaStream_t st)
+template <bool NHWC, int BITS>
+static int launch_bitpack_codes(const void* x, uint32_t* out, int N, int C, int HW, int sign, cudaStream_t st)
 {
     const int Cw = ceil_div(C, 32);
-    const int rec = Cw * q.bits;
-    const size_t smem = static_cast<size_t>(PACK_WARPS) * 32 * rec * 4;
+    const size_t smem = static_cast<size_t>(PACK_WARPS) * 32 * Cw * BITS * 4;
     if (smem > 200 * 1024) return BS_ERR_UNSUPPORTED;
-    auto kern = bitpack_kernel<T, NHWC, BITS, BOUNDS>;
+    auto kern = bitpack_codes_kernel<NHWC, BITS>;
     if (smem > 48 * 1024 &&
         cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)) != cudaSuccess)
         return BS_ERR_CUDA;
@@ -573,8 +514,8 @@ static int launch_bitpack_one(const void* x, uint32_t* out, int N, int C, int HW
     const long long ntiles = static_cast<long long>(N) * tiles_per_img;
     const long long blocks = ceil_div_ll(ntiles, PACK_WARPS);
     if (blocks > 0x7fffffffLL) return BS_ERR_UNSUPPORTED;
-    kern<<<static_cast<unsigned>(blocks), PACK_THREADS, smem, st>>>(static_cast<const T*>(x), out, C, HW, Cw, ntiles,
-                                                                  tiles_per_img, q);
+    kern<<<static_cast<unsigned>(blocks), PACK_THREADS, smem, st>>>(static_cast<const int8_t*>(x), out, C, HW, Cw, ntiles,
+                                                                  tiles_per_img, sign);
     return cudaGetLastError() == cudaSuccess ? BS_OK : BS_ERR_CUDA;
 }
 
@@ -609,36 +550,33 @@ static int launch_bitpack_i8(const void* x, uint32_t* out, int N, int C, int HW,
     }
 }
 
-template <typename T, bool NHWC>
-static int launch_bitpack(const void* x, uint32_t* out, int N, int C, int HW, const QuantParams& q, cudaStream_t st)
+// fp32 tensors: comparison-form kernels with one (32 pixels, channel word) unit per warp.
+template <bool NHWC>
+static int launch_bitpack_f32(const void* x, uint32_t* out, int N, int C, int HW, const QuantParams& q, cudaStream_t st)
 {
-    if constexpr (sizeof(T) == 4) {
-        // fp32 tensors take the comparison-form kernels with one (pixels, channel word) unit per warp
-        if (!NHWC && q.have_bounds) {
-            switch (q.bits) {
-                case 1: return launch_units(bitpack_nchw_f32_kernel<1>, x, out, N, C, HW, 32, st, q);
-                case 2: return launch_units(bitpack_nchw_f32_kernel<2>, x, out, N, C, HW, 32, st, q);
-                case 3: return launch_units(bitpack_nchw_f32_kernel<3>, x, out, N, C, HW, 32, st, q);
-                default: return launch_units(bitpack_nchw_f32_kernel<4>, x, out, N, C, HW, 32, st, q);
-            }
-        }
-        if (NHWC && q.have_bounds) {
-            switch (q.bits) {
-                case 1: return launch_units(bitpack_nhwc_f32_kernel<1>, x, out, N, C, HW, 32, st, q);
-                case 2: return launch_units(bitpack_nhwc_f32_kernel<2>, x, out, N, C, HW, 32, st, q);
-                case 3: return launch_units(bitpack_nhwc_f32_kernel<3>, x, out, N, C, HW, 32, st, q);
-                default: return launch_units(bitpack_nhwc_f32_kernel<4>, x, out, N, C, HW, 32, st, q);
-            }
-        }
-    } else {
-        // int8 codes whose planes are the low bits of the byte, in shapes that allow aligned vector loads
-        if (q.sign != BS_BIPOLAR && (NHWC ? C % 32 == 0 : HW % 4 == 0)) return launch_bitpack_i8<NHWC>(x, out, N, C, HW, q.bits, st);
-    }
     switch (q.bits) {
-        case 1: return launch_bitpack_one<T, NHWC, 1, true>(x, out, N, C, HW, q, st);
-        case 2: return launch_bitpack_one<T, NHWC, 2, true>(x, out, N, C, HW, q, st);
-        case 3: return launch_bitpack_one<T, NHWC, 3, false>(x, out, N, C, HW, q, st);
-        default: return launch_bitpack_one<T, NHWC, 4, false>(x, out, N, C, HW, q, st);
+        case 1: return NHWC ? launch_units(bitpack_nhwc_f32_kernel<1>, x, out, N, C, HW, 32, st, q)
+                            : launch_units(bitpack_nchw_f32_kernel<1>, x, out, N, C, HW, 32, st, q);
+        case 2: return NHWC ? launch_units(bitpack_nhwc_f32_kernel<2>, x, out, N, C, HW, 32, st, q)
+                            : launch_units(bitpack_nchw_f32_kernel<2>, x, out, N, C, HW, 32, st, q);
+        case 3: return NHWC ? launch_units(bitpack_nhwc_f32_kernel<3>, x, out, N, C, HW, 32, st, q)
+                            : launch_units(bitpack_nchw_f32_kernel<3>, x, out, N, C, HW, 32, st, q);
+        default: return NHWC ? launch_units(bitpack_nhwc_f32_kernel<4>, x, out, N, C, HW, 32, st, q)
+                             : launch_units(bitpack_nchw_f32_kernel<4>, x, out, N, C, HW, 32, st, q);
+    }
+}
+
+// int8 codes: the vector kernels where the shape allows aligned vector loads and the planes are the low bits of the byte,
+// else the fallback.
+template <bool NHWC>
+static int launch_bitpack_codes_any(const void* x, uint32_t* out, int N, int C, int HW, int bits, int sign, cudaStream_t st)
+{
+    if (sign != BS_BIPOLAR && (NHWC ? C % 32 == 0 : HW % 4 == 0)) return launch_bitpack_i8<NHWC>(x, out, N, C, HW, bits, st);
+    switch (bits) {
+        case 1: return launch_bitpack_codes<NHWC, 1>(x, out, N, C, HW, sign, st);
+        case 2: return launch_bitpack_codes<NHWC, 2>(x, out, N, C, HW, sign, st);
+        case 3: return launch_bitpack_codes<NHWC, 3>(x, out, N, C, HW, sign, st);
+        default: return launch_bitpack_codes<NHWC, 4>(x, out, N, C, HW, sign, st);
     }
 }
 
@@ -652,12 +590,13 @@ extern "C" int bitpack_activations(const void* x, int x_is_fp32, bs_layout_t lay
     if (static_cast<long long>(H) * W > 0x7fffffffLL) return BS_ERR_UNSUPPORTED;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const int HW = H * W;
-    const QuantParams q = make_quant_params(x_is_fp32 ? act_scale : 1.0f, a_bits, a_sign, x_is_fp32 != 0);
-    if (x_is_fp32)
-        return layout == BS_NHWC ? launch_bitpack<float, true>(x, packed_out, N, C, HW, q, st)
-                                 : launch_bitpack<float, false>(x, packed_out, N, C, HW, q, st);
-    return layout == BS_NHWC ? launch_bitpack<int8_t, true>(x, packed_out, N, C, HW, q, st)
-                             : launch_bitpack<int8_t, false>(x, packed_out, N, C, HW, q, st);
+    if (x_is_fp32) {
+        const QuantParams q = make_quant_params(act_scale, a_bits, a_sign);
+        return layout == BS_NHWC ? launch_bitpack_f32<true>(x, packed_out, N, C, HW, q, st)
+                                 : launch_bitpack_f32<false>(x, packed_out, N, C, HW, q, st);
+    }
+    return layout == BS_NHWC ? launch_bitpack_codes_any<true>(x, packed_out, N, C, HW, a_bits, a_sign, st)
+                             : launch_bitpack_codes_any<false>(x, packed_out, N, C, HW, a_bits, a_sign, st);
 }
 
 extern "C" int bitunpack_activations(const uint32_t* packed, int N, int C, int H, int W, int a_bits, bs_sign_t a_sign,
