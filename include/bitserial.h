@@ -68,10 +68,20 @@ size_t bs_packed_rows_bytes(int rows, int K, int bits);
  *   act_scale  the step s of the quantiser (> 0, finite); ignored for int8 input.
  *              Bipolar: code = +1 when x >= 0 else -1.
  *   packed_out device, bs_packed_act_bytes(N, C, H, W, a_bits) bytes, fully overwritten.
- * Inputs must be finite.  One pass over x; bound by HBM bandwidth.
+ * The quantiser is evaluated in its comparison form (bs_quantiser_bounds), which takes the formula's decision for every
+ * float32 input: +-inf clip to the limits, a NaN gets the lowest code.  One pass over x; bound by HBM bandwidth.
  */
 int bitpack_activations(const void* x, int x_is_fp32, bs_layout_t layout, int N, int C, int H, int W,
                         float act_scale, int a_bits, bs_sign_t a_sign, uint32_t* packed_out, void* stream);
+
+/*
+ * bs_quantiser_bounds -- the comparison form of the Section IV quantiser that bitpack_activations evaluates.  Host call,
+ * no device work.  Writes to bounds_out[k] (HOST memory, 2^a_bits - 1 floats; one for bipolar codes) the smallest
+ * float32 input whose code is >= qmin + k + 1 under round_half_even(clip(x / act_scale, qmin, qmax)), found by bisection
+ * with that very formula, so that  code = qmin + #{k : x >= bounds_out[k]}  for every float32 x (a NaN reaches no
+ * level).  Returns BS_ERR_INVALID_ARG for a null pointer, a scale that is not positive and finite, or a bad width/sign.
+ */
+int bs_quantiser_bounds(float act_scale, int a_bits, bs_sign_t a_sign, float* bounds_out);
 
 /* Inverse of the plane split (test and debugging aid): packed activations -> int8 codes in `layout`. */
 int bitunpack_activations(const uint32_t* packed, int N, int C, int H, int W, int a_bits, bs_sign_t a_sign,
@@ -237,6 +247,18 @@ int bitserial_gemm_tc(const uint32_t* a_packed, const int8_t* w_tc, int M, int N
  * outputs are then undefined), BS_ERR_CUDA if the stream reports an error, else BS_OK.
  */
 int bs_check_status(void* stream);
+
+/*
+ * bs_requant_bounds -- the comparison form of the requantisation epilogue for 1- and 2-bit outputs (the paper gives no
+ * epilogue; this is the library's fixed order fma, residual fma, ReLU, clip, round-half-even).  Host call, no device
+ * work.  With t = fmaf((float)acc, scale[o], bias[o]) the output code is  qmin + #{k : t >= bound[r][k]}  where r is
+ * the stored pattern of the residual code (0 when there is none); writes bound[r][0..2] to bounds_out[3 r + k] (HOST
+ * memory, 3 floats per residual pattern, 2^res_bits patterns; +inf for levels that do not exist).  Returns
+ * BS_ERR_UNSUPPORTED for outputs wider than 2 bits (the kernels evaluate the formula there), BS_ERR_INVALID_ARG for a
+ * null pointer or a bad width/sign.
+ */
+int bs_requant_bounds(int has_residual, float res_scale, int res_bits, bs_sign_t res_sign, int relu, int out_bits,
+                      bs_sign_t out_sign, float* bounds_out);
 
 /*
  * bs_selftest_wait_timeout -- exercises the failure path of the kernels' device-side waits without any fault (the paper

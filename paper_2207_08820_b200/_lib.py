@@ -91,6 +91,10 @@ def lib() -> ctypes.CDLL:
     L.bitserial_gemm_tc.argtypes = [vp, vp, i, i, i, i, i, i, i, vp, vp, i, i, i, vp, vp, vp]
     L.bs_check_status.restype = i
     L.bs_check_status.argtypes = [vp]
+    L.bs_quantiser_bounds.restype = i
+    L.bs_quantiser_bounds.argtypes = [ctypes.c_float, i, i, ctypes.POINTER(ctypes.c_float)]
+    L.bs_requant_bounds.restype = i
+    L.bs_requant_bounds.argtypes = [i, ctypes.c_float, i, i, i, i, i, ctypes.POINTER(ctypes.c_float)]
     L.bs_selftest_wait_timeout.restype = i
     L.bs_selftest_wait_timeout.argtypes = [i, vp]
     L.bs_popc_rate.restype = i
@@ -106,4 +110,4 @@ EXPORTED = ("bs_packed_act_bytes", "bs_packed_wgt_bytes", "bs_packed_rows_bytes"
             "bitserial_conv2d_ws", "bitserial_gemm_ws", "bs_conv_workspace_bytes", "bs_gemm_workspace_bytes",
             "bitserial_gemm_noalloc", "bs_gemm_noalloc_max_scratch_bytes",
             "bs_tc_weights_bytes", "bs_tc_prepare_weights", "bs_tc_supported", "bitserial_conv2d_tc", "bitserial_conv2d_tc_chained", "bitserial_gemm_tc", "bs_l2_prefetch",
-            "bs_check_status", "bs_selftest_wait_timeout", "bs_popc_rate", "bs_status_string")
+            "bs_check_status", "bs_quantiser_bounds", "bs_requant_bounds", "bs_selftest_wait_timeout", "bs_popc_rate", "bs_status_string")

@@ -7,6 +7,7 @@
 #include <mutex>
 
 #include "conv_launch.cuh"
+#include "requant_bounds.h"
 
 namespace bs {
 
@@ -503,4 +504,18 @@ extern "C" int bs_selftest_wait_timeout(int polls, void* stream)
     if (!status) return BS_ERR_CUDA;
     bs::wait_timeout_selftest_kernel<<<1, 32, 0, static_cast<cudaStream_t>(stream)>>>(static_cast<unsigned>(polls), status);
     return cudaGetLastError() == cudaSuccess ? BS_OK : BS_ERR_CUDA;
+}
+
+// ---- host-side view of the epilogue's comparison form (no device work) ------------------------------------------
+extern "C" int bs_requant_bounds(int has_residual, float res_scale, int res_bits, bs_sign_t res_sign, int relu, int out_bits,
+                                 bs_sign_t out_sign, float* bounds_out)
+{
+    if (!bounds_out || !bs::bits_ok(out_bits, out_sign)) return BS_ERR_INVALID_ARG;
+    if (has_residual && !bs::bits_ok(res_bits, res_sign)) return BS_ERR_INVALID_ARG;
+    const bs::RequantBounds rb = bs::make_requant_bounds(has_residual != 0, res_scale, res_bits, res_sign, relu, out_bits, out_sign);
+    if (!rb.enabled) return BS_ERR_UNSUPPORTED;
+    const int npat = has_residual ? (1 << res_bits) : 1;
+    for (int r = 0; r < npat; ++r)
+        for (int k = 0; k < 3; ++k) bounds_out[r * 3 + k] = rb.bound[r][k];
+    return BS_OK;
 }

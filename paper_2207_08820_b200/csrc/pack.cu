@@ -469,35 +469,51 @@ static float key_float(uint32_t k)
 
 // Comparison-form quantiser for scale s: below[k] = the binary32 value just under bound[k], the smallest input whose code
 // is >= qmin + k + 1 (bounds are never -inf: -inf always quantises to the lowest code; unreachable levels get +inf).
+// bound[k], k = 0 .. 14: smallest binary32 input whose code is >= qmin + k + 1; +inf for levels that do not exist.
+static void quantiser_bounds(float s, int bits, int sign, float (&bound)[15])
+{
+    int qmin, qmax;
+    code_limits(bits, sign, qmin, qmax);
+    for (int k = 0; k < 15; ++k) bound[k] = INFINITY;
+    if (sign == BS_BIPOLAR) {                 // +1 iff x >= 0
+        bound[0] = 0.0f;
+        return;
+    }
+    const uint32_t lo_key = float_key(-INFINITY), hi_key = float_key(INFINITY);
+    for (int k = 1; k <= qmax - qmin; ++k) {
+        // smallest x (in float order) with code >= qmin + k; the code is monotone in x and reaches qmax at +inf
+        uint32_t lo = lo_key, hi = hi_key;
+        while (lo < hi) {
+            const uint32_t mid = lo + (hi - lo) / 2;
+            if (host_quantize(key_float(mid), s, qmin, qmax) >= qmin + k) hi = mid;
+            else lo = mid + 1;
+        }
+        bound[k - 1] = key_float(lo);
+    }
+}
+
 static QuantParams make_quant_params(float s, int bits, int sign)
 {
     QuantParams q{};
     q.bits = bits; q.sign = sign;
-    int qmin, qmax;
-    code_limits(bits, sign, qmin, qmax);
     float bound[15];
-    for (int k = 0; k < 15; ++k) bound[k] = INFINITY;
-    if (sign == BS_BIPOLAR) {                 // +1 iff x >= 0
-        bound[0] = 0.0f;
-    } else {
-        const uint32_t lo_key = float_key(-INFINITY), hi_key = float_key(INFINITY);
-        for (int k = 1; k <= qmax - qmin; ++k) {
-            // smallest x (in float order) with code >= qmin + k; the code is monotone in x and reaches qmax at +inf
-            uint32_t lo = lo_key, hi = hi_key;
-            while (lo < hi) {
-                const uint32_t mid = lo + (hi - lo) / 2;
-                if (host_quantize(key_float(mid), s, qmin, qmax) >= qmin + k) hi = mid;
-                else lo = mid + 1;
-            }
-            bound[k - 1] = key_float(lo);
-        }
-    }
+    quantiser_bounds(s, bits, sign, bound);
     for (int k = 0; k < 15; ++k) {
         float p = bound[k] == 0.0f ? -1.401298464e-45f : key_float(float_key(bound[k]) - 1u);
         if (p == 0.0f) p = fabsf(p);          // drops the sign of a zero
         q.below[k] = p;
     }
     return q;
+}
+
+extern "C" int bs_quantiser_bounds(float act_scale, int a_bits, bs_sign_t a_sign, float* bounds_out)
+{
+    if (!bounds_out || !bits_ok(a_bits, a_sign) || !(act_scale > 0.0f && act_scale < 3.0e38f)) return BS_ERR_INVALID_ARG;
+    float bound[15];
+    quantiser_bounds(act_scale, a_bits, a_sign, bound);
+    const int n = a_sign == BS_BIPOLAR ? 1 : (1 << a_bits) - 1;
+    for (int k = 0; k < n; ++k) bounds_out[k] = bound[k];
+    return BS_OK;
 }
 
 template <bool NHWC, int BITS>
