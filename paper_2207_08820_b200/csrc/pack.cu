@@ -291,57 +291,98 @@ bitpack_nhwc_f32_kernel(const float* __restrict__ x, uint32_t* __restrict__ out,
 // highest down, leaves in byte k of a the eight channel bits of pixel k.  A byte permute drops each finished byte into
 // the plane word of its pixel.  About 1.8 instructions per element for 2-bit codes.  Needs H*W to be a multiple of 4
 // (aligned 32-bit loads); work unit of a warp = 128 pixels x one 32-channel word.
-template <int BITS>
+// Stores: with CW = 0 every lane writes the plane words of its pixels straight to the records (8-byte pieces of 32-byte
+// sectors, four partial writes per sector).  When the channel words of a record number CW = 1, 2 or 4, the four warps of
+// a block hold complete records of 4 / CW tiles: they park their words in shared memory as [warp][plane][pixel] (128-bit
+// stores, no bank conflicts), and after one barrier the block writes the records as whole 128-bit pieces.
+template <int BITS, int CW>
 __global__ void __launch_bounds__(FAST_THREADS, 8)
 bitpack_nchw_i8_kernel(const int8_t* __restrict__ x, uint32_t* __restrict__ out, int C, int HW, int Cw, long long nunits,
                        int units_per_img)
 {
+    constexpr bool STAGED = CW != 0;
+    __shared__ __align__(16) uint32_t stage[STAGED ? FAST_WARPS * BITS * 128 : 4];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const long long unit = static_cast<long long>(blockIdx.x) * FAST_WARPS + warp;
-    if (unit >= nunits) return;
-    const long long n = unit / units_per_img;
-    const int rem = static_cast<int>(unit % units_per_img);
-    const int cw = rem % Cw;
-    const int hw0 = (rem / Cw) * 128;
-    const int pix = hw0 + 4 * lane;
-    const bool pvalid = pix < HW;          // H*W is a multiple of 4: the four pixels of a lane are inside or outside together
-    const uint32_t* xin = reinterpret_cast<const uint32_t*>(x + (static_cast<size_t>(n) * C + cw * 32) * HW + (pvalid ? pix : hw0));
-    const int nvalid = min(32, C - cw * 32);
-    const size_t row = static_cast<size_t>(HW / 4);
-    uint32_t v[32];
-    if (nvalid == 32) {
+    const bool active = unit < nunits;
+    if (!STAGED && !active) return;
+    if (active) {
+        const long long n = unit / units_per_img;
+        const int rem = static_cast<int>(unit % units_per_img);
+        const int cw = rem % Cw;
+        const int hw0 = (rem / Cw) * 128;
+        const int pix = hw0 + 4 * lane;
+        const bool pvalid = pix < HW;      // H*W is a multiple of 4: the four pixels of a lane are inside or outside together
+        const uint32_t* xin = reinterpret_cast<const uint32_t*>(x + (static_cast<size_t>(n) * C + cw * 32) * HW + (pvalid ? pix : hw0));
+        const int nvalid = min(32, C - cw * 32);
+        const size_t row = static_cast<size_t>(HW / 4);
+        uint32_t v[32];
+        if (nvalid == 32) {
 #pragma unroll
-        for (int u = 0; u < 32; ++u) v[u] = __ldcs(xin + u * row);
-    } else {
+            for (int u = 0; u < 32; ++u) v[u] = __ldcs(xin + u * row);
+        } else {
 #pragma unroll
-        for (int u = 0; u < 32; ++u) v[u] = u < nvalid ? __ldcs(xin + u * row) : 0u;
-    }
-    uint32_t w[4][BITS];
-#pragma unroll
-    for (int k = 0; k < 4; ++k)
-#pragma unroll
-        for (int j = 0; j < BITS; ++j) w[k][j] = 0u;
-#pragma unroll
-    for (int g = 0; g < 4; ++g) {
-        uint32_t a[BITS];
-#pragma unroll
-        for (int j = 0; j < BITS; ++j) a[j] = 0u;
-#pragma unroll
-        for (int i = 7; i >= 0; --i) {
-            const uint32_t r = v[8 * g + i];
-#pragma unroll
-            for (int j = 0; j < BITS; ++j) a[j] = a[j] * 2u + ((r >> j) & 0x01010101u);
+            for (int u = 0; u < 32; ++u) v[u] = u < nvalid ? __ldcs(xin + u * row) : 0u;
         }
+        uint32_t w[4][BITS];
 #pragma unroll
         for (int k = 0; k < 4; ++k)
 #pragma unroll
-            for (int j = 0; j < BITS; ++j)      // byte k of a[j] becomes byte g of the plane word of pixel k
-                w[k][j] = __byte_perm(w[k][j], a[j], (0x3210u & ~(0xfu << (4 * g))) | ((4u + k) << (4 * g)));
-    }
-    if (!pvalid) return;
+            for (int j = 0; j < BITS; ++j) w[k][j] = 0u;
 #pragma unroll
-    for (int k = 0; k < 4; ++k)
-        store_planes<BITS>(out + ((static_cast<size_t>(n) * HW + pix + k) * Cw + cw) * BITS, w[k]);
+        for (int g = 0; g < 4; ++g) {
+            uint32_t a[BITS];
+#pragma unroll
+            for (int j = 0; j < BITS; ++j) a[j] = 0u;
+#pragma unroll
+            for (int i = 7; i >= 0; --i) {
+                const uint32_t r = v[8 * g + i];
+#pragma unroll
+                for (int j = 0; j < BITS; ++j) a[j] = a[j] * 2u + ((r >> j) & 0x01010101u);
+            }
+#pragma unroll
+            for (int k = 0; k < 4; ++k)
+#pragma unroll
+                for (int j = 0; j < BITS; ++j)      // byte k of a[j] becomes byte g of the plane word of pixel k
+                    w[k][j] = __byte_perm(w[k][j], a[j], (0x3210u & ~(0xfu << (4 * g))) | ((4u + k) << (4 * g)));
+        }
+        if constexpr (STAGED) {
+#pragma unroll
+            for (int j = 0; j < BITS; ++j)
+                *reinterpret_cast<uint4*>(stage + (warp * BITS + j) * 128 + 4 * lane) = make_uint4(w[0][j], w[1][j], w[2][j], w[3][j]);
+        } else {
+            if (!pvalid) return;
+#pragma unroll
+            for (int k = 0; k < 4; ++k)
+                store_planes<BITS>(out + ((static_cast<size_t>(n) * HW + pix + k) * Cw + cw) * BITS, w[k]);
+        }
+    }
+    if constexpr (STAGED) {
+        __syncthreads();
+        // the block's first unit is a multiple of 4, hence of CW: warp t * CW + c holds channel word c of the block's tile t
+        constexpr int REC = CW * BITS;                 // words of a pixel record
+        constexpr int PIECE = REC % 4 == 0 ? 4 : (REC % 2 == 0 ? 2 : 1);     // words per store
+#pragma unroll
+        for (int t = 0; t < FAST_WARPS / CW; ++t) {
+            const long long unit_t = static_cast<long long>(blockIdx.x) * FAST_WARPS + t * CW;
+            if (unit_t >= nunits) break;
+            const long long n = unit_t / units_per_img;
+            const int hw0 = (static_cast<int>(unit_t % units_per_img) / CW) * 128;
+            const int nwords = min(128, HW - hw0) * REC;            // a multiple of 4: H*W and the tile start are
+            uint32_t* dst = out + (static_cast<size_t>(n) * HW + hw0) * REC;
+            for (int i = threadIdx.x * PIECE; i < nwords; i += FAST_THREADS * PIECE) {
+                uint32_t piece[PIECE];
+#pragma unroll
+                for (int e = 0; e < PIECE; ++e) {
+                    const int idx = i + e, p = idx / REC, r = idx % REC;          // (pixel, word of its record)
+                    piece[e] = stage[((t * CW + r / BITS) * BITS + r % BITS) * 128 + p];
+                }
+                if constexpr (PIECE == 4) *reinterpret_cast<uint4*>(dst + i) = make_uint4(piece[0], piece[1], piece[2], piece[3]);
+                else if constexpr (PIECE == 2) *reinterpret_cast<uint2*>(dst + i) = make_uint2(piece[0], piece[1]);
+                else dst[i] = piece[0];
+            }
+        }
+    }
 }
 
 // int8 codes, NHWC, C a multiple of 32: the 32 channels of a (pixel, channel word) are 32 contiguous, aligned bytes.
@@ -551,18 +592,25 @@ static int launch_units(K kern, const void* x, uint32_t* out, int N, int C, int 
     return cudaGetLastError() == cudaSuccess ? BS_OK : BS_ERR_CUDA;
 }
 
+template <int BITS>
+static int launch_bitpack_nchw_i8(const void* x, uint32_t* out, int N, int C, int HW, cudaStream_t st)
+{
+    switch (ceil_div(C, 32)) {      // records of 1, 2 or 4 channel words leave through the block-staged stores
+        case 1: return launch_units(bitpack_nchw_i8_kernel<BITS, 1>, x, out, N, C, HW, 128, st);
+        case 2: return launch_units(bitpack_nchw_i8_kernel<BITS, 2>, x, out, N, C, HW, 128, st);
+        case 4: return launch_units(bitpack_nchw_i8_kernel<BITS, 4>, x, out, N, C, HW, 128, st);
+        default: return launch_units(bitpack_nchw_i8_kernel<BITS, 0>, x, out, N, C, HW, 128, st);
+    }
+}
+
 template <bool NHWC>
 static int launch_bitpack_i8(const void* x, uint32_t* out, int N, int C, int HW, int bits, cudaStream_t st)
 {
     switch (bits) {
-        case 1: return NHWC ? launch_units(bitpack_nhwc_i8_kernel<1>, x, out, N, C, HW, 128, st)
-                            : launch_units(bitpack_nchw_i8_kernel<1>, x, out, N, C, HW, 128, st);
-        case 2: return NHWC ? launch_units(bitpack_nhwc_i8_kernel<2>, x, out, N, C, HW, 128, st)
-                            : launch_units(bitpack_nchw_i8_kernel<2>, x, out, N, C, HW, 128, st);
-        case 3: return NHWC ? launch_units(bitpack_nhwc_i8_kernel<3>, x, out, N, C, HW, 128, st)
-                            : launch_units(bitpack_nchw_i8_kernel<3>, x, out, N, C, HW, 128, st);
-        default: return NHWC ? launch_units(bitpack_nhwc_i8_kernel<4>, x, out, N, C, HW, 128, st)
-                             : launch_units(bitpack_nchw_i8_kernel<4>, x, out, N, C, HW, 128, st);
+        case 1: return NHWC ? launch_units(bitpack_nhwc_i8_kernel<1>, x, out, N, C, HW, 128, st) : launch_bitpack_nchw_i8<1>(x, out, N, C, HW, st);
+        case 2: return NHWC ? launch_units(bitpack_nhwc_i8_kernel<2>, x, out, N, C, HW, 128, st) : launch_bitpack_nchw_i8<2>(x, out, N, C, HW, st);
+        case 3: return NHWC ? launch_units(bitpack_nhwc_i8_kernel<3>, x, out, N, C, HW, 128, st) : launch_bitpack_nchw_i8<3>(x, out, N, C, HW, st);
+        default: return NHWC ? launch_units(bitpack_nhwc_i8_kernel<4>, x, out, N, C, HW, 128, st) : launch_bitpack_nchw_i8<4>(x, out, N, C, HW, st);
     }
 }
 
