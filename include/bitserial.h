@@ -167,7 +167,9 @@ int bitserial_gemm(const uint32_t* a_packed, const uint32_t* w_packed, int M, in
  *                    first call and every call leaves it zero again, so one cudaMemset at allocation suffices.
  *                    Calls that share a workspace must not overlap on the GPU (use one stream, or one workspace
  *                    per stream).  A NULL or too small workspace falls back to the unsplit kernel.
- *   bs_*_workspace_bytes  bytes the planner wants for this shape (0: no split would be used).  Host-only, no launch.
+ *   bs_*_workspace_bytes  bytes the planner wants for this shape on the CURRENT device (0: no split would be used).
+ *                    Plans depend on the multiprocessor count, which is looked up per device: ask with the device
+ *                    current on which the call will run.  No launch.
  */
 size_t bs_conv_workspace_bytes(const bs_conv_params* p);
 size_t bs_gemm_workspace_bytes(int M, int N, int K, int a_bits, bs_sign_t a_sign, int w_bits, bs_sign_t w_sign);
@@ -196,11 +198,16 @@ int bitserial_gemm_ws(const uint32_t* a_packed, const uint32_t* w_packed, int M,
  *   Shapes the planner does not split run the ordinary kernel and touch no scratch.
  *   First call on a device: looks up the device address of the built-in array (once per device, with that device
  *   current).  Make that first call before starting any stream capture.
- *   Sharing: all calls on a device use the same array, which keeps the previous call's contents; each call clears
- *   the part it needs on `stream` before its kernel.  Two calls that overlap on the GPU (different streams without
- *   ordering) race on the array and give wrong results; serialise them.
+ *   Sharing: all calls on a device use the same array, which keeps the previous call's contents.  A call that ran to
+ *   completion leaves the part it used zero again (the last block of a tile restores it), so the clearing each call
+ *   does on `stream` before its kernel is a guard against a predecessor that did NOT complete normally (one that ended
+ *   with BS_ERR_TIMEOUT) and against a caller that wrote to the array.  Two calls that overlap on the GPU (different
+ *   streams without ordering) race on the array and give wrong results; serialise them.
  */
 size_t bs_gemm_noalloc_max_scratch_bytes(void);
+/* Test aid (no counterpart in the paper): fills the built-in scratch with `byte_value` on `stream`, as a predecessor that
+ * ended half-way would leave it.  A following bitserial_gemm_noalloc on the same stream must still be exact. */
+int bs_selftest_dirty_noalloc_scratch(int byte_value, void* stream);
 int bitserial_gemm_noalloc(const uint32_t* a_packed, const uint32_t* w_packed, int M, int N, int K, int a_bits,
                            bs_sign_t a_sign, int w_bits, bs_sign_t w_sign, const float* scale, const float* bias,
                            int relu, int out_bits, bs_sign_t out_sign, int32_t* out_i32, uint32_t* out_packed,

@@ -75,6 +75,8 @@ def lib() -> ctypes.CDLL:
     L.bitserial_gemm_noalloc.argtypes = [vp, vp, i, i, i, i, i, i, i, vp, vp, i, i, i, vp, vp, vp]
     L.bs_gemm_noalloc_max_scratch_bytes.restype = ctypes.c_size_t
     L.bs_gemm_noalloc_max_scratch_bytes.argtypes = []
+    L.bs_selftest_dirty_noalloc_scratch.restype = i
+    L.bs_selftest_dirty_noalloc_scratch.argtypes = [i, vp]
     L.bs_tc_weights_bytes.restype = ctypes.c_size_t
     L.bs_tc_weights_bytes.argtypes = [i] * 4
     L.bs_tc_prepare_weights.restype = i
@@ -108,6 +110,6 @@ def lib() -> ctypes.CDLL:
 EXPORTED = ("bs_packed_act_bytes", "bs_packed_wgt_bytes", "bs_packed_rows_bytes", "bitpack_activations",
             "bitunpack_activations", "pack_weights", "bs_pack_rows", "bitserial_conv2d", "bitserial_gemm",
             "bitserial_conv2d_ws", "bitserial_gemm_ws", "bs_conv_workspace_bytes", "bs_gemm_workspace_bytes",
-            "bitserial_gemm_noalloc", "bs_gemm_noalloc_max_scratch_bytes",
+            "bitserial_gemm_noalloc", "bs_gemm_noalloc_max_scratch_bytes", "bs_selftest_dirty_noalloc_scratch",
             "bs_tc_weights_bytes", "bs_tc_prepare_weights", "bs_tc_supported", "bitserial_conv2d_tc", "bitserial_conv2d_tc_chained", "bitserial_gemm_tc", "bs_l2_prefetch",
             "bs_check_status", "bs_quantiser_bounds", "bs_requant_bounds", "bs_selftest_wait_timeout", "bs_popc_rate", "bs_status_string")

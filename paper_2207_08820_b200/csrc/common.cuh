@@ -10,6 +10,7 @@ namespace bs {
 // Device status word: kernels OR error bits into it when a bounded wait runs out.
 enum : int { STATUS_TIMEOUT = 1 };
 int* status_device_ptr();   // device address of the status word of the current device (host call)
+int device_sm_count();      // multiprocessors of the CURRENT device (looked up once per device ordinal; 0 on error)
 
 inline int ceil_div(int a, int b) { return (a + b - 1) / b; }
 inline long long ceil_div_ll(long long a, long long b) { return (a + b - 1) / b; }

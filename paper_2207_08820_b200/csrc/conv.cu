@@ -29,18 +29,6 @@ static EncodeTiledFn encode_fn()
     return fn;
 }
 
-static int sm_count()
-{
-    static int sms = 0;
-    if (sms == 0) {
-        int dev = 0;
-        if (cudaGetDevice(&dev) != cudaSuccess ||
-            cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms <= 0)
-            sms = 148;
-    }
-    return sms;
-}
-
 static int round_up(int v, int m) { return (v + m - 1) / m * m; }
 
 struct Plan {
@@ -109,10 +97,9 @@ static const int kTiles[][2] = {{8, 8}, {7, 8}, {4, 8}, {8, 4}, {7, 4}, {4, 4}, 
 //   - the busiest SM runs ceil(tiles / SMs) CTAs one after the other on its four sub-partitions;
 //   - fewer than 8 resident warps leave the pipe partly idle.
 static bool search_plan(Plan& best, int N, int P, int Q, int O, int Cw, int R, int S, int stride, int A, int WB,
-                        bool allow_split)
+                        bool allow_split, int sms)
 {
     const int RS = R * S;
-    const int sms = sm_count();
     const int pairs = A * WB;
     bool found = false;
     for (const auto& tile : kTiles) {
@@ -198,14 +185,17 @@ static bool make_plan(Plan& out, int N, int P, int Q, int O, int Cw, int R, int 
         }
     }
 #endif
-    static std::map<std::array<int, 11>, std::pair<bool, Plan>> cache;
+    // the plan (tiling, reduction split, workspace size) also depends on the multiprocessor count of the current device
+    const int sms = device_sm_count();
+    if (sms <= 0) return false;
+    static std::map<std::array<int, 12>, std::pair<bool, Plan>> cache;
     static std::mutex mu;
-    const std::array<int, 11> key = {N, P, Q, O, Cw, R, S, stride, A, WB, allow_split ? 1 : 0};
+    const std::array<int, 12> key = {N, P, Q, O, Cw, R, S, stride, A, WB, allow_split ? 1 : 0, sms};
     std::lock_guard<std::mutex> lock(mu);
     auto it = cache.find(key);
     if (it == cache.end()) {
         Plan pl{};
-        const bool ok = search_plan(pl, N, P, Q, O, Cw, R, S, stride, A, WB, allow_split);
+        const bool ok = search_plan(pl, N, P, Q, O, Cw, R, S, stride, A, WB, allow_split, sms);
         it = cache.emplace(key, std::make_pair(ok, pl)).first;
     }
     out = it->second.second;
@@ -475,10 +465,25 @@ extern "C" int bitserial_gemm_noalloc(const uint32_t* a_packed, const uint32_t* 
     if (need > 0) {
         scratch = bs::static_scratch_ptr(&st);
         if (!scratch) return st;
-        // the array keeps whatever the previous call left; partial sums and arrival counters must start at zero
+        // Partial sums and arrival counters must start at zero.  A call that completed leaves them zero again, so this
+        // clearing is defensive: it covers a predecessor that gave up on a bounded wait (BS_ERR_TIMEOUT) half-way.
         if (cudaMemsetAsync(scratch, 0, need, cs) != cudaSuccess) { cudaGetLastError(); return BS_ERR_CUDA; }
     }
     return bs::conv_impl(a_packed, w_packed, &p, out_i32, out_packed, scratch, need, cs);
+}
+
+// Test aid: fills the built-in scratch with a byte value, standing in for a predecessor that did not finish cleanly,
+// so that a test can show the clearing in bitserial_gemm_noalloc is what makes the next call right.
+extern "C" int bs_selftest_dirty_noalloc_scratch(int byte_value, void* stream)
+{
+    int st = BS_OK;
+    void* scratch = bs::static_scratch_ptr(&st);
+    if (!scratch) return st;
+    if (cudaMemsetAsync(scratch, byte_value & 0xFF, BS_STATIC_SCRATCH_BYTES, static_cast<cudaStream_t>(stream)) != cudaSuccess) {
+        cudaGetLastError();
+        return BS_ERR_CUDA;
+    }
+    return BS_OK;
 }
 
 // ---- self-test of the failure path: a wait that runs out ------------------------------------------------------------

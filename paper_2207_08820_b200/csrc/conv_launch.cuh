@@ -24,7 +24,8 @@ inline int launch_conv_one(const ConvArgs& args, unsigned grid, unsigned block, 
 template <int A, int WB, int FB>
 inline int launch_conv_pb(int PB, const ConvArgs& args, unsigned grid, unsigned block, size_t smem, cudaStream_t st)
 {
-#define BS_CASE(P_, F_) if (FB == F_ && PB == P_) return launch_conv_one<A, WB, P_, F_>(args, grid, block, smem, st);
+    // the filter block is a compile-time choice of the translation unit: only its own kernels are instantiated
+#define BS_CASE(P_, F_) if constexpr (FB == F_) { if (PB == P_) return launch_conv_one<A, WB, P_, F_>(args, grid, block, smem, st); }
     BS_TILE_LIST(BS_CASE)
 #undef BS_CASE
     return BS_ERR_UNSUPPORTED;

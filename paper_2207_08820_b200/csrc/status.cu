@@ -1,4 +1,6 @@
 // Device status word, status strings and the popcount-pipe micro-benchmark.
+#include <atomic>
+
 #include "common.cuh"
 
 namespace bs {
@@ -10,6 +12,24 @@ int* status_device_ptr()
     int* p = nullptr;
     if (cudaGetSymbolAddress(reinterpret_cast<void**>(&p), g_status) != cudaSuccess) return nullptr;
     return p;
+}
+
+// Multiprocessor count of the current device.  Tile plans depend on it, so it is kept per device ordinal: a process
+// that drives GPUs of different sizes gets the right plan on each.
+int device_sm_count()
+{
+    constexpr int kMax = 64;
+    static std::atomic<int> cache[kMax];
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0) { cudaGetLastError(); return 0; }
+    if (dev < kMax) {
+        const int c = cache[dev].load(std::memory_order_relaxed);
+        if (c > 0) return c;
+    }
+    int sms = 0;
+    if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms <= 0) { cudaGetLastError(); return 0; }
+    if (dev < kMax) cache[dev].store(sms, std::memory_order_relaxed);
+    return sms;
 }
 
 // Register-only chains of acc += popc(x & y).  Operands change every round so nothing folds.

@@ -67,6 +67,36 @@ struct TcArgs {
     RequantBounds rb;                 // comparison form of the epilogue (1- and 2-bit outputs)
 };
 
+// ----------------------------------------------------------------------------- timeline trace (tuning builds only)
+//
+// Built with -DBS_TUNING, the first 148 CTAs of a launch record the SM cycle counter at the hand-offs between their roles
+// (per tile, for the first 8 tiles); bs_tc_trace_read copies the table to the host.  Compiled out of the normal library.
+enum { TR_START = 0, TR_SETUP, TR_PDL, TR_WGT, TR_LOAD, TR_XBEG, TR_XEND, TR_MBEG, TR_MEND, TR_EBEG, TR_EEND, TR_END, TR_E_LD, TR_E_CMP,
+       TR_E_ST, TR_E_LOOP, TR_M_ISSUED, TR_X_DONE0, TR_X_BEG0 };
+#ifdef BS_TUNING
+constexpr int TC_TRACE_EVENTS = 24, TC_TRACE_TILES = 8, TC_TRACE_CTAS = 148;
+__device__ long long g_tc_trace[TC_TRACE_CTAS * TC_TRACE_EVENTS * TC_TRACE_TILES];
+__device__ __forceinline__ void tc_trace(int ev, int tile)
+{
+    if (blockIdx.x < TC_TRACE_CTAS && tile >= 0 && tile < TC_TRACE_TILES)
+        g_tc_trace[(blockIdx.x * TC_TRACE_EVENTS + ev) * TC_TRACE_TILES + tile] = clock64();
+}
+#define TC_TRACE(ev, tile) tc_trace(ev, tile)
+#else
+#define TC_TRACE(ev, tile) do { } while (0)
+#endif
+
+// Position in a ring of `n` stages guarded by mbarriers: stage index and phase bit, advanced without any division (a
+// division by a run-time ring size costs a lone issuing thread hundreds of cycles per hand-off).  A consumer waits for
+// full[idx] with `phase`; a producer waits for empty[idx] with `phase ^ 1`, which a freshly initialised barrier already
+// satisfies, so the first round needs no special case.
+struct TcRing {
+    int idx;
+    unsigned phase;
+    __device__ __forceinline__ TcRing() : idx(0), phase(0) {}
+    __device__ __forceinline__ void advance(int n) { if (++idx == n) { idx = 0; phase ^= 1u; } }
+};
+
 // ----------------------------------------------------------------------------- tcgen05 wrappers
 
 __device__ __forceinline__ void mbar_arrive(uint64_t* bar)
@@ -75,12 +105,13 @@ __device__ __forceinline__ void mbar_arrive(uint64_t* bar)
 }
 // Barrier among the threads of one warp group (expanders or epilogue); ids 1 and 2, id 0 is __syncthreads.
 __device__ __forceinline__ void group_sync(int id, int nthreads = 128) { asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(nthreads) : "memory"); }
-// Low-latency bounded wait for the tensor-core pipeline: non-blocking test_wait in a spin loop (try_wait may park the
-// thread and wake it late, which costs microseconds per hand-off between the roles).  About a second at most.
+// Bounded wait for the tensor-core pipeline: try_wait parks the thread for at most ~2 us per attempt (measured: a
+// shorter hint, no hint or a test_wait spin make no difference to the layer times); 2^20 attempts bound a wait that
+// nothing satisfies to about two seconds, after which the caller sets the status word and the CTA drains.
 __device__ __forceinline__ bool mbar_spin_bounded(uint64_t* bar, unsigned parity)
 {
     const uint32_t addr = smem_u32(bar);
-    for (unsigned it = 0; it < (1u << 24); ++it) {
+    for (unsigned it = 0; it < (1u << 20); ++it) {
         unsigned ok;
         asm volatile(
             "{\n\t.reg .pred p;\n\t"
@@ -186,6 +217,40 @@ __device__ __forceinline__ TcTile tc_decode_tile(const TcArgs& g, int mt)
     t.p0 = (mt % g.tiles_p) * 16;                    mt /= g.tiles_p;
     t.n0 = mt * g.TNI;
     return t;
+}
+
+// Walks the pixel tiles first, first + step, ... of a CTA: the decomposition of the step is found once, each further
+// tile costs a few additions and carries instead of two divisions.
+struct TcTileWalker {
+    int iq, ip, in;            // tile coordinates
+    int dq, dp, dn;            // decomposition of the step
+    int mt;                    // linear tile index
+    int step;
+};
+
+__device__ __forceinline__ TcTileWalker tc_walk_init(const TcArgs& g, int first, int step)
+{
+    TcTileWalker w;
+    w.mt = first; w.step = step;
+    int t = first;
+    w.iq = t % g.tiles_q; t /= g.tiles_q; w.ip = t % g.tiles_p; w.in = t / g.tiles_p;
+    t = step;
+    w.dq = t % g.tiles_q; t /= g.tiles_q; w.dp = t % g.tiles_p; w.dn = t / g.tiles_p;
+    return w;
+}
+__device__ __forceinline__ TcTile tc_walk_tile(const TcArgs& g, const TcTileWalker& w)
+{
+    TcTile t;
+    if (g.flat) { t.q0 = w.mt * TC_M; t.p0 = 0; t.n0 = 0; return t; }
+    t.q0 = w.iq * 8; t.p0 = w.ip * 16; t.n0 = w.in * g.TNI;
+    return t;
+}
+__device__ __forceinline__ void tc_walk_next(const TcArgs& g, TcTileWalker& w)
+{
+    w.mt += w.step;
+    w.iq += w.dq; w.ip += w.dp; w.in += w.dn;
+    if (w.iq >= g.tiles_q) { w.iq -= g.tiles_q; ++w.ip; }
+    if (w.ip >= g.tiles_p) { w.ip -= g.tiles_p; ++w.in; }
 }
 
 // Fetch the packed halo of one tile (whole pixel records, all channel chunks) and arm `bar` with its byte count.
@@ -629,9 +694,23 @@ __device__ __forceinline__ void tc_epilogue_tables(const TcArgs& g, unsigned cha
     if (t == 32 && g.off_thr) *reinterpret_cast<int*>(tc_smem + g.off_thr + g.thr_pats * g.TN * 16) = 1;
 }
 
+// Where accumulator row m (= tensor-memory lane = tile pixel) sits inside a 2-D tile: image of the stack, row, column.
+// Depends on the thread only, so it is found once per kernel (stacked small images need a division).
+struct TcEpiThread { int ni, ty, tx; };
+
+__device__ __forceinline__ TcEpiThread tc_epi_thread(const TcArgs& g, int m)
+{
+    TcEpiThread t;
+    const int grp = m >> 3;
+    t.tx = m & 7; t.ni = 0; t.ty = grp;
+    if (!g.flat && g.GI != 16) { t.ni = grp / g.GI; t.ty = grp - t.ni * g.GI; }
+    return t;
+}
+
 // Epilogue of one tile: thread `tid` (0..127, warp = TMEM lane quadrant) owns accumulator row tid = one output pixel.
-__device__ __forceinline__ void tc_epilogue_tile(const TcArgs& g, uint32_t tmem_acc, int tid, int warp, const TcTile& tile, int o0,
-                                                 const float2* s_sb, const float4* s_bounds, uint32_t thr_addr, int cc0 = 0, int ccstep = 1)
+__device__ __forceinline__ void tc_epilogue_tile(const TcArgs& g, uint32_t tmem_acc, int tid, int warp, const TcTile& tile, const TcEpiThread& et,
+                                                 int o0, const float2* s_sb, const float4* s_bounds, uint32_t thr_addr, int cc0 = 0,
+                                                 int ccstep = 1, int trace_tile = -1)
 {
     const int n0 = tile.n0, p0 = tile.p0, q0 = tile.q0;
     const int m = tid;                               // TMEM lane = tile pixel
@@ -652,9 +731,7 @@ __device__ __forceinline__ void tc_epilogue_tile(const TcArgs& g, uint32_t tmem_
             q = static_cast<int>(rem - static_cast<unsigned>(p) * static_cast<unsigned>(g.Q));
         }
     } else {
-        const int grp = m >> 3, tx = m & 7;
-        int ni = 0, ty = grp;
-        if (g.GI != 16) { ni = grp / g.GI; ty = grp - ni * g.GI; }          // stacked small images
+        const int ni = et.ni, ty = et.ty, tx = et.tx;                        // stacked small images: ni > 0
         n = n0 + ni; p = p0 + ty; q = q0 + tx;
         valid = n < g.N && p < g.P && q < g.Q && ni < g.TNI && (g.GI == 16 || ty < g.P);
         pix = (static_cast<size_t>(n) * g.P + p) * g.Q + q;
@@ -667,6 +744,7 @@ __device__ __forceinline__ void tc_epilogue_tile(const TcArgs& g, uint32_t tmem_
         uint32_t v[32];
         tmem_ld32(tmem_acc + (static_cast<uint32_t>(warp * 32) << 16) + static_cast<uint32_t>(cc * 32), v);
         tmem_ld_wait();
+        if (tid == 0 && cc == cc0) TC_TRACE(TR_E_LD, trace_tile);
         const int ob = o0 + cc * 32;
         if (valid && ob < g.O) {
         if (g.out_i32) {
@@ -742,6 +820,7 @@ __device__ __forceinline__ void tc_epilogue_tile(const TcArgs& g, uint32_t tmem_
         }
         }
         __syncwarp();                 // the next tcgen05.ld is warp-collective
+        if (tid == 0 && cc == cc0) TC_TRACE(TR_E_ST, trace_tile);
     }
 }
 
@@ -801,19 +880,20 @@ __global__ void __launch_bounds__(TC_THREADS) bitserial_conv_tc_kernel(const __g
         if (lane == 0) {
             // the first ring of filter chunks does not depend on the preceding kernel: fetch it before waiting for it
             const int early = g.nchunks < g.nsp ? g.nchunks : g.nsp;
+            const int blk_bytes = g.b_bytes / g.MB;
+            const size_t blk_stride = static_cast<size_t>(g.opad8) * RS * (g.CK >> 4) * 128;      // one layout block, all filters
+            const int8_t* src = g.wgt + static_cast<size_t>(o0 >> 3) * RS * (g.CK >> 4) * 128;
+            TcRing rp;
             for (int c = 0; c < g.nchunks; ++c) {
-                const int s = c % g.nsp, k = c / g.nsp;
                 if (c == early) {
                     pdl_acquire();
                     for (int t = 0; t < nt; ++t) tc_load_tile(g, tc_smem + g.off_p + t * g.pa_bytes, full_a, tc_decode_tile(g, mt0 + t));
                 }
-                if (k >= 1 && !mbar_spin_bounded(&empty_p[s], (k - 1) & 1)) { atomicOr(g.status, STATUS_TIMEOUT); break; }
-                mbar_expect_tx(&full_p[s], static_cast<unsigned>(g.b_bytes));
-                const int blk_bytes = g.b_bytes / g.MB;
-                for (int j = 0; j < g.MB; ++j) {
-                    const size_t src = (static_cast<size_t>(c * g.MB + j) * g.opad8 + (o0 >> 3)) * RS * (g.CK >> 4) * 128;
-                    bulk_load(tc_smem + s * stage_p_bytes + j * blk_bytes, g.wgt + src, static_cast<unsigned>(blk_bytes), &full_p[s]);
-                }
+                if (!mbar_spin_bounded(&empty_p[rp.idx], rp.phase ^ 1u)) { atomicOr(g.status, STATUS_TIMEOUT); break; }
+                mbar_expect_tx(&full_p[rp.idx], static_cast<unsigned>(g.b_bytes));
+                for (int j = 0; j < g.MB; ++j, src += blk_stride)
+                    bulk_load(tc_smem + rp.idx * stage_p_bytes + j * blk_bytes, src, static_cast<unsigned>(blk_bytes), &full_p[rp.idx]);
+                rp.advance(g.nsp);
             }
             if (early == g.nchunks) {
                 pdl_acquire();
@@ -824,20 +904,22 @@ __global__ void __launch_bounds__(TC_THREADS) bitserial_conv_tc_kernel(const __g
     } else if (warp == 5) {
         // ------------------------------------------------------------------ MMA issuer
         if (lane == 0) {
-            const uint32_t e_base = smem_u32(tc_smem + g.off_e);
+            const uint32_t e_base = smem_u32(tc_smem + g.off_e), p_base = smem_u32(tc_smem);
             const TcIssue is = tc_make_issue(g);
+            TcRing rp, re;
             for (int c = 0; c < g.nchunks; ++c) {
-                const int s = c % g.nsp, e = c % g.nse;
-                if (!(mbar_spin_bounded(&full_p[s], (c / g.nsp) & 1) && mbar_spin_bounded(&full_e[e], (c / g.nse) & 1))) {
+                if (!(mbar_spin_bounded(&full_p[rp.idx], rp.phase) && mbar_spin_bounded(&full_e[re.idx], re.phase))) {
                     atomicOr(g.status, STATUS_TIMEOUT);
                     break;
                 }
                 tc_fence_after();
                 for (int t = 0; t < nt; ++t)
-                    tc_issue_chunk(is, e_base + static_cast<uint32_t>(e * e_stage + t * g.e_bytes), smem_u32(tc_smem + s * stage_p_bytes),
+                    tc_issue_chunk(is, e_base + static_cast<uint32_t>(re.idx * e_stage + t * g.e_bytes), p_base + static_cast<uint32_t>(rp.idx * stage_p_bytes),
                                    tmem_base + static_cast<uint32_t>(t * g.TN), c == 0);
-                umma_commit(&empty_e[e]);
-                umma_commit(&empty_p[s]);
+                umma_commit(&empty_e[re.idx]);
+                umma_commit(&empty_p[rp.idx]);
+                rp.advance(g.nsp);
+                re.advance(g.nse);
             }
             umma_commit(accum_full);      // arrives when every MMA issued above has completed
         }
@@ -850,17 +932,19 @@ __global__ void __launch_bounds__(TC_THREADS) bitserial_conv_tc_kernel(const __g
         tc_epilogue_tables(g, tc_smem, s_sb, s_bounds, o0, ct, TC_WORKERS);
         group_sync(1, TC_WORKERS);
         const TcExpand xp = tc_expand_init(g, ct, TC_WORKERS);
+        const TcEpiThread eth = tc_epi_thread(g, (warp & 3) * 32 + lane);
         bool ok = mbar_wait_warp(full_a, 0, lane);
+        TcRing re;
         for (int c = 0; c < g.nchunks; ++c) {
-            const int e = c % g.nse, k = c / g.nse;
-            if (ok && k >= 1) ok = mbar_wait_warp(&empty_e[e], (k - 1) & 1, lane);
+            if (ok) ok = mbar_wait_warp(&empty_e[re.idx], re.phase ^ 1u, lane);
             if (!ok) atomicOr(g.status, STATUS_TIMEOUT);
             for (int t = 0; t < nt; ++t)
                 tc_expand_chunk<A>(g, xp, reinterpret_cast<const uint32_t*>(tc_smem + g.off_p + t * g.pa_bytes),
-                                   tc_smem + g.off_e + e * e_stage + t * g.e_bytes, s_lut, ct, c);
+                                   tc_smem + g.off_e + re.idx * e_stage + t * g.e_bytes, s_lut, ct, c);
             fence_proxy_async();          // make the generic-proxy writes visible to the tensor core's reads
             group_sync(1, TC_WORKERS);
-            if (tid == 0) mbar_arrive(&full_e[e]);
+            if (tid == 0) mbar_arrive(&full_e[re.idx]);
+            re.advance(g.nse);
         }
         // the last chunks are still in the tensor core: time to turn the comparison bounds into integer thresholds
         uint32_t thr = 0;                 // shared-memory address of the thresholds, 0: floating-point comparison
@@ -877,7 +961,7 @@ __global__ void __launch_bounds__(TC_THREADS) bitserial_conv_tc_kernel(const __g
         for (int t = 0; t < nt; ++t)
             // a warp reads the tensor-memory lanes of quadrant (warp % 4): warps 0-3 take the even groups of 32 filters,
             // warps 6-9 (quadrants 2, 3, 0, 1) the odd ones
-            tc_epilogue_tile(g, tmem_base + static_cast<uint32_t>(t * g.TN), (warp & 3) * 32 + lane, warp & 3, tc_decode_tile(g, mt0 + t), o0,
+            tc_epilogue_tile(g, tmem_base + static_cast<uint32_t>(t * g.TN), (warp & 3) * 32 + lane, warp & 3, tc_decode_tile(g, mt0 + t), eth, o0,
                              s_sb, s_bounds, thr, warp < 4 ? 0 : 1, 2);
         tc_fence_before();
     }
@@ -931,6 +1015,7 @@ bitserial_conv_tc_persistent_kernel(const __grid_constant__ TcArgs g)
     const int tile_step = static_cast<int>(gridDim.x / static_cast<unsigned>(g.tiles_o));
     const int tiles_m = g.tiles_q * g.tiles_p * g.tiles_n;
 
+    if (tid == 0) TC_TRACE(TR_START, 0);
     pdl_release();
     if (tid == 0) {
         for (int s = 0; s < TCP_NSP; ++s) { mbar_init(&full_p[s], 1); mbar_init(&empty_p[s], 1); }
@@ -956,17 +1041,22 @@ bitserial_conv_tc_persistent_kernel(const __grid_constant__ TcArgs g)
         if (lane == 0) {
             mbar_expect_tx(wgt_full, static_cast<unsigned>(g.nchunks * g.b_bytes));
             const int blk_bytes = g.b_bytes / g.MB;
-            for (int c = 0; c < g.nchunks * g.MB; ++c) {       // layout blocks, consecutive in shared memory
-                const size_t src = (static_cast<size_t>(c) * g.opad8 + (o0 >> 3)) * RS * (g.CK >> 4) * 128;
-                bulk_load(s_w + static_cast<size_t>(c) * blk_bytes, g.wgt + src, static_cast<unsigned>(blk_bytes), wgt_full);
-            }
+            const size_t blk_stride = static_cast<size_t>(g.opad8) * RS * (g.CK >> 4) * 128;      // one layout block, all filters
+            const int8_t* src = g.wgt + static_cast<size_t>(o0 >> 3) * RS * (g.CK >> 4) * 128;
+            unsigned char* dst = s_w;
+            for (int c = 0; c < g.nchunks * g.MB; ++c, src += blk_stride, dst += blk_bytes)       // layout blocks, consecutive in shared memory
+                bulk_load(dst, src, static_cast<unsigned>(blk_bytes), wgt_full);
+            TC_TRACE(TR_SETUP, 0);
             pdl_acquire();                // activations come from the preceding kernel; the filters above do not
-            int i = 0;
+            TC_TRACE(TR_PDL, 0);
+            TcTileWalker tw = tc_walk_init(g, first_tile, tile_step);
+            TcRing rp;
             bool ok = true;
-            for (int mt = first_tile; mt < tiles_m && ok; mt += tile_step, ++i) {
-                const int s = i % g.nsp, k = i / g.nsp;
-                if (k >= 1 && !mbar_spin_bounded(&empty_p[s], (k - 1) & 1)) { ok = false; break; }
-                tc_load_tile(g, s_p + s * g.pa_bytes, &full_p[s], tc_decode_tile(g, mt));
+            for (int i = 0; tw.mt < tiles_m; tc_walk_next(g, tw), ++i) {
+                if (!mbar_spin_bounded(&empty_p[rp.idx], rp.phase ^ 1u)) { ok = false; break; }
+                TC_TRACE(TR_LOAD, i);
+                tc_load_tile(g, s_p + rp.idx * g.pa_bytes, &full_p[rp.idx], tc_walk_tile(g, tw));
+                rp.advance(g.nsp);
             }
             if (!ok) atomicOr(g.status, STATUS_TIMEOUT);
         }
@@ -975,22 +1065,32 @@ bitserial_conv_tc_persistent_kernel(const __grid_constant__ TcArgs g)
         // ------------------------------------------------------------------ MMA issuer
         if (lane == 0) {
             const TcIssue is = tc_make_issue(g);
+            const uint32_t e_base = smem_u32(s_e), w_base = smem_u32(s_w);
             bool ok = mbar_spin_bounded(wgt_full, 0);       // also keeps the CTA alive until the filter copy has landed
-            int it = 0, i = 0;
+            TC_TRACE(TR_WGT, 0);
+            TcRing re, ra;                                  // expanded chunks; accumulator buffers
+            int i = 0;
             for (int mt = first_tile; mt < tiles_m && ok; mt += tile_step, ++i) {
-                const int buf = i & 1, use = i >> 1;
-                if (use >= 1) ok = mbar_spin_bounded(&empty_acc[buf], (use - 1) & 1);
+                ok = mbar_spin_bounded(&empty_acc[ra.idx], ra.phase ^ 1u);
                 if (!ok) break;
                 tc_fence_after();
-                const uint32_t tmem_acc = tmem_base + static_cast<uint32_t>(buf * g.TN);
-                for (int c = 0; c < g.nchunks; ++c, ++it) {
-                    const int e = it % g.nse;
-                    if (!mbar_spin_bounded(&full_e[e], (it / g.nse) & 1)) { ok = false; break; }
+                const uint32_t tmem_acc = tmem_base + static_cast<uint32_t>(ra.idx * g.TN);
+                uint32_t wa = w_base;
+                for (int c = 0; c < g.nchunks; ++c, wa += static_cast<uint32_t>(g.b_bytes)) {
+                    if (!mbar_spin_bounded(&full_e[re.idx], re.phase)) { ok = false; break; }
+                    if (c == 0) TC_TRACE(TR_MBEG, i);
                     tc_fence_after();
-                    tc_issue_chunk(is, smem_u32(s_e + e * g.e_bytes), smem_u32(s_w + static_cast<size_t>(c) * g.b_bytes), tmem_acc, c == 0);
-                    umma_commit(&empty_e[e]);
+                    tc_issue_chunk(is, e_base + static_cast<uint32_t>(re.idx * g.e_bytes), wa, tmem_acc, c == 0);
+                    if (c == 0) TC_TRACE(TR_M_ISSUED, i);
+#ifdef BS_TC_DBG_DRAIN
+                    if (c == 0 && i < 2) { umma_commit(wgt_full); mbar_spin_bounded(wgt_full, (i + 1) & 1); TC_TRACE(19, i); }
+#endif
+                    umma_commit(&empty_e[re.idx]);
+                    re.advance(g.nse);
                 }
-                if (ok) umma_commit(&full_acc[buf]);
+                if (ok) umma_commit(&full_acc[ra.idx]);
+                TC_TRACE(TR_MEND, i);
+                ra.advance(2);
             }
             if (!ok) atomicOr(g.status, STATUS_TIMEOUT);
         }
@@ -1001,22 +1101,28 @@ bitserial_conv_tc_persistent_kernel(const __grid_constant__ TcArgs g)
         tc_build_lut(g, s_lut, et, 128);
         group_sync(1);
         const TcExpand xp = tc_expand_init(g, et, 128);
-        int it = 0, i = 0;
+        TcRing rp, re;
+        int i = 0;
         bool ok = true;
         for (int mt = first_tile; mt < tiles_m && ok; mt += tile_step, ++i) {
-            const int s = i % g.nsp;
-            ok = mbar_wait_warp(&full_p[s], (i / g.nsp) & 1, lane);
-            for (int c = 0; c < g.nchunks; ++c, ++it) {
-                const int e = it % g.nse, k = it / g.nse;
-                if (ok && k >= 1) ok = mbar_wait_warp(&empty_e[e], (k - 1) & 1, lane);
+            ok = mbar_wait_warp(&full_p[rp.idx], rp.phase, lane);
+            if (et == 0) TC_TRACE(TR_XBEG, i);
+            const uint32_t* pa = reinterpret_cast<const uint32_t*>(s_p + rp.idx * g.pa_bytes);
+            for (int c = 0; c < g.nchunks; ++c) {
+                if (ok) ok = mbar_wait_warp(&empty_e[re.idx], re.phase ^ 1u, lane);
                 ok = group_all(1, ok);
                 if (!ok) break;
-                tc_expand_chunk<A>(g, xp, reinterpret_cast<const uint32_t*>(s_p + s * g.pa_bytes), s_e + e * g.e_bytes, s_lut, et, c);
+                if (et == 0 && c == 0) TC_TRACE(TR_X_BEG0, i);
+                tc_expand_chunk<A>(g, xp, pa, s_e + re.idx * g.e_bytes, s_lut, et, c);
                 fence_proxy_async();
                 group_sync(1);                       // all 128 expander threads have written and fenced
-                if (et == 0) mbar_arrive(&full_e[e]);
+                if (et == 0 && c == 0) TC_TRACE(TR_X_DONE0, i);
+                if (et == 0) mbar_arrive(&full_e[re.idx]);
+                re.advance(g.nse);
             }
-            if (ok && et == 0) mbar_arrive(&empty_p[s]);   // ordered after the last group_sync: every thread is done reading
+            if (et == 0) TC_TRACE(TR_XEND, i);
+            if (ok && et == 0) mbar_arrive(&empty_p[rp.idx]);   // ordered after the last group_sync: every thread is done reading
+            rp.advance(g.nsp);
         }
         if (!ok) atomicOr(g.status, STATUS_TIMEOUT);
     } else {
@@ -1034,25 +1140,29 @@ bitserial_conv_tc_persistent_kernel(const __grid_constant__ TcArgs g)
             group_sync(2, EPI_THREADS);
             if (*thr_ok) thr = smem_u32(s_thr);
         }
+        const TcEpiThread eth = tc_epi_thread(g, (warp & 3) * 32 + lane);
+        TcTileWalker tw = tc_walk_init(g, first_tile, tile_step);
         pdl_acquire();                    // the epilogue reads the residual and overwrites buffers the preceding kernel may use
-        int i = 0;
+        TcRing ra;
         bool ok = true;
-        for (int mt = first_tile; mt < tiles_m && ok; mt += tile_step, ++i) {
-            const int buf = i & 1, use = i >> 1;
-            ok = group_all(2, mbar_wait_warp(&full_acc[buf], use & 1, lane), EPI_THREADS);
+        for (int i = 0; tw.mt < tiles_m; tc_walk_next(g, tw), ++i) {
+            ok = group_all(2, mbar_wait_warp(&full_acc[ra.idx], ra.phase, lane), EPI_THREADS);
             if (!ok) break;
+            if (tid == 0) TC_TRACE(TR_EBEG, i);
             tc_fence_after();
-            const TcTile tile = tc_decode_tile(g, mt);
-            tc_epilogue_tile(g, tmem_base + static_cast<uint32_t>(buf * g.TN), (warp & 3) * 32 + lane, warp & 3, tile, o0, s_sb, s_bounds, thr,
-                             WIDE ? second : 0, WIDE ? 2 : 1);
+            tc_epilogue_tile(g, tmem_base + static_cast<uint32_t>(ra.idx * g.TN), (warp & 3) * 32 + lane, warp & 3, tc_walk_tile(g, tw), eth, o0,
+                             s_sb, s_bounds, thr, WIDE ? second : 0, WIDE ? 2 : 1, i);
             tc_fence_before();
             group_sync(2, EPI_THREADS);              // every epilogue warp has read its accumulator rows
-            if (tid == 0) mbar_arrive(&empty_acc[buf]);
+            if (tid == 0) TC_TRACE(TR_EEND, i);
+            if (tid == 0) mbar_arrive(&empty_acc[ra.idx]);
+            ra.advance(2);
         }
         if (!ok) atomicOr(g.status, STATUS_TIMEOUT);
     }
     tc_fence_before();
     __syncthreads();
+    if (tid == 0) TC_TRACE(TR_END, 0);
     if (warp == 9) {
         tc_fence_after();
         tmem_dealloc(tmem_base, static_cast<unsigned>(g.tmem_cols));
@@ -1277,7 +1387,8 @@ static int tc_conv_impl(const uint32_t* act, const int8_t* wgt, const bs_conv_pa
     }
     g.pa_bytes = round_up_i(g.pa_tx_bytes, 128);
     g.e_bytes = round_up_i((CKP / 16) * g.HPE * 16, 128);
-    const int sms = 148;
+    const int sms = device_sm_count();
+    if (sms <= 0) return BS_ERR_CUDA;
     // Persistent plan: the filters of a tile (all channel chunks) stay resident in shared memory.  Largest filter tile
     // that fits and still leaves one (pixel tile, filter tile) pair per SM.
     size_t smem = 0;
@@ -1494,6 +1605,20 @@ static int tc_conv_impl(const uint32_t* act, const int8_t* wgt, const bs_conv_pa
 }
 
 }  // namespace bs
+
+#ifdef BS_TUNING
+// Tuning builds: copies the timeline table of the last tensor-core launches to `out` (HOST, 148 x 24 x 8 cycle counts).
+extern "C" int bs_tc_trace_read(long long* out, int clear)
+{
+    if (cudaDeviceSynchronize() != cudaSuccess) return BS_ERR_CUDA;
+    if (cudaMemcpyFromSymbol(out, bs::g_tc_trace, sizeof(bs::g_tc_trace)) != cudaSuccess) return BS_ERR_CUDA;
+    if (clear) {
+        void* p = nullptr;
+        if (cudaGetSymbolAddress(&p, bs::g_tc_trace) != cudaSuccess || cudaMemset(p, 0, sizeof(bs::g_tc_trace)) != cudaSuccess) return BS_ERR_CUDA;
+    }
+    return BS_OK;
+}
+#endif
 
 extern "C" size_t bs_tc_weights_bytes(int O, int C, int R, int S)
 {

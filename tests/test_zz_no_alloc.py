@@ -1,20 +1,25 @@
-"""`bitserial_gemm_noalloc` against `bitserial_gemm`, through the C ABI.
+"""`bitserial_gemm_noalloc` against `bitserial_gemm` and against the CPU oracle, through the C ABI.
 
 The no-allocation entry point exists for callers that are not allowed to call cudaMalloc (a host that gave all
 device memory to its own pool, an inference loop that must not allocate after start-up, a plugin inside someone
 else's stream).  It keeps its scratch in an array built into the library, shared by every call, so the test runs
-it twice in a row on different data: the second call must not see anything the first one left behind.  Outputs
-must equal the ordinary entry point's exactly (integer accumulators and packed codes; the GPU tests' tolerance
-for codes is at most 1e-4 of elements off by one level, and equality satisfies it).
+it several times in a row on different data and on shapes with different split plans.  Outputs must equal the
+ordinary entry point's exactly, and both must equal the oracle's integer product and requantised codes (integer
+accumulators and packed codes; the GPU tests' tolerance for codes is at most 1e-4 of elements off by one level,
+and equality satisfies it).
+
+A call that completes leaves the scratch zero again, so back-to-back calls alone would also pass without the
+clearing the entry point does before its kernel.  One case therefore fills the built-in array with a byte
+pattern first (the library's test aid), as a predecessor that ended half-way would leave it: only the clearing
+makes the call after that exact.
 
 This file is named to be collected last, so a run that stops at the first failure has already run everything else.
 """
-import ctypes
-
 import numpy as np
 import pytest
 import torch
 
+import oracle
 from paper_2207_08820_b200 import workloads as wl
 from paper_2207_08820_b200._lib import lib
 
@@ -44,21 +49,48 @@ def _run(L, fn, ap, wp, M, N, K, scale, bias):
     return acc, packed
 
 
-def test_noalloc_matches_regular_entry_point_twice_in_a_row():
+def _check_case(L, M, N, K, seed, dirty=None):
+    c = wl.gemm_case(M, N, K, seed=seed)
+    scale, bias = wl.calibrated_scale_bias(c["w"], 2, 0, 2)
+    ap, wp = _pack_rows(L, c["a"], 2, 0), _pack_rows(L, c["w"], 1, 2)
+    sc, bi = _dev(scale), _dev(bias)
+    want_acc, want_packed = _run(L, L.bitserial_gemm, ap, wp, M, N, K, sc, bi)
+    if dirty is not None:
+        assert L.bs_selftest_dirty_noalloc_scratch(dirty, None) == 0
+    got_acc, got_packed = _run(L, L.bitserial_gemm_noalloc, ap, wp, M, N, K, sc, bi)
+    assert torch.equal(got_acc, want_acc)
+    assert torch.equal(got_packed, want_packed)
+    # and against the oracle: plain integer product, then the epilogue formula and the plane split
+    acc = oracle.gemm_i32(c["a"], c["w"])
+    assert np.array_equal(got_acc.cpu().numpy(), acc)
+    codes = oracle.requantize(acc, scale, bias, True, 2, oracle.UNSIGNED, channel_axis=1)
+    assert len(np.unique(codes)) == 4                     # all four levels in use: the epilogue check has teeth
+    assert np.array_equal(got_packed.cpu().numpy().view(np.uint32).reshape(M, -1, 2), oracle.pack_rows(codes, 2, oracle.UNSIGNED))
+    assert len(np.unique(acc)) > 100                      # a real product, not a constant
+
+
+def test_noalloc_matches_regular_entry_point_and_oracle_on_calls_in_a_row():
     L = lib()
     assert L.bs_gemm_noalloc_max_scratch_bytes() == 2 * 1024 * 1024
-    M, N, K = 256, 256, 4608                  # few output tiles, long reduction: the planner splits it
-    assert 0 < L.bs_gemm_workspace_bytes(M, N, K, 2, 0, 1, 2) <= L.bs_gemm_noalloc_max_scratch_bytes()
-    for seed in (11, 12):                     # two calls in a row, different data, same built-in scratch
-        c = wl.gemm_case(M, N, K, seed=seed)
-        scale, bias = wl.calibrated_scale_bias(c["w"], 2, 0, 2)
-        ap, wp = _pack_rows(L, c["a"], 2, 0), _pack_rows(L, c["w"], 1, 2)
-        sc, bi = _dev(scale), _dev(bias)
-        want_acc, want_packed = _run(L, L.bitserial_gemm, ap, wp, M, N, K, sc, bi)
-        got_acc, got_packed = _run(L, L.bitserial_gemm_noalloc, ap, wp, M, N, K, sc, bi)
-        assert torch.equal(got_acc, want_acc)
-        assert torch.equal(got_packed, want_packed)
-        assert len(torch.unique(want_acc)) > 100          # a real product, not a constant
+    shapes = [(256, 256, 4608), (256, 256, 4608), (128, 320, 2304), (96, 64, 9216)]   # few output tiles, long reductions
+    split = 0
+    for k, (M, N, K) in enumerate(shapes):    # calls in a row, different data and plans, same built-in scratch
+        need = L.bs_gemm_workspace_bytes(M, N, K, 2, 0, 1, 2)
+        assert need <= L.bs_gemm_noalloc_max_scratch_bytes()
+        split += need > 0
+        _check_case(L, M, N, K, seed=11 + k)
+    assert split >= 2                         # the planner really split (and used the scratch for) several of them
+
+
+@pytest.mark.parametrize("byte", [0xFF, 0x01])
+def test_noalloc_clears_a_dirty_scratch(byte):
+    """The built-in array is filled with a byte pattern before the call: partial sums would start from garbage and
+    the arrival counters would never reach their target unless the entry point cleared what it uses."""
+    L = lib()
+    M, N, K = 256, 256, 4608
+    assert L.bs_gemm_workspace_bytes(M, N, K, 2, 0, 1, 2) > 0
+    _check_case(L, M, N, K, seed=21, dirty=byte)
+    _check_case(L, M, N, K, seed=22)          # and an undisturbed call right after it
 
 
 def test_noalloc_rejects_shapes_beyond_the_builtin_scratch():
