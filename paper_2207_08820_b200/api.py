@@ -206,12 +206,17 @@ def tc_supported(N, C, H, W, O, k, stride, pad, a_bits, a_sign, w_bits, w_sign) 
 
 def bitserial_gemm_tc(a_packed: torch.Tensor, w_tc: torch.Tensor, N: int, K: int, w_bits: int, *, a_sign: int = UNSIGNED,
                       w_sign: int = SIGNED, scale=None, bias=None, relu: bool = False, out_bits: int = 0,
-                      out_sign: int = UNSIGNED, want_i32: bool = True, stream=None):
+                      out_sign: int = UNSIGNED, want_i32: bool = True, out_i32: Optional[torch.Tensor] = None,
+                      out_packed: Optional[torch.Tensor] = None, stream=None):
     """Tensor-core matrix product: a_packed [M,Kw,a_bits], w_tc from tc_prepare_weights on the [N,1,1,Kw,w_bits] rows."""
     M, Kw, a_bits = a_packed.shape
     dev = a_packed.device
-    out_i32 = torch.empty(M, N, dtype=torch.int32, device=dev) if want_i32 else None
-    out_packed = torch.zeros(M, (N + 31) // 32, out_bits, dtype=torch.int32, device=dev) if out_bits > 0 else None
+    if want_i32 and out_i32 is None:
+        out_i32 = torch.empty(M, N, dtype=torch.int32, device=dev)
+    if out_bits > 0 and out_packed is None:
+        out_packed = torch.zeros(M, (N + 31) // 32, out_bits, dtype=torch.int32, device=dev)
+    if out_bits <= 0:
+        out_packed = None
     st = lib().bitserial_gemm_tc(_ptr(a_packed), _ptr(w_tc), M, N, K, a_bits, a_sign, w_bits, w_sign, _ptr(scale), _ptr(bias),
                                  int(relu), out_bits, out_sign, _ptr(out_i32), _ptr(out_packed), _stream_ptr(stream))
     _check(st, "bitserial_gemm_tc")

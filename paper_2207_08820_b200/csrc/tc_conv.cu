@@ -1280,14 +1280,17 @@ static cudaError_t tc_launch(void (*kern)(TcArgs), unsigned grid, unsigned block
     return cudaLaunchKernelEx(&cfg, kern, g);
 }
 
+// plan_only: validate and plan (tiles, shared memory) without touching any tensor or launching: the support query.
 static int tc_conv_impl(const uint32_t* act, const int8_t* wgt, const bs_conv_params* p, int32_t* out_i32, uint32_t* out_packed,
-                        cudaStream_t st, bool chained = false)
+                        cudaStream_t st, bool chained = false, bool plan_only = false)
 {
     int rc = tc_validate(p);
     if (rc != BS_OK) return rc;
-    if (!act || !wgt || (!out_i32 && !out_packed)) return BS_ERR_INVALID_ARG;
-    if (!aligned16(act) || !aligned16(wgt) || (out_i32 && !aligned16(out_i32)) || (out_packed && !aligned16(out_packed)))
-        return BS_ERR_ALIGNMENT;
+    if (!plan_only) {
+        if (!act || !wgt || (!out_i32 && !out_packed)) return BS_ERR_INVALID_ARG;
+        if (!aligned16(act) || !aligned16(wgt) || (out_i32 && !aligned16(out_i32)) || (out_packed && !aligned16(out_packed)))
+            return BS_ERR_ALIGNMENT;
+    }
     TcArgs g{};
     g.P = (p->H + 2 * p->pad - p->R) / p->stride + 1;
     g.Q = (p->W + 2 * p->pad - p->S) / p->stride + 1;
@@ -1307,8 +1310,10 @@ static int tc_conv_impl(const uint32_t* act, const int8_t* wgt, const bs_conv_pa
     const int A = p->a_bits, RS = p->R * p->S, Cw = p->C / 32;
     g.wgt = wgt; g.out_i32 = out_i32; g.out_packed = out_packed; g.scale = p->scale; g.bias = p->bias;
     g.residual = out_packed ? p->residual : nullptr; g.res_scale = p->res_scale;
-    g.status = status_device_ptr();
-    if (!g.status) return BS_ERR_CUDA;
+    if (!plan_only) {
+        g.status = status_device_ptr();
+        if (!g.status) return BS_ERR_CUDA;
+    }
     g.N = p->N; g.H = p->H; g.W = p->W; g.O = p->O; g.R = p->R; g.S = p->S; g.stride = p->stride; g.pad = p->pad; g.A = A;
     g.relu = p->relu; g.out_bits = p->out_bits; g.out_sign = p->out_sign;
     g.out_cw_off = p->out_c_offset / 32; g.out_cw_total = ceil_div(p->out_c_total > 0 ? p->out_c_total : 1, 32);
@@ -1387,8 +1392,11 @@ static int tc_conv_impl(const uint32_t* act, const int8_t* wgt, const bs_conv_pa
     }
     g.pa_bytes = round_up_i(g.pa_tx_bytes, 128);
     g.e_bytes = round_up_i((CKP / 16) * g.HPE * 16, 128);
-    const int sms = device_sm_count();
-    if (sms <= 0) return BS_ERR_CUDA;
+    int sms = device_sm_count();
+    if (sms <= 0) {
+        if (!plan_only) return BS_ERR_CUDA;
+        sms = 148;                     // support query without a device: plan for a full B200
+    }
     // Persistent plan: the filters of a tile (all channel chunks) stay resident in shared memory.  Largest filter tile
     // that fits and still leaves one (pixel tile, filter tile) pair per SM.
     size_t smem = 0;
@@ -1468,6 +1476,13 @@ static int tc_conv_impl(const uint32_t* act, const int8_t* wgt, const bs_conv_pa
         };
         if (stream_tn) TN = stream_tn;
         while (PT > 1 && (PT * TN > 512 || stream_bytes(TN, PT) > 220 * 1024)) PT /= 2;
+        // Large kernels (5x5, 7x7) over many channels: a 128-wide filter chunk of 64 channels does not fit the ring;
+        // halve the chunk to one layout block before narrowing the filter tile.
+        if (g.MB > 1 && stream_bytes(TN, PT) > 200 * 1024) {
+            g.MB = 1; CKP = g.CK; g.CWC = CKP / 32; g.nchunks = p->C / CKP;
+            g.e_bytes = round_up_i((CKP / 16) * g.HPE * 16, 128);
+            g.nsp = g.nse = g.nchunks < 2 ? g.nchunks : 2;
+        }
         while (TN > 32 && stream_bytes(TN, PT) > 200 * 1024) TN /= 2;
         // More CTAs than SMs: halve the chunk if that lets two CTAs share an SM (one wave instead of two)
         if (g.MB == 2 && RS > 1 && ceil_div_ll(tiles_m, PT) * ceil_div(p->O, TN) > sms) {
@@ -1521,6 +1536,7 @@ static int tc_conv_impl(const uint32_t* act, const int8_t* wgt, const bs_conv_pa
         }
     }
 
+    if (plan_only) return BS_OK;
     auto enc = tc_encode_fn();
     if (!enc) return BS_ERR_CUDA;
     const cuuint64_t fullA = static_cast<cuuint64_t>(Cw) * A;
@@ -1643,7 +1659,15 @@ extern "C" int bs_tc_prepare_weights(const uint32_t* wgt_packed, int O, int C, i
     return cudaGetLastError() == cudaSuccess ? BS_OK : BS_ERR_CUDA;
 }
 
-extern "C" int bs_tc_supported(const bs_conv_params* p) { return bs::tc_validate(p) == BS_OK ? 1 : 0; }
+extern "C" int bs_tc_supported(const bs_conv_params* p)
+{
+    if (bs::tc_validate(p) != BS_OK) return 0;
+    // the answer of the planner itself (a shape may pass validation and still find no tiling that fits shared memory);
+    // the epilogue fields do not change the tiling, so the query plans for raw accumulators
+    bs_conv_params q = *p;
+    q.scale = nullptr; q.bias = nullptr; q.residual = nullptr; q.out_bits = 0;
+    return bs::tc_conv_impl(nullptr, nullptr, &q, nullptr, nullptr, nullptr, false, true) == BS_OK ? 1 : 0;
+}
 
 extern "C" int bitserial_conv2d_tc(const uint32_t* act_packed, const int8_t* wgt_tc, const bs_conv_params* p, int32_t* out_i32,
                                    uint32_t* out_packed, void* stream)

@@ -4,7 +4,7 @@ import pytest
 
 import oracle
 from paper_2207_08820_b200 import api, workloads as wl
-from gpu_util import dev, words
+from gpu_util import Guarded, dev, words
 
 pytestmark = pytest.mark.gpu
 
@@ -12,8 +12,14 @@ pytestmark = pytest.mark.gpu
 def run_gemm(c, **kw):
     ap = api.bs_pack_rows(dev(c["a"]), c["a_bits"], c["a_sign"])
     wp = api.bs_pack_rows(dev(c["w"]), c["w_bits"], c["w_sign"])
-    out, packed = api.bitserial_gemm(ap, wp, c["K"], a_sign=c["a_sign"], w_sign=c["w_sign"], **kw)
+    guard = Guarded()
+    M, N = c["a"].shape[0], c["w"].shape[0]
+    out_i32 = guard.empty((M, N))
+    out_packed = guard.empty((M, (N + 31) // 32, kw["out_bits"]), fill=0) if kw.get("out_bits", 0) else None
+    out, packed = api.bitserial_gemm(ap, wp, c["K"], a_sign=c["a_sign"], w_sign=c["w_sign"], out_i32=out_i32,
+                                     out_packed=out_packed, **kw)
     api.bs_check_status()
+    guard.check()
     return out, packed
 
 

@@ -9,7 +9,7 @@ import oracle
 from oracle import network as onet
 from paper_2207_08820_b200 import api, workloads as wl
 from paper_2207_08820_b200.net import BitserialNet
-from gpu_util import dev
+from gpu_util import Guarded, dev
 
 pytestmark = pytest.mark.gpu
 
@@ -20,6 +20,9 @@ def compare_stack(net, batch, seed, sample=None, graph=False, engine="popc"):
     params = wl.network_params(net, seed)
     x = wl.network_input(net, seed, ACT_SCALE, batch=batch)
     runner = BitserialNet(net, params, ACT_SCALE, batch=batch, engine=engine)
+    guard = Guarded()                      # every activation buffer of the runner gets guard words around it
+    for name, buf in list(runner.bufs.items()):
+        runner.bufs[name] = guard.empty(tuple(buf.shape), fill=0)
     xd = dev(x)
     if graph:
         runner.capture(xd)
@@ -27,6 +30,7 @@ def compare_stack(net, batch, seed, sample=None, graph=False, engine="popc"):
     else:
         runner.forward(xd)
     api.bs_check_status()
+    guard.check()
     idx = list(range(batch)) if sample is None else sample
     want = onet.run_stack(net, params, x[idx], ACT_SCALE)
     levels = set()

@@ -7,7 +7,7 @@ import torch
 
 import oracle
 from paper_2207_08820_b200 import api, workloads as wl
-from gpu_util import dev, words
+from gpu_util import Guarded, conv_out_shapes, dev, words
 
 pytestmark = pytest.mark.gpu
 
@@ -20,12 +20,18 @@ def run_tc(c, residual=None, res_scale=0.0, want_packed=True, i32_layout=api.NCH
     if residual is not None:
         res_t = api.bitpack_activations(dev(residual), 1.0, 2, 0, api.NCHW)
         res_total = residual.shape[1]
+    guard = Guarded()                      # guard words around both outputs, checked after the call
+    acc_shape, npq = conv_out_shapes(c, i32_layout)
+    out_i32 = guard.empty(acc_shape)
+    out_packed = guard.empty((*npq, (c["w"].shape[0] + 31) // 32, c["out_bits"]), fill=0) if want_packed else None
     acc, packed = api.bitserial_conv2d(
         xa, wp, C=c["C"], stride=c["stride"], pad=c["pad"], a_sign=c["a_sign"], w_sign=c["w_sign"],
         scale=dev(c["scale"]) if want_packed else None, bias=dev(c["bias"]) if want_packed else None, relu=c["relu"],
         out_bits=c["out_bits"] if want_packed else 0, out_sign=0, residual=res_t, res_scale=res_scale,
-        res_bits=2 if residual is not None else 0, res_c_total=res_total, want_i32=True, i32_layout=i32_layout, wgt_tc=wt)
+        res_bits=2 if residual is not None else 0, res_c_total=res_total, out_i32=out_i32, out_packed=out_packed,
+        i32_layout=i32_layout, wgt_tc=wt)
     api.bs_check_status()
+    guard.check()
     return acc.cpu().numpy(), (words(packed) if packed is not None else None)
 
 
@@ -177,9 +183,43 @@ def test_tc_gemm(M, N, K):
     ap = api.bs_pack_rows(dev(c["a"]), 2, 0)
     wp = api.bs_pack_rows(dev(c["w"]), 1, 2)
     wt = api.tc_prepare_weights(wp.view(N, 1, 1, -1, 1), K, 2, 2)
-    out, _ = api.bitserial_gemm_tc(ap, wt, N, K, 1, a_sign=0, w_sign=2)
+    guard = Guarded()
+    out, _ = api.bitserial_gemm_tc(ap, wt, N, K, 1, a_sign=0, w_sign=2, out_i32=guard.empty((M, N)))
     api.bs_check_status()
+    guard.check()
     assert np.array_equal(out.cpu().numpy(), oracle.gemm_i32(c["a"], c["w"]))
+
+
+@pytest.mark.parametrize("K", [576, 4608])
+def test_tc_gemm_4096_sampled(K):
+    """The largest shapes of the matrix-product sweep on the tensor-core entry point: the oracle evaluates sampled rows
+    and columns; row and column sums of the whole product are checked against sums formed from the operands (a property
+    that holds at any size); the requantised output is compared on the sampled rows."""
+    M = N = 4096
+    c = wl.gemm_case(M, N, K, seed=wl.gemm_sweep_seed(M, K))
+    scale, bias = wl.calibrated_scale_bias(c["w"], 2, 0, 2)
+    ap = api.bs_pack_rows(dev(c["a"]), 2, 0)
+    wp = api.bs_pack_rows(dev(c["w"]), 1, 2)
+    wt = api.tc_prepare_weights(wp.view(N, 1, 1, -1, 1), K, 2, 2)
+    guard = Guarded()
+    out, packed = api.bitserial_gemm_tc(ap, wt, N, K, 1, a_sign=0, w_sign=2, scale=dev(scale), bias=dev(bias), relu=True, out_bits=2,
+                                        out_i32=guard.empty((M, N)), out_packed=guard.empty((M, N // 32, 2), fill=0))
+    api.bs_check_status()
+    guard.check()
+    out = out.cpu().numpy()
+    rng = np.random.default_rng(2)
+    rows = np.sort(rng.choice(M, 48, replace=False))
+    cols = np.sort(rng.choice(N, 48, replace=False))
+    want_rows = oracle.gemm_i32(c["a"][rows], c["w"])
+    assert np.array_equal(out[rows], want_rows)
+    assert np.array_equal(out[:, cols], oracle.gemm_i32(c["a"], c["w"][cols]))
+    wsum = c["w"].astype(np.int64).sum(axis=0)
+    assert np.array_equal(out.astype(np.int64).sum(axis=1), c["a"].astype(np.int64) @ wsum)
+    asum = c["a"].astype(np.int64).sum(axis=0)
+    assert np.array_equal(out.astype(np.int64).sum(axis=0), c["w"].astype(np.int64) @ asum)
+    codes = oracle.requantize(want_rows, scale, bias, True, 2, 0, channel_axis=1)
+    assert len(np.unique(codes)) == 4
+    assert np.array_equal(words(packed)[rows], oracle.pack_rows(codes, 2, 0))
 
 
 def test_tc_unsupported_shape_is_refused():
