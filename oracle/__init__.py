@@ -17,15 +17,17 @@ UNSIGNED, SIGNED, BIPOLAR = 0, 1, 2
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
 _SRC = os.path.join(_HERE, "bitserial_oracle.c")
+_SRC_FP32 = os.path.join(_HERE, "fp32_layers_oracle.c")
 _SO = os.path.join(_HERE, "libbitserial_oracle.so")
 _lib = None
 
 
 def build(force: bool = False) -> str:
     """Compile the oracle with gcc (no fast-math, no FMA contraction) and return the .so path."""
-    if force or not os.path.exists(_SO) or os.path.getmtime(_SO) < os.path.getmtime(_SRC):
+    newest = max(os.path.getmtime(_SRC), os.path.getmtime(_SRC_FP32))
+    if force or not os.path.exists(_SO) or os.path.getmtime(_SO) < newest:
         cmd = ["gcc", "-O2", "-std=c11", "-fPIC", "-shared", "-fopenmp", "-ffp-contract=off",
-               "-fno-fast-math", "-o", _SO, _SRC, "-lm"]
+               "-fno-fast-math", "-o", _SO, _SRC, _SRC_FP32, "-lm"]
         subprocess.run(cmd, check=True)
     return _SO
 
@@ -159,4 +161,50 @@ def pack_rows(codes, bits: int, sign: int) -> np.ndarray:
     rows, K = codes.shape
     out = np.empty((rows, (K + 31) // 32, bits), dtype=np.uint32)
     lib().oracle_pack_rows(_p(codes), rows, K, bits, sign, _p(out))
+    return out
+
+
+# ---- layers kept in floating point (fp32_layers_oracle.c) -----------------------------------------------------------
+
+def _f32(a) -> np.ndarray:
+    return np.ascontiguousarray(a, dtype=np.float32)
+
+
+def conv2d_f32(x, w, bias=None, stride: int = 1, pad: int = 0, relu: bool = False) -> np.ndarray:
+    x, w = _f32(x), _f32(w)
+    N, C, H, W = x.shape
+    O, C2, R, S = w.shape
+    assert C == C2
+    P, Q = out_hw(H, W, R, S, stride, pad)
+    out = np.empty((N, O, P, Q), dtype=np.float32)
+    b = _f32(bias) if bias is not None else None
+    lib().oracle_conv2d_f32(_p(x), _p(w), _p(b) if b is not None else None, N, C, H, W, O, R, S, stride, pad, int(bool(relu)), _p(out))
+    return out
+
+
+def maxpool2d_f32(x, k: int, stride: int, pad: int) -> np.ndarray:
+    x = _f32(x)
+    N, C, H, W = x.shape
+    P, Q = out_hw(H, W, k, k, stride, pad)
+    out = np.empty((N, C, P, Q), dtype=np.float32)
+    lib().oracle_maxpool2d_f32(_p(x), N, C, H, W, k, stride, pad, _p(out))
+    return out
+
+
+def avgpool_codes(codes, inv: float) -> np.ndarray:
+    codes = _i8(codes)
+    N, C, H, W = codes.shape
+    out = np.empty((N, C), dtype=np.float32)
+    lib().oracle_avgpool_codes(_p(codes), N, C, H, W, ctypes.c_float(inv), _p(out))
+    return out
+
+
+def fc_f32(x, w, bias=None) -> np.ndarray:
+    x, w = _f32(x), _f32(w)
+    N, K = x.shape
+    J, K2 = w.shape
+    assert K == K2
+    out = np.empty((N, J), dtype=np.float32)
+    b = _f32(bias) if bias is not None else None
+    lib().oracle_fc_f32(_p(x), _p(w), _p(b) if b is not None else None, N, K, J, _p(out))
     return out

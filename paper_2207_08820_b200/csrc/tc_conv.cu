@@ -46,6 +46,7 @@ struct TcArgs {
     int thr_packed;                   // thresholds stored for two filters per entry (16-bit lanes), see tc_compare_pairs
     // tiling
     int flat;                         // 1: 128 consecutive pixels of the flattened image (1x1, stride 1)
+    int NM;                           // filters of one MMA (TN when TN <= 128, else 256: a wider tile issues TN / NM MMAs per step)
     int TN, CK, MB, CWC, nchunks, nsp, nse;   // CK: channels per filter-layout block, MB: blocks per pipeline chunk, CWC: words per chunk
     int fullA;                        // words of one packed pixel record (Cw * A)
     int pmode;                        // how a tile's packed halo is fetched: 0 flat bulk copy, 1 rows merged with W, 2 4-D box
@@ -748,12 +749,19 @@ __device__ __forceinline__ void tc_epilogue_tile(const TcArgs& g, uint32_t tmem_
         const int ob = o0 + cc * 32;
         if (valid && ob < g.O) {
         if (g.out_i32) {
+            if (g.i32_nhwc && (g.O & 3) == 0 && g.O - ob >= 32) {
+                // channel-innermost accumulators: the 32 values of this thread are 128 contiguous, 16-byte aligned bytes
+                uint4* dst4 = reinterpret_cast<uint4*>(g.out_i32 + pix * g.O + ob);
 #pragma unroll
-            for (int f = 0; f < 32; ++f) {
-                const int o = ob + f;
-                if (o < g.O) {
-                    const size_t idx = g.i32_nhwc ? pix * g.O + o : ((static_cast<size_t>(n) * g.O + o) * g.P + p) * g.Q + q;
-                    g.out_i32[idx] = static_cast<int>(v[f]);
+                for (int f = 0; f < 8; ++f) dst4[f] = make_uint4(v[4 * f], v[4 * f + 1], v[4 * f + 2], v[4 * f + 3]);
+            } else {
+#pragma unroll
+                for (int f = 0; f < 32; ++f) {
+                    const int o = ob + f;
+                    if (o < g.O) {
+                        const size_t idx = g.i32_nhwc ? pix * g.O + o : ((static_cast<size_t>(n) * g.O + o) * g.P + p) * g.Q + q;
+                        g.out_i32[idx] = static_cast<int>(v[f]);
+                    }
                 }
             }
         }
@@ -906,6 +914,8 @@ __global__ void __launch_bounds__(TC_THREADS) bitserial_conv_tc_kernel(const __g
         if (lane == 0) {
             const uint32_t e_base = smem_u32(tc_smem + g.off_e), p_base = smem_u32(tc_smem);
             const TcIssue is = tc_make_issue(g);
+            const int nmt = g.TN / g.NM;
+            const uint32_t nm_b_bytes = static_cast<uint32_t>(g.NM >> 3) * static_cast<uint32_t>(RS * (g.CK >> 4)) * 128u;   // NM / 8 groups of 8 filters
             TcRing rp, re;
             for (int c = 0; c < g.nchunks; ++c) {
                 if (!(mbar_spin_bounded(&full_p[rp.idx], rp.phase) && mbar_spin_bounded(&full_e[re.idx], re.phase))) {
@@ -914,8 +924,10 @@ __global__ void __launch_bounds__(TC_THREADS) bitserial_conv_tc_kernel(const __g
                 }
                 tc_fence_after();
                 for (int t = 0; t < nt; ++t)
-                    tc_issue_chunk(is, e_base + static_cast<uint32_t>(re.idx * e_stage + t * g.e_bytes), p_base + static_cast<uint32_t>(rp.idx * stage_p_bytes),
-                                   tmem_base + static_cast<uint32_t>(t * g.TN), c == 0);
+                    for (int nm = 0; nm < nmt; ++nm)      // a tile wider than one MMA: the same expanded chunk against each slice of NM filters
+                        tc_issue_chunk(is, e_base + static_cast<uint32_t>(re.idx * e_stage + t * g.e_bytes),
+                                       p_base + static_cast<uint32_t>(rp.idx * stage_p_bytes) + static_cast<uint32_t>(nm) * nm_b_bytes,
+                                       tmem_base + static_cast<uint32_t>(t * g.TN + nm * g.NM), c == 0);
                 umma_commit(&empty_e[re.idx]);
                 umma_commit(&empty_p[rp.idx]);
                 rp.advance(g.nsp);
@@ -1457,6 +1469,9 @@ static int tc_conv_impl(const uint32_t* act, const int8_t* wgt, const bs_conv_pa
         if (per_o > tiles_m) per_o = tiles_m;
         if (2 * tiles_m <= 3 * per_o) g.persistent = 0;       // at most 1.5 pixel tiles per CTA
     }
+    // Wide matrix products (see the streaming plan below): a resident 128-filter tile would expand every pixel tile once per
+    // filter tile; with four or more filter tiles the streaming kernel with 256- or 512-filter tiles does less work.
+    if (!keep_narrow && g.persistent && g.flat && p->O >= 512 && p->O % 256 == 0 && tiles_m * (p->O / 256) >= sms) g.persistent = 0;
     if (force_stream) g.persistent = 0;
     g.PT = 1;
     if (!g.persistent) {
@@ -1474,6 +1489,30 @@ static int tc_conv_impl(const uint32_t* act, const int8_t* wgt, const bs_conv_pa
                    static_cast<size_t>(g.nse) * pt * g.e_bytes + 2 * tn * 4 + 256 + (4 * TC_MAX_STAGES + 3) * 8 + 128 +
                    16 + static_cast<size_t>(A) * TC_LUT_BYTES_PER_PLANE;
         };
+        // Matrix products and 1x1 layers with many filters: every filter tile of a pixel tile expands the same packed rows
+        // again, and one K = 32 step is a single MMA, so the expansion, not the tensor core, sets the pace.  A CTA then
+        // takes 256 or 512 filters (N = 256 MMAs, 256 or 512 accumulator columns) as long as a full wave of CTAs remains.
+        if (g.flat && PT == 1 && !stream_tn) {
+            for (int wide = 512; wide > 128; wide /= 2) {
+                if (p->O % wide != 0 || tiles_m * (p->O / wide) < sms) continue;
+                int mb = g.MB;
+                auto bytes_mb = [&](int m) {
+                    const int ckp = g.CK * m;
+                    return static_cast<size_t>(2) * wide * RS * ckp + g.pa_bytes + static_cast<size_t>(2) * round_up_i((ckp / 16) * g.HPE * 16, 128) +
+                           2 * wide * 4 + 256 + (4 * TC_MAX_STAGES + 3) * 8 + 128 + 16 + static_cast<size_t>(A) * TC_LUT_BYTES_PER_PLANE +
+                           static_cast<size_t>(wide) * 16 + 16;
+                };
+                while (mb > 1 && bytes_mb(mb) > 200 * 1024) mb /= 2;
+                if (bytes_mb(mb) > 200 * 1024) continue;
+                if (mb != g.MB) {
+                    g.MB = mb; CKP = g.CK * mb; g.CWC = CKP / 32; g.nchunks = p->C / CKP;
+                    g.e_bytes = round_up_i((CKP / 16) * g.HPE * 16, 128);
+                    g.nsp = g.nse = g.nchunks < 2 ? g.nchunks : 2;
+                }
+                TN = wide;
+                break;
+            }
+        }
         if (stream_tn) TN = stream_tn;
         while (PT > 1 && (PT * TN > 512 || stream_bytes(TN, PT) > 220 * 1024)) PT /= 2;
         // Large kernels (5x5, 7x7) over many channels: a 128-wide filter chunk of 64 channels does not fit the ring;
@@ -1508,7 +1547,8 @@ static int tc_conv_impl(const uint32_t* act, const int8_t* wgt, const bs_conv_pa
     }
     g.tiles_o = ceil_div(p->O, g.TN);
     g.tmem_cols = g.persistent ? 2 * g.TN : g.PT * g.TN;      // TN is 32, 64 or 128, PT 1, 2 or 4: powers of two, 32..512 columns
-    g.idesc = (2u << 4) | (1u << 7) | (1u << 10) | (static_cast<unsigned>(g.TN >> 3) << 17) | (static_cast<unsigned>(TC_M >> 4) << 24);
+    g.NM = g.TN > 128 ? 256 : g.TN;
+    g.idesc = (2u << 4) | (1u << 7) | (1u << 10) | (static_cast<unsigned>(g.NM >> 3) << 17) | (static_cast<unsigned>(TC_M >> 4) << 24);
     for (int j = 0; j < 4; ++j) g.mul[j] = 1u << j;
     g.xormask = 0;
     if (p->a_sign == BS_SIGNED) g.mul[A - 1] = 256u - (1u << (A - 1));

@@ -5,6 +5,7 @@ import os
 
 import numpy as np
 import pytest
+import torch
 
 import oracle
 from oracle import BIPOLAR, SIGNED, UNSIGNED
@@ -302,3 +303,94 @@ def test_popcount_form_on_packed_words_matches_dot():
                     pc = sum(bin(int(pa[m, kw, j]) & int(pw[n, kw, i])).count("1") for kw in range(pa.shape[1]))
                     tot += (-1 if i == wb - 1 else 1) * (pc << (i + j))
             assert tot == want[m, n]
+
+
+# ---------------------------------------------------------------- layers kept in floating point
+
+def _fp32_rows():
+    for row in _rows("fp32_layers_worked.txt"):
+        yield row
+
+
+@pytest.mark.parametrize("row", list(_fp32_rows()), ids=lambda r: r[0].strip() + ":" + r[1].strip().replace(" ", "x"))
+def test_fp32_layers_worked(row):
+    kind = row[0].strip()
+    f = lambda s: np.array(s.split(), dtype=np.float64).astype(np.float32)
+    if kind == "conv":
+        C, H, W = map(int, row[1].split())
+        O, R, S = map(int, row[2].split())
+        stride, pad, relu = map(int, row[3].split())
+        got = oracle.conv2d_f32(f(row[4]).reshape(1, C, H, W), f(row[5]).reshape(O, C, R, S), f(row[6]), stride, pad, bool(relu))
+        assert np.array_equal(got.reshape(-1), f(row[7]))
+    elif kind == "maxpool":
+        C, H, W = map(int, row[1].split())
+        k, stride, pad = map(int, row[2].split())
+        got = oracle.maxpool2d_f32(f(row[3]).reshape(1, C, H, W), k, stride, pad)
+        assert np.array_equal(got.reshape(-1), f(row[4]))
+    elif kind == "avgpool":
+        C, H, W = map(int, row[1].split())
+        got = oracle.avgpool_codes(np.array(row[3].split(), dtype=np.int8).reshape(1, C, H, W), float(row[2]))
+        assert np.array_equal(got.reshape(-1), f(row[4]))
+    else:
+        K, J = map(int, row[1].split())
+        got = oracle.fc_f32(f(row[2]).reshape(1, K), f(row[3]).reshape(J, K), f(row[4]))
+        assert np.array_equal(got.reshape(-1), f(row[5]))
+
+
+@pytest.mark.parametrize("k,stride,pad", [(7, 2, 3), (3, 1, 1), (1, 1, 0), (5, 2, 0)])
+def test_conv_f32_against_float64_library_within_chain_bound(k, stride, pad):
+    """A chain of K fused multiply-adds differs from the exact sum by at most K * 2^-24 * sum|x w| (plus the bias term)."""
+    rng = np.random.default_rng(k + stride)
+    x = rng.normal(0, 1, (2, 3, 19, 23)).astype(np.float32)
+    w = rng.normal(0, 0.2, (5, 3, k, k)).astype(np.float32)
+    b = rng.normal(0, 1, 5).astype(np.float32)
+    got = oracle.conv2d_f32(x, w, b, stride, pad)
+    t = lambda a: torch.from_numpy(a.astype(np.float64))
+    want = torch.nn.functional.conv2d(t(x), t(w), t(b), stride=stride, padding=pad).numpy()
+    mag = torch.nn.functional.conv2d(t(np.abs(x)), t(np.abs(w)), t(np.abs(b)), stride=stride, padding=pad).numpy()
+    K = 3 * k * k + 1
+    assert np.all(np.abs(got - want) <= K * 2.0 ** -24 * mag)
+    assert np.abs(got - want).max() > 0            # binary32 all the way: not a float64 computation rounded at the end
+    relu = oracle.conv2d_f32(x, w, b, stride, pad, relu=True)
+    assert np.array_equal(relu, np.maximum(got, 0))
+
+
+def test_conv_f32_single_tap_shift_and_axes():
+    """One non-zero weight at (c, r, s) copies a shifted channel: pins the correlation direction, the stride/pad arithmetic
+    and the channel / filter axes."""
+    rng = np.random.default_rng(3)
+    x = rng.normal(0, 1, (2, 3, 9, 11)).astype(np.float32)
+    w = np.zeros((4, 3, 3, 3), dtype=np.float32)
+    w[2, 1, 0, 2] = 1.0
+    got = oracle.conv2d_f32(x, w, None, 2, 1)
+    assert not got[:, [0, 1, 3]].any()
+    P, Q = got.shape[2:]
+    for p in range(P):
+        for q in range(Q):
+            y, xx = 2 * p - 1 + 0, 2 * q - 1 + 2
+            want = x[:, 1, y, xx] if (0 <= y < 9 and 0 <= xx < 11) else 0.0
+            assert np.array_equal(got[:, 2, p, q], np.broadcast_to(want, (2,)).astype(np.float32))
+
+
+def test_pooling_against_library_routines():
+    rng = np.random.default_rng(8)
+    x = rng.normal(0, 1, (2, 5, 13, 10)).astype(np.float32)
+    for k, s, p in ((3, 2, 1), (2, 2, 0), (3, 1, 1)):
+        want = torch.nn.functional.max_pool2d(torch.from_numpy(x), k, s, p).numpy()
+        assert np.array_equal(oracle.maxpool2d_f32(x, k, s, p), want)
+    codes = rng.integers(0, 4, (3, 6, 7, 7)).astype(np.int8)
+    inv = np.float32(0.25 / 49)
+    want = (codes.astype(np.int64).sum(axis=(2, 3)).astype(np.float32) * inv).astype(np.float32)
+    assert np.array_equal(oracle.avgpool_codes(codes, float(inv)), want)
+    assert np.allclose(oracle.avgpool_codes(codes, float(inv)), codes.astype(np.float64).mean(axis=(2, 3)) * 0.25, rtol=1e-6)
+
+
+def test_fc_f32_against_float64_within_chain_bound():
+    rng = np.random.default_rng(12)
+    x = rng.normal(0, 1, (4, 512)).astype(np.float32)
+    w = rng.normal(0, 0.05, (10, 512)).astype(np.float32)
+    b = rng.normal(0, 1, 10).astype(np.float32)
+    got = oracle.fc_f32(x, w, b)
+    want = x.astype(np.float64) @ w.astype(np.float64).T + b.astype(np.float64)
+    mag = np.abs(x).astype(np.float64) @ np.abs(w).astype(np.float64).T + np.abs(b)
+    assert np.all(np.abs(got - want) <= 513 * 2.0 ** -24 * mag)
