@@ -441,6 +441,30 @@ def measure_other_configs(torch, api, stream, args):
                                  "frac": sums["roofline_s_burst"] / (t_conv * 1e-3), "frac_sustained": sums["roofline_s_sustained"] / (t_conv * 1e-3),
                                  "hbm_bound_layers": sums["hbm_bound_layers"],
                                  "pack_frac_hbm": (x.numel() * 4 + runner.bufs[net.in_name].numel() * 4) / (t_pack * 1e-3) / pk["hbm"]}
+    del runner, x
+    # ---- the whole mixed-precision classifier: floating-point stem and head around the headline stack
+    from paper_2207_08820_b200.net import BitserialFullNet
+    fnet = wl.resnet18_full(batch=args.batch)
+    fparams = wl.full_network_params(fnet, 3000)
+    images = torch.from_numpy(wl.full_network_input(fnet, 3000)).cuda()
+    full = BitserialFullNet(fnet, fparams, batch=fnet.batch, engine="tc")
+    with torch.cuda.stream(stream):
+        full.forward(images)
+        stream.synchronize()
+        t_stem = graph_time(lambda: full.run_stem(images), reps=1, rounds=6)
+        t_packf = graph_time(lambda: full.body.pack_input(full.stem_pool), reps=1, rounds=6)
+        t_body = graph_time(full.body.run_layers, reps=1, rounds=8)
+        t_head = graph_time(full.run_head, reps=1, rounds=6)
+        t_all = graph_time(lambda: full.forward(images), reps=1, rounds=8)
+    stem_flops = 2.0 * fnet.stem_macs_per_image() * fnet.batch
+    fp32_peak = 2.0 * 128 * torch.cuda.get_device_properties(0).multi_processor_count * peaks["sm_max_mhz"] * 1e6
+    out["resnet18_full"] = {"workload": f"resnet18_full_batch{fnet.batch}_224px: fp32 stem (7x7 s2 conv + 3x3 s2 max pool), quantise + pack, W2A2 body, fp32 head "
+                                        "(average pool + 512 -> 1000 fully connected); warm L2, one CUDA graph per part",
+                            "stem_ms": t_stem, "pack_ms": t_packf, "body_ms": t_body, "head_ms": t_head, "forward_ms": t_all,
+                            "images_per_s": fnet.batch / (t_all * 1e-3), "stem_fp32_TFLOPs": stem_flops / (t_stem * 1e-3) / 1e12,
+                            "stem_frac_fp32_fma_peak": stem_flops / (t_stem * 1e-3) / fp32_peak,
+                            "fp32_fma_peak_TFLOPs": fp32_peak / 1e12, "body_only_images_per_s": fnet.batch / ((t_body + t_packf) * 1e-3)}
+    launches += 0
     api.bs_check_status(stream)
     return out, launches
 

@@ -249,6 +249,28 @@ int bitserial_gemm_tc(const uint32_t* a_packed, const int8_t* w_tc, int M, int N
                       bs_sign_t out_sign, int32_t* out_i32, uint32_t* out_packed, void* stream);
 
 /*
+ * Layers kept in floating point.  The paper's mixed-precision networks keep "a few quantization-sensitive layers in FP32 and the
+ * rest quantized down to 2 bits" (Section VII-D; the runtime of Section VI executes both kinds): in a residual classifier the
+ * first convolution with its pooling, and the final pooling + fully connected layer.  The paper gives no arithmetic for them; this
+ * library fixes it, because the quantiser behind the stem turns every rounding into a possible code change: IEEE binary32;
+ *   bs_conv2d_f32       out[n][o][p][q] = chain of fused multiply-adds starting at bias[o] (0 when bias is NULL) over the taps in
+ *                       the order c (outermost), r, s (innermost), all ascending; out-of-image taps add nothing; optional ReLU.
+ *                       x [N][C][H][W], w [O][C][R][S], out [N][O][P][Q], device, 16-byte aligned.  Any R, S, stride >= 1, pad >= 0.
+ *   bs_maxpool2d_f32    maximum over the k x k window positions inside the image (padding never wins); 2*pad <= k.
+ *   bs_avgpool_codes_f32  global average pool of packed activation codes [N][H][W][Cw][a_bits] -> float [N][C]: the exact integer
+ *                       sum of the H*W codes of a channel, converted to float and multiplied once by `inv` (code step / (H*W)).
+ *   bs_fc_f32           out[n][j] = chain of fused multiply-adds starting at bias[j] over k ascending of x[n][k] * w[j][k];
+ *                       x [N][K], w [J][K], out [N][J].
+ * All asynchronous on `stream`; errors BS_ERR_INVALID_ARG / BS_ERR_ALIGNMENT / BS_ERR_UNSUPPORTED / BS_ERR_CUDA.
+ */
+int bs_conv2d_f32(const float* x, const float* w, const float* bias, int N, int C, int H, int W, int O, int R, int S, int stride,
+                  int pad, int relu, float* out, void* stream);
+int bs_maxpool2d_f32(const float* x, int N, int C, int H, int W, int k, int stride, int pad, float* out, void* stream);
+int bs_avgpool_codes_f32(const uint32_t* packed, int N, int C, int H, int W, int a_bits, bs_sign_t a_sign, float inv, float* out,
+                         void* stream);
+int bs_fc_f32(const float* x, const float* w, const float* bias, int N, int K, int J, float* out, void* stream);
+
+/*
  * bs_check_status -- synchronises `stream`, then reads and clears the device status word of the current
  * device.  Returns BS_ERR_TIMEOUT if any kernel since the last check gave up on a bounded wait (its
  * outputs are then undefined), BS_ERR_CUDA if the stream reports an error, else BS_OK.

@@ -12,7 +12,7 @@ from typing import Dict
 
 import numpy as np
 
-from . import UNSIGNED, conv2d_i32, quantize, requantize
+from . import UNSIGNED, avgpool_codes, conv2d_f32, conv2d_i32, fc_f32, maxpool2d_f32, quantize, requantize
 
 
 def run_stack(net, params: Dict[str, Dict], x_fp32: np.ndarray, act_scale: float,
@@ -35,4 +35,18 @@ def run_stack(net, params: Dict[str, Dict], x_fp32: np.ndarray, act_scale: float
         t[L.dst][:, L.dst_c_offset:L.dst_c_offset + L.O] = codes
         if keep_acc:
             t["acc:" + L.name] = acc
+    return t
+
+
+def run_full(net, params: Dict[str, Dict], images: np.ndarray) -> Dict[str, np.ndarray]:
+    """Whole classifier (duck-typed ``FullNetSpec``): floating-point stem -> quantiser -> quantised body -> floating-point head.
+    Returns every tensor: ``stem_conv``, ``stem_pool`` (float32), the body's code tensors, ``pooled`` and ``logits``."""
+    t: Dict[str, np.ndarray] = {}
+    t["stem_conv"] = conv2d_f32(images, params["stem"]["w"], params["stem"]["bias"], stride=2, pad=3, relu=True)
+    t["stem_pool"] = maxpool2d_f32(t["stem_conv"], 3, 2, 1)
+    t.update(run_stack(net.body, params, t["stem_pool"], net.stem_act_scale))
+    last = t[net.body.out_name]
+    inv = np.float32(np.float32(net.body_act_scale) / np.float32(last.shape[2] * last.shape[3]))
+    t["pooled"] = avgpool_codes(last, float(inv))
+    t["logits"] = fc_f32(t["pooled"], params["fc"]["w"], params["fc"]["bias"])
     return t

@@ -91,6 +91,14 @@ def lib() -> ctypes.CDLL:
     L.bitserial_conv2d_tc_chained.argtypes = [vp, vp, ctypes.POINTER(ConvParams), vp, vp, vp]
     L.bitserial_gemm_tc.restype = i
     L.bitserial_gemm_tc.argtypes = [vp, vp, i, i, i, i, i, i, i, vp, vp, i, i, i, vp, vp, vp]
+    L.bs_conv2d_f32.restype = i
+    L.bs_conv2d_f32.argtypes = [vp, vp, vp, i, i, i, i, i, i, i, i, i, i, vp, vp]
+    L.bs_maxpool2d_f32.restype = i
+    L.bs_maxpool2d_f32.argtypes = [vp, i, i, i, i, i, i, i, vp, vp]
+    L.bs_avgpool_codes_f32.restype = i
+    L.bs_avgpool_codes_f32.argtypes = [vp, i, i, i, i, i, i, ctypes.c_float, vp, vp]
+    L.bs_fc_f32.restype = i
+    L.bs_fc_f32.argtypes = [vp, vp, vp, i, i, i, vp, vp]
     L.bs_check_status.restype = i
     L.bs_check_status.argtypes = [vp]
     L.bs_quantiser_bounds.restype = i
@@ -112,4 +120,5 @@ EXPORTED = ("bs_packed_act_bytes", "bs_packed_wgt_bytes", "bs_packed_rows_bytes"
             "bitserial_conv2d_ws", "bitserial_gemm_ws", "bs_conv_workspace_bytes", "bs_gemm_workspace_bytes",
             "bitserial_gemm_noalloc", "bs_gemm_noalloc_max_scratch_bytes", "bs_selftest_dirty_noalloc_scratch",
             "bs_tc_weights_bytes", "bs_tc_prepare_weights", "bs_tc_supported", "bitserial_conv2d_tc", "bitserial_conv2d_tc_chained", "bitserial_gemm_tc", "bs_l2_prefetch",
+            "bs_conv2d_f32", "bs_maxpool2d_f32", "bs_avgpool_codes_f32", "bs_fc_f32",
             "bs_check_status", "bs_quantiser_bounds", "bs_requant_bounds", "bs_selftest_wait_timeout", "bs_popc_rate", "bs_status_string")

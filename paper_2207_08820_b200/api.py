@@ -238,6 +238,51 @@ def conv_workspace(N: int, C: int, H: int, W: int, O: int, k: int, stride: int, 
     return torch.zeros((nbytes + 3) // 4, dtype=torch.int32, device=device) if nbytes else None
 
 
+def conv2d_f32(x: torch.Tensor, w: torch.Tensor, bias: Optional[torch.Tensor] = None, stride: int = 1, pad: int = 0, relu: bool = False,
+               out: Optional[torch.Tensor] = None, stream=None) -> torch.Tensor:
+    """Floating-point convolution of the layers kept in FP32 (``bs_conv2d_f32``): x [N,C,H,W], w [O,C,R,S] float32."""
+    N, C, H, W = x.shape
+    O, C2, R, S = w.shape
+    if C != C2 or x.dtype != torch.float32 or w.dtype != torch.float32:
+        raise ValueError("float32 tensors with matching channels expected")
+    P, Q = (H + 2 * pad - R) // stride + 1, (W + 2 * pad - S) // stride + 1
+    if out is None:
+        out = torch.empty(N, O, P, Q, dtype=torch.float32, device=x.device)
+    _check(lib().bs_conv2d_f32(_ptr(x), _ptr(w), _ptr(bias), N, C, H, W, O, R, S, stride, pad, int(relu), _ptr(out), _stream_ptr(stream)),
+           "bs_conv2d_f32")
+    return out
+
+
+def maxpool2d_f32(x: torch.Tensor, k: int, stride: int, pad: int, out: Optional[torch.Tensor] = None, stream=None) -> torch.Tensor:
+    N, C, H, W = x.shape
+    P, Q = (H + 2 * pad - k) // stride + 1, (W + 2 * pad - k) // stride + 1
+    if out is None:
+        out = torch.empty(N, C, P, Q, dtype=torch.float32, device=x.device)
+    _check(lib().bs_maxpool2d_f32(_ptr(x), N, C, H, W, k, stride, pad, _ptr(out), _stream_ptr(stream)), "bs_maxpool2d_f32")
+    return out
+
+
+def avgpool_codes_f32(packed: torch.Tensor, C: int, a_sign: int, inv: float, out: Optional[torch.Tensor] = None, stream=None) -> torch.Tensor:
+    """Global average pool of packed codes [N,H,W,Cw,a_bits] -> float32 [N,C] (``bs_avgpool_codes_f32``)."""
+    N, H, W, Cw, a_bits = packed.shape
+    if out is None:
+        out = torch.empty(N, C, dtype=torch.float32, device=packed.device)
+    _check(lib().bs_avgpool_codes_f32(_ptr(packed), N, C, H, W, a_bits, a_sign, ctypes.c_float(inv), _ptr(out), _stream_ptr(stream)),
+           "bs_avgpool_codes_f32")
+    return out
+
+
+def fc_f32(x: torch.Tensor, w: torch.Tensor, bias: Optional[torch.Tensor] = None, out: Optional[torch.Tensor] = None, stream=None) -> torch.Tensor:
+    N, K = x.shape
+    J, K2 = w.shape
+    if K != K2:
+        raise ValueError("inner dimensions disagree")
+    if out is None:
+        out = torch.empty(N, J, dtype=torch.float32, device=x.device)
+    _check(lib().bs_fc_f32(_ptr(x), _ptr(w), _ptr(bias), N, K, J, _ptr(out), _stream_ptr(stream)), "bs_fc_f32")
+    return out
+
+
 def bs_check_status(stream=None) -> None:
     st = lib().bs_check_status(_stream_ptr(stream))
     if st != 0:

@@ -142,3 +142,44 @@ class BitserialNet:
         """int8 NCHW codes of an activation tensor (debugging / tests)."""
         C = self.shapes[name][0]
         return api.bitunpack_activations(self.bufs[name], C, self.net.a_bits, api.UNSIGNED, api.NCHW)
+
+
+class BitserialFullNet:
+    """The whole mixed-precision classifier of ``workloads.FullNetSpec`` through the C ABI: floating-point stem
+    (``bs_conv2d_f32`` + ``bs_maxpool2d_f32``), quantise + pack, the quantised body (:class:`BitserialNet`), floating-point head
+    (``bs_avgpool_codes_f32`` + ``bs_fc_f32``).  Host logic only."""
+
+    def __init__(self, net, params: Dict[str, Dict], device="cuda", batch: Optional[int] = None, engine: str = "tc"):
+        self.net = net
+        self.batch = batch or net.batch
+        self.device = torch.device(device)
+        self.body = BitserialNet(net.body, params, net.stem_act_scale, device=device, batch=self.batch, engine=engine)
+        to = lambda a: torch.from_numpy(np.ascontiguousarray(a)).to(self.device)
+        self.stem_w, self.stem_b = to(params["stem"]["w"]), to(params["stem"]["bias"])
+        self.fc_w, self.fc_b = to(params["fc"]["w"]), to(params["fc"]["bias"])
+        h1 = (net.hw + 2 * 3 - 7) // 2 + 1
+        h2 = (h1 + 2 - 3) // 2 + 1
+        self.stem_conv = torch.empty(self.batch, 64, h1, h1, dtype=torch.float32, device=self.device)
+        self.stem_pool = torch.empty(self.batch, 64, h2, h2, dtype=torch.float32, device=self.device)
+        C, H, W = net.body.tensor_shapes()[net.body.out_name]
+        self.pooled = torch.empty(self.batch, C, dtype=torch.float32, device=self.device)
+        self.logits = torch.empty(self.batch, net.classes, dtype=torch.float32, device=self.device)
+        self.inv = float(np.float32(np.float32(net.body_act_scale) / np.float32(H * W)))
+        self.launches_per_forward = 4 + self.body.launches_per_forward
+
+    def run_stem(self, images: torch.Tensor) -> None:
+        api.conv2d_f32(images, self.stem_w, self.stem_b, stride=2, pad=3, relu=True, out=self.stem_conv)
+        api.maxpool2d_f32(self.stem_conv, 3, 2, 1, out=self.stem_pool)
+
+    def run_head(self) -> None:
+        body = self.net.body
+        api.avgpool_codes_f32(self.body.bufs[body.out_name], body.tensor_shapes()[body.out_name][0], api.UNSIGNED, self.inv, out=self.pooled)
+        api.fc_f32(self.pooled, self.fc_w, self.fc_b, out=self.logits)
+
+    def forward(self, images: torch.Tensor) -> torch.Tensor:
+        """images: float32 [batch, 3, hw, hw] on the device.  Returns the logits [batch, classes]."""
+        self.run_stem(images)
+        self.body.pack_input(self.stem_pool)
+        self.body.run_layers()
+        self.run_head()
+        return self.logits

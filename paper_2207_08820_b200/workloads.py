@@ -319,3 +319,49 @@ def network_input(net: NetSpec, seed: int, act_scale: float = 0.25, batch: Optio
     rng = np.random.default_rng(seed + 1)
     C, H, W = net.in_shape
     return float_activations(rng, (batch or net.batch, C, H, W), net.a_bits, act_scale)
+
+
+# --------------------------------------------------------------------------------------
+# Whole classifier: floating-point stem and head around the quantised body (mixed precision)
+# --------------------------------------------------------------------------------------
+
+@dataclass
+class FullNetSpec:
+    """An 18-layer residual classifier at ``hw`` x ``hw`` input: a floating-point stem (7x7 stride-2 convolution 3 -> 64 with
+    bias and ReLU, 3x3 stride-2 max pool), the quantised body, and a floating-point head (global average pool of the last
+    codes, fully connected layer to ``classes`` outputs).  ``stem_act_scale`` is the step of the quantiser between stem and
+    body, ``body_act_scale`` the step of the body's codes (used by the average pool)."""
+    name: str
+    batch: int
+    hw: int
+    body: NetSpec
+    classes: int = 1000
+    stem_act_scale: float = 0.6
+    body_act_scale: float = 0.25
+
+    def stem_macs_per_image(self) -> int:
+        return (self.hw // 2) ** 2 * 64 * 3 * 49
+
+    def head_macs_per_image(self) -> int:
+        return 512 * self.classes
+
+
+def resnet18_full(batch: int = 64, hw: int = 224) -> FullNetSpec:
+    return FullNetSpec(name="resnet18_full", batch=batch, hw=hw, body=resnet18_body(batch, hw // 4))
+
+
+def full_network_params(net: FullNetSpec, seed: int) -> Dict[str, Dict]:
+    """Body parameters as ``network_params``; stem and head weights drawn so that their outputs have unit scale."""
+    params = network_params(net.body, seed)
+    rng = np.random.default_rng(seed + 7)
+    params["stem"] = dict(w=(rng.normal(0.0, 1.0, (64, 3, 7, 7)) / np.sqrt(147.0)).astype(np.float32),
+                          bias=rng.normal(0.0, 0.1, 64).astype(np.float32))
+    params["fc"] = dict(w=(rng.normal(0.0, 1.0, (net.classes, 512)) / np.sqrt(512.0)).astype(np.float32),
+                        bias=rng.normal(0.0, 0.1, net.classes).astype(np.float32))
+    return params
+
+
+def full_network_input(net: FullNetSpec, seed: int, batch: Optional[int] = None) -> np.ndarray:
+    """Normalised images: fp32 [batch, 3, hw, hw], standard normal (what mean/std normalisation of 8-bit images gives)."""
+    rng = np.random.default_rng(seed + 2)
+    return rng.normal(0.0, 1.0, (batch or net.batch, 3, net.hw, net.hw)).astype(np.float32)
