@@ -10,12 +10,13 @@ namespace bs {
 
 // ----------------------------------------------------------------------------- convolution, register-tiled
 //
-// CTA tile: TH x TW output pixels of one image x 64 filters; thread = 4 filters x 8 consecutive output columns.
+// CTA tile: TH x TW output pixels of one image x 64 filters; thread = 8 filters x 8 consecutive output columns.
 // Weights of the 64 filters ([c][r][s][64], 16-byte vectors of four filters) and the input halo sit in shared memory.  For a
-// fixed (c, r) a thread keeps the input row segment of its eight outputs in registers and walks the S columns: per column one
-// 128-bit weight load feeds 32 fused multiply-adds.  A warp is 16 filter quads x 2 strips: its weight loads are 16 distinct
-// consecutive vectors (no bank conflict), its input loads two broadcasts.
-constexpr int F32_TH = 4, F32_TW = 32, F32_STRIP = 8, F32_OT = 64, F32_THREADS = 256;
+// fixed (c, r) a thread keeps the input row segment of its eight outputs in registers and walks the S columns: per column two
+// 128-bit weight loads feed 64 fused multiply-adds (with four filters per thread the shared-memory pipe, not the FMA pipe, set
+// the pace: 22 TFLOP/s).  A warp is 8 filter octets x 4 strips: its weight loads are 8 distinct vectors, its input loads four
+// broadcasts.
+constexpr int F32_TH = 8, F32_TW = 32, F32_STRIP = 8, F32_OT = 64, F32_THREADS = 256, F32_FPT = 8;
 
 struct ConvF32Args {
     const float* x;
@@ -28,12 +29,12 @@ struct ConvF32Args {
 };
 
 template <int S, int STRIDE>
-__global__ void __launch_bounds__(F32_THREADS) conv2d_f32_tiled_kernel(const ConvF32Args g)
+__global__ void __launch_bounds__(F32_THREADS, 2) conv2d_f32_tiled_kernel(const ConvF32Args g)
 {
     extern __shared__ __align__(16) float f32_smem[];
     constexpr int WIN = (F32_STRIP - 1) * STRIDE + S;            // input columns one strip needs
     constexpr int WIN4 = (WIN + 3) / 4;
-    float* s_w = f32_smem;                                       // [C][R][S][64]
+    float* s_w = f32_smem;                                       // [C][R][S][2][8][4]
     float* s_x = f32_smem + g.C * g.R * S * F32_OT;              // [C][in_h][pitch]
     const int tid = threadIdx.x;
     const int to = blockIdx.y, o0 = to * F32_OT;
@@ -43,8 +44,10 @@ __global__ void __launch_bounds__(F32_THREADS) conv2d_f32_tiled_kernel(const Con
     // (the filter bank is a few tens of KB) and are amortised over all the tiles the CTA walks.
     const int taps = g.C * g.R * S;
     for (int i = tid; i < taps * F32_OT; i += F32_THREADS) {
+        // filter o = 8 * octet + k sits at [tap][k / 4][octet][k % 4]: the eight threads of a quarter warp, one octet each, read
+        // 128 contiguous bytes with each of their two vector loads
         const int t = i >> 6, o = i & 63;
-        s_w[i] = (o0 + o < g.O) ? g.w[static_cast<size_t>(o0 + o) * taps + t] : 0.0f;
+        s_w[t * F32_OT + ((o & 7) >> 2) * 32 + (o >> 3) * 4 + (o & 3)] = (o0 + o < g.O) ? g.w[static_cast<size_t>(o0 + o) * taps + t] : 0.0f;
     }
     const int tiles = g.N * g.tiles_p * g.tiles_q;
     for (int tile = blockIdx.x; tile < tiles; tile += gridDim.x) {
@@ -66,17 +69,17 @@ __global__ void __launch_bounds__(F32_THREADS) conv2d_f32_tiled_kernel(const Con
     }
     __syncthreads();
 
-    const int cq = tid & 15, strip = tid >> 4;                   // filter quad, strip (row-major over TH x TW / 8)
+    const int cq = tid & 7, strip = tid >> 3;                    // filter octet, strip (row-major over TH x TW / 8)
     const int sp = strip / (F32_TW / F32_STRIP), sq = strip % (F32_TW / F32_STRIP);
-    float acc[F32_STRIP][4];
+    float acc[F32_STRIP][F32_FPT];
     {
-        float bq[4];
+        float bq[F32_FPT];
 #pragma unroll
-        for (int k = 0; k < 4; ++k) bq[k] = (g.bias && o0 + cq * 4 + k < g.O) ? g.bias[o0 + cq * 4 + k] : 0.0f;
+        for (int k = 0; k < F32_FPT; ++k) bq[k] = (g.bias && o0 + cq * F32_FPT + k < g.O) ? g.bias[o0 + cq * F32_FPT + k] : 0.0f;
 #pragma unroll
         for (int j = 0; j < F32_STRIP; ++j)
 #pragma unroll
-            for (int k = 0; k < 4; ++k) acc[j][k] = bq[k];       // the chain starts at the bias
+            for (int k = 0; k < F32_FPT; ++k) acc[j][k] = bq[k];  // the chain starts at the bias
     }
     for (int c = 0; c < g.C; ++c) {
         for (int r = 0; r < g.R; ++r) {
@@ -90,22 +93,27 @@ __global__ void __launch_bounds__(F32_THREADS) conv2d_f32_tiled_kernel(const Con
             const float* wrow = s_w + ((c * g.R + r) * S) * F32_OT + cq * 4;
 #pragma unroll
             for (int s = 0; s < S; ++s) {
-                const float4 w4 = *reinterpret_cast<const float4*>(wrow + s * F32_OT);
+                const float4 wa = *reinterpret_cast<const float4*>(wrow + s * F32_OT);
+                const float4 wb = *reinterpret_cast<const float4*>(wrow + s * F32_OT + 32);
 #pragma unroll
                 for (int j = 0; j < F32_STRIP; ++j) {
                     const float xv = xr[j * STRIDE + s];
-                    acc[j][0] = fmaf(xv, w4.x, acc[j][0]);
-                    acc[j][1] = fmaf(xv, w4.y, acc[j][1]);
-                    acc[j][2] = fmaf(xv, w4.z, acc[j][2]);
-                    acc[j][3] = fmaf(xv, w4.w, acc[j][3]);
+                    acc[j][0] = fmaf(xv, wa.x, acc[j][0]);
+                    acc[j][1] = fmaf(xv, wa.y, acc[j][1]);
+                    acc[j][2] = fmaf(xv, wa.z, acc[j][2]);
+                    acc[j][3] = fmaf(xv, wa.w, acc[j][3]);
+                    acc[j][4] = fmaf(xv, wb.x, acc[j][4]);
+                    acc[j][5] = fmaf(xv, wb.y, acc[j][5]);
+                    acc[j][6] = fmaf(xv, wb.z, acc[j][6]);
+                    acc[j][7] = fmaf(xv, wb.w, acc[j][7]);
                 }
             }
         }
     }
     const int p = p0 + sp, qb = q0 + sq * F32_STRIP;
 #pragma unroll
-    for (int k = 0; k < 4; ++k) {
-        const int o = o0 + cq * 4 + k;
+    for (int k = 0; k < F32_FPT; ++k) {
+        const int o = o0 + cq * F32_FPT + k;
         if (o >= g.O || p >= g.P) continue;
         float* dst = g.out + ((static_cast<size_t>(n) * g.O + o) * g.P + p) * g.Q + qb;
         float v[F32_STRIP];
@@ -169,6 +177,35 @@ __global__ void maxpool2d_f32_kernel(const float* __restrict__ x, float* __restr
             }
         }
         out[i] = m;
+    }
+}
+
+// 3x3 window, stride 2, pad 1 on rows whose width is a multiple of 8 (the stem's pooling): a thread produces four consecutive
+// outputs from three rows of eight inputs read as 128-bit vectors plus the column to their left.  The maximum does not depend
+// on the order of its operands, so this is the same result as the generic kernel.
+__global__ void maxpool3x3s2p1_f32_kernel(const float* __restrict__ x, float* __restrict__ out, long long planes, int H, int W, int P, int Q)
+{
+    const int q4n = Q >> 2;
+    const long long total = planes * P * q4n;
+    for (long long i = static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x; i < total; i += static_cast<long long>(gridDim.x) * blockDim.x) {
+        const int q4 = static_cast<int>(i % q4n);
+        const int p = static_cast<int>((i / q4n) % P);
+        const long long pl = i / (static_cast<long long>(P) * q4n);
+        const float* src = x + pl * H * W;
+        float m[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+#pragma unroll
+        for (int r = 0; r < 3; ++r) {
+            const int y = 2 * p - 1 + r;
+            if (y < 0 || y >= H) continue;
+            const float* row = src + static_cast<size_t>(y) * W + 8 * q4;
+            const float4 a = *reinterpret_cast<const float4*>(row), b = *reinterpret_cast<const float4*>(row + 4);
+            const float left = q4 > 0 ? row[-1] : -INFINITY;
+            m[0] = fmaxf(m[0], fmaxf(left, fmaxf(a.x, a.y)));
+            m[1] = fmaxf(m[1], fmaxf(a.y, fmaxf(a.z, a.w)));
+            m[2] = fmaxf(m[2], fmaxf(a.w, fmaxf(b.x, b.y)));
+            m[3] = fmaxf(m[3], fmaxf(b.y, fmaxf(b.z, b.w)));
+        }
+        *reinterpret_cast<float4*>(out + (pl * P + p) * Q + 4 * q4) = make_float4(m[0], m[1], m[2], m[3]);
     }
 }
 
@@ -282,6 +319,12 @@ extern "C" int bs_maxpool2d_f32(const float* x, int N, int C, int H, int W, int 
     if (H + 2 * pad < k || W + 2 * pad < k) return BS_ERR_INVALID_ARG;
     const int P = (H + 2 * pad - k) / stride + 1, Q = (W + 2 * pad - k) / stride + 1;
     const long long planes = static_cast<long long>(N) * C, total = planes * P * Q;
+    if (k == 3 && stride == 2 && pad == 1 && W % 8 == 0 && Q * 2 == W && bs::aligned16(x) && bs::aligned16(out)) {
+        long long blocks4 = (total / 4 + 255) / 256;
+        if (blocks4 > 148 * 64) blocks4 = 148 * 64;
+        bs::maxpool3x3s2p1_f32_kernel<<<static_cast<unsigned>(blocks4), 256, 0, static_cast<cudaStream_t>(stream)>>>(x, out, planes, H, W, P, Q);
+        return cudaGetLastError() == cudaSuccess ? BS_OK : BS_ERR_CUDA;
+    }
     long long blocks = (total + 255) / 256;
     if (blocks > 148 * 64) blocks = 148 * 64;
     bs::maxpool2d_f32_kernel<<<static_cast<unsigned>(blocks), 256, 0, static_cast<cudaStream_t>(stream)>>>(x, out, planes, H, W, k, stride, pad, P, Q);

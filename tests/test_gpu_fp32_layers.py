@@ -57,6 +57,10 @@ def test_maxpool_bit_exact(k, stride, pad):
     x = rng.normal(-1, 1, (3, 6, 29, 18)).astype(np.float32)
     got = api.maxpool2d_f32(dev(x), k, stride, pad).cpu().numpy()
     assert same_bits(got, oracle.maxpool2d_f32(x, k, stride, pad))
+    # a row width that is a multiple of 8 takes the vectorised kernel when the window is 3x3, stride 2, pad 1
+    x8 = rng.normal(-1, 1, (2, 5, 13, 24)).astype(np.float32)
+    got8 = api.maxpool2d_f32(dev(x8), k, stride, pad).cpu().numpy()
+    assert same_bits(got8, oracle.maxpool2d_f32(x8, k, stride, pad))
 
 
 @pytest.mark.parametrize("bits,sign,C", [(2, 0, 512), (3, 1, 70), (1, 2, 33), (4, 0, 64)])
