@@ -244,6 +244,35 @@ int bitserial_conv2d_tc(const uint32_t* act_packed, const int8_t* wgt_tc, const 
  */
 int bitserial_conv2d_tc_chained(const uint32_t* act_packed, const int8_t* wgt_tc, const bs_conv_params* p,
                                 int32_t* out_i32, uint32_t* out_packed, void* stream);
+/*
+ * bitserial_conv2d_tc_chain -- 2 to 4 consecutive layers of a network in ONE launch (the paper runs a network layer by layer
+ * and names tiling and parallelisation as the source of its speed, Section V; running several layers as one grid whose tiles
+ * wait for the tiles they depend on, instead of one grid per layer, is this library's addition).  Every layer computes exactly
+ * what bitserial_conv2d_tc computes for its bs_conv_params; results are identical.
+ *   layers[l]        bs_conv_params of layer l.  All layers share N, C, H, W, O = C, R = S, pad = (R-1)/2, stride 1 (the output
+ *                    is as large as the input), the activation and weight formats, and a packed output (out_bits > 0, no
+ *                    channel offset: out_c_offset 0, out_c_total O) whose format is the next layer's activation format; a
+ *                    residual, if any, has res_c_offset 0 and res_c_total O.  scale, bias and residual are DEVICE pointers.
+ *   act_packed[l], wgt_tc[l], out_packed[l]   HOST arrays of `nlayers` DEVICE pointers: packed input, prepared filters
+ *                    (bs_tc_prepare_weights) and packed output of layer l.  A layer may read -- as input or residual -- the
+ *                    output of any EARLIER layer of the chain, or tensors that were final before the launch; an output must
+ *                    not overlap a tensor the same chain reads unless that tensor is the output of an earlier layer or the
+ *                    input of one.  Outputs of all layers are materialised in full.
+ *   workspace        DEVICE, 16-byte aligned, at least bs_tc_chain_workspace_bytes(layers, nlayers) bytes, zero-filled by the
+ *                    caller once before its first use (and again after a launch that ended with BS_ERR_TIMEOUT); the library
+ *                    keeps per-tile progress counters in it from launch to launch.  One workspace serves one chain; launches
+ *                    that share a workspace must not overlap on the GPU.
+ *   chained          non-zero: launched like bitserial_conv2d_tc_chained (same promise by the caller, for every layer).
+ * bs_tc_chain_workspace_bytes returns 0 when the layers cannot run as one chain (shapes differ, a layer does not take the
+ * resident-filter plan, more than 4 layers); bitserial_conv2d_tc_chain then returns BS_ERR_UNSUPPORTED and launches nothing:
+ * call bitserial_conv2d_tc per layer.  Other errors: BS_ERR_INVALID_ARG (null pointer, workspace too small),
+ * BS_ERR_ALIGNMENT, BS_ERR_CUDA.  Every device-side wait is bounded (about a second); one that runs out sets the status
+ * word read by bs_check_status.  Asynchronous on `stream`; works under stream capture.
+ */
+size_t bs_tc_chain_workspace_bytes(const bs_conv_params* layers, int nlayers);
+int bitserial_conv2d_tc_chain(int nlayers, const uint32_t* const* act_packed, const int8_t* const* wgt_tc,
+                              const bs_conv_params* layers, uint32_t* const* out_packed, void* workspace,
+                              size_t workspace_bytes, int chained, void* stream);
 int bitserial_gemm_tc(const uint32_t* a_packed, const int8_t* w_tc, int M, int N, int K, int a_bits, bs_sign_t a_sign,
                       int w_bits, bs_sign_t w_sign, const float* scale, const float* bias, int relu, int out_bits,
                       bs_sign_t out_sign, int32_t* out_i32, uint32_t* out_packed, void* stream);

@@ -89,6 +89,11 @@ def lib() -> ctypes.CDLL:
     L.bs_l2_prefetch.argtypes = [ctypes.POINTER(ctypes.c_void_p), ctypes.POINTER(ctypes.c_size_t), ctypes.c_int, vp]
     L.bitserial_conv2d_tc_chained.restype = i
     L.bitserial_conv2d_tc_chained.argtypes = [vp, vp, ctypes.POINTER(ConvParams), vp, vp, vp]
+    L.bs_tc_chain_workspace_bytes.restype = ctypes.c_size_t
+    L.bs_tc_chain_workspace_bytes.argtypes = [ctypes.POINTER(ConvParams), i]
+    L.bitserial_conv2d_tc_chain.restype = i
+    L.bitserial_conv2d_tc_chain.argtypes = [i, ctypes.POINTER(ctypes.c_void_p), ctypes.POINTER(ctypes.c_void_p), ctypes.POINTER(ConvParams),
+                                            ctypes.POINTER(ctypes.c_void_p), vp, ctypes.c_size_t, i, vp]
     L.bitserial_gemm_tc.restype = i
     L.bitserial_gemm_tc.argtypes = [vp, vp, i, i, i, i, i, i, i, vp, vp, i, i, i, vp, vp, vp]
     L.bs_conv2d_f32.restype = i
@@ -119,6 +124,6 @@ EXPORTED = ("bs_packed_act_bytes", "bs_packed_wgt_bytes", "bs_packed_rows_bytes"
             "bitunpack_activations", "pack_weights", "bs_pack_rows", "bitserial_conv2d", "bitserial_gemm",
             "bitserial_conv2d_ws", "bitserial_gemm_ws", "bs_conv_workspace_bytes", "bs_gemm_workspace_bytes",
             "bitserial_gemm_noalloc", "bs_gemm_noalloc_max_scratch_bytes", "bs_selftest_dirty_noalloc_scratch",
-            "bs_tc_weights_bytes", "bs_tc_prepare_weights", "bs_tc_supported", "bitserial_conv2d_tc", "bitserial_conv2d_tc_chained", "bitserial_gemm_tc", "bs_l2_prefetch",
+            "bs_tc_weights_bytes", "bs_tc_prepare_weights", "bs_tc_supported", "bitserial_conv2d_tc", "bitserial_conv2d_tc_chained", "bs_tc_chain_workspace_bytes", "bitserial_conv2d_tc_chain", "bitserial_gemm_tc", "bs_l2_prefetch",
             "bs_conv2d_f32", "bs_maxpool2d_f32", "bs_avgpool_codes_f32", "bs_fc_f32",
             "bs_check_status", "bs_quantiser_bounds", "bs_requant_bounds", "bs_selftest_wait_timeout", "bs_popc_rate", "bs_status_string")

@@ -204,6 +204,47 @@ def tc_supported(N, C, H, W, O, k, stride, pad, a_bits, a_sign, w_bits, w_sign) 
     return bool(lib().bs_tc_supported(ctypes.byref(p)))
 
 
+def conv_params(act_shape, wgt_shape, *, C: int, stride: int = 1, pad: int = 0, a_sign: int = UNSIGNED, w_sign: int = SIGNED,
+                scale: Optional[torch.Tensor] = None, bias: Optional[torch.Tensor] = None, relu: bool = False, out_bits: int = 0,
+                out_sign: int = UNSIGNED, residual: Optional[torch.Tensor] = None, res_scale: float = 0.0, res_bits: int = 0,
+                res_sign: int = UNSIGNED) -> ConvParams:
+    """``bs_conv_params`` of a layer whose packed output is a whole tensor (no channel offset), from the shapes of the packed
+    operands; for :func:`tc_chain_workspace_bytes` and :func:`bitserial_conv2d_tc_chain`."""
+    N, H, W, Cw, a_bits = act_shape
+    O, R, S, Cw2, w_bits = wgt_shape
+    if Cw != Cw2 or Cw != (C + 31) // 32:
+        raise ValueError("channel words of activations and weights disagree")
+    return ConvParams(N=N, C=C, H=H, W=W, O=O, R=R, S=S, stride=stride, pad=pad, a_bits=a_bits, a_sign=a_sign, w_bits=w_bits,
+                      w_sign=w_sign, scale=_ptr(scale), bias=_ptr(bias), relu=int(relu), out_bits=out_bits, out_sign=out_sign,
+                      residual=_ptr(residual), res_scale=res_scale, res_bits=res_bits, res_sign=res_sign, res_c_offset=0,
+                      res_c_total=O, out_c_offset=0, out_c_total=O, i32_layout=NCHW)
+
+
+def _params_array(params):
+    arr = (ConvParams * len(params))()
+    for k, q in enumerate(params):
+        ctypes.memmove(ctypes.addressof(arr[k]), ctypes.addressof(q), ctypes.sizeof(ConvParams))
+    return arr
+
+
+def tc_chain_workspace_bytes(params) -> int:
+    """Bytes of the (zero-filled) workspace ``bitserial_conv2d_tc_chain`` needs for these layers; 0 when they cannot run as
+    one launch."""
+    return int(lib().bs_tc_chain_workspace_bytes(_params_array(params), len(params)))
+
+
+def bitserial_conv2d_tc_chain(acts, wgts_tc, params, outs, workspace: torch.Tensor, chained: bool = False, stream=None) -> None:
+    """Several same-shaped layers in one launch (``bitserial_conv2d_tc_chain``): per layer the packed input, the prepared
+    filters, the :func:`conv_params` and the packed output tensor.  ``workspace``: device tensor of
+    :func:`tc_chain_workspace_bytes` bytes, zero-filled once before its first use."""
+    n = len(params)
+    vp = ctypes.c_void_p * n
+    st = lib().bitserial_conv2d_tc_chain(n, vp(*[_ptr(t) for t in acts]), vp(*[_ptr(t) for t in wgts_tc]), _params_array(params),
+                                         vp(*[_ptr(t) for t in outs]), _ptr(workspace), workspace.numel() * workspace.element_size(),
+                                         int(chained), _stream_ptr(stream))
+    _check(st, "bitserial_conv2d_tc_chain")
+
+
 def bitserial_gemm_tc(a_packed: torch.Tensor, w_tc: torch.Tensor, N: int, K: int, w_bits: int, *, a_sign: int = UNSIGNED,
                       w_sign: int = SIGNED, scale=None, bias=None, relu: bool = False, out_bits: int = 0,
                       out_sign: int = UNSIGNED, want_i32: bool = True, out_i32: Optional[torch.Tensor] = None,

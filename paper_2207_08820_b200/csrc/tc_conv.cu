@@ -11,6 +11,7 @@
 //   - four warps read the accumulator rows back with tcgen05.ld (one pixel per thread), apply the same fused
 //     requantisation epilogue as the popcount kernel and build the output plane words thread-locally.
 // Every wait on an mbarrier is bounded; a wait that runs out sets the device status word and the CTA drains.
+#include <cstdio>
 #include <cstdlib>
 #include <array>
 #include <map>
@@ -71,11 +72,11 @@ struct TcArgs {
 // ----------------------------------------------------------------------------- timeline trace (tuning builds only)
 //
 // Built with -DBS_TUNING, the first 148 CTAs of a launch record the SM cycle counter at the hand-offs between their roles
-// (per tile, for the first 8 tiles); bs_tc_trace_read copies the table to the host.  Compiled out of the normal library.
+// (per tile, for the first 24 tiles); bs_tc_trace_read copies the table to the host.  Compiled out of the normal library.
 enum { TR_START = 0, TR_SETUP, TR_PDL, TR_WGT, TR_LOAD, TR_XBEG, TR_XEND, TR_MBEG, TR_MEND, TR_EBEG, TR_EEND, TR_END, TR_E_LD, TR_E_CMP,
        TR_E_ST, TR_E_LOOP, TR_M_ISSUED, TR_X_DONE0, TR_X_BEG0 };
 #ifdef BS_TUNING
-constexpr int TC_TRACE_EVENTS = 24, TC_TRACE_TILES = 8, TC_TRACE_CTAS = 148;
+constexpr int TC_TRACE_EVENTS = 24, TC_TRACE_TILES = 24, TC_TRACE_CTAS = 148;
 __device__ long long g_tc_trace[TC_TRACE_CTAS * TC_TRACE_EVENTS * TC_TRACE_TILES];
 __device__ __forceinline__ void tc_trace(int ev, int tile)
 {
@@ -711,7 +712,7 @@ __device__ __forceinline__ TcEpiThread tc_epi_thread(const TcArgs& g, int m)
 // Epilogue of one tile: thread `tid` (0..127, warp = TMEM lane quadrant) owns accumulator row tid = one output pixel.
 __device__ __forceinline__ void tc_epilogue_tile(const TcArgs& g, uint32_t tmem_acc, int tid, int warp, const TcTile& tile, const TcEpiThread& et,
                                                  int o0, const float2* s_sb, const float4* s_bounds, uint32_t thr_addr, int cc0 = 0,
-                                                 int ccstep = 1, int trace_tile = -1)
+                                                 int ccstep = 1, int trace_tile = -1, bool res_l2 = false)
 {
     const int n0 = tile.n0, p0 = tile.p0, q0 = tile.q0;
     const int m = tid;                               // TMEM lane = tile pixel
@@ -771,7 +772,7 @@ __device__ __forceinline__ void tc_epilogue_tile(const TcArgs& g, uint32_t tmem_
                 const uint32_t* rp = g.residual + (pix * g.res_cw_total + ((g.res_c_off + ob) >> 5)) * g.res_bits;
 #pragma unroll
                 for (int j = 0; j < 4; ++j)
-                    if (j < g.res_bits) rw[j] = rp[j];
+                    if (j < g.res_bits) rw[j] = res_l2 ? __ldcg(rp + j) : rp[j];     // inside a chain another SM may just have written it: read at L2
             }
             uint32_t ow[4] = {0, 0, 0, 0};
             if (g.rb.enabled) {
@@ -859,6 +860,7 @@ __global__ void __launch_bounds__(TC_THREADS) bitserial_conv_tc_kernel(const __g
     const int nt = tiles_m - mt0 < g.PT ? tiles_m - mt0 : g.PT;                                   // 1..PT pixel tiles
     const int e_stage = g.PT * g.e_bytes;
 
+    if (tid == 0) TC_TRACE(TR_START, 0);
     pdl_release();
     if (tid == 0) {
         for (int s = 0; s < TC_MAX_STAGES; ++s) {
@@ -898,6 +900,7 @@ __global__ void __launch_bounds__(TC_THREADS) bitserial_conv_tc_kernel(const __g
                     for (int t = 0; t < nt; ++t) tc_load_tile(g, tc_smem + g.off_p + t * g.pa_bytes, full_a, tc_decode_tile(g, mt0 + t));
                 }
                 if (!mbar_spin_bounded(&empty_p[rp.idx], rp.phase ^ 1u)) { atomicOr(g.status, STATUS_TIMEOUT); break; }
+                TC_TRACE(TR_LOAD, c);
                 mbar_expect_tx(&full_p[rp.idx], static_cast<unsigned>(g.b_bytes));
                 for (int j = 0; j < g.MB; ++j, src += blk_stride)
                     bulk_load(tc_smem + rp.idx * stage_p_bytes + j * blk_bytes, src, static_cast<unsigned>(blk_bytes), &full_p[rp.idx]);
@@ -922,6 +925,7 @@ __global__ void __launch_bounds__(TC_THREADS) bitserial_conv_tc_kernel(const __g
                     atomicOr(g.status, STATUS_TIMEOUT);
                     break;
                 }
+                TC_TRACE(TR_MBEG, c);
                 tc_fence_after();
                 for (int t = 0; t < nt; ++t)
                     for (int nm = 0; nm < nmt; ++nm)      // a tile wider than one MMA: the same expanded chunk against each slice of NM filters
@@ -930,6 +934,7 @@ __global__ void __launch_bounds__(TC_THREADS) bitserial_conv_tc_kernel(const __g
                                        tmem_base + static_cast<uint32_t>(t * g.TN + nm * g.NM), c == 0);
                 umma_commit(&empty_e[re.idx]);
                 umma_commit(&empty_p[rp.idx]);
+                TC_TRACE(TR_MEND, c);
                 rp.advance(g.nsp);
                 re.advance(g.nse);
             }
@@ -945,16 +950,20 @@ __global__ void __launch_bounds__(TC_THREADS) bitserial_conv_tc_kernel(const __g
         group_sync(1, TC_WORKERS);
         const TcExpand xp = tc_expand_init(g, ct, TC_WORKERS);
         const TcEpiThread eth = tc_epi_thread(g, (warp & 3) * 32 + lane);
+        if (tid == 0) TC_TRACE(TR_SETUP, 0);
         bool ok = mbar_wait_warp(full_a, 0, lane);
+        if (tid == 0) TC_TRACE(TR_PDL, 0);
         TcRing re;
         for (int c = 0; c < g.nchunks; ++c) {
             if (ok) ok = mbar_wait_warp(&empty_e[re.idx], re.phase ^ 1u, lane);
             if (!ok) atomicOr(g.status, STATUS_TIMEOUT);
+            if (tid == 0) TC_TRACE(TR_XBEG, c);
             for (int t = 0; t < nt; ++t)
                 tc_expand_chunk<A>(g, xp, reinterpret_cast<const uint32_t*>(tc_smem + g.off_p + t * g.pa_bytes),
                                    tc_smem + g.off_e + re.idx * e_stage + t * g.e_bytes, s_lut, ct, c);
             fence_proxy_async();          // make the generic-proxy writes visible to the tensor core's reads
             group_sync(1, TC_WORKERS);
+            if (tid == 0) TC_TRACE(TR_XEND, c);
             if (tid == 0) mbar_arrive(&full_e[re.idx]);
             re.advance(g.nse);
         }
@@ -967,17 +976,21 @@ __global__ void __launch_bounds__(TC_THREADS) bitserial_conv_tc_kernel(const __g
             group_sync(1, TC_WORKERS);
             if (*thr_ok) thr = smem_u32(s_thr);
         }
+        if (tid == 0) TC_TRACE(TR_E_CMP, 0);
         if (ok) ok = mbar_wait_warp(accum_full, 0, lane);
         if (!ok) atomicOr(g.status, STATUS_TIMEOUT);
+        if (tid == 0) TC_TRACE(TR_EBEG, 0);
         tc_fence_after();
         for (int t = 0; t < nt; ++t)
             // a warp reads the tensor-memory lanes of quadrant (warp % 4): warps 0-3 take the even groups of 32 filters,
             // warps 6-9 (quadrants 2, 3, 0, 1) the odd ones
             tc_epilogue_tile(g, tmem_base + static_cast<uint32_t>(t * g.TN), (warp & 3) * 32 + lane, warp & 3, tc_decode_tile(g, mt0 + t), eth, o0,
                              s_sb, s_bounds, thr, warp < 4 ? 0 : 1, 2);
+        if (tid == 0) TC_TRACE(TR_EEND, 0);
         tc_fence_before();
     }
     __syncthreads();
+    if (tid == 0) TC_TRACE(TR_END, 0);
     if (warp == 5) {
         tc_fence_after();
         tmem_dealloc(tmem_base, static_cast<unsigned>(g.tmem_cols));
@@ -987,6 +1000,64 @@ __global__ void __launch_bounds__(TC_THREADS) bitserial_conv_tc_kernel(const __g
 // ----------------------------------------------------------------------------- persistent CTAs, filters resident
 //
 // A CTA keeps the int8 filters of its filter tile (all channel chunks) in shared memory and walks over pixel tiles.
+// A chain of layers run by one launch: the same geometry in every layer (stride 1, output as large as the input, same
+// channels and filters), so that all layers share one shared-memory plan and one tiling, and a pixel tile of layer l + 1
+// reads only its own and the adjacent pixel tiles of layer l.  The work items (layer, pixel tile) are numbered layer by
+// layer and dealt to the CTAs round-robin; every role of a CTA walks its items in that order, the pipeline rings simply
+// continue across a layer boundary and only the filters are swapped.  What keeps the order of the layers is a counter
+// per (layer, pixel tile) in global memory, raised by the epilogue once the tile's outputs are stored; the producer
+// of a CTA waits (bounded) for the up to nine counters its next halo depends on.  All CTAs of the grid are resident
+// at once (the host sizes the grid by the occupancy of the kernel), and an item only ever waits for items that come
+// earlier in the common order, so the CTA holding the earliest unfinished item can always proceed.
+// MAXL = 1 is the plain one-layer kernel: no counters, no waits.
+constexpr int TC_CHAIN_MAX = 4;
+
+template <int MAXL>
+struct TcChainArgs {
+    TcArgs L[MAXL];
+    int nlayers;
+    unsigned* flags;       // [nlayers][pixel tiles] filter tiles finished, summed over all launches on this workspace
+    unsigned* ctl;         // [0] launches completed on this workspace, [1] CTAs of the running launch that have finished
+};
+
+__device__ __forceinline__ unsigned ld_acquire_gpu(const unsigned* p)
+{
+    unsigned v;
+    asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+    return v;
+}
+__device__ __forceinline__ void fence_proxy_async_global() { asm volatile("fence.proxy.async.global;" ::: "memory"); }
+
+// Bounded wait until the counter has reached `target` (wrap-safe).  About a second before it gives up.
+__device__ __forceinline__ bool tc_flag_wait(const unsigned* flag, unsigned target)
+{
+    for (unsigned it = 0; it < (1u << 22); ++it) {
+        if (static_cast<int>(ld_acquire_gpu(flag) - target) >= 0) return true;
+        __nanosleep(200);
+    }
+    return false;
+}
+
+// Position of a role in the item sequence of its CTA: layer and pixel tile, advanced without divisions.
+struct TcItemWalker {
+    TcTileWalker w;            // tile within the layer (w.mt is the tile index inside the layer)
+    int l, dl;                 // layer, and whole layers per step
+};
+
+__device__ __forceinline__ TcItemWalker tc_item_init(const TcArgs& g, int first, int step, int tiles_m)
+{
+    TcItemWalker x;
+    x.l = first / tiles_m; x.dl = step / tiles_m;
+    x.w = tc_walk_init(g, first - x.l * tiles_m, step - x.dl * tiles_m);
+    return x;
+}
+__device__ __forceinline__ void tc_item_next(const TcArgs& g, TcItemWalker& x, int tiles_m)
+{
+    tc_walk_next(g, x.w);
+    x.l += x.dl;
+    if (x.w.mt >= tiles_m) { x.w.mt -= tiles_m; x.w.in -= g.tiles_n; ++x.l; }
+}
+
 // Warps 0-3: epilogue (TMEM lane quadrants), warps 4-7: bitplane expansion, warp 8: TMA producer, warp 9: MMA issuer.
 // Packed and expanded activation chunks travel through two mbarrier rings; two TMEM accumulator buffers let the
 // epilogue of tile i overlap the MMAs of tile i + 1.
@@ -999,33 +1070,37 @@ constexpr int TCP_NSE = 3;            // expanded-chunk ring (at most)
 // CPS: CTAs per SM the registers are budgeted for (3: 64 registers per thread; 1: no cap, for plans whose shared memory
 // leaves room for one or two CTAs anyway).
 // WIDE: eight epilogue warps (0-3 and 10-13, two per tensor-memory lane quadrant, sharing the groups of 32 filters).
-template <int A, int CPS, bool WIDE = false>
+template <int A, int CPS, bool WIDE, int MAXL>
 __global__ void __launch_bounds__(WIDE ? TCP_THREADS_WIDE : TCP_THREADS, CPS)
-bitserial_conv_tc_persistent_kernel(const __grid_constant__ TcArgs g)
+bitserial_conv_tc_persistent_kernel(const __grid_constant__ TcChainArgs<MAXL> ch)
 {
     extern __shared__ __align__(128) unsigned char tc_smem[];
+    const TcArgs& g0 = ch.L[0];                     // geometry, tiling and shared-memory plan: the same in every layer
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const int RS = g.R * g.S;
-    unsigned char* s_w = tc_smem;                                              // [nchunks][b_bytes]
-    unsigned char* s_p = tc_smem + g.off_p;                                    // [nsp][pa_bytes] packed tiles
-    unsigned char* s_e = tc_smem + g.off_e;                                    // [nse][e_bytes]
-    float2* s_sb = reinterpret_cast<float2*>(tc_smem + g.off_sb);
-    float4* s_bounds = reinterpret_cast<float4*>(tc_smem + g.off_sb + g.TN * 8);
-    uint2* s_lut = reinterpret_cast<uint2*>(tc_smem + g.off_lut);
-    uint64_t* bars = reinterpret_cast<uint64_t*>(tc_smem + g.off_bar);
+    const int RS = g0.R * g0.S;
+    unsigned char* s_w = tc_smem;                                               // [nchunks][b_bytes]
+    unsigned char* s_p = tc_smem + g0.off_p;                                    // [nsp][pa_bytes] packed tiles
+    unsigned char* s_e = tc_smem + g0.off_e;                                    // [nse][e_bytes]
+    float2* s_sb = reinterpret_cast<float2*>(tc_smem + g0.off_sb);
+    float4* s_bounds = reinterpret_cast<float4*>(tc_smem + g0.off_sb + g0.TN * 8);
+    uint2* s_lut = reinterpret_cast<uint2*>(tc_smem + g0.off_lut);
+    uint64_t* bars = reinterpret_cast<uint64_t*>(tc_smem + g0.off_bar);
     uint64_t* full_p = bars;                        // [TCP_NSP]
     uint64_t* empty_p = bars + TCP_NSP;             // [TCP_NSP]
     uint64_t* full_e = bars + 2 * TCP_NSP;          // [TCP_NSE]
     uint64_t* empty_e = full_e + TCP_NSE;           // [TCP_NSE]
     uint64_t* full_acc = empty_e + TCP_NSE;         // [2]
     uint64_t* empty_acc = full_acc + 2;             // [2]
-    uint64_t* wgt_full = empty_acc + 2;             // [1]
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(wgt_full + 1);
+    uint64_t* wgt_full = empty_acc + 2;             // [1] filters of the current layer have landed
+    uint64_t* wgt_free = wgt_full + 1;              // [1] every MMA that reads the filters of the layer just finished has completed
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(wgt_free + 1);
 
-    const int o0 = static_cast<int>(blockIdx.x % static_cast<unsigned>(g.tiles_o)) * g.TN;
-    const int first_tile = static_cast<int>(blockIdx.x / static_cast<unsigned>(g.tiles_o));
-    const int tile_step = static_cast<int>(gridDim.x / static_cast<unsigned>(g.tiles_o));
-    const int tiles_m = g.tiles_q * g.tiles_p * g.tiles_n;
+    const int nlayers = MAXL > 1 ? ch.nlayers : 1;
+    const int o0 = static_cast<int>(blockIdx.x % static_cast<unsigned>(g0.tiles_o)) * g0.TN;
+    const int first_tile = static_cast<int>(blockIdx.x / static_cast<unsigned>(g0.tiles_o));
+    const int tile_step = static_cast<int>(gridDim.x / static_cast<unsigned>(g0.tiles_o));
+    const int tiles_m = g0.tiles_q * g0.tiles_p * g0.tiles_n;
+    const int items = nlayers * tiles_m;
 
     if (tid == 0) TC_TRACE(TR_START, 0);
     pdl_release();
@@ -1034,11 +1109,12 @@ bitserial_conv_tc_persistent_kernel(const __grid_constant__ TcArgs g)
         for (int s = 0; s < TCP_NSE; ++s) { mbar_init(&full_e[s], 1); mbar_init(&empty_e[s], 1); }
         for (int s = 0; s < 2; ++s) { mbar_init(&full_acc[s], 1); mbar_init(&empty_acc[s], 1); }
         mbar_init(wgt_full, 1);
+        mbar_init(wgt_free, 1);
         fence_barrier_init();
         fence_proxy_async();
     }
     if (warp == 9) {
-        tmem_alloc(tmem_slot, static_cast<unsigned>(g.tmem_cols));
+        tmem_alloc(tmem_slot, static_cast<unsigned>(g0.tmem_cols));
         tmem_relinquish();
     }
     // Only the barriers and the tensor-memory address are needed by every role: the producer starts fetching right
@@ -1048,35 +1124,83 @@ bitserial_conv_tc_persistent_kernel(const __grid_constant__ TcArgs g)
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
 
-    if (warp == 8) {
-        // ------------------------------------------------------------------ producer: filters once, then packed chunks
+    if (MAXL == 1 && warp == 8) {
+        // ------------------------------------------------------------------ producer of the one-layer kernel: filters once, then packed tiles
         if (lane == 0) {
-            mbar_expect_tx(wgt_full, static_cast<unsigned>(g.nchunks * g.b_bytes));
-            const int blk_bytes = g.b_bytes / g.MB;
-            const size_t blk_stride = static_cast<size_t>(g.opad8) * RS * (g.CK >> 4) * 128;      // one layout block, all filters
-            const int8_t* src = g.wgt + static_cast<size_t>(o0 >> 3) * RS * (g.CK >> 4) * 128;
+            mbar_expect_tx(wgt_full, static_cast<unsigned>(g0.nchunks * g0.b_bytes));
+            const int blk_bytes = g0.b_bytes / g0.MB;
+            const size_t blk_stride = static_cast<size_t>(g0.opad8) * RS * (g0.CK >> 4) * 128;     // one layout block, all filters
+            const int8_t* src = g0.wgt + static_cast<size_t>(o0 >> 3) * RS * (g0.CK >> 4) * 128;
             unsigned char* dst = s_w;
-            for (int c = 0; c < g.nchunks * g.MB; ++c, src += blk_stride, dst += blk_bytes)       // layout blocks, consecutive in shared memory
+            for (int c = 0; c < g0.nchunks * g0.MB; ++c, src += blk_stride, dst += blk_bytes)      // layout blocks, consecutive in shared memory
                 bulk_load(dst, src, static_cast<unsigned>(blk_bytes), wgt_full);
             TC_TRACE(TR_SETUP, 0);
             pdl_acquire();                // activations come from the preceding kernel; the filters above do not
             TC_TRACE(TR_PDL, 0);
-            TcTileWalker tw = tc_walk_init(g, first_tile, tile_step);
+            TcTileWalker tw = tc_walk_init(g0, first_tile, tile_step);
             TcRing rp;
             bool ok = true;
-            for (int i = 0; tw.mt < tiles_m; tc_walk_next(g, tw), ++i) {
+            for (int i = 0; tw.mt < tiles_m; tc_walk_next(g0, tw), ++i) {
                 if (!mbar_spin_bounded(&empty_p[rp.idx], rp.phase ^ 1u)) { ok = false; break; }
                 TC_TRACE(TR_LOAD, i);
-                tc_load_tile(g, s_p + rp.idx * g.pa_bytes, &full_p[rp.idx], tc_walk_tile(g, tw));
-                rp.advance(g.nsp);
+                tc_load_tile(g0, s_p + rp.idx * g0.pa_bytes, &full_p[rp.idx], tc_walk_tile(g0, tw));
+                rp.advance(g0.nsp);
             }
-            if (!ok) atomicOr(g.status, STATUS_TIMEOUT);
+            if (!ok) atomicOr(g0.status, STATUS_TIMEOUT);
         }
         __syncwarp();
+    } else if (warp == 8) {
+        // ------------------------------------------------------------------ producer of a chain: packed tiles, in item order
+        if (lane == 0) TC_TRACE(TR_SETUP, 0);
+        pdl_acquire();                    // activations come from the preceding kernel
+        if (lane == 0) TC_TRACE(TR_PDL, 0);
+        unsigned target = 0;
+        if (MAXL > 1 && nlayers > 1) target = (ld_acquire_gpu(ch.ctl) + 1u) * static_cast<unsigned>(g0.tiles_o);
+        TcItemWalker x = tc_item_init(g0, first_tile, tile_step, tiles_m);
+        TcRing rp;
+        bool ok = true;
+        int i = 0;
+        // One copy of the loop per layer: the layer's arguments are then read at fixed offsets of the parameter block
+        // (operands of the instructions) instead of being fetched through a run-time index after every barrier.
+#pragma unroll
+        for (int l = 0; l < MAXL; ++l) {
+            const TcArgs& g = ch.L[l];
+            for (; ok && x.l == l && l < nlayers; tc_item_next(g0, x, tiles_m), ++i) {
+                if (MAXL > 1 && l > 0) {
+                    // the halo of this tile was written by the tile itself and its neighbours in the preceding layer
+                    bool mine = true;
+                    if (lane < 9) {
+                        const int dy = g.flat ? 0 : lane / 3 - 1, dx = g.flat ? 0 : lane % 3 - 1;
+                        const int ip = x.w.ip + dy, iq = x.w.iq + dx;
+                        const bool exists = g.flat ? lane == 4 : (ip >= 0 && ip < g.tiles_p && iq >= 0 && iq < g.tiles_q);
+                        if (exists) {
+                            const int nb = g.flat ? x.w.mt : (x.w.in * g.tiles_p + ip) * g.tiles_q + iq;
+                            mine = tc_flag_wait(ch.flags + static_cast<size_t>(l - 1) * tiles_m + nb, target);
+                        }
+                    }
+                    ok = __all_sync(0xffffffffu, mine);
+                    if (!ok) break;
+                }
+                unsigned mine_ok = 1;
+                if (lane == 0) {
+                    if (MAXL > 1 && l > 0) fence_proxy_async_global();       // stores of other SMs, read by the copy engine
+                    mine_ok = mbar_spin_bounded(&empty_p[rp.idx], rp.phase ^ 1u) ? 1u : 0u;
+                    if (mine_ok) {
+                        TC_TRACE(TR_LOAD, i);
+                        tc_load_tile(g, s_p + rp.idx * g.pa_bytes, &full_p[rp.idx], tc_walk_tile(g, x.w));
+                    }
+                }
+                ok = __shfl_sync(0xffffffffu, mine_ok, 0) != 0;
+                if (!ok) break;
+                rp.advance(g0.nsp);
+            }
+        }
+        if (!ok && lane == 0) atomicOr(g0.status, STATUS_TIMEOUT);
+        __syncwarp();
     } else if (warp == 9) {
-        // ------------------------------------------------------------------ MMA issuer
-        if (lane == 0) {
-            const TcIssue is = tc_make_issue(g);
+        // ------------------------------------------------------------------ MMA issuer (in a chain it also fetches the filters of each layer)
+        if (MAXL == 1 && lane == 0) {
+            const TcIssue is = tc_make_issue(g0);
             const uint32_t e_base = smem_u32(s_e), w_base = smem_u32(s_w);
             bool ok = mbar_spin_bounded(wgt_full, 0);       // also keeps the CTA alive until the filter copy has landed
             TC_TRACE(TR_WGT, 0);
@@ -1086,98 +1210,201 @@ bitserial_conv_tc_persistent_kernel(const __grid_constant__ TcArgs g)
                 ok = mbar_spin_bounded(&empty_acc[ra.idx], ra.phase ^ 1u);
                 if (!ok) break;
                 tc_fence_after();
-                const uint32_t tmem_acc = tmem_base + static_cast<uint32_t>(ra.idx * g.TN);
+                const uint32_t tmem_acc = tmem_base + static_cast<uint32_t>(ra.idx * g0.TN);
                 uint32_t wa = w_base;
-                for (int c = 0; c < g.nchunks; ++c, wa += static_cast<uint32_t>(g.b_bytes)) {
+                for (int c = 0; c < g0.nchunks; ++c, wa += static_cast<uint32_t>(g0.b_bytes)) {
                     if (!mbar_spin_bounded(&full_e[re.idx], re.phase)) { ok = false; break; }
                     if (c == 0) TC_TRACE(TR_MBEG, i);
                     tc_fence_after();
-                    tc_issue_chunk(is, e_base + static_cast<uint32_t>(re.idx * g.e_bytes), wa, tmem_acc, c == 0);
+                    tc_issue_chunk(is, e_base + static_cast<uint32_t>(re.idx * g0.e_bytes), wa, tmem_acc, c == 0);
                     if (c == 0) TC_TRACE(TR_M_ISSUED, i);
-#ifdef BS_TC_DBG_DRAIN
-                    if (c == 0 && i < 2) { umma_commit(wgt_full); mbar_spin_bounded(wgt_full, (i + 1) & 1); TC_TRACE(19, i); }
-#endif
                     umma_commit(&empty_e[re.idx]);
-                    re.advance(g.nse);
+                    re.advance(g0.nse);
                 }
                 if (ok) umma_commit(&full_acc[ra.idx]);
                 TC_TRACE(TR_MEND, i);
                 ra.advance(2);
             }
-            if (!ok) atomicOr(g.status, STATUS_TIMEOUT);
+            if (!ok) atomicOr(g0.status, STATUS_TIMEOUT);
+        } else if (lane == 0) {
+            const TcIssue is = tc_make_issue(g0);
+            const uint32_t e_base = smem_u32(s_e), w_base = smem_u32(s_w);
+            const int blk_bytes = g0.b_bytes / g0.MB;
+            const size_t blk_stride = static_cast<size_t>(g0.opad8) * RS * (g0.CK >> 4) * 128;    // one layout block, all filters
+            TcRing re, ra;                                  // expanded chunks; accumulator buffers
+            bool ok = true;
+            int cur_l = -1;
+            unsigned wphase = 0;
+            int l = first_tile / tiles_m, rem = first_tile - l * tiles_m;
+            const int dl = tile_step / tiles_m, drem = tile_step - dl * tiles_m;
+            for (int i = 0; l < nlayers && ok; ++i) {
+                if (l != cur_l) {
+                    if (cur_l >= 0) {       // the filters in shared memory are still being read: wait for those MMAs
+                        umma_commit(wgt_free);
+                        ok = mbar_spin_bounded(wgt_free, wphase ^ 1u);
+                        if (!ok) break;
+                    }
+                    const TcArgs& g = ch.L[MAXL > 1 ? l : 0];
+                    mbar_expect_tx(wgt_full, static_cast<unsigned>(g0.nchunks * g0.b_bytes));
+                    const int8_t* src = g.wgt + static_cast<size_t>(o0 >> 3) * RS * (g0.CK >> 4) * 128;
+                    unsigned char* dst = s_w;
+                    for (int c = 0; c < g0.nchunks * g0.MB; ++c, src += blk_stride, dst += blk_bytes)   // layout blocks, consecutive in shared memory
+                        bulk_load(dst, src, static_cast<unsigned>(blk_bytes), wgt_full);
+                    ok = mbar_spin_bounded(wgt_full, wphase);       // also keeps the CTA alive until the filter copy has landed
+                    if (!ok) break;
+                    if (cur_l < 0) TC_TRACE(TR_WGT, 0);
+                    wphase ^= 1u;
+                    cur_l = l;
+                }
+                ok = mbar_spin_bounded(&empty_acc[ra.idx], ra.phase ^ 1u);
+                if (!ok) break;
+                tc_fence_after();
+                const uint32_t tmem_acc = tmem_base + static_cast<uint32_t>(ra.idx * g0.TN);
+                uint32_t wa = w_base;
+                for (int c = 0; c < g0.nchunks; ++c, wa += static_cast<uint32_t>(g0.b_bytes)) {
+                    if (!mbar_spin_bounded(&full_e[re.idx], re.phase)) { ok = false; break; }
+                    if (c == 0) TC_TRACE(TR_MBEG, i);
+                    tc_fence_after();
+                    tc_issue_chunk(is, e_base + static_cast<uint32_t>(re.idx * g0.e_bytes), wa, tmem_acc, c == 0);
+                    if (c == 0) TC_TRACE(TR_M_ISSUED, i);
+                    umma_commit(&empty_e[re.idx]);
+                    re.advance(g0.nse);
+                }
+                if (ok) umma_commit(&full_acc[ra.idx]);
+                TC_TRACE(TR_MEND, i);
+                ra.advance(2);
+                l += dl; rem += drem;
+                if (rem >= tiles_m) { rem -= tiles_m; ++l; }
+            }
+            if (!ok) atomicOr(g0.status, STATUS_TIMEOUT);
         }
         __syncwarp();
     } else if (warp >= 4 && warp < 8) {
         // ------------------------------------------------------------------ expanders (warps 4-7)
         const int et = tid - 128;
-        tc_build_lut(g, s_lut, et, 128);
+        tc_build_lut(g0, s_lut, et, 128);
         group_sync(1);
-        const TcExpand xp = tc_expand_init(g, et, 128);
+        const TcExpand xp = tc_expand_init(g0, et, 128);
         TcRing rp, re;
-        int i = 0;
         bool ok = true;
-        for (int mt = first_tile; mt < tiles_m && ok; mt += tile_step, ++i) {
+        for (int i = 0, it = first_tile; it < items && ok; it += tile_step, ++i) {
             ok = mbar_wait_warp(&full_p[rp.idx], rp.phase, lane);
             if (et == 0) TC_TRACE(TR_XBEG, i);
-            const uint32_t* pa = reinterpret_cast<const uint32_t*>(s_p + rp.idx * g.pa_bytes);
-            for (int c = 0; c < g.nchunks; ++c) {
+            const uint32_t* pa = reinterpret_cast<const uint32_t*>(s_p + rp.idx * g0.pa_bytes);
+            for (int c = 0; c < g0.nchunks; ++c) {
                 if (ok) ok = mbar_wait_warp(&empty_e[re.idx], re.phase ^ 1u, lane);
                 ok = group_all(1, ok);
                 if (!ok) break;
                 if (et == 0 && c == 0) TC_TRACE(TR_X_BEG0, i);
-                tc_expand_chunk<A>(g, xp, pa, s_e + re.idx * g.e_bytes, s_lut, et, c);
+                tc_expand_chunk<A>(g0, xp, pa, s_e + re.idx * g0.e_bytes, s_lut, et, c);
                 fence_proxy_async();
                 group_sync(1);                       // all 128 expander threads have written and fenced
                 if (et == 0 && c == 0) TC_TRACE(TR_X_DONE0, i);
                 if (et == 0) mbar_arrive(&full_e[re.idx]);
-                re.advance(g.nse);
+                re.advance(g0.nse);
             }
             if (et == 0) TC_TRACE(TR_XEND, i);
             if (ok && et == 0) mbar_arrive(&empty_p[rp.idx]);   // ordered after the last group_sync: every thread is done reading
-            rp.advance(g.nsp);
+            rp.advance(g0.nsp);
         }
-        if (!ok) atomicOr(g.status, STATUS_TIMEOUT);
+        if (!ok) atomicOr(g0.status, STATUS_TIMEOUT);
     } else {
         // ------------------------------------------------------------------ epilogue (warps 0-3, and 10-13 when WIDE)
         constexpr int EPI_THREADS = WIDE ? 256 : 128;
         const int second = warp >= 10 ? 1 : 0;                 // second set: the odd groups of 32 filters
         const int ei = second ? tid - 192 : tid;               // 0 .. EPI_THREADS-1
-        tc_epilogue_tables(g, tc_smem, s_sb, s_bounds, o0, ei, EPI_THREADS);
-        group_sync(2, EPI_THREADS);
-        uint32_t thr = 0;                 // shared-memory address of the thresholds, 0: floating-point comparison
-        if (g.off_thr) {                  // while the pipeline fills: comparison bounds -> integer thresholds
-            int4* s_thr = reinterpret_cast<int4*>(tc_smem + g.off_thr);
-            int* thr_ok = reinterpret_cast<int*>(s_thr + g.thr_pats * g.TN);
-            tc_build_thresholds(g, s_thr, thr_ok, s_sb, s_bounds, o0, ei, EPI_THREADS);
+        if constexpr (MAXL == 1) {
+            // the one-layer kernel keeps its own, simpler loop: the chain form of it below measured 1.5 % slower on a whole network
+            tc_epilogue_tables(g0, tc_smem, s_sb, s_bounds, o0, ei, EPI_THREADS);
             group_sync(2, EPI_THREADS);
-            if (*thr_ok) thr = smem_u32(s_thr);
+            uint32_t thr = 0;                 // shared-memory address of the thresholds, 0: floating-point comparison
+            if (g0.off_thr) {                  // while the pipeline fills: comparison bounds -> integer thresholds
+                int4* s_thr = reinterpret_cast<int4*>(tc_smem + g0.off_thr);
+                int* thr_ok = reinterpret_cast<int*>(s_thr + g0.thr_pats * g0.TN);
+                tc_build_thresholds(g0, s_thr, thr_ok, s_sb, s_bounds, o0, ei, EPI_THREADS);
+                group_sync(2, EPI_THREADS);
+                if (*thr_ok) thr = smem_u32(s_thr);
+            }
+            const TcEpiThread eth = tc_epi_thread(g0, (warp & 3) * 32 + lane);
+            TcTileWalker tw = tc_walk_init(g0, first_tile, tile_step);
+            pdl_acquire();                    // the epilogue reads the residual and overwrites buffers the preceding kernel may use
+            TcRing ra;
+            bool ok = true;
+            for (int i = 0; tw.mt < tiles_m; tc_walk_next(g0, tw), ++i) {
+                ok = group_all(2, mbar_wait_warp(&full_acc[ra.idx], ra.phase, lane), EPI_THREADS);
+                if (!ok) break;
+                if (tid == 0) TC_TRACE(TR_EBEG, i);
+                tc_fence_after();
+                tc_epilogue_tile(g0, tmem_base + static_cast<uint32_t>(ra.idx * g0.TN), (warp & 3) * 32 + lane, warp & 3, tc_walk_tile(g0, tw), eth, o0,
+                                 s_sb, s_bounds, thr, WIDE ? second : 0, WIDE ? 2 : 1, i);
+                tc_fence_before();
+                group_sync(2, EPI_THREADS);              // every epilogue warp has read its accumulator rows
+                if (tid == 0) TC_TRACE(TR_EEND, i);
+                if (tid == 0) mbar_arrive(&empty_acc[ra.idx]);
+                ra.advance(2);
+            }
+            if (!ok) atomicOr(g0.status, STATUS_TIMEOUT);
+        } else {
+            const TcEpiThread eth = tc_epi_thread(g0, (warp & 3) * 32 + lane);
+            TcItemWalker x = tc_item_init(g0, first_tile, tile_step, tiles_m);
+            TcRing ra;
+            bool ok = true;
+            int i = 0;
+#pragma unroll
+            for (int l = 0; l < MAXL; ++l) {          // one copy of the loop per layer, see the producer
+                const TcArgs& g = ch.L[l];
+                if (!ok || x.l != l || l >= nlayers) continue;
+                // tables of the layer (the preceding tile's group_sync has every thread past its last use of the old ones)
+                tc_epilogue_tables(g, tc_smem, s_sb, s_bounds, o0, ei, EPI_THREADS);
+                group_sync(2, EPI_THREADS);
+                uint32_t thr = 0;                 // shared-memory address of the thresholds, 0: floating-point comparison
+                if (g.off_thr) {                  // while the pipeline fills: comparison bounds -> integer thresholds
+                    int4* s_thr = reinterpret_cast<int4*>(tc_smem + g.off_thr);
+                    int* thr_ok = reinterpret_cast<int*>(s_thr + g.thr_pats * g.TN);
+                    tc_build_thresholds(g, s_thr, thr_ok, s_sb, s_bounds, o0, ei, EPI_THREADS);
+                    group_sync(2, EPI_THREADS);
+                    if (*thr_ok) thr = smem_u32(s_thr);
+                }
+                if (i == 0) pdl_acquire();        // the epilogue reads the residual and overwrites buffers the preceding kernel may use
+                for (; x.l == l; tc_item_next(g0, x, tiles_m), ++i) {
+                    ok = group_all(2, mbar_wait_warp(&full_acc[ra.idx], ra.phase, lane), EPI_THREADS);
+                    if (!ok) break;
+                    if (tid == 0) TC_TRACE(TR_EBEG, i);
+                    tc_fence_after();
+                    tc_epilogue_tile(g, tmem_base + static_cast<uint32_t>(ra.idx * g0.TN), (warp & 3) * 32 + lane, warp & 3, tc_walk_tile(g, x.w), eth, o0,
+                                     s_sb, s_bounds, thr, WIDE ? second : 0, WIDE ? 2 : 1, i, true);
+                    if (l + 1 < nlayers) fence_proxy_async_global();     // the next layer reads these stores through the copy engine
+                    tc_fence_before();
+                    group_sync(2, EPI_THREADS);              // every epilogue warp has read its accumulator rows
+                    if (tid == 0) TC_TRACE(TR_EEND, i);
+                    if (tid == 0) {
+                        mbar_arrive(&empty_acc[ra.idx]);
+                        if (l + 1 < nlayers) {
+                            __threadfence();                 // cumulative: orders the stores of the whole group (seen through the barrier) before the counter
+                            atomicAdd(ch.flags + static_cast<size_t>(l) * tiles_m + x.w.mt, 1u);
+                        }
+                    }
+                    ra.advance(2);
+                }
+            }
+            if (!ok) atomicOr(g0.status, STATUS_TIMEOUT);
         }
-        const TcEpiThread eth = tc_epi_thread(g, (warp & 3) * 32 + lane);
-        TcTileWalker tw = tc_walk_init(g, first_tile, tile_step);
-        pdl_acquire();                    // the epilogue reads the residual and overwrites buffers the preceding kernel may use
-        TcRing ra;
-        bool ok = true;
-        for (int i = 0; tw.mt < tiles_m; tc_walk_next(g, tw), ++i) {
-            ok = group_all(2, mbar_wait_warp(&full_acc[ra.idx], ra.phase, lane), EPI_THREADS);
-            if (!ok) break;
-            if (tid == 0) TC_TRACE(TR_EBEG, i);
-            tc_fence_after();
-            tc_epilogue_tile(g, tmem_base + static_cast<uint32_t>(ra.idx * g.TN), (warp & 3) * 32 + lane, warp & 3, tc_walk_tile(g, tw), eth, o0,
-                             s_sb, s_bounds, thr, WIDE ? second : 0, WIDE ? 2 : 1, i);
-            tc_fence_before();
-            group_sync(2, EPI_THREADS);              // every epilogue warp has read its accumulator rows
-            if (tid == 0) TC_TRACE(TR_EEND, i);
-            if (tid == 0) mbar_arrive(&empty_acc[ra.idx]);
-            ra.advance(2);
-        }
-        if (!ok) atomicOr(g.status, STATUS_TIMEOUT);
     }
     tc_fence_before();
     __syncthreads();
     if (tid == 0) TC_TRACE(TR_END, 0);
     if (warp == 9) {
         tc_fence_after();
-        tmem_dealloc(tmem_base, static_cast<unsigned>(g.tmem_cols));
+        tmem_dealloc(tmem_base, static_cast<unsigned>(g0.tmem_cols));
+    }
+    if (MAXL > 1 && nlayers > 1 && tid == 0) {
+        // the last CTA out counts the launch: every CTA has read ctl[0] long before
+        __threadfence();
+        if (atomicAdd(ch.ctl + 1, 1u) == gridDim.x - 1) {
+            atomicExch(ch.ctl + 1, 0u);
+            __threadfence();
+            atomicAdd(ch.ctl, 1u);
+        }
     }
 }
 
@@ -1273,28 +1500,12 @@ static int tc_validate(const bs_conv_params* p)
     return BS_OK;
 }
 
-// Launch with or without the programmatic-serialisation attribute.  With it, the grid may begin (barrier and TMEM
-// set-up, byte table, filter fetch) while the preceding kernel of the stream drains; everything it reads before
-// pdl_acquire() must therefore have been final before that preceding kernel was launched.
-static cudaError_t tc_launch(void (*kern)(TcArgs), unsigned grid, unsigned block, size_t smem, cudaStream_t st, bool chained,
-                             const TcArgs& g)
-{
-    cudaLaunchConfig_t cfg{};
-    cfg.gridDim = dim3(grid);
-    cfg.blockDim = dim3(block);
-    cfg.dynamicSmemBytes = smem;
-    cfg.stream = st;
-    cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    attr[0].val.programmaticStreamSerializationAllowed = 1;
-    cfg.attrs = attr;
-    cfg.numAttrs = chained ? 1 : 0;
-    return cudaLaunchKernelEx(&cfg, kern, g);
-}
-
-// plan_only: validate and plan (tiles, shared memory) without touching any tensor or launching: the support query.
-static int tc_conv_impl(const uint32_t* act, const int8_t* wgt, const bs_conv_params* p, int32_t* out_i32, uint32_t* out_packed,
-                        cudaStream_t st, bool chained = false, bool plan_only = false)
+// Validates and plans one layer: tiles, shared-memory layout, kernel arguments (and the tensor map unless plan_only, which
+// touches no tensor: the support query).  `smem` receives the dynamic shared memory of the plan.
+// chain_n > 1: the layer is one of chain_n same-shaped layers run by one launch, which needs the resident-filter plan and has
+// chain_n times the pixel tiles to spread over the SMs.
+static int tc_plan(const uint32_t* act, const int8_t* wgt, const bs_conv_params* p, int32_t* out_i32, uint32_t* out_packed,
+                   bool plan_only, TcArgs& g, size_t& smem_out, int chain_n = 1)
 {
     int rc = tc_validate(p);
     if (rc != BS_OK) return rc;
@@ -1303,7 +1514,7 @@ static int tc_conv_impl(const uint32_t* act, const int8_t* wgt, const bs_conv_pa
         if (!aligned16(act) || !aligned16(wgt) || (out_i32 && !aligned16(out_i32)) || (out_packed && !aligned16(out_packed)))
             return BS_ERR_ALIGNMENT;
     }
-    TcArgs g{};
+    g = TcArgs{};
     g.P = (p->H + 2 * p->pad - p->R) / p->stride + 1;
     g.Q = (p->W + 2 * p->pad - p->S) / p->stride + 1;
     if (out_packed) {
@@ -1428,7 +1639,7 @@ static int tc_conv_impl(const uint32_t* act, const int8_t* wgt, const bs_conv_pa
     for (int TN = 128; TN >= 32; TN /= 2) {
         if (TN > tn_max) continue;
         if (TN / 2 >= round_up_i(p->O, 32)) continue;                      // tile twice as wide as the filter bank
-        const long long pairs = tiles_m * ceil_div(p->O, TN);
+        const long long pairs = tiles_m * chain_n * ceil_div(p->O, TN);
         if (TN > 32 && pairs < sms) continue;
         const size_t wbytes = static_cast<size_t>(g.nchunks) * TN * RS * CKP;
         const int shapes[4][2] = {{2, 2}, {2, 2}, {2, 2}, {1, 2}};      // (packed-tile stages, expanded-chunk stages)
@@ -1458,7 +1669,7 @@ static int tc_conv_impl(const uint32_t* act, const int8_t* wgt, const bs_conv_pa
     // A resident plan also loses when its CTAs see hardly more than one pixel tile each: nothing amortises the filter
     // fetch, and the streaming kernel has twice the expand/epilogue warps.  Measured on the bottleneck stack for
     // reductions of 512 and more (shallower ones are epilogue-bound and stay resident).
-    if (!keep_narrow && g.persistent && kred >= 512) {
+    if (!keep_narrow && chain_n == 1 && g.persistent && kred >= 512) {        // (a chain exists to save launches: it stays resident)
         int cps_est = static_cast<int>((225 * 1024) / (smem + 1024));
         if (cps_est > 3) cps_est = 3;
         if (cps_est * 2 * g.TN > 512) cps_est = 512 / (2 * g.TN);
@@ -1576,6 +1787,7 @@ static int tc_conv_impl(const uint32_t* act, const int8_t* wgt, const bs_conv_pa
         }
     }
 
+    smem_out = smem;
     if (plan_only) return BS_OK;
     auto enc = tc_encode_fn();
     if (!enc) return BS_ERR_CUDA;
@@ -1599,46 +1811,92 @@ static int tc_conv_impl(const uint32_t* act, const int8_t* wgt, const bs_conv_pa
                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     }
     if (cr != CUDA_SUCCESS) return BS_ERR_CUDA;
+    return BS_OK;
+}
 
-    if (g.persistent) {
-        int cps = ctas_per_sm(smem);                                       // CTAs that fit on one SM: shared memory,
-        if (cps > 3) cps = 3;                                              // registers (launch bounds) and
-        if (cps * 2 * g.TN > 512) cps = 512 / (2 * g.TN);                  // tensor-memory columns
+// CTAs of the resident-filter kernel that fit on one SM: shared memory, registers (launch bounds) and tensor-memory columns.
+static int tcp_ctas_per_sm(size_t smem, int TN)
+{
+    int cps = static_cast<int>((225 * 1024) / (smem + 1024));
+    if (cps > 3) cps = 3;
+    if (cps * 2 * TN > 512) cps = 512 / (2 * TN);
 #ifdef BS_TUNING
-        if (const char* e = getenv("BS_TC_CPSMAX")) { const int m = atoi(e); if (cps > m) cps = m; }
+    if (const char* e = getenv("BS_TC_CPSMAX")) { const int m = atoi(e); if (cps > m) cps = m; }
 #endif
-        if (cps < 1) cps = 1;
+    return cps < 1 ? 1 : cps;
+}
+
+// The instantiation for a plan: CTAs per SM and whether registers allow eight epilogue warps (one or two CTAs per SM and
+// at least two groups of 32 filters in the tile).
+template <int MAXL>
+static void (*tcp_pick(int A, int cps, bool wide))(TcChainArgs<MAXL>)
+{
+    switch (A) {
+#define BS_TCP_PICK(ABITS) (cps >= 3 ? bitserial_conv_tc_persistent_kernel<ABITS, 3, false, MAXL> \
+                          : cps == 2 ? (wide ? bitserial_conv_tc_persistent_kernel<ABITS, 2, true, MAXL> : bitserial_conv_tc_persistent_kernel<ABITS, 2, false, MAXL>) \
+                                     : (wide ? bitserial_conv_tc_persistent_kernel<ABITS, 1, true, MAXL> : bitserial_conv_tc_persistent_kernel<ABITS, 1, false, MAXL>))
+        case 1: return BS_TCP_PICK(1);
+        case 2: return BS_TCP_PICK(2);
+        case 3: return BS_TCP_PICK(3);
+        default: return BS_TCP_PICK(4);
+#undef BS_TCP_PICK
+    }
+}
+
+// Launch with or without the programmatic-serialisation attribute.  With it, the grid may begin (barrier and TMEM
+// set-up, byte table, filter fetch) while the preceding kernel of the stream drains; everything it reads before
+// pdl_acquire() must therefore have been final before that preceding kernel was launched.
+template <typename Args>
+static cudaError_t tc_launch(void (*kern)(Args), unsigned grid, unsigned block, size_t smem, cudaStream_t st, bool chained, const Args& g)
+{
+    cudaLaunchConfig_t cfg{};
+    cfg.gridDim = dim3(grid);
+    cfg.blockDim = dim3(block);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = chained ? 1 : 0;
+    return cudaLaunchKernelEx(&cfg, kern, g);
+}
+
+static int tc_conv_impl(const uint32_t* act, const int8_t* wgt, const bs_conv_params* p, int32_t* out_i32, uint32_t* out_packed,
+                        cudaStream_t st, bool chained = false, bool plan_only = false)
+{
+    TcArgs g;
+    size_t smem = 0;
+    const int rc = tc_plan(act, wgt, p, out_i32, out_packed, plan_only, g, smem);
+    if (rc != BS_OK || plan_only) return rc;
+    const int A = p->a_bits;
+    if (g.persistent) {
+        const int sms = device_sm_count();
+        const long long tiles_m = static_cast<long long>(g.tiles_q) * g.tiles_p * g.tiles_n;
+        const int cps = tcp_ctas_per_sm(smem, g.TN);
         long long per_o = (static_cast<long long>(sms) * cps) / g.tiles_o;
         if (per_o < 1) per_o = 1;
         if (per_o > tiles_m) per_o = tiles_m;
         const long long grid = per_o * g.tiles_o;
-        // eight epilogue warps when registers allow (one or two CTAs per SM) and the tile has at least two groups of 32 filters
         bool wide = cps <= 2 && g.TN >= 64;
 #ifdef BS_TUNING
         if (const char* e = getenv("BS_TC_WIDE")) wide = wide && atoi(e) != 0;
 #endif
-        void (*kern)(TcArgs) = nullptr;
-        switch (A) {
-#define BS_TCP_PICK(ABITS) (cps >= 3 ? bitserial_conv_tc_persistent_kernel<ABITS, 3> \
-                          : cps == 2 ? (wide ? bitserial_conv_tc_persistent_kernel<ABITS, 2, true> : bitserial_conv_tc_persistent_kernel<ABITS, 2>) \
-                                     : (wide ? bitserial_conv_tc_persistent_kernel<ABITS, 1, true> : bitserial_conv_tc_persistent_kernel<ABITS, 1>))
-            case 1: kern = BS_TCP_PICK(1); break;
-            case 2: kern = BS_TCP_PICK(2); break;
-            case 3: kern = BS_TCP_PICK(3); break;
-            default: kern = BS_TCP_PICK(4); break;
-#undef BS_TCP_PICK
-        }
+        void (*kern)(TcChainArgs<1>) = tcp_pick<1>(A, cps, wide);
         if (smem > 48 * 1024 &&
             cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)) != cudaSuccess) {
             cudaGetLastError();
             return BS_ERR_CUDA;
         }
-        if (tc_launch(kern, static_cast<unsigned>(grid), wide ? TCP_THREADS_WIDE : TCP_THREADS, smem, st, chained, g) != cudaSuccess) {
+        TcChainArgs<1> ch{};
+        ch.L[0] = g; ch.nlayers = 1; ch.flags = nullptr; ch.ctl = nullptr;
+        if (tc_launch(kern, static_cast<unsigned>(grid), wide ? TCP_THREADS_WIDE : TCP_THREADS, smem, st, chained, ch) != cudaSuccess) {
             cudaGetLastError();
             return BS_ERR_CUDA;
         }
         return BS_OK;
     }
+    const long long tiles_m = static_cast<long long>(g.tiles_q) * g.tiles_p * g.tiles_n;
     const long long grid = ceil_div_ll(tiles_m, g.PT) * g.tiles_o;
     if (grid > 0x7fffffffLL) return BS_ERR_UNSUPPORTED;
     void (*kern)(TcArgs) = nullptr;
@@ -1660,10 +1918,109 @@ static int tc_conv_impl(const uint32_t* act, const int8_t* wgt, const bs_conv_pa
     return BS_OK;
 }
 
+// ----------------------------------------------------------------------------- several layers in one launch
+
+// Pixel tiles of one layer of a chain, or 0 when the layers cannot run as one chain: 2..TC_CHAIN_MAX layers that all take
+// the resident-filter plan with the same geometry (batch, image, channels = filters, kernel, stride 1, output as large as the
+// input), the same activation and weight formats, and packed outputs whose width is the next layer's activation width.
+static long long tc_chain_plan(int n, const uint32_t* const* act, const int8_t* const* wgt, const bs_conv_params* params,
+                               uint32_t* const* out, bool plan_only, TcArgs* L, size_t& smem)
+{
+    if (n < 2 || n > TC_CHAIN_MAX || !params) return 0;
+    smem = 0;
+    for (int l = 0; l < n; ++l) {
+        const bs_conv_params* p = &params[l];
+        bs_conv_params q = *p;
+        if (plan_only) {                        // the epilogue's kind (thresholds, residual patterns) still shapes the plan
+            static const float dummy = 0.f;
+            q.scale = &dummy; q.bias = &dummy;
+        }
+        size_t s = 0;
+        // a non-null placeholder stands for the output in a query: only "packed output wanted" matters to the plan
+        uint32_t* o = plan_only ? reinterpret_cast<uint32_t*>(16) : out[l];
+        if (tc_plan(plan_only ? nullptr : act[l], plan_only ? nullptr : wgt[l], &q, nullptr, o, plan_only, L[l], s, n) != BS_OK) return 0;
+        if (!L[l].persistent || q.out_bits <= 0) return 0;
+        if (p->stride != 1 || L[l].P != p->H || L[l].Q != p->W || p->O != p->C) return 0;
+        if (s > smem) smem = s;
+        if (l == 0) continue;
+        const bs_conv_params* p0 = &params[0];
+        if (p->N != p0->N || p->C != p0->C || p->H != p0->H || p->W != p0->W || p->O != p0->O || p->R != p0->R || p->S != p0->S ||
+            p->pad != p0->pad || p->a_bits != p0->a_bits || p->a_sign != p0->a_sign || p->w_bits != p0->w_bits || p->w_sign != p0->w_sign)
+            return 0;
+        if (params[l - 1].out_bits != p->a_bits || params[l - 1].out_sign != p->a_sign) return 0;
+        const TcArgs &a = L[0], &b = L[l];
+        if (a.TN != b.TN || a.MB != b.MB || a.nchunks != b.nchunks || a.nsp != b.nsp || a.nse != b.nse || a.off_p != b.off_p ||
+            a.off_e != b.off_e || a.off_sb != b.off_sb || a.off_bar != b.off_bar || a.off_lut != b.off_lut || a.tmem_cols != b.tmem_cols ||
+            a.b_bytes != b.b_bytes || a.pa_bytes != b.pa_bytes || a.e_bytes != b.e_bytes || a.pmode != b.pmode || a.flat != b.flat)
+            return 0;
+    }
+    for (int l = 0; l < n; ++l) {
+        if (params[l].out_c_offset != 0 || params[l].out_c_total != params[l].O) return 0;       // a layer's output is a whole tensor
+        if (params[l].residual && (params[l].res_c_offset != 0 || params[l].res_c_total != params[l].O)) return 0;
+    }
+    if (!plan_only) {
+        // a layer may read (activations, residual) what an EARLIER layer of the chain wrote, or tensors final before the launch
+        for (int l = 0; l < n; ++l)
+            for (int k = l; k < n; ++k)
+                if (act[l] == out[k] || (params[l].residual && params[l].residual == out[k])) return 0;
+    }
+    return static_cast<long long>(L[0].tiles_q) * L[0].tiles_p * L[0].tiles_n;
+}
+
+static size_t tc_chain_ws_bytes(int n, long long tiles_m) { return (static_cast<size_t>(n) * tiles_m + 4) * sizeof(unsigned); }
+
+static int tc_chain_impl(int n, const uint32_t* const* act, const int8_t* const* wgt, const bs_conv_params* params,
+                         uint32_t* const* out, void* workspace, size_t workspace_bytes, cudaStream_t st, bool chained)
+{
+    if (!act || !wgt || !params || !out || !workspace) return BS_ERR_INVALID_ARG;
+    if (n < 2 || n > TC_CHAIN_MAX) return BS_ERR_UNSUPPORTED;
+    for (int l = 0; l < n; ++l)
+        if (!act[l] || !wgt[l] || !out[l]) return BS_ERR_INVALID_ARG;
+    TcChainArgs<TC_CHAIN_MAX> ch{};
+    size_t smem = 0;
+    const long long tiles_m = tc_chain_plan(n, act, wgt, params, out, false, ch.L, smem);
+    if (tiles_m <= 0) return BS_ERR_UNSUPPORTED;
+    if (workspace_bytes < tc_chain_ws_bytes(n, tiles_m)) return BS_ERR_INVALID_ARG;
+    if (!aligned16(workspace)) return BS_ERR_ALIGNMENT;
+    ch.nlayers = n;
+    ch.ctl = static_cast<unsigned*>(workspace);
+    ch.flags = ch.ctl + 4;
+    const TcArgs& g = ch.L[0];
+    const int A = params[0].a_bits;
+    const int sms = device_sm_count();
+    if (sms <= 0) return BS_ERR_CUDA;
+    const int cps = tcp_ctas_per_sm(smem, g.TN);
+    const bool wide = cps <= 2 && g.TN >= 64;
+    void (*kern)(TcChainArgs<TC_CHAIN_MAX>) = tcp_pick<TC_CHAIN_MAX>(A, cps, wide);
+    if (smem > 48 * 1024 &&
+        cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)) != cudaSuccess) {
+        cudaGetLastError();
+        return BS_ERR_CUDA;
+    }
+    // Every CTA of the grid must be resident at once (tiles wait for tiles of other CTAs).  The grid is sized by the same
+    // count the one-layer kernel uses -- shared memory with the largest carve-out, which the kernel asks for here, registers
+    // through the launch bounds, tensor-memory columns -- because the runtime's occupancy query answers one CTA per SM for
+    // every kernel that allocates tensor memory, whatever its shared memory and block size.  Should fewer CTAs be resident
+    // than counted, the bounded waits end the launch with BS_ERR_TIMEOUT instead of hanging.
+    if (cudaFuncSetAttribute(kern, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared) != cudaSuccess) {
+        cudaGetLastError();
+        return BS_ERR_CUDA;
+    }
+    long long per_o = (static_cast<long long>(sms) * cps) / g.tiles_o;
+    if (per_o < 1) return BS_ERR_UNSUPPORTED;                       // more filter tiles than resident CTAs
+    if (per_o > n * tiles_m) per_o = n * tiles_m;
+    const long long grid = per_o * g.tiles_o;
+    if (tc_launch(kern, static_cast<unsigned>(grid), wide ? TCP_THREADS_WIDE : TCP_THREADS, smem, st, chained, ch) != cudaSuccess) {
+        cudaGetLastError();
+        return BS_ERR_CUDA;
+    }
+    return BS_OK;
+}
+
 }  // namespace bs
 
 #ifdef BS_TUNING
-// Tuning builds: copies the timeline table of the last tensor-core launches to `out` (HOST, 148 x 24 x 8 cycle counts).
+// Tuning builds: copies the timeline table of the last tensor-core launches to `out` (HOST, 148 x 24 x 24 cycle counts).
 extern "C" int bs_tc_trace_read(long long* out, int clear)
 {
     if (cudaDeviceSynchronize() != cudaSuccess) return BS_ERR_CUDA;
@@ -1713,6 +2070,23 @@ extern "C" int bitserial_conv2d_tc(const uint32_t* act_packed, const int8_t* wgt
                                    uint32_t* out_packed, void* stream)
 {
     return bs::tc_conv_impl(act_packed, wgt_tc, p, out_i32, out_packed, static_cast<cudaStream_t>(stream));
+}
+
+extern "C" size_t bs_tc_chain_workspace_bytes(const bs_conv_params* layers, int nlayers)
+{
+    if (!layers || nlayers < 2 || nlayers > bs::TC_CHAIN_MAX) return 0;
+    bs::TcArgs L[bs::TC_CHAIN_MAX];
+    size_t smem = 0;
+    const long long tiles_m = bs::tc_chain_plan(nlayers, nullptr, nullptr, layers, nullptr, true, L, smem);
+    return tiles_m > 0 ? bs::tc_chain_ws_bytes(nlayers, tiles_m) : 0;
+}
+
+extern "C" int bitserial_conv2d_tc_chain(int nlayers, const uint32_t* const* act_packed, const int8_t* const* wgt_tc,
+                                         const bs_conv_params* layers, uint32_t* const* out_packed, void* workspace,
+                                         size_t workspace_bytes, int chained, void* stream)
+{
+    return bs::tc_chain_impl(nlayers, act_packed, wgt_tc, layers, out_packed, workspace, workspace_bytes,
+                             static_cast<cudaStream_t>(stream), chained != 0);
 }
 
 extern "C" int bitserial_conv2d_tc_chained(const uint32_t* act_packed, const int8_t* wgt_tc, const bs_conv_params* p,

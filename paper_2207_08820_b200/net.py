@@ -1,11 +1,12 @@
 """Runs a stack of quantised conv layers (``workloads.NetSpec``) through the C ABI.
 
-Host logic only: buffer planning, weight packing at set-up, one ``bitserial_conv2d`` call per layer
-(residual adds and concatenations are epilogue arguments), optional CUDA-graph replay.
+Host logic only: buffer planning, weight packing at set-up, one ``bitserial_conv2d`` call per layer -- or one
+``bitserial_conv2d_tc_chain`` call per run of same-shaped layers -- (residual adds and concatenations are epilogue
+arguments), optional CUDA-graph replay.
 """
 from __future__ import annotations
 
-from typing import Dict, Optional
+from typing import Dict, List, Optional
 
 import numpy as np
 import torch
@@ -15,11 +16,16 @@ from .workloads import NetSpec
 
 
 class BitserialNet:
+    MAX_CHAIN = 4
+
     def __init__(self, net: NetSpec, params: Dict[str, Dict], act_scale: float, device="cuda", batch: Optional[int] = None,
-                 engine: str = "popc", concurrent: bool = True):
+                 engine: str = "popc", concurrent: bool = True, chains="auto"):
         """engine: "popc" = popcount kernels on the integer pipes; "tc" = tensor-core entry point for every layer it
         supports (others fall back to the popcount kernel).  concurrent: launch independent neighbouring layers on
-        two streams (see :meth:`run_layers`)."""
+        two streams (see :meth:`run_layers`).  chains: with the "tc" engine, runs of consecutive same-shaped layers can go
+        through ``bitserial_conv2d_tc_chain`` (one launch per run) where the library accepts them: True = always,
+        False = never, "auto" = each such run is timed both ways at set-up and the faster form is kept (the chain wins
+        where launches dominate -- small batches -- and loses where every layer already fills the GPU)."""
         self.net = net
         self.engine = engine
         self.act_scale = float(act_scale)
@@ -44,12 +50,59 @@ class BitserialNet:
         self.bufs: Dict[str, torch.Tensor] = {}
         for name, (C, H, W) in self.shapes.items():
             self.bufs[name] = torch.zeros(self.batch, H, W, (C + 31) // 32, net.a_bits, dtype=torch.int32, device=self.device)
+        self.units = self._plan_units(bool(chains) and engine == "tc")
         torch.cuda.synchronize(self.device)   # chained layers fetch filters, scale and bias ahead of stream order
+        if chains == "auto":
+            self.units = self._keep_faster_units(self.units)
         self.concurrent = concurrent
         self.side = torch.cuda.Stream(device=self.device)
         self.graph = None
         self.static_in = None
-        self.launches_per_forward = 2 + len(self.layers)
+        self.launches_per_forward = 2 + len(self.units)
+
+    def _layer_params(self, item):
+        """``bs_conv_params`` of a layer as a chain would run it, or None when its output is a slice of a wider tensor."""
+        net, L = self.net, item["spec"]
+        if L.dst_c_offset != 0 or self.shapes[L.dst][0] != L.O or (L.res and self.shapes[L.res][0] != L.O):
+            return None
+        return api.conv_params(
+            self.bufs[L.src].shape, item["w"].shape, C=L.C, stride=L.stride, pad=L.pad, a_sign=api.UNSIGNED, w_sign=item["w_sign"],
+            scale=item["scale"], bias=item["bias"], relu=L.relu, out_bits=net.a_bits, out_sign=api.UNSIGNED,
+            residual=self.bufs[L.res] if L.res else None, res_scale=L.res_scale, res_bits=net.a_bits if L.res else 0,
+            res_sign=api.UNSIGNED)
+
+    def _plan_units(self, chains: bool) -> List[Dict]:
+        """The launches of a forward pass: single layers, and runs of up to MAX_CHAIN consecutive layers that the library
+        accepts as one chain (same shape, resident-filter plan) and whose inputs come from outside the run or from an
+        earlier layer of it.  Longest run first, greedily from the front."""
+        units, i, n = [], 0, len(self.layers)
+        while i < n:
+            took = 0
+            if chains:
+                for length in range(min(self.MAX_CHAIN, n - i), 1, -1):
+                    items = self.layers[i:i + length]
+                    if any(it["w_tc"] is None for it in items):
+                        continue
+                    prm = [self._layer_params(it) for it in items]
+                    if any(q is None for q in prm):
+                        continue
+                    dsts = [it["spec"].dst for it in items]
+                    if len(set(dsts)) != length:
+                        continue
+                    if any(t in dsts[k:] for k, it in enumerate(items) for t in (it["spec"].src, it["spec"].res) if t):
+                        continue
+                    nbytes = api.tc_chain_workspace_bytes(prm)
+                    if nbytes == 0:
+                        continue
+                    ws = torch.zeros((nbytes + 3) // 4, dtype=torch.int32, device=self.device)
+                    units.append(dict(items=items, params=prm, workspace=ws))
+                    took = length
+                    break
+            if not took:
+                units.append(dict(items=[self.layers[i]], params=None, workspace=None))
+                took = 1
+            i += took
+        return units
 
     def _run(self, x: torch.Tensor) -> torch.Tensor:
         self.pack_input(x)
@@ -71,6 +124,41 @@ class BitserialNet:
         api.bitpack_activations(x, self.act_scale, net.a_bits, api.UNSIGNED, api.NCHW, out=self.bufs[net.in_name].view(-1))
         main.wait_event(done)
 
+    def _time_units(self, units, reps: int = 8) -> float:
+        """Microseconds per pass of `units` launched back to back (as inside a forward pass), from a CUDA graph of `reps` passes."""
+        stream = torch.cuda.Stream(device=self.device)
+        with torch.cuda.stream(stream):
+            for u in units:
+                self.run_unit(u, chained=False)
+            stream.synchronize()
+            graph = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(graph, stream=stream):
+                for _ in range(reps):
+                    for u in units:
+                        self.run_unit(u)
+            best = float("inf")
+            for _ in range(4):
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0.record(stream)
+                graph.replay()
+                e1.record(stream)
+                e1.synchronize()
+                best = min(best, e0.elapsed_time(e1) * 1e3 / reps)
+        return best
+
+    def _keep_faster_units(self, units):
+        out = []
+        for u in units:
+            if u["params"] is None:
+                out.append(u)
+                continue
+            singles = [dict(items=[it], params=None, workspace=None) for it in u["items"]]
+            t_chain, t_single = self._time_units([u]), self._time_units(singles)
+            u["timing_us"] = (t_chain, t_single)
+            out.extend([u] if t_chain < t_single else singles)
+        torch.cuda.synchronize(self.device)
+        return out
+
     def run_layer(self, item, chained: bool = True) -> None:
         """One conv layer through the C ABI on the current stream."""
         net, L = self.net, item["spec"]
@@ -83,35 +171,56 @@ class BitserialNet:
             out_packed=self.bufs[L.dst], out_c_offset=L.dst_c_offset, out_c_total=self.shapes[L.dst][0],
             wgt_tc=item["w_tc"], chained=chained and item["w_tc"] is not None)
 
+    def run_unit(self, unit, chained: bool = True) -> None:
+        """One launch on the current stream: a layer, or a chain of layers."""
+        if unit["params"] is None:
+            self.run_layer(unit["items"][0], chained=chained)
+            return
+        items = unit["items"]
+        params = [self._layer_params(it) for it in items]       # pointers of the buffers as they are now (tests swap them)
+        api.bitserial_conv2d_tc_chain([self.bufs[it["spec"].src] for it in items], [it["w_tc"] for it in items], params,
+                                      [self.bufs[it["spec"].dst] for it in items], unit["workspace"], chained=chained)
+
     def run_layers(self) -> None:
-        """All conv layers in order.  With ``concurrent`` a layer whose successor in the list neither reads nor
-        overwrites its output (a projection shortcut beside the first conv of its block, the two 1x1 branches of a
-        cross-stage block) is launched on a side stream, so the two kernels share the GPU; events carry the
-        dependencies, and under stream capture they become the edges of the graph."""
+        """All launches in order.  With ``concurrent`` a single layer whose successor neither reads nor overwrites its
+        output (a projection shortcut beside the first conv of its block, the two 1x1 branches of a cross-stage block) is
+        launched on a side stream, so the two kernels share the GPU; events carry the dependencies, and under stream
+        capture they become the edges of the graph."""
         main = torch.cuda.current_stream(self.device)
         pending: Dict[str, torch.cuda.Event] = {}
-        n = len(self.layers)
-        for i, item in enumerate(self.layers):
-            L = item["spec"]
-            nxt = self.layers[i + 1]["spec"] if i + 1 < n else None
-            aside = (self.concurrent and nxt is not None and L.dst not in (nxt.src, nxt.res)
-                     and nxt.dst not in (L.src, L.res)
-                     and (nxt.dst != L.dst or nxt.dst_c_offset != L.dst_c_offset) and L.src not in pending
-                     and (L.res is None or L.res not in pending))
+        n = len(self.units)
+
+        def touched(unit):
+            reads, writes = set(), set()
+            for it in unit["items"]:
+                L = it["spec"]
+                reads.update(t for t in (L.src, L.res) if t)
+                writes.add((L.dst, L.dst_c_offset))
+            return reads, writes
+
+        for i, unit in enumerate(self.units):
+            reads, writes = touched(unit)
+            wnames = {d for d, _ in writes}
+            aside = False
+            if self.concurrent and i + 1 < n and len(unit["items"]) == 1:
+                nreads, nwrites = touched(self.units[i + 1])
+                aside = (not (wnames & nreads) and not ({d for d, _ in nwrites} & reads) and not (writes & nwrites)
+                         and not (reads & set(pending)))
             if aside:
                 fork = torch.cuda.Event()
                 fork.record(main)
                 self.side.wait_event(fork)
                 with torch.cuda.stream(self.side):
-                    self.run_layer(item, chained=False)
+                    self.run_unit(unit, chained=False)
                     done = torch.cuda.Event()
                     done.record(self.side)
-                pending[L.dst] = done
+                for d in wnames:
+                    pending[d] = done
                 continue
-            for t in (L.src, L.res, L.dst):
-                if t is not None and t in pending:
+            for t in reads | wnames:
+                if t in pending:
                     main.wait_event(pending.pop(t))
-            self.run_layer(item)
+            self.run_unit(unit)
         for ev in pending.values():
             main.wait_event(ev)
 

@@ -1,8 +1,9 @@
-"""Per-CTA timeline of the persistent tensor-core kernel (tuning builds only).
+"""Per-CTA timeline of the tensor-core kernels (tuning builds only).
 
 A library built with ``BS_EXTRA_NVCC_FLAGS=-DBS_TUNING python -m paper_2207_08820_b200.build --force`` records, for the first
-148 CTAs of a launch and the first eight pixel tiles of each, the SM cycle counter at the hand-offs between the kernel's roles
-(packed tile requested / landed, expansion begin / end, MMA issue begin / end, epilogue begin / end).  This tool runs chosen layers
+148 CTAs of a launch and the first 24 pixel tiles of each, the SM cycle counter at the hand-offs between the kernel's roles
+(packed tile requested / landed, expansion begin / end, MMA issue begin / end, epilogue begin / end; per channel chunk instead of
+per tile for the kernel that streams its filters).  This tool runs chosen layers
 of a layer stack once and prints those timelines:
 
     python -m paper_2207_08820_b200.timeline resnet18_body 0,7 [cta,cta,...]
@@ -44,7 +45,7 @@ def main(argv) -> int:
     runner = BitserialNet(net, params, 0.25, batch=batch, engine="tc")
     runner.forward(x)
     api.bs_check_status()
-    buf = np.zeros((148, 24, 8), dtype=np.int64)
+    buf = np.zeros((148, 24, 24), dtype=np.int64)
     for li in layers:
         item = runner.layers[li]
         for _ in range(3):
@@ -57,10 +58,20 @@ def main(argv) -> int:
         for c in ctas:
             t0 = buf[c, 0, 0]
             if t0 == 0:
-                print(f"  CTA {c}: no timeline (not the persistent kernel, or fewer CTAs)")
+                print(f"  CTA {c}: no timeline (fewer CTAs in this launch)")
+                continue
+            if buf[c, 3, 0] == 0:
+                # the streaming kernel (one pixel-tile group per CTA, filters fetched chunk by chunk): one line per channel chunk
+                rel = lambda e, t=0: buf[c, e, t] - t0
+                print(f"  CTA {c} (filters streamed): ends at {rel(11)} cycles; tables built {rel(1)}, packed tile landed {rel(2)}, "
+                      f"expansion finished {rel(13)}, accumulators ready {rel(9)}, epilogue done {rel(10)}")
+                for t in range(24):
+                    if buf[c, 5, t] == 0:
+                        break
+                    print(f"    chunk {t}: filters requested {rel(4, t)}  expand {rel(5, t)}..{rel(6, t)}  mma issue {rel(7, t)}..{rel(8, t)}")
                 continue
             print(f"  CTA {c}: ends at {buf[c, 11, 0] - t0} cycles; set-up {buf[c, 1, 0] - t0}, filters landed {buf[c, 3, 0] - t0}")
-            for t in range(8):
+            for t in range(24):
                 if buf[c, 4, t] == 0 and buf[c, 5, t] == 0:
                     break
                 rel = lambda e: buf[c, e, t] - t0
