@@ -49,13 +49,35 @@ static int largest_unit(int a, int b)
 }
 
 // Fill the staging part of a plan; returns false if the tile cannot be staged in shared memory.
-static bool plan_staging(Plan& pl, int Cw, int RS, int R, int S, int stride, int A, int WB)
+static bool plan_staging(Plan& pl, int Cw, int RS, int R, int S, int stride, int A, int WB, bool many_tiles = false)
 {
     const int TN = pl.NFG * pl.FB;
     const int TW = pl.TWB * pl.PB;
     pl.hh = (pl.TH - 1) * stride + R;
     pl.hw = (TW - 1) * stride + S;
     pl.CWC = Cw < (RS == 1 ? 8 : 4) ? Cw : (RS == 1 ? 8 : 4);
+    if (RS == 1 && Cw > 8) {
+        // 1x1 layers and matrix products: channel words per chunk among 8, 6 and 4.  The reduction loop takes the words of
+        // a chunk three at a time through the carry-save adder (two counts per three words, one count per left-over
+        // word) and a chunk costs about 0.85 counts of hand-off (fitted to 4096 x 4096 products with 72 words: 640 / 605 /
+        // 709 us for 8 / 6 / 4); six words are two clean triples, and 18 words (576 channels) are three full chunks of six
+        // instead of 8 + 8 + 2.  A width that would take the activations off the TMA path (record not a multiple of
+        // 16 bytes) is not considered; the filters may fall back to the gather.  More chunks are only accepted when the
+        // tiles fill the machine several times over (`many_tiles`): with one or two tiles per SM every extra hand-off is
+        // exposed latency (1024 x 1024 x 2304: 0.058 ms with chunks of 8, 0.065 ms with chunks of 6).
+        double best_cost = 0.0;
+        const int chunks8 = ceil_div(Cw, 8);
+        for (int cwc = 8; cwc >= 4; cwc -= 2) {
+            if ((cwc * A) % 4 != 0 && (8 * A) % 4 == 0) continue;
+            const int full = Cw / cwc, tail = Cw % cwc;
+            if (!many_tiles && full + (tail ? 1 : 0) > chunks8) continue;
+            const double cost = full * (2 * (cwc / 3) + cwc % 3) + (tail ? 2 * (tail / 3) + tail % 3 : 0) + 0.85 * (full + (tail ? 1 : 0));
+            if (cwc == 8 || cost < 0.95 * best_cost) { best_cost = cost; pl.CWC = cwc; }      // a clear gain only
+        }
+    }
+#ifdef BS_TUNING
+    if (const char* e = getenv("BS_CWC")) { const int v = atoi(e); if (v >= 1 && v <= 8 && v <= Cw) pl.CWC = v; }
+#endif
     pl.nchunks = ceil_div(Cw, pl.CWC);
     const int recA = pl.CWC * A, recW = pl.CWC * WB;
     pl.tma_a = (recA % 4 == 0) && ((Cw * A) % 4 == 0);
@@ -126,8 +148,8 @@ static bool search_plan(Plan& best, int N, int P, int Q, int O, int Cw, int R, i
                         Plan pl{};
                         pl.PB = PB; pl.FB = FB; pl.NFG = NFG; pl.TWB = TWB; pl.TH = TH; pl.TNI = TNI;
                         pl.NT = round_up(used * NFG, 32);
-                        if (!plan_staging(pl, Cw, RS, R, S, stride, A, WB)) continue;
                         pl.tiles = tiles_o * ceil_div(qb, TWB) * ceil_div(P, TH) * ceil_div(N, TNI);
+                        if (!plan_staging(pl, Cw, RS, R, S, stride, A, WB, pl.tiles >= 8LL * sms)) continue;
                         const double cta_warps = pl.NT / 32.0;
                         // warps of a CTA spread over the four sub-partitions; the fullest one sets the pace
                         double per_subpartition = 0.5 * (ceil(cta_warps / 4.0) + cta_warps / 4.0);

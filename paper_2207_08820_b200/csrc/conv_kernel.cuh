@@ -319,11 +319,15 @@ __global__ void __launch_bounds__(256, (PB * FB <= 32) ? 3 : 1) bitserial_conv_k
         //     popc(x0) + popc(x1) + popc(x2) = popc(x0 ^ x1 ^ x2) + 2 * popc(maj(x0, x1, x2)),
         // i.e. two population counts (the scarce pipe: 16 lanes per clock per SM) and two 3-input logic operations
         // instead of three counts.  A remainder of one or two words takes the plain form.
+        // A 1x1 layer (a matrix product) whose channel words do not fill the last chunk: the staged words past the
+        // end are zero and add nothing, so the loops stop at the last live word (576 channels = 18 words in chunks of 8
+        // would otherwise pay for 24).  With several taps the zero words sit between the taps and are kept.
+        const int cw_live = RS == 1 ? min(g.CWC, g.Cw - (c_begin + c) * g.CWC) : g.CWC;
         if (pg_used)
         for (int r = 0; r < g.R; ++r) {
             const uint32_t* par = sA + a_off0 + r * g.hw * recA;
             const uint32_t* pwr = sW + w_off0 + r * g.S * recW;
-            const int M = g.S * g.CWC;
+            const int M = g.S * cw_live;
             int m = 0;
             for (; m + 3 <= M; m += 3) {
                 uint32_t w[3][FB][WB];
@@ -378,7 +382,7 @@ __global__ void __launch_bounds__(256, (PB * FB <= 32) ? 3 : 1) bitserial_conv_k
                     for (int tap = 0; tap < RS; ++tap) {
                         const int r = tap / g.S, sx = tap - r * g.S;
                         const uint32_t* p = base + (r * g.hw + sx) * recA;
-                        for (int cw = 0; cw < g.CWC; ++cw)
+                        for (int cw = 0; cw < cw_live; ++cw)
 #pragma unroll
                             for (int j = 0; j < A; ++j) sum += g.rs_coef[j] * __popc(p[cw * A + j]);
                     }
@@ -389,7 +393,7 @@ __global__ void __launch_bounds__(256, (PB * FB <= 32) ? 3 : 1) bitserial_conv_k
         if (g.need_cs && tid < TN) {
             const uint32_t* base = sW + tid * RS * recW;
             int sum = 0;
-            for (int k = 0; k < RS * g.CWC; ++k)
+            for (int k = 0; k < (RS == 1 ? cw_live : RS * g.CWC); ++k)
 #pragma unroll
                 for (int i = 0; i < WB; ++i) sum += g.cs_coef[i] * __popc(base[k * WB + i]);
             cs_acc += sum;
