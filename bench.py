@@ -345,6 +345,8 @@ def measure_other_configs(torch, api, stream, args):
       gemm_sweep / bitwidth_sweep   as the stand-alone sweeps, fewer repetitions;
       detection_backbone            the detection-shaped stack at batch 16 on the tensor-core engine: conv time per pass under a
                                     CUDA graph, images/s, and sum(roofline time) / measured time over its layers;
+      layer_chains   the residual stack's conv layers at batch 16 and 64, one launch per layer against runs of same-shaped
+                     layers as one launch (bitserial_conv2d_tc_chain), and how many launches the runner's set-up timing keeps;
       pack_large     the pack kernels on inputs larger than L2 (fp32 NCHW and NHWC, 2 and 3 bits)."""
     from paper_2207_08820_b200.net import BitserialNet
     dev = lambda a: torch.from_numpy(np.ascontiguousarray(a)).cuda()
@@ -442,6 +444,25 @@ def measure_other_configs(torch, api, stream, args):
                                  "hbm_bound_layers": sums["hbm_bound_layers"],
                                  "pack_frac_hbm": (x.numel() * 4 + runner.bufs[net.in_name].numel() * 4) / (t_pack * 1e-3) / pk["hbm"]}
     del runner, x
+    # ---- runs of same-shaped layers as one launch (bitserial_conv2d_tc_chain) against one launch per layer
+    chain_rows = []
+    for b in (16, 64):
+        cnet, cseed = make_net("resnet18_body", b)
+        cparams = wl.network_params(cnet, cseed)
+        row = {"workload": f"resnet18_body_batch{b}_w2a2, conv layers only (warm L2, one CUDA graph per pass)"}
+        for key, mode in (("per_layer", False), ("chains", True)):
+            r = BitserialNet(cnet, cparams, ACT_SCALE, batch=b, engine="tc", chains=mode)
+            with torch.cuda.stream(stream):
+                r.run_layers()
+                stream.synchronize()
+                row[key + "_ms"] = graph_time(r.run_layers, reps=1, rounds=8)
+            row[key + "_launches"] = len(r.units)
+            del r
+        auto = BitserialNet(cnet, cparams, ACT_SCALE, batch=b, engine="tc", chains="auto")
+        row["auto_keeps_launches"] = len(auto.units)
+        del auto
+        chain_rows.append(row)
+    out["layer_chains"] = chain_rows
     # ---- the whole mixed-precision classifier: floating-point stem and head around the headline stack
     from paper_2207_08820_b200.net import BitserialFullNet
     fnet = wl.resnet18_full(batch=args.batch)
@@ -489,7 +510,8 @@ def run_ours(args):
     params = wl.network_params(net, seed)
     x_host = torch.from_numpy(wl.network_input(net, replicas.rank_seed(seed, rank), ACT_SCALE)).pin_memory()
     x_dev = x_host.cuda()
-    runner = BitserialNet(net, params, ACT_SCALE, batch=net.batch, engine=args.engine)
+    chains = False if args.eager or args.chains == "off" else (True if args.chains == "on" else "auto")
+    runner = BitserialNet(net, params, ACT_SCALE, batch=net.batch, engine=args.engine, chains=chains)
 
     stream = torch.cuda.Stream()
     with torch.cuda.stream(stream):
@@ -722,6 +744,7 @@ def run_ours(args):
             "clocks": clocks.summary(),
         }
         line["config"]["engine"] = args.engine
+        line["config"]["conv_launches_per_step"] = len(runner.units)
         if t_conv_other is not None:
             alt = popc_roofline(t_conv_other) if other == "popc" else tensor_roofline(t_conv_other)
             alt["engine"] = other
@@ -774,6 +797,8 @@ def main():
     ap.add_argument("--no-configs", action="store_true", help="leave out the compact measurements of the other workloads")
     ap.add_argument("--engine", default="tc", choices=["popc", "tc"],
                     help="popc: popcount kernels on the integer pipes; tc: exact int8 tensor-core formulation")
+    ap.add_argument("--chains", default="auto", choices=["auto", "on", "off"], help="runs of same-shaped layers as one launch: timed at set-up and "
+                    "kept where faster (auto), always, or never; --eager implies off")
     ap.add_argument("--eager", action="store_true", help="plain stream launches instead of CUDA graphs (for per-launch profiling)")
     args = ap.parse_args()
     if args.workload in ("bitwidth_sweep", "gemm_sweep"):
