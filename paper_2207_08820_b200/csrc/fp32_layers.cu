@@ -16,7 +16,7 @@ namespace bs {
 // 128-bit weight loads feed 64 fused multiply-adds (with four filters per thread the shared-memory pipe, not the FMA pipe, set
 // the pace: 22 TFLOP/s).  A warp is 8 filter octets x 4 strips: its weight loads are 8 distinct vectors, its input loads four
 // broadcasts.
-constexpr int F32_TH = 8, F32_TW = 32, F32_STRIP = 8, F32_OT = 64, F32_THREADS = 256, F32_FPT = 8;
+constexpr int F32_TH = 16, F32_TW = 16, F32_STRIP = 8, F32_OT = 64, F32_THREADS = 256, F32_FPT = 8;
 
 struct ConvF32Args {
     const float* x;
@@ -35,7 +35,8 @@ __global__ void __launch_bounds__(F32_THREADS, 2) conv2d_f32_tiled_kernel(const 
     constexpr int WIN = (F32_STRIP - 1) * STRIDE + S;            // input columns one strip needs
     constexpr int WIN4 = (WIN + 3) / 4;
     float* s_w = f32_smem;                                       // [C][R][S][2][8][4]
-    float* s_x = f32_smem + g.C * g.R * S * F32_OT;              // [C][in_h][pitch]
+    float* s_x0 = f32_smem + g.C * g.R * S * F32_OT;             // [2][C][in_h][pitch]: the halo of the next tile lands while this one is computed
+    const int halo_floats = g.C * g.in_h * g.pitch;
     const int tid = threadIdx.x;
     const int to = blockIdx.y, o0 = to * F32_OT;
 
@@ -50,22 +51,49 @@ __global__ void __launch_bounds__(F32_THREADS, 2) conv2d_f32_tiled_kernel(const 
         s_w[t * F32_OT + ((o & 7) >> 2) * 32 + (o >> 3) * 4 + (o & 3)] = (o0 + o < g.O) ? g.w[static_cast<size_t>(o0 + o) * taps + t] : 0.0f;
     }
     const int tiles = g.N * g.tiles_p * g.tiles_q;
-    for (int tile = blockIdx.x; tile < tiles; tile += gridDim.x) {
+    // Input halo of a tile, zero outside the image (a zero tap leaves the chain unchanged: fma(0, w, acc) == acc), fetched with
+    // 4-byte asynchronous copies (zero-filled where the source is outside): a thread owns column tid % 64 of every fourth
+    // halo row, so no division is needed per element, and the copies of tile k + 1 fly while tile k is computed.
+    auto stage = [&](int tile, float* dst) {
+        int b = tile;
+        const int tq = b % g.tiles_q; b /= g.tiles_q;
+        const int tp = b % g.tiles_p; b /= g.tiles_p;
+        const int n = b;
+        const int y0 = tp * F32_TH * STRIDE - g.pad, x0 = tq * F32_TW * STRIDE - g.pad;
+        const int rows = g.C * g.in_h;
+        int yy = tid >> 6, c = 0;
+        while (yy >= g.in_h) { yy -= g.in_h; ++c; }
+        for (int xx = tid & 63; xx < g.pitch; xx += 64) {
+            int y2 = yy, c2 = c;
+            const int x = x0 + xx;
+            const bool xok = xx < g.in_w && x >= 0 && x < g.W;
+            for (int row = tid >> 6; row < rows; row += F32_THREADS / 64) {
+                const int y = y0 + y2;
+                const bool ok = xok && y >= 0 && y < g.H;
+                const float* src = ok ? g.x + ((static_cast<size_t>(n) * g.C + c2) * g.H + y) * g.W + x : g.x;
+                const unsigned d = static_cast<unsigned>(__cvta_generic_to_shared(dst + row * g.pitch + xx));
+                asm volatile("cp.async.ca.shared.global [%0], [%1], 4, %2;" ::"r"(d), "l"(src), "r"(ok ? 4 : 0) : "memory");
+                y2 += F32_THREADS / 64;
+                while (y2 >= g.in_h) { y2 -= g.in_h; ++c2; }
+            }
+        }
+        asm volatile("cp.async.commit_group;" ::: "memory");
+    };
+    if (static_cast<int>(blockIdx.x) < tiles) stage(blockIdx.x, s_x0);
+    int buf = 0;
+    for (int tile = blockIdx.x; tile < tiles; tile += gridDim.x, buf ^= 1) {
     int b = tile;
     const int tq = b % g.tiles_q; b /= g.tiles_q;
     const int tp = b % g.tiles_p; b /= g.tiles_p;
     const int n = b;
     const int p0 = tp * F32_TH, q0 = tq * F32_TW;
-    __syncthreads();                                             // the previous tile's readers are done with s_x
-    // input halo, zero outside the image (a zero tap leaves the chain unchanged: fma(0, w, acc) == acc)
-    const int y0 = p0 * STRIDE - g.pad, x0 = q0 * STRIDE - g.pad;
-    for (int i = tid; i < g.C * g.in_h * g.pitch; i += F32_THREADS) {
-        const int xx = i % g.pitch, rest = i / g.pitch;
-        const int yy = rest % g.in_h, c = rest / g.in_h;
-        const int y = y0 + yy, x = x0 + xx;
-        float v = 0.0f;
-        if (xx < g.in_w && y >= 0 && y < g.H && x >= 0 && x < g.W) v = g.x[((static_cast<size_t>(n) * g.C + c) * g.H + y) * g.W + x];
-        s_x[i] = v;
+    const float* s_x = s_x0 + buf * halo_floats;
+    // the other buffer was read by the tile before this one: every thread is past that (barrier at the end of the loop body)
+    if (tile + static_cast<int>(gridDim.x) < tiles) {
+        stage(tile + gridDim.x, s_x0 + (buf ^ 1) * halo_floats);
+        asm volatile("cp.async.wait_group 1;" ::: "memory");     // this tile's copies have landed; the next tile's may still fly
+    } else {
+        asm volatile("cp.async.wait_group 0;" ::: "memory");
     }
     __syncthreads();
 
@@ -128,6 +156,7 @@ __global__ void __launch_bounds__(F32_THREADS, 2) conv2d_f32_tiled_kernel(const 
                 if (qb + j < g.Q) dst[j] = v[j];
         }
     }
+    __syncthreads();                                             // every thread is done reading this tile's halo buffer
     }   // tiles
 }
 
@@ -298,7 +327,7 @@ extern "C" int bs_conv2d_f32(const float* x, const float* w, const float* bias, 
         const int need = (bs::F32_TW / bs::F32_STRIP - 1) * bs::F32_STRIP * stride + win4;
         g.pitch = ((need > g.in_w ? need : g.in_w) + 3) / 4 * 4;
         g.tiles_p = bs::ceil_div(g.P, bs::F32_TH); g.tiles_q = bs::ceil_div(g.Q, bs::F32_TW); g.tiles_o = bs::ceil_div(O, bs::F32_OT);
-        const size_t smem = (static_cast<size_t>(C) * R * S * bs::F32_OT + static_cast<size_t>(C) * g.in_h * g.pitch) * 4;
+        const size_t smem = (static_cast<size_t>(C) * R * S * bs::F32_OT + 2 * static_cast<size_t>(C) * g.in_h * g.pitch) * 4;
         if (smem <= 200 * 1024) {
             if (S == 7) return bs::launch_conv_tiled<7, 2>(g, smem, st);
             if (S == 3 && stride == 1) return bs::launch_conv_tiled<3, 1>(g, smem, st);
