@@ -50,6 +50,8 @@ struct TcArgs {
     int NM;                           // filters of one MMA (TN when TN <= 128, else 256: a wider tile issues TN / NM MMAs per step)
     int TN, CK, MB, CWC, nchunks, nsp, nse;   // CK: channels per filter-layout block, MB: blocks per pipeline chunk, CWC: words per chunk
     int fullA;                        // words of one packed pixel record (Cw * A)
+    int pitchA;                       // words between the staged records of consecutive pixels (fullA, or seg_words)
+    int seg_words, seg_chunks, nseg;  // flat tiles with long records: the 128 rows are staged seg_words at a time (0: whole records)
     int pmode;                        // how a tile's packed halo is fetched: 0 flat bulk copy, 1 rows merged with W, 2 4-D box
     int TNI, GI, hh, hw;              // packed halo: TNI images x hh rows x hw columns; GI row groups per image
     int hwb, xsh;                     // row pitch of the staged halo in pixels, and pixels skipped at the start of a row
@@ -354,7 +356,7 @@ __device__ __forceinline__ void tc_expand_items(const TcArgs& g, const TcExpand&
             ep = hy * g.HWP + (MODE == 1 ? hx : (hx & 1) * g.HWH + (hx >> 1));
         }
         uint32_t w[A];
-        load_planes<A>(src_c + static_cast<size_t>(hp) * g.fullA, w);
+        load_planes<A>(src_c + static_cast<size_t>(hp) * g.pitchA, w);
         uint32_t out[8];
         if (A == 2) {
             // byte j of t / u: table index of nibble 2j / 2j+1 (plane 0 in the low four bits, plane 1 in the high four)
@@ -835,7 +837,10 @@ __device__ __forceinline__ void tc_epilogue_tile(const TcArgs& g, uint32_t tmem_
 
 // ----------------------------------------------------------------------------- one tile per CTA (filters streamed per chunk)
 
-template <int A>
+// SEG: the packed rows of a flat tile are staged in segments (matrix products with a long reduction, see the plan); a
+// template parameter so that the common instantiation carries none of that code (with a run-time switch the residual stack
+// measured 1.2 % slower).
+template <int A, bool SEG>
 __global__ void __launch_bounds__(TC_THREADS) bitserial_conv_tc_kernel(const __grid_constant__ TcArgs g)
 {
     extern __shared__ __align__(128) unsigned char tc_smem[];
@@ -851,8 +856,9 @@ __global__ void __launch_bounds__(TC_THREADS) bitserial_conv_tc_kernel(const __g
     uint64_t* full_e = bars + 2 * TC_MAX_STAGES;
     uint64_t* empty_e = bars + 3 * TC_MAX_STAGES;
     uint64_t* accum_full = bars + 4 * TC_MAX_STAGES;
-    uint64_t* full_a = bars + 4 * TC_MAX_STAGES + 1;      // packed tile landed
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 4 * TC_MAX_STAGES + 2);
+    uint64_t* full_a = bars + 4 * TC_MAX_STAGES + 1;      // [2] packed tile (or segment of its rows) landed
+    uint64_t* empty_a = bars + 4 * TC_MAX_STAGES + 3;     // [2] segment buffer expanded (segmented rows only)
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 4 * TC_MAX_STAGES + 5);
 
     const int o0 = static_cast<int>(blockIdx.x % static_cast<unsigned>(g.tiles_o)) * g.TN;   // filter tile fastest
     const int tiles_m = g.tiles_q * g.tiles_p * g.tiles_n;
@@ -870,7 +876,12 @@ __global__ void __launch_bounds__(TC_THREADS) bitserial_conv_tc_kernel(const __g
             mbar_init(&empty_e[s], 1);
         }
         mbar_init(accum_full, 1);
-        mbar_init(full_a, static_cast<unsigned>(nt));
+        mbar_init(&full_a[0], static_cast<unsigned>(nt));
+        if (SEG) {
+            mbar_init(&full_a[1], 1);
+            mbar_init(&empty_a[0], 1);
+            mbar_init(&empty_a[1], 1);
+        }
         fence_barrier_init();
         fence_proxy_async();
     }
@@ -885,7 +896,63 @@ __global__ void __launch_bounds__(TC_THREADS) bitserial_conv_tc_kernel(const __g
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
 
-    if (warp == 4) {
+    if (SEG && warp == 4) {
+        // ------------------------------------------------------------------ producer, rows staged in segments
+        // A matrix product with a long reduction: the packed rows of the tile are too large to stay resident (4608 channels at
+        // 2 bits: 147 KB), so they are fetched seg_words per row at a time into two buffers.  The 128 row pieces of a segment
+        // are separate bulk copies, four per lane, requested one segment ahead of the expanders.
+        const int early = g.nchunks < g.nsp ? g.nchunks : g.nsp;
+        const int blk_bytes = g.b_bytes / g.MB;
+        const size_t blk_stride = static_cast<size_t>(g.opad8) * RS * (g.CK >> 4) * 128;
+        const int8_t* src = g.wgt + static_cast<size_t>(o0 >> 3) * RS * (g.CK >> 4) * 128;
+        const int seg_bytes = g.pa_bytes / 2;
+        const TcTile tile = tc_decode_tile(g, mt0);
+        const long long npix = static_cast<long long>(g.N) * g.P * g.Q;
+        const int rows = static_cast<int>(npix - tile.q0 < TC_M ? npix - tile.q0 : TC_M);
+        auto load_segment = [&](int sg) {
+            const int w0 = sg * g.seg_words;
+            const int words = g.fullA - w0 < g.seg_words ? g.fullA - w0 : g.seg_words;
+            uint64_t* bar = &full_a[sg & 1];
+            if (lane == 0) mbar_expect_tx(bar, static_cast<unsigned>(rows) * static_cast<unsigned>(words) * 4u);
+            __syncwarp();
+            unsigned char* dst = tc_smem + g.off_p + (sg & 1) * seg_bytes;
+            for (int r = lane; r < rows; r += 32)
+                bulk_load(dst + static_cast<size_t>(r) * g.seg_words * 4, g.act + (static_cast<size_t>(tile.q0) + r) * g.fullA + w0,
+                          static_cast<unsigned>(words) * 4u, bar);
+        };
+        TcRing rp;
+        unsigned ok = 1;
+        for (int c = 0; c < g.nchunks; ++c) {
+            if (c == early) {
+                pdl_acquire();
+                load_segment(0);
+                if (g.nseg > 1) load_segment(1);
+            }
+            if (lane == 0) {
+                ok = mbar_spin_bounded(&empty_p[rp.idx], rp.phase ^ 1u) ? 1u : 0u;
+                if (ok) {
+                    TC_TRACE(TR_LOAD, c);
+                    mbar_expect_tx(&full_p[rp.idx], static_cast<unsigned>(g.b_bytes));
+                    for (int j = 0; j < g.MB; ++j, src += blk_stride)
+                        bulk_load(tc_smem + rp.idx * stage_p_bytes + j * blk_bytes, src, static_cast<unsigned>(blk_bytes), &full_p[rp.idx]);
+                }
+            }
+            ok = __shfl_sync(0xffffffffu, ok, 0);
+            if (!ok) break;
+            rp.advance(g.nsp);
+            if (c >= early && c % g.seg_chunks == 0 && c / g.seg_chunks >= 1 && c / g.seg_chunks + 1 < g.nseg) {
+                // the filters of the first chunk of segment c / seg_chunks are on their way, so the expanders are about to leave
+                // the segment before it: its buffer takes the segment after this one (needed a whole segment from now)
+                const int sg = c / g.seg_chunks + 1;
+                if (lane == 0) ok = mbar_spin_bounded(&empty_a[sg & 1], ((sg >> 1) - 1) & 1) ? 1u : 0u;
+                ok = __shfl_sync(0xffffffffu, ok, 0);
+                if (!ok) break;
+                load_segment(sg);
+            }
+        }
+        if (!ok && lane == 0) atomicOr(g.status, STATUS_TIMEOUT);
+        __syncwarp();
+    } else if (warp == 4) {
         // ------------------------------------------------------------------ producer
         if (lane == 0) {
             // the first ring of filter chunks does not depend on the preceding kernel: fetch it before waiting for it
@@ -951,21 +1018,33 @@ __global__ void __launch_bounds__(TC_THREADS) bitserial_conv_tc_kernel(const __g
         const TcExpand xp = tc_expand_init(g, ct, TC_WORKERS);
         const TcEpiThread eth = tc_epi_thread(g, (warp & 3) * 32 + lane);
         if (tid == 0) TC_TRACE(TR_SETUP, 0);
-        bool ok = mbar_wait_warp(full_a, 0, lane);
+        bool ok = SEG ? true : mbar_wait_warp(&full_a[0], 0, lane);
         if (tid == 0) TC_TRACE(TR_PDL, 0);
         TcRing re;
+        int sg = 0, cl = 0;               // segmented rows: segment and chunk within it
         for (int c = 0; c < g.nchunks; ++c) {
+            if (SEG && cl == 0 && ok) ok = mbar_wait_warp(&full_a[sg & 1], (sg >> 1) & 1, lane);
             if (ok) ok = mbar_wait_warp(&empty_e[re.idx], re.phase ^ 1u, lane);
             if (!ok) atomicOr(g.status, STATUS_TIMEOUT);
             if (tid == 0) TC_TRACE(TR_XBEG, c);
-            for (int t = 0; t < nt; ++t)
-                tc_expand_chunk<A>(g, xp, reinterpret_cast<const uint32_t*>(tc_smem + g.off_p + t * g.pa_bytes),
-                                   tc_smem + g.off_e + re.idx * e_stage + t * g.e_bytes, s_lut, ct, c);
+            if (SEG) {
+                tc_expand_chunk<A>(g, xp, reinterpret_cast<const uint32_t*>(tc_smem + g.off_p + (sg & 1) * (g.pa_bytes / 2)),
+                                   tc_smem + g.off_e + re.idx * e_stage, s_lut, ct, cl);
+            } else {
+                for (int t = 0; t < nt; ++t)
+                    tc_expand_chunk<A>(g, xp, reinterpret_cast<const uint32_t*>(tc_smem + g.off_p + t * g.pa_bytes),
+                                       tc_smem + g.off_e + re.idx * e_stage + t * g.e_bytes, s_lut, ct, c);
+            }
             fence_proxy_async();          // make the generic-proxy writes visible to the tensor core's reads
             group_sync(1, TC_WORKERS);
             if (tid == 0) TC_TRACE(TR_XEND, c);
             if (tid == 0) mbar_arrive(&full_e[re.idx]);
             re.advance(g.nse);
+            if (SEG && ++cl == g.seg_chunks) {
+                if (tid == 0) mbar_arrive(&empty_a[sg & 1]);      // after the group barrier: every thread has read the segment
+                cl = 0;
+                ++sg;
+            }
         }
         // the last chunks are still in the tensor core: time to turn the comparison bounds into integer thresholds
         uint32_t thr = 0;                 // shared-memory address of the thresholds, 0: floating-point comparison
@@ -1572,6 +1651,8 @@ static int tc_plan(const uint32_t* act, const int8_t* wgt, const bs_conv_params*
     int CKP = g.CK * g.MB;                        // channels per pipeline chunk
     g.CWC = CKP / 32;
     g.fullA = Cw * A;
+    g.pitchA = g.fullA;
+    g.seg_words = g.seg_chunks = g.nseg = 0;
     g.act = act;
     g.nchunks = p->C / CKP;
     g.nsp = g.nse = g.nchunks < 2 ? g.nchunks : 2;
@@ -1695,9 +1776,21 @@ static int tc_plan(const uint32_t* act, const int8_t* wgt, const bs_conv_params*
         int TN = 128;
         while (TN > 32 && (TN / 2 >= round_up_i(p->O, 32) || tiles_m * ceil_div(p->O, TN) < sms / 2)) TN /= 2;
         int PT = stream_pt;
+        // Matrix products with a long reduction: 128 packed rows of all K no longer fit beside useful filter and expansion stages
+        // (K = 4608 at 2 bits: 147 KB, which left room for 32-channel chunks only: one or two MMAs per hand-off).  Their rows are
+        // staged in segments of at most 72 words (a multiple of every chunk width), two buffers of 36 KB: 512-filter tiles with
+        // 64-channel chunks (four N = 256 MMAs per hand-off).  Segments of 32 words with 128-channel chunks in 214 KB measured
+        // slower (0.190 against 0.175 ms at 4096 x 4096 x 4608): the expansion of a chunk then takes longer than its MMAs.  Only for records that
+        // crowd the stages out (K = 2304, 74 KB resident, measured faster whole: 0.091 against 0.103 ms at 4096 x 4096) and only
+        // when the tiles fill the machine (1024 x 1024 x 4608 on 16 CTAs is latency-bound: 0.048 against 0.063 ms).
+        int seg_words = 0;
+        if (g.flat && PT == 1 && g.fullA % 4 == 0 && g.pa_tx_bytes > 96 * 1024 && tiles_m * ceil_div(p->O, 256) >= sms) {
+            seg_words = 72 / (4 * A) * (4 * A);
+            g.pa_bytes = 2 * round_up_i(TC_M * seg_words * 4, 128);
+        }
         auto stream_bytes = [&](int tn, int pt) {
             return static_cast<size_t>(g.nsp) * tn * RS * CKP + static_cast<size_t>(pt) * g.pa_bytes +
-                   static_cast<size_t>(g.nse) * pt * g.e_bytes + 2 * tn * 4 + 256 + (4 * TC_MAX_STAGES + 3) * 8 + 128 +
+                   static_cast<size_t>(g.nse) * pt * g.e_bytes + 2 * tn * 4 + 256 + (4 * TC_MAX_STAGES + 6) * 8 + 128 +
                    16 + static_cast<size_t>(A) * TC_LUT_BYTES_PER_PLANE;
         };
         // Matrix products and 1x1 layers with many filters: every filter tile of a pixel tile expands the same packed rows
@@ -1710,7 +1803,7 @@ static int tc_plan(const uint32_t* act, const int8_t* wgt, const bs_conv_params*
                 auto bytes_mb = [&](int m) {
                     const int ckp = g.CK * m;
                     return static_cast<size_t>(2) * wide * RS * ckp + g.pa_bytes + static_cast<size_t>(2) * round_up_i((ckp / 16) * g.HPE * 16, 128) +
-                           2 * wide * 4 + 256 + (4 * TC_MAX_STAGES + 3) * 8 + 128 + 16 + static_cast<size_t>(A) * TC_LUT_BYTES_PER_PLANE +
+                           2 * wide * 4 + 256 + (4 * TC_MAX_STAGES + 6) * 8 + 128 + 16 + static_cast<size_t>(A) * TC_LUT_BYTES_PER_PLANE +
                            static_cast<size_t>(wide) * 16 + 16;
                 };
                 while (mb > 1 && bytes_mb(mb) > 200 * 1024) mb /= 2;
@@ -1728,12 +1821,13 @@ static int tc_plan(const uint32_t* act, const int8_t* wgt, const bs_conv_params*
         while (PT > 1 && (PT * TN > 512 || stream_bytes(TN, PT) > 220 * 1024)) PT /= 2;
         // Large kernels (5x5, 7x7) over many channels: a 128-wide filter chunk of 64 channels does not fit the ring;
         // halve the chunk to one layout block before narrowing the filter tile.
-        if (g.MB > 1 && stream_bytes(TN, PT) > 200 * 1024) {
+        const size_t stream_cap = 200 * 1024;
+        if (g.MB > 1 && stream_bytes(TN, PT) > stream_cap) {
             g.MB = 1; CKP = g.CK; g.CWC = CKP / 32; g.nchunks = p->C / CKP;
             g.e_bytes = round_up_i((CKP / 16) * g.HPE * 16, 128);
             g.nsp = g.nse = g.nchunks < 2 ? g.nchunks : 2;
         }
-        while (TN > 32 && stream_bytes(TN, PT) > 200 * 1024) TN /= 2;
+        while (TN > 32 && stream_bytes(TN, PT) > stream_cap) TN /= 2;
         // More CTAs than SMs: halve the chunk if that lets two CTAs share an SM (one wave instead of two)
         if (g.MB == 2 && RS > 1 && ceil_div_ll(tiles_m, PT) * ceil_div(p->O, TN) > sms) {
             const int e_keep = g.e_bytes, n_keep = g.nchunks;
@@ -1745,6 +1839,13 @@ static int tc_plan(const uint32_t* act, const int8_t* wgt, const bs_conv_params*
                 g.nsp = g.nse = g.nchunks < 2 ? g.nchunks : 2;
             }
         }
+        if (seg_words) {
+            g.seg_words = seg_words;
+            g.pitchA = seg_words;
+            g.seg_chunks = seg_words / (g.CWC * A);
+            g.nseg = ceil_div(g.fullA, seg_words);
+            if (g.nchunks <= g.nsp || PT != 1) return BS_ERR_UNSUPPORTED;      // cannot happen: records of 64 KB / 128 rows are many chunks
+        }
         g.TN = TN;
         g.PT = PT;
         g.b_bytes = TN * RS * CKP;
@@ -1752,7 +1853,7 @@ static int tc_plan(const uint32_t* act, const int8_t* wgt, const bs_conv_params*
         g.off_e = g.off_p + PT * g.pa_bytes;
         g.off_sb = g.off_e + g.nse * PT * g.e_bytes;
         g.off_bar = round_up_i(g.off_sb + 2 * g.TN * 4 + 256, 16);
-        g.off_lut = round_up_i(g.off_bar + (4 * TC_MAX_STAGES + 3) * 8, 16);
+        g.off_lut = round_up_i(g.off_bar + (4 * TC_MAX_STAGES + 6) * 8, 16);
         smem = static_cast<size_t>(g.off_lut) + static_cast<size_t>(A) * TC_LUT_BYTES_PER_PLANE;
         if (smem > 220 * 1024) return BS_ERR_UNSUPPORTED;
     }
@@ -1901,10 +2002,10 @@ static int tc_conv_impl(const uint32_t* act, const int8_t* wgt, const bs_conv_pa
     if (grid > 0x7fffffffLL) return BS_ERR_UNSUPPORTED;
     void (*kern)(TcArgs) = nullptr;
     switch (A) {
-        case 1: kern = bitserial_conv_tc_kernel<1>; break;
-        case 2: kern = bitserial_conv_tc_kernel<2>; break;
-        case 3: kern = bitserial_conv_tc_kernel<3>; break;
-        default: kern = bitserial_conv_tc_kernel<4>; break;
+        case 1: kern = g.seg_words ? bitserial_conv_tc_kernel<1, true> : bitserial_conv_tc_kernel<1, false>; break;
+        case 2: kern = g.seg_words ? bitserial_conv_tc_kernel<2, true> : bitserial_conv_tc_kernel<2, false>; break;
+        case 3: kern = g.seg_words ? bitserial_conv_tc_kernel<3, true> : bitserial_conv_tc_kernel<3, false>; break;
+        default: kern = g.seg_words ? bitserial_conv_tc_kernel<4, true> : bitserial_conv_tc_kernel<4, false>; break;
     }
     if (smem > 48 * 1024 &&
         cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)) != cudaSuccess) {
