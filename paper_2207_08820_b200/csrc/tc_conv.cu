@@ -51,6 +51,8 @@ struct TcArgs {
     int TN, CK, MB, CWC, nchunks, nsp, nse;   // CK: channels per filter-layout block, MB: blocks per pipeline chunk, CWC: words per chunk
     int fullA;                        // words of one packed pixel record (Cw * A)
     int pitchA;                       // words between the staged records of consecutive pixels (fullA, or seg_words)
+    int ld_stride;                    // 2: a 1x1 stride-2 layer fetched through a tensor map that skips every other row and column
+                                      // (the kernels then see a stride-1 layer on the subsampled image: `stride` is 1)
     int seg_words, seg_chunks, nseg;  // flat tiles with long records: the 128 rows are staged seg_words at a time (0: whole records)
     int pmode;                        // how a tile's packed halo is fetched: 0 flat bulk copy, 1 rows merged with W, 2 4-D box
     int TNI, GI, hh, hw;              // packed halo: TNI images x hh rows x hw columns; GI row groups per image
@@ -271,7 +273,7 @@ __device__ __forceinline__ void tc_load_tile(const TcArgs& g, void* dst, uint64_
         bulk_load(dst, g.act + static_cast<size_t>(tile.q0) * g.fullA, bytes, bar);
     } else {
         mbar_expect_tx(bar, static_cast<unsigned>(g.pa_tx_bytes));
-        const int x0 = tile.q0 * g.stride - g.pad, y0 = tile.p0 * g.stride - g.pad;
+        const int x0 = tile.q0 * g.stride * g.ld_stride - g.pad, y0 = tile.p0 * g.stride * g.ld_stride - g.pad;
         if (g.pmode == 1) tma_load_3d(dst, &g.tmA, bar, (x0 - g.xsh) * g.fullA, y0, tile.n0);
         else tma_load_4d(dst, &g.tmA, bar, 0, x0, y0, tile.n0);
     }
@@ -1617,6 +1619,11 @@ static int tc_plan(const uint32_t* act, const int8_t* wgt, const bs_conv_params*
         if (!g.status) return BS_ERR_CUDA;
     }
     g.N = p->N; g.H = p->H; g.W = p->W; g.O = p->O; g.R = p->R; g.S = p->S; g.stride = p->stride; g.pad = p->pad; g.A = A;
+    // A 1x1 stride-2 layer (projection shortcut) reads one pixel in four: its tensor map traverses rows and columns with element
+    // stride 2, so the tile arrives dense and everything after the fetch is a stride-1 1x1 layer on the subsampled image.
+    g.ld_stride = 1;
+    if (RS == 1 && p->stride == 2 && p->pad == 0 && (Cw * A) % 4 == 0 && Cw * A <= 256) { g.ld_stride = 2; g.stride = 1; }
+    const int st = g.stride;          // the stride the tiling sees
     g.relu = p->relu; g.out_bits = p->out_bits; g.out_sign = p->out_sign;
     g.out_cw_off = p->out_c_offset / 32; g.out_cw_total = ceil_div(p->out_c_total > 0 ? p->out_c_total : 1, 32);
     g.res_bits = p->res_bits; g.res_sign = p->res_sign; g.res_c_off = p->res_c_offset;
@@ -1640,7 +1647,7 @@ static int tc_plan(const uint32_t* act, const int8_t* wgt, const bs_conv_params*
 #ifdef BS_TUNING
         if (const char* e = getenv("BS_TC_MB")) wide = atoi(e);
 #endif
-        if (RS == 1 && p->stride == 1 && p->pad == 0)
+        if (RS == 1 && p->pad == 0 && (p->stride == 1 || g.ld_stride == 2))
             for (int mb = wide; mb > 1; mb /= 2)
                 if (p->C % (g.CK * mb) == 0) { g.MB = mb; break; }
         if (RS > 1 && p->stride == 2 && p->C >= 128) g.MB = 1;
@@ -1668,29 +1675,29 @@ static int tc_plan(const uint32_t* act, const int8_t* wgt, const bs_conv_params*
         g.pmode = 0;
         tiles_m = g.tiles_q;
     } else {
-        g.hw = 7 * p->stride + p->S;
+        g.hw = 7 * st + p->S;
         g.xsh = (g.fullA % 4 != 0 && (p->pad & 1)) ? 1 : 0;
         g.hwb = g.fullA % 4 != 0 ? round_up_i(g.hw + g.xsh, 2) : g.hw;
         g.HWH = (g.hw + 1) / 2;
-        g.HWP = p->stride == 2 ? 2 * g.HWH : g.hw;
+        g.HWP = st == 2 ? 2 * g.HWH : g.hw;
         if (g.P <= 16) {        // whole image height in one tile; stack as many images as fit in the 16 row groups
-            g.hh = round_up_i((g.P - 1) * p->stride + p->R, p->stride);
-            g.GI = g.hh / p->stride;
+            g.hh = round_up_i((g.P - 1) * st + p->R, st);
+            g.GI = g.hh / st;
             g.TNI = (16 - g.P) / g.GI + 1;
             if (g.TNI > p->N) g.TNI = p->N;
             g.tiles_p = 1;
         } else {
-            g.hh = round_up_i(15 * p->stride + p->R, p->stride);
+            g.hh = round_up_i(15 * st + p->R, st);
             g.GI = 16; g.TNI = 1;
             g.tiles_p = ceil_div(g.P, 16);
         }
         g.tiles_q = ceil_div(g.Q, 8);
         g.tiles_n = ceil_div(p->N, g.TNI);
         const int rows_box = g.TNI * g.hh;
-        const int rows_read = 15 * p->stride + p->R;
+        const int rows_read = 15 * st + p->R;
         g.HPE = (rows_box > rows_read ? rows_box : rows_read) * g.HWP;
         g.pa_tx_bytes = g.TNI * g.hh * g.hwb * g.fullA * 4;
-        g.pmode = (g.hwb * g.fullA <= 256) ? 1 : 2;
+        g.pmode = (g.hwb * g.fullA <= 256 && g.ld_stride == 1) ? 1 : 2;      // columns can only be skipped as a dimension of their own
         if (g.pmode == 2 && (g.fullA > 256 || g.fullA % 4 != 0)) return BS_ERR_UNSUPPORTED;
         tiles_m = static_cast<long long>(g.tiles_q) * g.tiles_p * g.tiles_n;
     }
@@ -1905,8 +1912,11 @@ static int tc_plan(const uint32_t* act, const int8_t* wgt, const bs_conv_params*
     } else if (g.pmode == 2) {
         cuuint64_t dims[4] = {fullA, static_cast<cuuint64_t>(p->W), static_cast<cuuint64_t>(p->H), static_cast<cuuint64_t>(p->N)};
         cuuint64_t strides[3] = {fullA * 4, fullA * 4 * p->W, fullA * 4 * p->W * p->H};
-        cuuint32_t box[4] = {static_cast<cuuint32_t>(g.fullA), static_cast<cuuint32_t>(g.hw), static_cast<cuuint32_t>(g.hh),
+        // with an element stride s a box dimension counts the elements TRAVERSED: s * n of them deliver n
+        const cuuint32_t ls = static_cast<cuuint32_t>(g.ld_stride);
+        cuuint32_t box[4] = {static_cast<cuuint32_t>(g.fullA), static_cast<cuuint32_t>(g.hw) * ls, static_cast<cuuint32_t>(g.hh) * ls,
                              static_cast<cuuint32_t>(g.TNI)};
+        estr[1] = estr[2] = ls;
         cr = enc(&g.tmA, CU_TENSOR_MAP_DATA_TYPE_UINT32, 4, const_cast<uint32_t*>(act), dims, strides, box, estr,
                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
