@@ -190,13 +190,13 @@ def test_tc_gemm(M, N, K):
     assert np.array_equal(out.cpu().numpy(), oracle.gemm_i32(c["a"], c["w"]))
 
 
-@pytest.mark.parametrize("K", [576, 4608])
-def test_tc_gemm_4096_sampled(K):
+@pytest.mark.parametrize("M,N,K", [(4096, 4096, 576), (4096, 4096, 4608), (4000, 4608, 3200)])
+def test_tc_gemm_4096_sampled(M, N, K):
     """The largest shapes of the matrix-product sweep on the tensor-core entry point: the oracle evaluates sampled rows
     and columns; row and column sums of the whole product are checked against sums formed from the operands (a property
-    that holds at any size); the requantised output is compared on the sampled rows."""
-    M = N = 4096
-    c = wl.gemm_case(M, N, K, seed=wl.gemm_sweep_seed(M, K))
+    that holds at any size); the requantised output is compared on the sampled rows.  K = 4608 and 3200 stage the packed
+    rows in segments; 4000 x 4608 x 3200 has a last pixel tile of 32 rows and a last segment of 56 of 72 words."""
+    c = wl.gemm_case(M, N, K, seed=wl.gemm_sweep_seed(M, K) if M == 4096 else 2100 + K)
     scale, bias = wl.calibrated_scale_bias(c["w"], 2, 0, 2)
     ap = api.bs_pack_rows(dev(c["a"]), 2, 0)
     wp = api.bs_pack_rows(dev(c["w"]), 1, 2)
