@@ -221,6 +221,13 @@ static bool make_plan(Plan& out, int N, int P, int Q, int O, int Cw, int R, int 
         it = cache.emplace(key, std::make_pair(ok, pl)).first;
     }
     out = it->second.second;
+#ifdef BS_TUNING
+    if (getenv("BS_PLAN_VERBOSE")) {
+        const Plan& q = out;
+        fprintf(stderr, "popc plan: N%d %dx%d O%d Cw%d k%d s%d A%d W%d -> PB %d FB %d NFG %d NT %d TWB %d TH %d TNI %d CWC %d chunks %d stages %d split %d tiles %lld smem %zu cost %.0f\n",
+                N, P, Q, O, Cw, R, stride, A, WB, q.PB, q.FB, q.NFG, q.NT, q.TWB, q.TH, q.TNI, q.CWC, q.nchunks, q.nstage, q.ksplit, q.tiles, q.smem, q.cost);
+    }
+#endif
     return it->second.first;
 }
 
