@@ -107,6 +107,49 @@ def test_bad_arguments_are_rejected_on_the_host(L):
     assert L.bs_tc_weights_bytes(200, 64, 3, 3) == 256 * 9 * 64
 
 
+def test_chain_query_and_refusals_on_the_host(L):
+    """The chain planner answers without a device (it plans for a full B200): same-shaped stride-1 layers with packed outputs
+    are accepted, anything else gives 0 bytes, and the launch entry point refuses bad arguments before touching the GPU."""
+    from paper_2207_08820_b200._lib import ConvParams
+    buf = (ctypes.c_char * 4096)()
+    addr = (ctypes.addressof(buf) + 255) & ~255      # stands for device pointers; never dereferenced on these paths
+    INVALID, UNSUPPORTED = 1, 2
+
+    def layer(**kw):
+        d = dict(N=8, C=64, H=56, W=56, O=64, R=3, S=3, stride=1, pad=1, a_bits=2, a_sign=0, w_bits=2, w_sign=1, scale=addr, bias=addr,
+                 relu=1, out_bits=2, out_sign=0, out_c_offset=0, out_c_total=64, i32_layout=0)
+        d.update(kw)
+        return ConvParams(**d)
+
+    def arr(*layers):
+        a = (ConvParams * len(layers))()
+        for k, q in enumerate(layers):
+            ctypes.memmove(ctypes.addressof(a[k]), ctypes.addressof(q), ctypes.sizeof(ConvParams))
+        return a
+
+    four = arr(layer(), layer(residual=addr, res_bits=2, res_scale=0.5, res_c_total=64), layer(), layer())
+    nbytes = L.bs_tc_chain_workspace_bytes(four, 4)
+    tiles = 8 * 4 * 7                                   # 56 x 56 in tiles of 16 x 8 pixels
+    assert nbytes == (4 * tiles + 4) * 4
+    assert L.bs_tc_chain_workspace_bytes(four, 2) == (2 * tiles + 4) * 4
+    assert L.bs_tc_chain_workspace_bytes(four, 1) == 0 and L.bs_tc_chain_workspace_bytes(four, 5) == 0
+    assert L.bs_tc_chain_workspace_bytes(None, 2) == 0
+    assert L.bs_tc_chain_workspace_bytes(arr(layer(), layer(stride=2)), 2) == 0            # output smaller than input
+    assert L.bs_tc_chain_workspace_bytes(arr(layer(), layer(O=128, out_c_total=128)), 2) == 0
+    assert L.bs_tc_chain_workspace_bytes(arr(layer(), layer(R=1, S=1, pad=0)), 2) == 0     # kernel sizes differ
+    assert L.bs_tc_chain_workspace_bytes(arr(layer(out_bits=3), layer()), 2) == 0          # next layer reads 2-bit activations
+    assert L.bs_tc_chain_workspace_bytes(arr(layer(out_bits=0), layer()), 2) == 0          # a layer without packed output
+    assert L.bs_tc_chain_workspace_bytes(arr(layer(out_c_total=96), layer()), 2) == 0      # output is a slice of a wider tensor
+    vp = ctypes.c_void_p * 2
+    two = arr(layer(), layer())
+    ptrs = vp(addr, addr + 1024)
+    assert L.bitserial_conv2d_tc_chain(2, None, ptrs, two, ptrs, addr, 1 << 20, 0, None) == INVALID
+    assert L.bitserial_conv2d_tc_chain(2, ptrs, ptrs, two, ptrs, None, 1 << 20, 0, None) == INVALID
+    assert L.bitserial_conv2d_tc_chain(2, vp(addr, None), ptrs, two, ptrs, addr, 1 << 20, 0, None) == INVALID
+    assert L.bitserial_conv2d_tc_chain(1, ptrs, ptrs, two, ptrs, addr, 1 << 20, 0, None) == UNSUPPORTED
+    assert L.bitserial_conv2d_tc_chain(5, ptrs, ptrs, two, ptrs, addr, 1 << 20, 0, None) == UNSUPPORTED
+
+
 def test_binding_fails_loudly_without_library(tmp_path):
     """Importing the binding with the shared library absent must raise, not fall back."""
     code = ("import sys; sys.path.insert(0, %r)\n"
