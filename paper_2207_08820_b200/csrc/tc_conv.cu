@@ -1806,6 +1806,10 @@ static int tc_plan(const uint32_t* act, const int8_t* wgt, const bs_conv_params*
         if (g.flat && PT == 1 && !stream_tn) {
             for (int wide = 512; wide > 128; wide /= 2) {
                 if (p->O % wide != 0 || tiles_m * (p->O / wide) < sms) continue;
+                // int32 outputs of a short reduction are bound by their own stores (four bytes per output against 2 K operations:
+                // K below ~1000): two CTAs of 256 filters per SM then overlap one's stores with the other's MMAs
+                // (4096 x 4096 x 576: 64 against 72 us; at K = 2304 the 512-filter tile wins, 106 against 126 us)
+                if (wide == 512 && out_i32 && !out_packed && kred < 1024 && p->O % 256 == 0) continue;
                 int mb = g.MB;
                 auto bytes_mb = [&](int m) {
                     const int ckp = g.CK * m;
