@@ -18,24 +18,25 @@ pytestmark = pytest.mark.gpu
 A_BITS, W_BITS = 2, 2
 
 
-def make_chain(seed, N, C, H, W, k, nlayers, res_scale=0.75):
+def make_chain(seed, N, C, H, W, k, nlayers, res_scale=0.75, a_bits=A_BITS):
     """Seeded layers shaped like consecutive residual blocks: layer l reads layer l - 1; odd layers add the input of their block
     (the chain's input for layer 1, the output of layer 1 for layer 3).  Scale and bias are set from the oracle's accumulators
     so that all four codes occur.  Returns the input codes, the per-layer dicts and the oracle's codes per layer."""
     rng = np.random.default_rng(seed)
-    x = rng.integers(0, 4, size=(N, C, H, W), dtype=np.int8)
+    top = (1 << a_bits) - 1
+    x = rng.integers(0, top + 1, size=(N, C, H, W), dtype=np.int8)
     layers, want = [], []
     cur, block_in = x, x
     for l in range(nlayers):
         w = rng.integers(-2, 2, size=(C, C, k, k), dtype=np.int8)
         acc = oracle.conv2d_i32(cur, w, stride=1, pad=k // 2)
         sd = float(acc.std()) + 1.0
-        scale = (rng.uniform(0.8, 1.6, size=C) / sd).astype(np.float32)
-        bias = (1.5 - acc.mean(axis=(0, 2, 3)) * scale + rng.normal(0, 0.3, size=C)).astype(np.float32)
+        scale = (rng.uniform(0.8, 1.6, size=C) * (top / 3.0) / sd).astype(np.float32)
+        bias = (top / 2.0 - acc.mean(axis=(0, 2, 3)) * scale + rng.normal(0, 0.3, size=C)).astype(np.float32)
         res = block_in if l % 2 == 1 else None
         if res is not None:
-            bias -= np.float32(res_scale * 1.5)
-        codes = oracle.requantize(acc, scale, bias, True, A_BITS, oracle.UNSIGNED, res=res, res_scale=res_scale if res is not None else 0.0)
+            bias -= np.float32(res_scale * top / 2.0)
+        codes = oracle.requantize(acc, scale, bias, True, a_bits, oracle.UNSIGNED, res=res, res_scale=res_scale if res is not None else 0.0)
         layers.append(dict(w=w, scale=scale, bias=bias, res=(-1 if l == 1 else l - 2) if res is not None else None,
                            res_scale=res_scale if res is not None else 0.0))
         want.append(codes)
@@ -46,26 +47,26 @@ def make_chain(seed, N, C, H, W, k, nlayers, res_scale=0.75):
 
 
 class ChainOnGpu:
-    def __init__(self, x, layers, k):
+    def __init__(self, x, layers, k, a_bits=A_BITS):
         N, C, H, W = x.shape
-        self.k, self.C = k, C
+        self.k, self.C, self.a_bits = k, C, a_bits
         self.guard = Guarded()
-        self.x = api.bitpack_activations(dev(x.astype(np.float32)), 1.0, A_BITS, api.UNSIGNED, api.NCHW)
-        self.x = self.x.view(N, H, W, C // 32, A_BITS)
-        self.outs = [self.guard.empty((N, H, W, C // 32, A_BITS), fill=-1) for _ in layers]
+        self.x = api.bitpack_activations(dev(x.astype(np.float32)), 1.0, a_bits, api.UNSIGNED, api.NCHW)
+        self.x = self.x.view(N, H, W, C // 32, a_bits)
+        self.outs = [self.guard.empty((N, H, W, C // 32, a_bits), fill=-1) for _ in layers]
         self.wp, self.wtc, self.params, self.acts, self.keep = [], [], [], [], []
         for l, L in enumerate(layers):
             wp = api.pack_weights(dev(L["w"]), W_BITS, api.SIGNED)
             self.wp.append(wp)
-            self.wtc.append(api.tc_prepare_weights(wp, C, api.SIGNED, A_BITS))
+            self.wtc.append(api.tc_prepare_weights(wp, C, api.SIGNED, a_bits))
             act = self.x if l == 0 else self.outs[l - 1]
             res = None if L["res"] is None else (self.x if L["res"] < 0 else self.outs[L["res"]])
             scale, bias = dev(L["scale"]), dev(L["bias"])
             self.keep += [scale, bias]
             self.acts.append(act)
             self.params.append(api.conv_params(act.shape, wp.shape, C=C, stride=1, pad=k // 2, a_sign=api.UNSIGNED, w_sign=api.SIGNED,
-                                               scale=scale, bias=bias, relu=True, out_bits=A_BITS, out_sign=api.UNSIGNED, residual=res,
-                                               res_scale=L["res_scale"], res_bits=A_BITS if res is not None else 0, res_sign=api.UNSIGNED))
+                                               scale=scale, bias=bias, relu=True, out_bits=a_bits, out_sign=api.UNSIGNED, residual=res,
+                                               res_scale=L["res_scale"], res_bits=a_bits if res is not None else 0, res_sign=api.UNSIGNED))
         self.nbytes = api.tc_chain_workspace_bytes(self.params)
         self.ws = torch.zeros(max(self.nbytes, 4) // 4, dtype=torch.int32, device="cuda")
         torch.cuda.synchronize()
@@ -78,7 +79,7 @@ class ChainOnGpu:
         self.guard.check()
         for l, codes in enumerate(want):
             got = words(self.outs[l]).reshape(-1)
-            ref = oracle.pack_activations(codes, A_BITS, oracle.UNSIGNED).reshape(-1)
+            ref = oracle.pack_activations(codes, self.a_bits, oracle.UNSIGNED).reshape(-1)
             assert np.array_equal(got, ref), f"layer {l}: {(got != ref).sum()} of {ref.size} words differ"
 
 
@@ -103,6 +104,19 @@ def test_chain_matches_oracle(seed, N, C, H, W, k, nlayers):
     g = ChainOnGpu(x, layers, k)
     if g.nbytes == 0:
         pytest.skip("the planner does not run this shape with resident filters")
+    g.run()
+    g.check(want)
+
+
+@pytest.mark.parametrize("a_bits", [1, 3, 4])
+def test_chain_other_activation_widths(a_bits):
+    """The 1-, 3- and 4-bit instantiations of the chain kernel (3- and 4-bit outputs take the formula epilogue, 4-bit records are
+    twice as long): same comparison with the oracle, layer by layer."""
+    x, layers, want = make_chain(30 + a_bits, 3, 64, 24, 24, 3, 3, a_bits=a_bits)
+    assert len(np.unique(want[-1])) >= min(3, 1 << a_bits)
+    g = ChainOnGpu(x, layers, 3, a_bits=a_bits)
+    if g.nbytes == 0:
+        pytest.skip("the tensor-core path does not take this activation width at this shape")
     g.run()
     g.check(want)
 
