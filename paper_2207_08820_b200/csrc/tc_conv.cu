@@ -716,7 +716,7 @@ __device__ __forceinline__ TcEpiThread tc_epi_thread(const TcArgs& g, int m)
 // Epilogue of one tile: thread `tid` (0..127, warp = TMEM lane quadrant) owns accumulator row tid = one output pixel.
 __device__ __forceinline__ void tc_epilogue_tile(const TcArgs& g, uint32_t tmem_acc, int tid, int warp, const TcTile& tile, const TcEpiThread& et,
                                                  int o0, const float2* s_sb, const float4* s_bounds, uint32_t thr_addr, int cc0 = 0,
-                                                 int ccstep = 1, int trace_tile = -1, bool res_l2 = false)
+                                                 int ccstep = 1, int trace_tile = -1, bool res_l2 = false, unsigned char* stage = nullptr)
 {
     const int n0 = tile.n0, p0 = tile.p0, q0 = tile.q0;
     const int m = tid;                               // TMEM lane = tile pixel
@@ -752,8 +752,29 @@ __device__ __forceinline__ void tc_epilogue_tile(const TcArgs& g, uint32_t tmem_
         tmem_ld_wait();
         if (tid == 0 && cc == cc0) TC_TRACE(TR_E_LD, trace_tile);
         const int ob = o0 + cc * 32;
+        // Flat tiles with channel-innermost int32 outputs (matrix products): the 32 x 32 block of this warp goes through 4 KB of
+        // shared memory so that a store instruction writes four whole 128-byte lines (eight lanes per row) instead of 16 bytes of 32
+        // different lines.  16-byte chunks are swizzled by the row, which keeps both passes free of bank conflicts.
+        const bool staged = stage != nullptr && g.out_i32 && g.i32_nhwc && g.flat && (g.O & 3) == 0 && g.O - ob >= 32;      // warp-uniform
+        if (staged) {
+            uint4* sw = reinterpret_cast<uint4*>(stage);
+            const int l = tid & 31;
+#pragma unroll
+            for (int c = 0; c < 8; ++c) sw[l * 8 + (c ^ (l & 7))] = make_uint4(v[4 * c], v[4 * c + 1], v[4 * c + 2], v[4 * c + 3]);
+            __syncwarp();
+            const unsigned row0 = static_cast<unsigned>(q0) + static_cast<unsigned>(tid & ~31);
+            const unsigned npix = static_cast<unsigned>(g.N) * static_cast<unsigned>(g.P * g.Q);
+#pragma unroll
+            for (int it = 0; it < 8; ++it) {
+                const int rr = it * 4 + (l >> 3), ch = l & 7;
+                const uint4 val = sw[rr * 8 + (ch ^ (rr & 7))];
+                const unsigned upix = row0 + static_cast<unsigned>(rr);
+                if (upix < npix) *reinterpret_cast<uint4*>(g.out_i32 + static_cast<size_t>(upix) * g.O + ob + ch * 4) = val;
+            }
+            __syncwarp();                 // the next group of 32 filters reuses the block
+        }
         if (valid && ob < g.O) {
-        if (g.out_i32) {
+        if (g.out_i32 && !staged) {
             if (g.i32_nhwc && (g.O & 3) == 0 && g.O - ob >= 32) {
                 // channel-innermost accumulators: the 32 values of this thread are 128 contiguous, 16-byte aligned bytes
                 uint4* dst4 = reinterpret_cast<uint4*>(g.out_i32 + pix * g.O + ob);
@@ -1062,11 +1083,17 @@ __global__ void __launch_bounds__(TC_THREADS) bitserial_conv_tc_kernel(const __g
         if (!ok) atomicOr(g.status, STATUS_TIMEOUT);
         if (tid == 0) TC_TRACE(TR_EBEG, 0);
         tc_fence_after();
+        // every MMA has completed, so the filter ring is free: each of the eight warps takes 4 KB of it to stage its int32 stores
+        unsigned char* i32_stage = nullptr;
+        if (g.flat && g.out_i32 && g.nsp * g.b_bytes >= 8 * 4096) {
+            fence_proxy_async();          // the ring was last written by bulk copies
+            i32_stage = tc_smem + (warp < 4 ? warp : warp - 2) * 4096;
+        }
         for (int t = 0; t < nt; ++t)
             // a warp reads the tensor-memory lanes of quadrant (warp % 4): warps 0-3 take the even groups of 32 filters,
             // warps 6-9 (quadrants 2, 3, 0, 1) the odd ones
             tc_epilogue_tile(g, tmem_base + static_cast<uint32_t>(t * g.TN), (warp & 3) * 32 + lane, warp & 3, tc_decode_tile(g, mt0 + t), eth, o0,
-                             s_sb, s_bounds, thr, warp < 4 ? 0 : 1, 2);
+                             s_sb, s_bounds, thr, warp < 4 ? 0 : 1, 2, -1, false, i32_stage);
         if (tid == 0) TC_TRACE(TR_EEND, 0);
         tc_fence_before();
     }
